@@ -1,0 +1,174 @@
+/*
+ * oled.h — C ABI of the B200 MoE denoise-step library.
+ *
+ * One context holds, for an L-layer MoE stack, a bounded per-layer GPU expert cache
+ * ("each MoE layer owns an independent cache pool", paper Sec. 4.1), the host expert store
+ * (borrowed pinned host memory; "the rest reside in host CPU memory", Sec. 2.2) and the
+ * scratch the step needs.  A call to oled_denoise_step() performs one layer execution of one
+ * denoising iteration over a block of tokens (Sec. 2.1, Sec. 4.1 per-layer flow):
+ *
+ *   gate -> top-k expert ids + gate scores -> token->expert permutation -> hits/misses
+ *   against the resident set before execution (Sec. 4.2: A, R, M = A \ R) -> misses copied
+ *   host->HBM on a side stream -> grouped SwiGLU expert FFN through the expert->slot table
+ *   -> gate-weighted combine -> reuse priority (Sec. 4.3 priority equation) and the cache
+ *   update R' = Top_C(R u G, p) (Sec. 4.2 cache-update equation) with G = M.
+ *
+ * There is no CPU execution path for misses: every missed expert is fetched and computed on
+ * the GPU.  Offloading is lossless (Sec. 5.1): the output does not depend on the capacity.
+ *
+ * Conventions
+ *   - Every function returns OLED_OK (0) or a negative oled_status; nothing aborts or throws.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary host memory unless "pinned" is stated.
+ *   - bf16 tensors are row-major arrays of 16-bit bfloat16 values.
+ *   - One context is used by one host thread at a time.  Work is ordered on the stream given
+ *     to oled_create(); oled_denoise_step() blocks the host until the gate results of the step
+ *     are known (a few hundred bytes are read back to plan the copies), not until the step ends.
+ *   - Shape limits: hidden a multiple of 256; intermediate a multiple of 128;
+ *     1 <= top_k <= 32, top_k <= n_experts <= OLED_MAX_EXPERTS.
+ */
+#ifndef OLED_H_
+#define OLED_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OLED_MAX_EXPERTS 512
+#define OLED_MAX_TOPK 32
+
+typedef enum {
+  OLED_OK = 0,
+  OLED_ERR_INVALID_ARG = -1,    /* null pointer, bad shape, layer out of range, aliasing       */
+  OLED_ERR_NOT_PINNED = -2,     /* host expert store is not page-locked host memory             */
+  OLED_ERR_NOT_REGISTERED = -3, /* step before the layer's router / experts were registered    */
+  OLED_ERR_TOO_MANY_TOKENS = -4,/* n_tokens > max_tokens                                        */
+  OLED_ERR_OOM = -5,            /* device or host allocation failed                             */
+  OLED_ERR_CUDA = -6,           /* a CUDA call failed; see oled_last_cuda_error()               */
+  OLED_ERR_TIMEOUT = -7,        /* a bounded device-side wait ran out; the step's out is invalid */
+  OLED_ERR_NO_SLOT = -8,        /* staging_slots too small for this step's misses               */
+  OLED_ERR_STALE_DEBUG = -9     /* oled_debug_last(): the last step was on another layer        */
+} oled_status;
+
+typedef struct oled_ctx oled_ctx; /* opaque, owned by the library */
+
+typedef struct {
+  int32_t n_layers;
+  int32_t hidden;          /* H */
+  int32_t n_experts;       /* E */
+  int32_t top_k;           /* k */
+  int32_t intermediate;    /* I (SwiGLU) */
+  int32_t max_tokens;      /* upper bound on n_tokens of any step */
+  int32_t has_router_bias; /* 1: oled_register_router() takes a per-expert fp32 bias */
+  int32_t staging_slots;   /* transient slots for misses beyond capacity; 0 = E - min capacity */
+} oled_model_shape;
+
+/* Cumulative counters (Sec. 5.1 metrics: cache utilisation = hits / capacity per execution). */
+typedef struct {
+  uint64_t steps;          /* layer executions                                   */
+  uint64_t hits;           /* sum of #(A n R), R taken before execution (Sec. 4.2) */
+  uint64_t misses;         /* sum of #(A \ R)                                    */
+  uint64_t bytes_moved;    /* host->HBM bytes: misses * 3*H*I*2                  */
+  uint64_t evictions;      /* sum of #(R \ R')                                   */
+  uint64_t active_experts; /* sum of #A                                          */
+  uint64_t assignments;    /* sum of n_tokens * k                                */
+} oled_stats_t;
+
+/* Create a context on the current CUDA device.
+ *   shape           host; copied.
+ *   cache_capacity  host int32[n_layers]; slots C_l per layer, 1 <= C_l <= E ("Cache" in Sec. 5.1).
+ *   cuda_stream     a cudaStream_t (may be 0) on which every step is enqueued; borrowed.
+ *   out_ctx         receives the context; the library owns it until oled_destroy().
+ * Allocates the slot pool (sum C_l + staging slots, each 3*H*I*2 bytes), router weights and
+ * scratch in device memory.  Errors: INVALID_ARG, OOM, CUDA. */
+int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, void* cuda_stream,
+                oled_ctx** out_ctx);
+
+/* Give a layer its gate (Sec. 4.1: "the MoE gate first produces the routed expert IDs, gate
+ * scores").  w_router: [E,H] bf16, host or device, copied by the call.  bias: fp32[E] host or
+ * device, or NULL (must be non-NULL iff has_router_bias). */
+int oled_register_router(oled_ctx* ctx, int32_t layer, const void* w_router, const float* bias);
+
+/* Give a layer its host expert store (Sec. 2.2, Sec. 4.1).  host_blob is PINNED host memory,
+ * borrowed until oled_destroy() and never written; expert e starts at
+ * host_blob + e*expert_stride_bytes and holds gate[I,H] | up[I,H] | down[H,I] in bf16
+ * (3*H*I*2 bytes; stride >= that and a multiple of 16).  Errors: NOT_PINNED, INVALID_ARG. */
+int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob,
+                          size_t expert_stride_bytes);
+
+/* One layer execution of one denoising iteration (Sec. 4.1 per-layer flow; Sec. 4.2-4.3).
+ *   hidden       device [n_tokens,H] bf16, read only.
+ *   confidences  device fp32[n_tokens], token confidences c_t in [0,1] (Sec. 4.3).
+ *   n_tokens     0 <= n_tokens <= max_tokens.
+ *   out          device [n_tokens,H] bf16: sum_j g[t,j]*FFN_{e(t,j)}(hidden[t]); must not alias hidden.
+ * Buffers are borrowed until the enqueued work completes on the context's stream.  The layer's
+ * resident set and the counters are updated before the call returns.
+ * Errors: INVALID_ARG, NOT_REGISTERED, TOO_MANY_TOKENS, NO_SLOT, CUDA, TIMEOUT (reported by
+ * the next call that synchronises). */
+int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
+                      int32_t n_tokens, void* out);
+
+/* Same step with HOST buffers: hidden/confidences are copied host->device, out device->host,
+ * on the context's stream; the call returns after out has arrived.  Pinned buffers make the
+ * copies asynchronous with respect to the expert fills. */
+int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden,
+                           const float* host_confidences, int32_t n_tokens, void* host_out);
+
+/* Counters of one layer, or summed over layers for layer = -1.  Synchronises the stream. */
+int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out);
+
+/* Parity aid: results of the most recent step, which must have been on `layer`.  All outputs
+ * are host buffers and may be NULL to skip: ids int32[T*k], gate fp32[T*k], perm int32[T*k]
+ * (perm[r] = t*k+j of sorted row r), counts int32[E], scores uint64[E] (integer numerators of
+ * the Sec. 4.3 priority), resident_before / resident_after uint8[E] (0/1).  Synchronises. */
+int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int32_t* perm,
+                    int32_t* counts, uint64_t* scores, uint8_t* resident_before,
+                    uint8_t* resident_after);
+
+/* Gate logits fp32[T*E] of the most recent step (host buffer).  Synchronises. */
+int oled_debug_logits(oled_ctx* ctx, int32_t layer, float* logits);
+
+/* Back to the cold state: every layer's resident set empty, counters zero.  Synchronises. */
+int oled_reset_cache(oled_ctx* ctx);
+
+/* y = bf16(x + r) elementwise over n bf16 values on the context's stream (the residual
+ * between the layers of a stack is the caller's; this is a convenience kernel). */
+int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size_t n);
+
+/* Options.  OLED_OPT_FFN_IMPL: 0 = tcgen05 tensor-core kernels (default), 1 = plain-FMA
+ * bring-up kernels.  OLED_OPT_MISS_CHUNK: experts per fill group (default 4). */
+#define OLED_OPT_FFN_IMPL 1
+#define OLED_OPT_MISS_CHUNK 2
+int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value);
+
+/* Number of kernels the library has launched on this context so far. */
+int oled_launch_count(oled_ctx* ctx, uint64_t* out);
+
+/* Wait for the context's streams; returns TIMEOUT if a device-side wait ran out. */
+int oled_synchronize(oled_ctx* ctx);
+
+void oled_destroy(oled_ctx* ctx);
+
+const char* oled_strerror(int code);
+
+/* The CUDA error code of the last OLED_ERR_CUDA on this context (cudaError_t as int). */
+int oled_last_cuda_error(oled_ctx* ctx);
+
+/* ---- host-only policy simulator (no GPU needed): the same C++ policy code the step uses,
+ * driven by recorded counts and integer scores.  For tests of the host logic. ---- */
+typedef struct oled_policy oled_policy;
+int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, oled_policy** out);
+/* counts int32[E], scores uint64[E] -> resident_before/after uint8[E], slot_of int32[E] (slot of
+ * every activated expert during the step, -1 otherwise), n_hits/n_misses/n_evictions. */
+int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scores,
+                     uint8_t* resident_before, uint8_t* resident_after, int32_t* slot_of,
+                     int32_t* n_hits, int32_t* n_misses, int32_t* n_evictions);
+void oled_policy_destroy(oled_policy* p);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OLED_H_ */

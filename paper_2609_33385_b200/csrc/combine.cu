@@ -1,0 +1,67 @@
+// Weighted un-permute / combine: the gate-weighted sum of the expert outputs of each token
+// (paper Sec. 2.1: the MoE layer output is the gate-score-weighted sum over the top-k experts).
+// Deterministic: ranks are added in ascending order in fp32, then rounded to bf16.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "kernels.h"
+
+namespace oled {
+namespace {
+
+__global__ void __launch_bounds__(256)
+combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
+               const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out) {
+  const int t = blockIdx.x;
+  __shared__ float s_g[OLED_MAX_TOPK];
+  __shared__ int s_r[OLED_MAX_TOPK];
+  if (threadIdx.x < K) {
+    s_g[threadIdx.x] = gate[(size_t)t * K + threadIdx.x];
+    s_r[threadIdx.x] = pos[(size_t)t * K + threadIdx.x];
+  }
+  __syncthreads();
+  for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < K; ++j) {
+      const float4 v = *reinterpret_cast<const float4*>(y + (size_t)s_r[j] * H + h);
+      const float g = s_g[j];
+      acc.x = fmaf(g, v.x, acc.x);
+      acc.y = fmaf(g, v.y, acc.y);
+      acc.z = fmaf(g, v.z, acc.z);
+      acc.w = fmaf(g, v.w, acc.w);
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + (size_t)t * H + h) = pk;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ r,
+                    uint16_t* __restrict__ y, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (size_t)gridDim.x * blockDim.x) {
+    const float a = __uint_as_float((uint32_t)x[i] << 16);
+    const float b = __uint_as_float((uint32_t)r[i] << 16);
+    const __nv_bfloat16 s = __float2bfloat16_rn(a + b);
+    y[i] = *reinterpret_cast<const uint16_t*>(&s);
+  }
+}
+
+}  // namespace
+
+void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
+                    int H, int K, uint16_t* out) {
+  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out);
+}
+
+void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {
+  const int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+  residual_add_kernel<<<blocks, 256, 0, st>>>(x, r, y, n);
+}
+
+}  // namespace oled

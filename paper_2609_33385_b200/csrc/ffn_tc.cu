@@ -1,0 +1,477 @@
+// Grouped SwiGLU expert FFN on the 5th-generation tensor cores (paper Sec. 4.1: "cache-hit
+// experts execute directly on the GPU"; misses follow once their weights have landed).
+//
+// Two persistent kernels per expert group, both "weights on M, tokens on N":
+//   KIND 1:  D_g[i,n] = sum_h Wg[i,h] x[n,h],  D_u likewise with Wu  (two TMEM accumulators),
+//            epilogue  hbuf[n,i] = bf16( silu(D_g) * D_u )
+//   KIND 2:  D[c,n]   = sum_i Wd[c,i] hbuf[n,i],  epilogue  y[n,c] = D   (fp32)
+// The 128 rows of a weight tile fill the MMA's M dimension whatever the number of tokens an
+// expert received, so that the few-tokens-per-expert regime of a denoising block streams each
+// resident expert's weights exactly once at HBM speed, and the many-token regime uses N up to
+// 256.  Weights are addressed through the expert->slot table: one 3-D tensor map covers the
+// whole slot pool and the slot number is a TMA coordinate.
+//
+// Warp roles (192 threads): warps 0-3 epilogue (TMEM lane quarter = warp id), warp 4 lane 0 TMA
+// producer, warp 5 lane 0 MMA issuer (warp 5 also owns the TMEM allocation).  Every mbarrier
+// wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
+// copies time to land, frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "kernels.h"
+
+namespace oled {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kBlockM = 128;
+constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
+constexpr uint32_t kATile = kBlockM * kBlockK * 2;
+constexpr int kMaxStages = 10;
+constexpr uint32_t kSmemMax = 232448;  // 227 KB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct __align__(16) SharedCtl {
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  uint32_t tmem_base;
+  int abort;
+  int n_tiles_total;
+  int pad;
+  int tile_prefix[OLED_MAX_EXPERTS + 1];
+  int row_start[OLED_MAX_EXPERTS];
+  int count[OLED_MAX_EXPERTS];
+};
+constexpr uint32_t kCtlBytes = (sizeof(SharedCtl) + 1023u) & ~1023u;
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting or the time limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t* status) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 1023u) == 1023u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = globaltimer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, (uint32_t)kStatusWaitTimeout);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(const CUtensorMap* map, uint32_t dst, uint32_t bar, int c0,
+                                            int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint32_t dst, uint32_t bar, int c0,
+                                            int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart (what a {64 x rows} bf16 TMA box with SWIZZLE_128B writes).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4)   // start address
+         | (1ull << 16)                         // leading byte offset (unused for this layout)
+         | ((uint64_t)(1024u >> 4) << 32)       // stride byte offset
+         | (1ull << 46)                         // descriptor version (sm_100)
+         | (2ull << 61);                        // SWIZZLE_128B
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+}
+
+struct Item {
+  int slot, m0, row0, valid;
+};
+__device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int m_tiles,
+                                            int n_box, int& g, Item& it) {
+  const int q = item / m_tiles;
+  const int m = item - q * m_tiles;
+  while (ctl->tile_prefix[g + 1] <= q) ++g;
+  const int nt = q - ctl->tile_prefix[g];
+  it.slot = grp.slot[g];
+  it.m0 = m * kBlockM;
+  it.row0 = ctl->row_start[g] + nt * n_box;
+  it.valid = min(n_box, ctl->count[g] - nt * n_box);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
+              const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
+  const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_box = grp.n_box;
+  constexpr uint32_t a_bytes = (KIND == 1 ? 2u : 1u) * kATile;
+  const uint32_t stage_bytes = a_bytes + (uint32_t)n_box * 128u;
+  const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
+  const int m_tiles = (KIND == 1 ? I : H) / kBlockM;
+  const int acc_cols = (KIND == 1 ? 2 : 1) * n_box;
+  const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
+
+  // ---- set-up: work table, barriers, TMEM
+  for (int g = threadIdx.x; g < grp.n; g += kThreads) {
+    const int e = grp.expert[g];
+    const int s = offsets[e];
+    ctl->row_start[g] = s;
+    ctl->count[g] = offsets[e + 1] - s;
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kMaxStages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[a]), 128);
+    }
+    ctl->abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int g = 0; g < grp.n; ++g) {
+      ctl->tile_prefix[g] = acc;
+      acc += (ctl->count[g] + n_box - 1) / n_box;
+    }
+    ctl->tile_prefix[grp.n] = acc;
+    ctl->n_tiles_total = acc;
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&ctl->tmem_base)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+
+  const uint32_t tmem_base = ctl->tmem_base;
+  const int total_items = ctl->n_tiles_total * m_tiles;
+  volatile int* abort_flag = &ctl->abort;
+
+  if (warp == 4 && lane == 0) {
+    // ------------------------------------------------------------ TMA producer
+    int stage = 0, g = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+      Item it;
+      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status)) {
+          ok = false;
+          break;
+        }
+        const uint32_t bar = smem_u32(&ctl->full[stage]);
+        const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
+        mbar_expect_tx(bar, stage_bytes);
+        if (KIND == 1) {
+          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // gate rows
+          tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
+        } else {
+          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // down rows
+        }
+        tma_load_2d(&tm_act, a_addr + a_bytes, bar, kb * kBlockK, it.row0);
+        if (++stage == n_stages) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+    }
+    if (!ok) {  // let copies already issued land before the CTA's shared memory is released
+      const unsigned long long t0 = globaltimer();
+      while (globaltimer() - t0 < 2000000ull) {
+      }
+    }
+  } else if (warp == 5 && lane == 0) {
+    // ------------------------------------------------------------ MMA issuer
+    int stage = 0, g = 0, local = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
+      Item it;
+      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      const int acc = local % acc_stages;
+      const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
+      if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
+      tc_fence_after();
+      const int n_mma = max(16, (it.valid + 15) & ~15);
+      const uint32_t idesc = make_idesc(n_mma);
+      const uint32_t d0 = tmem_base + (uint32_t)(acc * acc_cols);
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, status)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
+        const uint32_t b_addr = a_addr + a_bytes;
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k) {
+          const uint64_t db = make_smem_desc(b_addr + k * 32);
+          const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+          tc_mma(d0, make_smem_desc(a_addr + k * 32), db, idesc, accum);
+          if (KIND == 1) tc_mma(d0 + (uint32_t)n_box, make_smem_desc(a_addr + kATile + k * 32), db, idesc, accum);
+        }
+        tc_commit(smem_u32(&ctl->empty[stage]));
+        if (++stage == n_stages) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+      if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
+    }
+  } else if (warp < 4) {
+    // ------------------------------------------------------------ epilogue
+    int g = 0, local = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
+      Item it;
+      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      const int acc = local % acc_stages;
+      const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
+      // warp-uniform outcome: tcgen05.ld below is warp-collective
+      const bool ready = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, status);
+      if (!__all_sync(0xffffffffu, ready)) break;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * acc_cols);
+      const int n_mma = max(16, (it.valid + 15) & ~15);
+      const int col = it.m0 + warp * 32 + lane;  // output feature owned by this thread
+      for (int c = 0; c < n_mma; c += 16) {
+        uint32_t ra[16];
+        tmem_ld16(t_row + (uint32_t)c, ra);
+        if (KIND == 1) {
+          uint32_t rb[16];
+          tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
+          tmem_ld_wait();
+          uint16_t* hb = reinterpret_cast<uint16_t*>(out_ptr);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            if (c + j < it.valid) {
+              const float a = __uint_as_float(ra[j]);
+              const float u = __uint_as_float(rb[j]);
+              const float hm = __fdividef(a, 1.0f + __expf(-a)) * u;
+              const __nv_bfloat16 b = __float2bfloat16_rn(hm);
+              hb[(size_t)(it.row0 + c + j) * I + col] = *reinterpret_cast<const uint16_t*>(&b);
+            }
+          }
+        } else {
+          tmem_ld_wait();
+          float* y = reinterpret_cast<float*>(out_ptr);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c + j < it.valid) y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, const cuuint64_t* strides,
+            const cuuint32_t* box) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides,
+            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int stages_for(int kind, int n_box) {
+  const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+  const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
+  return (int)std::min<uint32_t>(kMaxStages, avail / stage);
+}
+uint32_t smem_for(int kind, int n_box, int stages) {
+  const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+  return kCtlBytes + 1024u + (uint32_t)stages * stage;
+}
+
+}  // namespace
+
+int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I,
+                 const uint16_t* xp, const uint16_t* hbuf, int rows) {
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
+    const cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)slot_bytes};
+    const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
+    if (!encode(&maps->w13, 3, pool, dims, strides, box)) return OLED_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)I, (cuuint64_t)H, (cuuint64_t)n_slots};
+    const cuuint64_t strides[2] = {(cuuint64_t)I * 2, (cuuint64_t)slot_bytes};
+    const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
+    if (!encode(&maps->w2, 3, pool + (size_t)2 * I * H * 2, dims, strides, box)) return OLED_ERR_CUDA;
+  }
+  for (int i = 0; i < 5; ++i) {
+    const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(16 << i)};
+    {
+      const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
+      const cuuint64_t strides[1] = {(cuuint64_t)H * 2};
+      if (!encode(&maps->xp[i], 2, xp, dims, strides, box)) return OLED_ERR_CUDA;
+    }
+    {
+      const cuuint64_t dims[2] = {(cuuint64_t)I, (cuuint64_t)rows};
+      const cuuint64_t strides[1] = {(cuuint64_t)I * 2};
+      if (!encode(&maps->hbuf[i], 2, hbuf, dims, strides, box)) return OLED_ERR_CUDA;
+    }
+  }
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) !=
+            cudaSuccess)
+      return OLED_ERR_CUDA;
+    attr_done = true;
+  }
+  return OLED_OK;
+}
+
+static int box_index(int max_count, int cap) {
+  int i = 0;
+  while ((16 << i) < max_count && (16 << i) < cap) ++i;
+  return i;
+}
+
+int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count,
+                  const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
+                  uint32_t* status) {
+  if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
+  FfnGroup grp = grp_in;
+  // KIND 1 holds two accumulators per tile: N <= 128 keeps them double-buffered in TMEM.
+  const int i1 = box_index(max_count, 128), i2 = box_index(max_count, 256);
+  {
+    grp.n_box = 16 << i1;
+    const int stages = stages_for(1, grp.n_box);
+    ffn_tc_kernel<1><<<n_sms, kThreads, smem_for(1, grp.n_box, stages), st>>>(
+        maps.w13, maps.xp[i1], grp, offsets, hbuf, H, I, stages, status);
+  }
+  {
+    grp.n_box = 16 << i2;
+    const int stages = stages_for(2, grp.n_box);
+    ffn_tc_kernel<2><<<n_sms, kThreads, smem_for(2, grp.n_box, stages), st>>>(
+        maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
+  }
+  return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
+}
+
+}  // namespace oled

@@ -1,0 +1,63 @@
+// Launch wrappers of the CUDA kernels of the denoise step (internal to the library).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/oled.h"
+
+namespace oled {
+
+// The experts one FFN launch works on and the slot each one's weights sit in: the per-launch
+// image of the expert->slot indirection table, passed by value in kernel-parameter space.
+struct FfnGroup {
+  int32_t n;
+  int32_t n_box;  // token rows per TMA box / MMA N tile of this launch
+  uint16_t expert[OLED_MAX_EXPERTS];
+  uint16_t slot[OLED_MAX_EXPERTS];
+};
+
+// Device status word values (0 = ok).
+enum : uint32_t { kStatusOk = 0, kStatusWaitTimeout = 1 };
+
+// ---- route.cu -------------------------------------------------------------------------
+// Gate logits in the contract order, top-k (ties to the lower index), softmax over the selected
+// logits, per-expert counts and integer reuse-score numerators (atomics on zeroed arrays).
+void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
+                  const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
+                  float* gate, int32_t* counts, unsigned long long* scores);
+// Offsets (exclusive scan), stable permutation by expert and its inverse.
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
+                    int32_t* offsets, int32_t* perm, int32_t* pos);
+// xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
+void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
+                   uint16_t* xp);
+
+// ---- combine.cu -----------------------------------------------------------------------
+// out[t,:] = bf16( sum_j gate[t,j] * y[pos[t*K+j],:] ), j ascending, fp32 accumulation.
+void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
+                    int H, int K, uint16_t* out);
+void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n);
+
+// ---- ffn_simple.cu (bring-up path, plain FMA) ---------------------------------------------
+void launch_ffn_simple(cudaStream_t st, const FfnGroup& grp, const uint8_t* pool, size_t slot_bytes,
+                       const int32_t* offsets, const uint16_t* xp, uint16_t* hbuf, float* y, int H,
+                       int I);
+
+// ---- ffn_tc.cu (tcgen05 / TMEM / TMA) ------------------------------------------------------
+struct FfnTcMaps {
+  CUtensorMap w13;       // [slots][2I][H] bf16, box {64,128,1}
+  CUtensorMap w2;        // [slots][H][I]  bf16, box {64,128,1}
+  CUtensorMap xp[5];     // [rows][H] bf16, box {64, 16<<i}
+  CUtensorMap hbuf[5];   // [rows][I] bf16, box {64, 16<<i}
+};
+// Builds the tensor maps; returns 0 or a negative oled_status.
+int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I,
+                 const uint16_t* xp, const uint16_t* hbuf, int rows);
+// Two launches: gate/up + SwiGLU into hbuf, then down projection into y.
+int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count,
+                  const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
+                  uint32_t* status);
+
+}  // namespace oled

@@ -1,0 +1,574 @@
+// C ABI of the MoE denoise-step library: context, host expert store, the per-step
+// orchestration (gate -> policy -> fills on a side stream -> grouped FFN -> combine) and the
+// counters.  The flow follows the paper's per-layer order (Sec. 4.1) with the sets of Sec. 4.2
+// and the retention rule of Sec. 4.2/4.3; every missed expert is fetched (no CPU execution).
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.h"
+#include "policy.h"
+
+using namespace oled;
+
+namespace {
+
+struct LayerData {
+  LayerCacheState cache;
+  const uint8_t* host_blob = nullptr;
+  size_t host_stride = 0;
+  uint16_t* w_router = nullptr;  // device [E,H]
+  float* bias = nullptr;         // device [E] or null
+  bool has_router = false;
+  oled_stats_t stats{};
+};
+
+}  // namespace
+
+struct oled_ctx {
+  oled_model_shape shape{};
+  cudaStream_t stream = nullptr;       // caller's
+  cudaStream_t copy_stream = nullptr;  // expert fills
+  std::vector<cudaEvent_t> fill_events;
+  cudaEvent_t gate_event = nullptr;
+  int n_sms = 148;
+  size_t slot_bytes = 0;
+  int n_slots = 0;
+  uint8_t* pool = nullptr;
+  SlotPool slots;
+  std::vector<LayerData> layers;
+  StepPlan plan;
+
+  // scratch (device)
+  unsigned long long* d_scores = nullptr;  // [E]   } one block, zeroed per step
+  int32_t* d_counts = nullptr;             // [E]   }
+  size_t ctrl_bytes = 0;
+  float* d_logits = nullptr;   // [T,E]
+  int32_t* d_ids = nullptr;    // [T,k]
+  float* d_gate = nullptr;     // [T,k]
+  int32_t* d_offsets = nullptr;// [E+1]
+  int32_t* d_perm = nullptr;   // [T*k]
+  int32_t* d_pos = nullptr;    // [T*k]
+  uint16_t* d_xp = nullptr;    // [T*k,H]
+  uint16_t* d_hbuf = nullptr;  // [T*k,I]
+  float* d_y = nullptr;        // [T*k,H]
+  uint32_t* d_status = nullptr;
+  uint16_t* d_hidden_stage = nullptr;  // for the host-buffer entry point
+  float* d_conf_stage = nullptr;
+  uint16_t* d_out_stage = nullptr;
+  // pinned host mirror of the control block
+  uint8_t* h_ctrl = nullptr;
+  uint32_t* h_status = nullptr;
+
+  FfnTcMaps maps;
+  int ffn_impl = 0;
+  int miss_chunk = 4;
+  uint64_t launches = 0;
+  int last_cuda_error = 0;
+  int last_layer = -1;
+  int last_tokens = 0;
+  std::vector<uint8_t> last_before, last_after;
+};
+
+namespace {
+
+#define OLED_CUDA(ctx, call)                      \
+  do {                                            \
+    cudaError_t err__ = (call);                   \
+    if (err__ != cudaSuccess) {                   \
+      (ctx)->last_cuda_error = (int)err__;        \
+      return OLED_ERR_CUDA;                       \
+    }                                             \
+  } while (0)
+
+template <typename T>
+int dev_alloc(oled_ctx* ctx, T** p, size_t n) {
+  void* q = nullptr;
+  cudaError_t err = cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T));
+  if (err != cudaSuccess) {
+    ctx->last_cuda_error = (int)err;
+    cudaGetLastError();
+    return OLED_ERR_OOM;
+  }
+  *p = static_cast<T*>(q);
+  return OLED_OK;
+}
+
+int check_status(oled_ctx* ctx) {
+  if (ctx->h_status && *ctx->h_status != kStatusOk) return OLED_ERR_TIMEOUT;
+  return OLED_OK;
+}
+
+int sync_all(oled_ctx* ctx) {
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                                 ctx->stream));
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  return check_status(ctx);
+}
+
+void free_ctx(oled_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->stream || ctx->copy_stream) cudaDeviceSynchronize();
+  for (auto& l : ctx->layers) {
+    cudaFree(l.w_router);
+    cudaFree(l.bias);
+  }
+  cudaFree(ctx->pool);
+  cudaFree(ctx->d_scores);
+  cudaFree(ctx->d_logits);
+  cudaFree(ctx->d_ids);
+  cudaFree(ctx->d_gate);
+  cudaFree(ctx->d_offsets);
+  cudaFree(ctx->d_perm);
+  cudaFree(ctx->d_pos);
+  cudaFree(ctx->d_xp);
+  cudaFree(ctx->d_hbuf);
+  cudaFree(ctx->d_y);
+  cudaFree(ctx->d_status);
+  cudaFree(ctx->d_hidden_stage);
+  cudaFree(ctx->d_conf_stage);
+  cudaFree(ctx->d_out_stage);
+  if (ctx->h_ctrl) cudaFreeHost(ctx->h_ctrl);
+  if (ctx->h_status) cudaFreeHost(ctx->h_status);
+  for (auto ev : ctx->fill_events) cudaEventDestroy(ev);
+  if (ctx->gate_event) cudaEventDestroy(ctx->gate_event);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  cudaGetLastError();
+  delete ctx;
+}
+
+// One FFN launch pair over `experts` (ids), weights through the layer's slot table.
+int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& experts, size_t begin, size_t end,
+                  const int32_t* counts) {
+  if (begin >= end) return OLED_OK;
+  FfnGroup grp;
+  grp.n = (int32_t)(end - begin);
+  grp.n_box = 16;
+  int max_count = 0;
+  for (size_t i = begin; i < end; ++i) {
+    const int32_t e = experts[i];
+    grp.expert[i - begin] = (uint16_t)e;
+    grp.slot[i - begin] = (uint16_t)L.cache.slot_of[e];
+    max_count = std::max(max_count, counts[e]);
+  }
+  const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
+  if (ctx->ffn_impl == 1) {
+    launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
+                      ctx->d_y, H, I);
+  } else {
+    const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, ctx->d_offsets, ctx->d_hbuf, ctx->d_y,
+                                 H, I, ctx->n_sms, ctx->d_status);
+    if (rc != OLED_OK) return rc;
+  }
+  ctx->launches += 2;
+  OLED_CUDA(ctx, cudaGetLastError());
+  return OLED_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* oled_strerror(int code) {
+  switch (code) {
+    case OLED_OK: return "ok";
+    case OLED_ERR_INVALID_ARG: return "invalid argument";
+    case OLED_ERR_NOT_PINNED: return "host expert store is not pinned host memory";
+    case OLED_ERR_NOT_REGISTERED: return "layer has no router or no expert store registered";
+    case OLED_ERR_TOO_MANY_TOKENS: return "n_tokens exceeds max_tokens";
+    case OLED_ERR_OOM: return "out of memory";
+    case OLED_ERR_CUDA: return "CUDA error (see oled_last_cuda_error)";
+    case OLED_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case OLED_ERR_NO_SLOT: return "not enough staging slots for this step's misses";
+    case OLED_ERR_STALE_DEBUG: return "the most recent step was on another layer";
+    default: return "unknown error";
+  }
+}
+
+int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, void* cuda_stream,
+                oled_ctx** out_ctx) {
+  if (!shape || !cache_capacity || !out_ctx) return OLED_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  const oled_model_shape& s = *shape;
+  if (s.n_layers <= 0 || s.hidden <= 0 || s.hidden % 256 != 0 || s.intermediate <= 0 ||
+      s.intermediate % 128 != 0 || s.n_experts <= 0 || s.n_experts > OLED_MAX_EXPERTS || s.top_k <= 0 ||
+      s.top_k > OLED_MAX_TOPK || s.top_k > s.n_experts || s.max_tokens <= 0 || s.staging_slots < 0)
+    return OLED_ERR_INVALID_ARG;
+  int min_cap = s.n_experts;
+  long long total_cap = 0;
+  for (int l = 0; l < s.n_layers; ++l) {
+    if (cache_capacity[l] <= 0 || cache_capacity[l] > s.n_experts) return OLED_ERR_INVALID_ARG;
+    min_cap = std::min(min_cap, cache_capacity[l]);
+    total_cap += cache_capacity[l];
+  }
+  oled_ctx* ctx = new (std::nothrow) oled_ctx();
+  if (!ctx) return OLED_ERR_OOM;
+  ctx->shape = s;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  int rc = OLED_OK;
+  auto fail = [&](int code) {
+    const int cu = ctx->last_cuda_error;
+    (void)cu;
+    free_ctx(ctx);
+    return code;
+  };
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(OLED_ERR_CUDA);
+  }
+  ctx->n_sms = prop.multiProcessorCount;
+  if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->gate_event, cudaEventDisableTiming) != cudaSuccess)
+    return fail(OLED_ERR_CUDA);
+  ctx->fill_events.resize(s.n_experts);
+  for (auto& ev : ctx->fill_events) {
+    ev = nullptr;
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(OLED_ERR_CUDA);
+  }
+
+  const int staging = s.staging_slots > 0 ? s.staging_slots : (s.n_experts - min_cap);
+  ctx->slot_bytes = (size_t)3 * s.hidden * s.intermediate * 2;
+  ctx->n_slots = (int)std::min<long long>(total_cap + staging, 65535);
+  if (total_cap + staging > 65535) return fail(OLED_ERR_INVALID_ARG);
+  ctx->slots.init(ctx->n_slots);
+  ctx->layers.resize(s.n_layers);
+  for (int l = 0; l < s.n_layers; ++l) ctx->layers[l].cache.init(s.n_experts, cache_capacity[l]);
+
+  const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
+  const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t));
+  uint8_t* ctrl = nullptr;
+  if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctrl, ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
+  ctx->d_scores = reinterpret_cast<unsigned long long*>(ctrl);
+  ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
+  if ((rc = dev_alloc(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_offsets, E + 1)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_perm, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_pos, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_xp, T * K * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_hbuf, T * K * I)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_y, T * K * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_status, 1)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_hidden_stage, T * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_conf_stage, T)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_out_stage, T * H)) != OLED_OK) return fail(rc);
+  for (int l = 0; l < s.n_layers; ++l) {
+    if ((rc = dev_alloc(ctx, &ctx->layers[l].w_router, E * H)) != OLED_OK) return fail(rc);
+    if (s.has_router_bias && (rc = dev_alloc(ctx, &ctx->layers[l].bias, E)) != OLED_OK) return fail(rc);
+  }
+  if (cudaMallocHost(reinterpret_cast<void**>(&ctx->h_ctrl), ctx->ctrl_bytes) != cudaSuccess ||
+      cudaMallocHost(reinterpret_cast<void**>(&ctx->h_status), sizeof(uint32_t)) != cudaSuccess)
+    return fail(OLED_ERR_OOM);
+  *ctx->h_status = kStatusOk;
+  if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->d_xp, 0, T * K * H * 2) != cudaSuccess ||
+      cudaMemset(ctx->d_hbuf, 0, T * K * I * 2) != cudaSuccess ||
+      cudaMemset(ctx->d_y, 0, T * K * H * 4) != cudaSuccess)
+    return fail(OLED_ERR_CUDA);
+  rc = ffn_tc_setup(&ctx->maps, ctx->pool, ctx->slot_bytes, ctx->n_slots, s.hidden, s.intermediate, ctx->d_xp,
+                    ctx->d_hbuf, (int)(T * K));
+  if (rc != OLED_OK) return fail(rc);
+  if (const char* env = getenv("OLED_FFN_IMPL")) ctx->ffn_impl = atoi(env) == 1 ? 1 : 0;
+  if (const char* env = getenv("OLED_MISS_CHUNK")) ctx->miss_chunk = std::max(1, atoi(env));
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(OLED_ERR_CUDA);
+  *out_ctx = ctx;
+  return OLED_OK;
+}
+
+int oled_register_router(oled_ctx* ctx, int32_t layer, const void* w_router, const float* bias) {
+  if (!ctx || !w_router || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  if ((bias != nullptr) != (ctx->shape.has_router_bias != 0)) return OLED_ERR_INVALID_ARG;
+  LayerData& L = ctx->layers[layer];
+  const size_t bytes = (size_t)ctx->shape.n_experts * ctx->shape.hidden * 2;
+  OLED_CUDA(ctx, cudaMemcpyAsync(L.w_router, w_router, bytes, cudaMemcpyDefault, ctx->stream));
+  if (bias)
+    OLED_CUDA(ctx, cudaMemcpyAsync(L.bias, bias, (size_t)ctx->shape.n_experts * sizeof(float),
+                                   cudaMemcpyDefault, ctx->stream));
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  L.has_router = true;
+  return OLED_OK;
+}
+
+int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob, size_t expert_stride_bytes) {
+  if (!ctx || !host_blob || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  if (expert_stride_bytes < ctx->slot_bytes || expert_stride_bytes % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(host_blob) % 16 != 0)
+    return OLED_ERR_INVALID_ARG;
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host_blob) != cudaSuccess) {
+    cudaGetLastError();
+    return OLED_ERR_NOT_PINNED;
+  }
+  if (a.type != cudaMemoryTypeHost) return OLED_ERR_NOT_PINNED;
+  // the last byte must be pinned too
+  const uint8_t* last = static_cast<const uint8_t*>(host_blob) +
+                        (size_t)(ctx->shape.n_experts - 1) * expert_stride_bytes + ctx->slot_bytes - 1;
+  if (cudaPointerGetAttributes(&a, last) != cudaSuccess || a.type != cudaMemoryTypeHost) {
+    cudaGetLastError();
+    return OLED_ERR_NOT_PINNED;
+  }
+  LayerData& L = ctx->layers[layer];
+  // a new store invalidates whatever this layer has cached
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  drop_all(L.cache, ctx->slots);
+  L.host_blob = static_cast<const uint8_t*>(host_blob);
+  L.host_stride = expert_stride_bytes;
+  return OLED_OK;
+}
+
+int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
+                      int32_t n_tokens, void* out) {
+  if (!ctx || layer < 0 || layer >= ctx->shape.n_layers || n_tokens < 0) return OLED_ERR_INVALID_ARG;
+  if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
+  LayerData& L = ctx->layers[layer];
+  if (!L.has_router || !L.host_blob) return OLED_ERR_NOT_REGISTERED;
+  const int T = n_tokens, H = ctx->shape.hidden, E = ctx->shape.n_experts, K = ctx->shape.top_k;
+  if (T > 0) {
+    if (!hidden || !confidences || !out) return OLED_ERR_INVALID_ARG;
+    const uint8_t* a = static_cast<const uint8_t*>(hidden);
+    const uint8_t* b = static_cast<const uint8_t*>(out);
+    const size_t bytes = (size_t)T * H * 2;
+    if (a < b + bytes && b < a + bytes) return OLED_ERR_INVALID_ARG;  // out aliases hidden
+  }
+  cudaStream_t st = ctx->stream;
+  ctx->last_layer = layer;
+  ctx->last_tokens = T;
+  if (T == 0) {  // nothing is activated: R' = R, only the step counter moves
+    ctx->last_before = L.cache.resident;
+    ctx->last_after = L.cache.resident;
+    L.stats.steps += 1;
+    return OLED_OK;
+  }
+
+  // 1. gate, counts and reuse-score numerators; read them back while the permutation runs
+  OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
+  launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
+               ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores);
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_ctrl, ctx->d_scores, ctx->ctrl_bytes, cudaMemcpyDeviceToHost, st));
+  OLED_CUDA(ctx, cudaEventRecord(ctx->gate_event, st));
+  launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos);
+  launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
+  ctx->launches += 3;
+  OLED_CUDA(ctx, cudaGetLastError());
+  OLED_CUDA(ctx, cudaEventSynchronize(ctx->gate_event));
+  // Everything enqueued before this step has completed, so slots released earlier are free to
+  // be overwritten by the side stream.
+  const unsigned long long* scores = reinterpret_cast<const unsigned long long*>(ctx->h_ctrl);
+  const int32_t* counts = reinterpret_cast<const int32_t*>(ctx->h_ctrl + (size_t)E * sizeof(unsigned long long));
+
+  // 2. hits / misses against the pre-step resident set, Top-C retention, slot plan
+  StepPlan& plan = ctx->plan;
+  if (!plan_step(L.cache, ctx->slots, counts, reinterpret_cast<const uint64_t*>(scores), plan))
+    return OLED_ERR_NO_SLOT;
+  ctx->last_before = plan.before;
+  ctx->last_after = plan.after;
+
+  // 3. fills: one pinned-host -> HBM copy per miss on the side stream, an event per chunk
+  const size_t n_miss = plan.misses.size();
+  const size_t chunk = (size_t)ctx->miss_chunk;
+  size_t n_chunks = 0;
+  for (size_t i = 0; i < n_miss; ++i) {
+    const int32_t e = plan.misses[i];
+    OLED_CUDA(ctx, cudaMemcpyAsync(ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes,
+                                   L.host_blob + (size_t)e * L.host_stride, ctx->slot_bytes,
+                                   cudaMemcpyHostToDevice, ctx->copy_stream));
+    if ((i + 1) % chunk == 0 || i + 1 == n_miss)
+      OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[n_chunks++], ctx->copy_stream));
+  }
+
+  // 4. grouped FFN: hits at once, misses chunk by chunk as their weights land
+  int rc = run_ffn_group(ctx, L, plan.hits, 0, plan.hits.size(), counts);
+  if (rc != OLED_OK) return rc;
+  for (size_t c = 0; c < n_chunks; ++c) {
+    OLED_CUDA(ctx, cudaStreamWaitEvent(st, ctx->fill_events[c], 0));
+    rc = run_ffn_group(ctx, L, plan.misses, c * chunk, std::min(n_miss, (c + 1) * chunk), counts);
+    if (rc != OLED_OK) return rc;
+  }
+
+  // 5. combine
+  launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out));
+  ctx->launches += 1;
+  OLED_CUDA(ctx, cudaGetLastError());
+
+  finish_step(L.cache, ctx->slots, plan);
+  L.stats.steps += 1;
+  L.stats.hits += plan.hits.size();
+  L.stats.misses += n_miss;
+  L.stats.bytes_moved += (uint64_t)n_miss * ctx->slot_bytes;
+  L.stats.evictions += (uint64_t)plan.n_evictions;
+  L.stats.active_experts += (uint64_t)plan.n_active;
+  L.stats.assignments += (uint64_t)T * K;
+  return OLED_OK;
+}
+
+int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden,
+                           const float* host_confidences, int32_t n_tokens, void* host_out) {
+  if (!ctx || n_tokens < 0) return OLED_ERR_INVALID_ARG;
+  if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
+  if (n_tokens > 0 && (!host_hidden || !host_confidences || !host_out)) return OLED_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)n_tokens * ctx->shape.hidden * 2;
+  if (n_tokens > 0) {
+    OLED_CUDA(ctx, cudaMemcpyAsync(ctx->d_hidden_stage, host_hidden, bytes, cudaMemcpyHostToDevice, ctx->stream));
+    OLED_CUDA(ctx, cudaMemcpyAsync(ctx->d_conf_stage, host_confidences, (size_t)n_tokens * sizeof(float),
+                                   cudaMemcpyHostToDevice, ctx->stream));
+  }
+  const int rc = oled_denoise_step(ctx, layer, ctx->d_hidden_stage, ctx->d_conf_stage, n_tokens, ctx->d_out_stage);
+  if (rc != OLED_OK) return rc;
+  if (n_tokens > 0) {
+    OLED_CUDA(ctx, cudaMemcpyAsync(host_out, ctx->d_out_stage, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  }
+  return OLED_OK;
+}
+
+int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out) {
+  if (!ctx || !out || layer < -1 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  const int rc = sync_all(ctx);
+  oled_stats_t acc{};
+  for (int l = 0; l < ctx->shape.n_layers; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    const oled_stats_t& s = ctx->layers[l].stats;
+    acc.steps += s.steps;
+    acc.hits += s.hits;
+    acc.misses += s.misses;
+    acc.bytes_moved += s.bytes_moved;
+    acc.evictions += s.evictions;
+    acc.active_experts += s.active_experts;
+    acc.assignments += s.assignments;
+  }
+  *out = acc;
+  return rc;
+}
+
+int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int32_t* perm, int32_t* counts,
+                    uint64_t* scores, uint8_t* resident_before, uint8_t* resident_after) {
+  if (!ctx || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  if (ctx->last_layer != layer) return OLED_ERR_STALE_DEBUG;
+  const int rc = sync_all(ctx);
+  if (rc != OLED_OK && rc != OLED_ERR_TIMEOUT) return rc;
+  const size_t n = (size_t)ctx->last_tokens * ctx->shape.top_k, E = (size_t)ctx->shape.n_experts;
+  if (n > 0) {
+    if (ids) OLED_CUDA(ctx, cudaMemcpy(ids, ctx->d_ids, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (gate) OLED_CUDA(ctx, cudaMemcpy(gate, ctx->d_gate, n * sizeof(float), cudaMemcpyDeviceToHost));
+    if (perm) OLED_CUDA(ctx, cudaMemcpy(perm, ctx->d_perm, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (counts) OLED_CUDA(ctx, cudaMemcpy(counts, ctx->d_counts, E * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (scores) OLED_CUDA(ctx, cudaMemcpy(scores, ctx->d_scores, E * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  } else {
+    if (counts) memset(counts, 0, E * sizeof(int32_t));
+    if (scores) memset(scores, 0, E * sizeof(uint64_t));
+  }
+  if (resident_before) memcpy(resident_before, ctx->last_before.data(), E);
+  if (resident_after) memcpy(resident_after, ctx->last_after.data(), E);
+  return rc;
+}
+
+int oled_debug_logits(oled_ctx* ctx, int32_t layer, float* logits) {
+  if (!ctx || !logits || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  if (ctx->last_layer != layer) return OLED_ERR_STALE_DEBUG;
+  const int rc = sync_all(ctx);
+  if (rc != OLED_OK && rc != OLED_ERR_TIMEOUT) return rc;
+  const size_t n = (size_t)ctx->last_tokens * ctx->shape.n_experts;
+  if (n > 0) OLED_CUDA(ctx, cudaMemcpy(logits, ctx->d_logits, n * sizeof(float), cudaMemcpyDeviceToHost));
+  return rc;
+}
+
+int oled_reset_cache(oled_ctx* ctx) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  const int rc = sync_all(ctx);
+  for (auto& L : ctx->layers) {
+    drop_all(L.cache, ctx->slots);
+    L.stats = oled_stats_t{};
+  }
+  ctx->last_layer = -1;
+  return rc;
+}
+
+int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size_t n) {
+  if (!ctx || !x || !r || !y) return OLED_ERR_INVALID_ARG;
+  if (n == 0) return OLED_OK;
+  launch_residual_add(ctx->stream, static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(r),
+                      static_cast<uint16_t*>(y), n);
+  ctx->launches += 1;
+  OLED_CUDA(ctx, cudaGetLastError());
+  return OLED_OK;
+}
+
+int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  switch (option) {
+    case OLED_OPT_FFN_IMPL:
+      if (value != 0 && value != 1) return OLED_ERR_INVALID_ARG;
+      ctx->ffn_impl = (int)value;
+      return OLED_OK;
+    case OLED_OPT_MISS_CHUNK:
+      if (value < 1) return OLED_ERR_INVALID_ARG;
+      ctx->miss_chunk = (int)std::min<int64_t>(value, OLED_MAX_EXPERTS);
+      return OLED_OK;
+    default:
+      return OLED_ERR_INVALID_ARG;
+  }
+}
+
+int oled_launch_count(oled_ctx* ctx, uint64_t* out) {
+  if (!ctx || !out) return OLED_ERR_INVALID_ARG;
+  *out = ctx->launches;
+  return OLED_OK;
+}
+
+int oled_synchronize(oled_ctx* ctx) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  return sync_all(ctx);
+}
+
+void oled_destroy(oled_ctx* ctx) { free_ctx(ctx); }
+
+int oled_last_cuda_error(oled_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+// ---- host-only policy simulator -----------------------------------------------------------
+struct oled_policy {
+  LayerCacheState cache;
+  SlotPool pool;
+  StepPlan plan;
+};
+
+int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, oled_policy** out) {
+  if (!out || n_experts <= 0 || n_experts > OLED_MAX_EXPERTS || capacity <= 0 || capacity > n_experts ||
+      pool_slots < capacity)
+    return OLED_ERR_INVALID_ARG;
+  oled_policy* p = new (std::nothrow) oled_policy();
+  if (!p) return OLED_ERR_OOM;
+  p->cache.init(n_experts, capacity);
+  p->pool.init(pool_slots);
+  *out = p;
+  return OLED_OK;
+}
+
+int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scores, uint8_t* resident_before,
+                     uint8_t* resident_after, int32_t* slot_of, int32_t* n_hits, int32_t* n_misses,
+                     int32_t* n_evictions) {
+  if (!p || !counts || !scores) return OLED_ERR_INVALID_ARG;
+  if (!plan_step(p->cache, p->pool, counts, scores, p->plan)) return OLED_ERR_NO_SLOT;
+  const size_t E = (size_t)p->cache.n_experts;
+  if (resident_before) memcpy(resident_before, p->plan.before.data(), E);
+  if (resident_after) memcpy(resident_after, p->plan.after.data(), E);
+  if (slot_of)
+    for (size_t e = 0; e < E; ++e) slot_of[e] = counts[e] > 0 ? p->cache.slot_of[e] : -1;
+  if (n_hits) *n_hits = (int32_t)p->plan.hits.size();
+  if (n_misses) *n_misses = (int32_t)p->plan.misses.size();
+  if (n_evictions) *n_evictions = p->plan.n_evictions;
+  finish_step(p->cache, p->pool, p->plan);
+  return OLED_OK;
+}
+
+void oled_policy_destroy(oled_policy* p) { delete p; }
+
+}  // extern "C"

@@ -1,0 +1,269 @@
+// Gate of the MoE layer (paper Sec. 2.1 / Sec. 4.1: "the MoE gate first produces the routed
+// expert IDs, gate scores"), token->expert permutation, and the integer numerators of the
+// expert reuse priority (Sec. 4.3 priority equation).
+//
+// Everything a keep/evict or routing decision depends on is computed in a fixed operation
+// order so that it can be reproduced bit for bit elsewhere:
+//   * logit(t,e): 32 chains, lane q owns h with (h/8) mod 32 == q, ascending h, one fused
+//     multiply-add per term (bf16*bf16 is exact in fp32, so the fma rounds once, like a plain
+//     add of the exact product); butterfly over xor distances 16,8,4,2,1; bias one rounded add.
+//   * top-k: logit descending, ties to the lower expert index.
+//   * gate scores: z_j = exp_spec(L_j - L_0); S = ((z_0+z_1)+z_2)...; g_j = z_j / S.
+//   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
+// The router stays off the tensor cores on purpose: their accumulation order is unspecified.
+#include <algorithm>
+
+#include "kernels.h"
+
+namespace oled {
+namespace {
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// exp(x) for x <= 0 from individually rounded fp32 operations (no contraction, no fast math).
+__device__ __forceinline__ float exp_spec(float x) {
+  if (x < -80.0f) return 0.0f;
+  const float kLog2e = __uint_as_float(0x3fb8aa3bu);  // fl32(1/ln 2)
+  const float kLn2Hi = __uint_as_float(0x3f317000u);  // fl32(ln 2), low 12 significand bits cleared
+  const float kLn2Lo = __uint_as_float(0x3805fdf4u);  // fl32(ln 2 - kLn2Hi)
+  const float n = rintf(__fmul_rn(x, kLog2e));
+  const float r = __fsub_rn(__fsub_rn(x, __fmul_rn(n, kLn2Hi)), __fmul_rn(n, kLn2Lo));
+  float p = __uint_as_float(0x39500d01u);                        // 1/5040
+  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3ab60b61u));  // 1/720
+  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3c088889u));  // 1/120
+  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3d2aaaabu));  // 1/24
+  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3e2aaaabu));  // 1/6
+  p = __fadd_rn(__fmul_rn(p, r), 0.5f);
+  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
+  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
+  const float scale = __int_as_float(((int)n + 127) << 23);  // 2^n, n >= -116
+  return __fmul_rn(p, scale);
+}
+
+constexpr int kRouteThreads = 256;
+constexpr int kRouteWarps = kRouteThreads / 32;
+constexpr int kEPerWarp = 4;                   // experts per warp per pass
+constexpr int kMaxEPerLane = OLED_MAX_EXPERTS / 32;
+
+template <int TT>
+__global__ void __launch_bounds__(kRouteThreads)
+route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
+             const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
+             int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
+             float* __restrict__ gate, int32_t* __restrict__ counts,
+             unsigned long long* __restrict__ scores) {
+  extern __shared__ float s_logits[];  // [TT][E]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = blockIdx.x * TT;
+
+  for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
+    float acc[TT][kEPerWarp];
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = 0.0f;
+
+    for (int hc = 0; hc < H; hc += 256) {
+      const int h = hc + lane * 8;
+      uint4 xv[TT], wv[kEPerWarp];
+#pragma unroll
+      for (int a = 0; a < TT; ++a) {
+        const int t = min(t0 + a, T - 1);
+        xv[a] = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+      }
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        const int e = min(eb + b, E - 1);
+        wv[b] = *reinterpret_cast<const uint4*>(wr + (size_t)e * H + h);
+      }
+      // elements j = 0..7 in ascending h: word0.lo, word0.hi, word1.lo, ...
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float wf[kEPerWarp];
+#pragma unroll
+        for (int b = 0; b < kEPerWarp; ++b) {
+          const uint32_t w32 = (j >> 1) == 0 ? wv[b].x : (j >> 1) == 1 ? wv[b].y
+                               : (j >> 1) == 2 ? wv[b].z : wv[b].w;
+          wf[b] = (j & 1) ? bf16_hi(w32) : bf16_lo(w32);
+        }
+#pragma unroll
+        for (int a = 0; a < TT; ++a) {
+          const uint32_t x32 = (j >> 1) == 0 ? xv[a].x : (j >> 1) == 1 ? xv[a].y
+                               : (j >> 1) == 2 ? xv[a].z : xv[a].w;
+          const float xf = (j & 1) ? bf16_hi(x32) : bf16_lo(x32);
+#pragma unroll
+          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf, wf[b], acc[a][b]);
+        }
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        float v = acc[a][b];
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, d));
+        const int e = eb + b;
+        if (lane == 0 && e < E && t0 + a < T) {
+          if (bias != nullptr) v = __fadd_rn(v, bias[e]);
+          s_logits[a * E + e] = v;
+          if (logits_out != nullptr) logits_out[(size_t)(t0 + a) * E + e] = v;
+        }
+      }
+  }
+  __syncthreads();
+
+  // top-k, gate scores, counts and reuse-score numerators: one warp per token
+  for (int a = warp; a < TT; a += kRouteWarps) {
+    const int t = t0 + a;
+    if (t >= T) continue;
+    float v[kMaxEPerLane];
+#pragma unroll
+    for (int i = 0; i < kMaxEPerLane; ++i) {
+      const int e = lane + 32 * i;
+      v[i] = e < E ? s_logits[a * E + e] : 0.0f;
+    }
+    uint32_t used = 0;
+    int my_id = 0;
+    float my_logit = 0.0f;
+    for (int r = 0; r < K; ++r) {
+      float bv = 0.0f;
+      int be = 0x7fffffff;
+#pragma unroll
+      for (int i = 0; i < kMaxEPerLane; ++i) {
+        const int e = lane + 32 * i;
+        if (e < E && !((used >> i) & 1u)) {
+          if (be == 0x7fffffff || v[i] > bv) {  // ascending e: strict > keeps the lower index
+            bv = v[i];
+            be = e;
+          }
+        }
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+        const int oe = __shfl_xor_sync(0xffffffffu, be, d);
+        const bool take = (oe != 0x7fffffff) &&
+                          (be == 0x7fffffff || ov > bv || (ov == bv && oe < be));
+        if (take) {
+          bv = ov;
+          be = oe;
+        }
+      }
+      if ((be & 31) == lane) used |= 1u << (be >> 5);
+      if (lane == r) {
+        my_id = be;
+        my_logit = bv;
+      }
+    }
+    const float top = __shfl_sync(0xffffffffu, my_logit, 0);
+    const float z = lane < K ? exp_spec(__fsub_rn(my_logit, top)) : 0.0f;
+    float s = __shfl_sync(0xffffffffu, z, 0);
+    for (int j = 1; j < K; ++j) s = __fadd_rn(s, __shfl_sync(0xffffffffu, z, j));
+    if (lane < K) {
+      const float g = __fdiv_rn(z, s);
+      ids[(size_t)t * K + lane] = my_id;
+      gate[(size_t)t * K + lane] = g;
+      float c = conf[t];
+      c = (c != c) ? 0.0f : fminf(fmaxf(c, 0.0f), 1.0f);  // psi(c) = c, clamped; NaN -> 0
+      const float pv = __fmul_rn(g, c);
+      const unsigned long long q = __float2ull_rz(__fmul_rn(pv, 4294967296.0f));
+      atomicAdd(&counts[my_id], 1);
+      atomicAdd(&scores[my_id], q);
+    }
+  }
+}
+
+// One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
+// assignment list (ascending t*K+j) hands out consecutive sorted rows.
+__global__ void __launch_bounds__(256)
+permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
+               int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos) {
+  __shared__ int s_red[8];
+  __shared__ int s_base;
+  const int e = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int part = 0;
+  for (int i = threadIdx.x; i < e; i += blockDim.x) part += counts[i];
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+  if (lane == 0) s_red[warp] = part;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int off = 0;
+    for (int w = 0; w < 8; ++w) off += s_red[w];
+    s_base = off;
+    offsets[e] = off;
+    if (e == E - 1) offsets[E] = off + counts[e];
+  }
+  __syncthreads();
+  if (counts[e] == 0) return;
+  int base = s_base;
+  for (int a0 = 0; a0 < n; a0 += blockDim.x) {
+    const int a = a0 + threadIdx.x;
+    const bool match = a < n && ids[a] == e;
+    const uint32_t bal = __ballot_sync(0xffffffffu, match);
+    __syncthreads();  // previous round's s_red fully consumed
+    if (lane == 0) s_red[warp] = __popc(bal);
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const int c = s_red[w];
+      if (w < warp) before += c;
+      total += c;
+    }
+    if (match) {
+      const int r = base + before + __popc(bal & ((1u << lane) - 1u));
+      perm[r] = a;
+      pos[a] = r;
+    }
+    base += total;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, int n_rows, int H,
+              int K, uint16_t* __restrict__ xp) {
+  const int vec_per_row = H / 8;
+  const size_t total = (size_t)n_rows * vec_per_row;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / vec_per_row);
+    const int c = (int)(i % vec_per_row);
+    const int t = perm[r] / K;
+    reinterpret_cast<uint4*>(xp)[(size_t)r * vec_per_row + c] =
+        reinterpret_cast<const uint4*>(x)[(size_t)t * vec_per_row + c];
+  }
+}
+
+}  // namespace
+
+void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
+                  const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
+                  float* gate, int32_t* counts, unsigned long long* scores) {
+  if (T <= 512) {
+    constexpr int TT = 2;
+    route_kernel<TT><<<(T + TT - 1) / TT, kRouteThreads, TT * E * sizeof(float), st>>>(
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+  } else {
+    constexpr int TT = 8;
+    route_kernel<TT><<<(T + TT - 1) / TT, kRouteThreads, TT * E * sizeof(float), st>>>(
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+  }
+}
+
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
+                    int32_t* offsets, int32_t* perm, int32_t* pos) {
+  permute_kernel<<<E, 256, 0, st>>>(ids, counts, T * K, E, offsets, perm, pos);
+}
+
+void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
+                   uint16_t* xp) {
+  const size_t total = (size_t)T * K * (H / 8);
+  const int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+  gather_kernel<<<blocks, 256, 0, st>>>(x, perm, T * K, H, K, xp);
+}
+
+}  // namespace oled

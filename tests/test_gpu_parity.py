@@ -1,0 +1,257 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle on seeded inputs.
+
+Discrete results (expert ids, permutation, counts, integer reuse scores, resident sets,
+counters) must match bit for bit; gate scores are fp32 values computed in the same operation
+order and must also match bit for bit; the layer output (bf16 on the GPU, fp64 in the oracle)
+must satisfy max-abs error <= 2e-2 and relative L2 error <= 1e-2.
+"""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import OracleStack  # noqa: E402
+from paper_2609_33385_b200 import synth  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, REL_L2 = 2e-2, 1e-2
+
+
+def _runner(w, **kw):
+    from paper_2609_33385_b200 import build
+    build.build()
+    from paper_2609_33385_b200.runner import StackRunner
+    return StackRunner(w, **kw)
+
+
+def _oracle_for(run, caps):
+    w = run.w
+    st = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, caps)
+    for l in range(w.n_layers):
+        st.register_router(l, run.router_bits[l], run.bias[l])
+        st.register_experts(l, run.layer_blobs(l))
+    return st
+
+
+def _check_out(out_bits, ref, what=""):
+    got = synth.bf16_bits_to_f32(out_bits).astype(np.float64)
+    err = np.abs(got - ref).max() if ref.size else 0.0
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30) if ref.size else 0.0
+    assert err <= MAX_ABS and rel <= REL_L2, f"{what}: max-abs {err:.3e}, rel-L2 {rel:.3e}"
+    return err, rel
+
+
+def _check_step(run, layer, n_tokens, out_t, ref, check_out=True):
+    from paper_2609_33385_b200.runner import dev_to_bits
+    dbg = run.ctx.debug_last(layer, n_tokens)
+    e = run.w.n_experts
+    assert np.array_equal(dbg["ids"], ref["ids"]), "expert ids differ"
+    assert np.array_equal(dbg["gate"].view(np.uint32), ref["gate"].view(np.uint32)), "gate scores differ"
+    assert np.array_equal(dbg["counts"], ref["counts"])
+    assert np.array_equal(dbg["perm"], ref["perm"]), "permutation differs"
+    assert [int(v) for v in dbg["scores"]] == list(ref["scores"]), "reuse scores differ"
+    assert set(np.flatnonzero(dbg["resident_before"])) == ref["resident_before"]
+    assert set(np.flatnonzero(dbg["resident_after"])) == ref["resident_after"]
+    if n_tokens:
+        logits = run.ctx.debug_logits(layer, n_tokens)
+        assert np.array_equal(logits.view(np.uint32), ref["logits"].view(np.uint32)), "logits differ"
+    if check_out:
+        _check_out(dev_to_bits(out_t), ref["out"], f"layer {layer}")
+    assert len(dbg["counts"]) == e
+
+
+def _check_stats(run, ora):
+    for l in range(run.w.n_layers):
+        a, b = run.ctx.stats(l), ora.stats(l)
+        assert (a.steps, a.hits, a.misses, a.bytes_moved, a.evictions, a.active_experts, a.assignments) == \
+               (b.steps, b.hits, b.misses, b.bytes_moved, b.evictions, b.active_experts, b.assignments)
+    a, b = run.ctx.stats(-1), ora.stats(-1)
+    assert (a.hits, a.misses, a.bytes_moved) == (b.hits, b.misses, b.bytes_moved)
+
+
+def _run_stack(run, ora, check_out=True):
+    """Replay mode: the oracle is fed the bf16 inputs the GPU saw at every call."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = run.w
+    dev = run.device
+    out = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=dev)
+    bufs = [torch.empty_like(out), torch.empty_like(out)]
+    for b, i, h_bits, conf in synth.denoise_inputs(w):
+        x = bits_to_dev(h_bits, dev)
+        c = torch.from_numpy(conf).to(dev)
+        for l in range(w.n_layers):
+            run.step(l, x, c, out)
+            ref = ora.denoise_step(l, dev_to_bits(x), conf)
+            _check_step(run, l, w.tokens, out, ref, check_out)
+            nxt = bufs[l & 1]
+            run.ctx.residual_add(x.data_ptr(), out.data_ptr(), nxt.data_ptr(), x.numel())
+            # the residual kernel: bf16(x + out) with one rounding
+            exp = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(dev_to_bits(x)) +
+                                         synth.bf16_bits_to_f32(dev_to_bits(out)))
+            assert np.array_equal(dev_to_bits(nxt), exp)
+            x = nxt
+    _check_stats(run, ora)
+
+
+@pytest.mark.parametrize("ffn_impl", [1, 0], ids=["ffn-plain", "ffn-tcgen05"])
+def test_tiny_stack_elementwise(ffn_impl):
+    w = synth.tiny()
+    run = _runner(w, capacity=[3, 5], ffn_impl=ffn_impl)
+    try:
+        _run_stack(run, _oracle_for(run, [3, 5]))
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("ffn_impl", [1, 0], ids=["ffn-plain", "ffn-tcgen05"])
+def test_config1_full_run(ffn_impl):
+    w = synth.config(0)                        # hidden 512, 16 experts top-2, I 1024, 32 tokens
+    run = _runner(w, ffn_impl=ffn_impl)
+    try:
+        _run_stack(run, _oracle_for(run, [w.capacity]))
+        st = run.ctx.stats()
+        assert st.steps == w.iters and st.misses > 0 and st.hits > 0
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("n_tokens", [0, 1, 7, 33, 150])
+def test_ragged_token_counts(n_tokens):
+    """Token counts that leave experts empty, span several 16-row tiles and end in a ragged tail."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=6, top_k=3, hidden=512, intermediate=256)
+    run = _runner(w, capacity=[2], max_tokens=160)
+    ora = _oracle_for(run, [2])
+    try:
+        for rep in range(2):
+            h_bits, conf = synth.flat_tokens(w, n_tokens, rep)
+            x = bits_to_dev(h_bits, run.device) if n_tokens else torch.empty((0, w.hidden), dtype=torch.bfloat16, device=run.device)
+            c = torch.from_numpy(conf).to(run.device)
+            out = torch.zeros((max(n_tokens, 1), w.hidden), dtype=torch.bfloat16, device=run.device)[:n_tokens]
+            run.step(0, x, c, out)
+            ref = ora.denoise_step(0, h_bits.reshape(n_tokens, w.hidden), conf)
+            _check_step(run, 0, n_tokens, out, ref)
+        _check_stats(run, ora)
+    finally:
+        run.close()
+
+
+def test_many_tokens_per_expert_multi_tile():
+    """More than 256 rows for one expert: several N tiles per expert in both FFN kernels."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=256, intermediate=128)
+    n = 700                                     # ~350 rows per expert on average
+    run = _runner(w, capacity=[4], max_tokens=n)
+    ora = _oracle_for(run, [4])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 7)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        ref = ora.denoise_step(0, h_bits, conf)
+        assert ref["counts"].max() > 256
+        _check_step(run, 0, n, out, ref)
+    finally:
+        run.close()
+
+
+def test_output_bit_identical_at_every_capacity():
+    """Offloading is lossless (Sec. 5.1): routing and output do not depend on the capacity."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1, blocks=1, iters=4, n_experts=8, top_k=2)
+    outs, miss = [], []
+    for cap in (1, 3, 8):
+        run = _runner(w, capacity=[cap])
+        try:
+            res = []
+            for _, _, h_bits, conf in synth.denoise_inputs(w):
+                x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+                out = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=run.device)
+                run.step(0, x, c, out)
+                res.append((dev_to_bits(out).copy(), run.ctx.debug_last(0, w.tokens)["ids"].copy()))
+            outs.append(res)
+            miss.append(run.ctx.stats().misses)
+        finally:
+            run.close()
+    for res in outs[1:]:
+        for (o0, i0), (o1, i1) in zip(outs[0], res):
+            assert np.array_equal(i0, i1) and np.array_equal(o0, o1)
+    assert miss[0] >= miss[1] >= miss[2]
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1)
+    run_d, run_h = _runner(w, capacity=[3]), _runner(w, capacity=[3])
+    try:
+        for _, _, h_bits, conf in synth.denoise_inputs(w):
+            x, c = bits_to_dev(h_bits, run_d.device), torch.from_numpy(conf).to(run_d.device)
+            out = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=run_d.device)
+            run_d.step(0, x, c, out)
+            hx = torch.from_numpy(h_bits.view(np.int16)).pin_memory()
+            hc = torch.from_numpy(conf).pin_memory()
+            ho = torch.empty((w.tokens, w.hidden), dtype=torch.int16).pin_memory()
+            run_h.step_host(0, hx, hc, ho)
+            assert np.array_equal(ho.numpy().view(np.uint16), dev_to_bits(out))
+        assert run_d.ctx.stats() == run_h.ctx.stats()
+    finally:
+        run_d.close()
+        run_h.close()
+
+
+def test_errors_are_codes_not_crashes():
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1)
+    ctx = binding.OledContext(1, w.hidden, w.n_experts, w.top_k, w.intermediate, 8, [2])
+    try:
+        x = torch.zeros((8, w.hidden), dtype=torch.bfloat16, device="cuda:0")
+        c = torch.zeros(8, device="cuda:0")
+        out = torch.zeros_like(x)
+        assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.ERR_NOT_REGISTERED
+        wr, _ = synth.router_weights(w, 0)
+        wr_d = bits_to_dev(wr, "cuda:0")
+        ctx.register_router(0, wr_d.data_ptr())
+        pageable = torch.zeros((w.n_experts, w.expert_elems), dtype=torch.int16)
+        with pytest.raises(binding.OledError) as ei:
+            ctx.register_experts(0, pageable.data_ptr(), w.expert_bytes)
+        assert ei.value.code == binding.ERR_NOT_PINNED
+        pinned = torch.zeros((w.n_experts, w.expert_elems), dtype=torch.int16).pin_memory()
+        with pytest.raises(binding.OledError) as ei:
+            ctx.register_experts(0, pinned.data_ptr(), w.expert_bytes - 16)
+        assert ei.value.code == binding.ERR_INVALID_ARG
+        ctx.register_experts(0, pinned.data_ptr(), w.expert_bytes)
+        assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 9, out.data_ptr()) == binding.ERR_TOO_MANY_TOKENS
+        assert ctx.denoise_step_rc(1, x.data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.ERR_INVALID_ARG
+        assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, x.data_ptr()) == binding.ERR_INVALID_ARG
+        assert ctx.denoise_step_rc(0, None, c.data_ptr(), 8, out.data_ptr()) == binding.ERR_INVALID_ARG
+        assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.OLED_OK
+        ctx.synchronize()
+        assert float(out.float().abs().max()) == 0.0          # zero weights -> zero output
+        with pytest.raises(binding.OledError):
+            binding.OledContext(1, 250, 8, 2, 128, 8, [2])     # hidden not a multiple of 256
+        with pytest.raises(binding.OledError):
+            binding.OledContext(1, 256, 8, 2, 128, 8, [9])     # capacity > E
+    finally:
+        ctx.destroy()
+
+
+def test_reset_cache_returns_to_cold_state():
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1)
+    run = _runner(w, capacity=[w.n_experts])
+    try:
+        h_bits, conf = synth.flat_tokens(w, 5)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((5, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        m1 = run.ctx.stats().misses
+        run.step(0, x, c, out)
+        assert run.ctx.stats().misses == m1 and m1 > 0        # second identical step: all hits
+        run.ctx.reset_cache()
+        assert run.ctx.stats().steps == 0
+        run.step(0, x, c, out)
+        assert run.ctx.stats().misses == m1
+    finally:
+        run.close()

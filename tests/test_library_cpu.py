@@ -1,0 +1,83 @@
+"""Host-side checks that need no GPU: the library loads, exports every symbol the header
+declares, and its C++ cache policy agrees with the oracle's policy decision for decision."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import cache_policy as cp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2609_33385_b200 import build
+    build.build()
+    from paper_2609_33385_b200 import binding as b
+    b.load()
+    return b
+
+
+def test_library_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "oled.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(oled_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    lib = binding.load()
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} declared in include/oled.h but not exported"
+    assert declared == set(binding.EXPORTS)
+
+
+def test_strerror_and_arg_checks_without_gpu(binding):
+    assert binding.strerror(0) == "ok"
+    assert "pinned" in binding.strerror(binding.ERR_NOT_PINNED)
+    assert binding.strerror(-12345) == "unknown error"
+    with pytest.raises(binding.OledError):
+        binding.PolicySim(8, 0, 8)            # capacity 0
+    with pytest.raises(binding.OledError):
+        binding.PolicySim(8, 4, 3)            # pool smaller than capacity
+    lib = binding.load()
+    assert lib.oled_denoise_step(None, 0, None, None, 1, None) == binding.ERR_INVALID_ARG
+    assert lib.oled_stats(None, 0, None) == binding.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("e,cap,seed", [(16, 8, 0), (64, 26, 1), (12, 1, 2), (9, 9, 3), (128, 51, 4)])
+def test_host_policy_matches_oracle(binding, e, cap, seed):
+    rng = np.random.default_rng(seed)
+    sim = binding.PolicySim(e, cap, e)        # worst-case pool: E slots
+    ref = cp.LayerCache(e, cap, 100)
+    for step in range(60):
+        t, k = int(rng.integers(1, 12)), int(rng.integers(1, min(4, e) + 1))
+        ids = np.stack([rng.permutation(e)[:k] for _ in range(t)]).astype(np.int32)
+        gate = rng.dirichlet(np.ones(k), size=t).astype(np.float32)
+        conf = rng.choice([0.0, 0.25, 0.5, 1.0], size=t).astype(np.float32)   # many ties, zeros
+        r = ref.step(ids, gate, conf)
+        counts = np.bincount(ids.reshape(-1), minlength=e).astype(np.int32)
+        got = sim.step(counts, np.array(r["scores"], dtype=np.uint64))
+        assert set(np.flatnonzero(got["resident_before"])) == r["resident_before"]
+        assert set(np.flatnonzero(got["resident_after"])) == r["resident_after"]
+        assert got["hits"] == len(r["hits"]) and got["misses"] == len(r["misses"])
+        assert got["evictions"] == len(r["resident_before"] - r["resident_after"])
+        # slot table: every activated expert has a distinct slot during the step
+        slots = got["slot_of"][counts > 0]
+        assert np.all(slots >= 0) and len(set(slots.tolist())) == len(slots)
+        assert np.all(got["slot_of"][counts == 0] == -1)
+
+
+def test_host_policy_pool_exhaustion_is_an_error_not_a_crash(binding):
+    sim = binding.PolicySim(8, 2, 3)          # capacity 2 plus one transient slot
+    counts = np.zeros(8, np.int32)
+    counts[[0, 1, 2]] = 1
+    sim.step(counts, np.arange(8, dtype=np.uint64) + 1)    # 3 misses fit in 3 slots
+    counts[:] = 0
+    counts[[3, 4, 5, 6]] = 1                                # 4 misses: 2 stale slots + 1 free < 4
+    with pytest.raises(binding.OledError) as ei:
+        sim.step(counts, np.arange(8, dtype=np.uint64) + 1)
+    assert ei.value.code == binding.ERR_NO_SLOT
+    counts[:] = 0
+    counts[[3, 4, 5]] = 1                                   # the failed step changed nothing
+    got = sim.step(counts, np.arange(8, dtype=np.uint64) + 1)
+    assert got["misses"] == 3
