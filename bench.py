@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE denoise step against a bounded expert cache.
+
+A "step" is one denoising iteration of the whole stack over one block of tokens: every layer
+runs gate -> top-k -> permutation -> hit/miss + fills -> grouped SwiGLU FFN -> combine ->
+retention once (the residual between layers included).  The headline workload is the 16-layer,
+hidden-2048, 64-expert top-8 stack with a 32-token block at 40 % expert residency.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle as it stands.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "moe_denoise_step_tokens_per_s_at_40pct_residency"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.proc = None
+        self.gpu_id = gpu_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+                pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ oracle legs
+def oracle_layer_steps(w, budget_s: float, max_steps: int, distinct_layers: int = 1):
+    """Time the CPU oracle, as it stands, on layer executions of the workload.
+
+    Returns (seconds per layer execution, layer executions timed, BLAS threads)."""
+    from oracle import OracleStack
+    from paper_2609_33385_b200 import synth
+    caps = [w.capacity] * w.n_layers
+    ora = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, caps)
+    blobs = []
+    for d in range(distinct_layers):
+        b = np.empty((w.n_experts, w.expert_elems), np.uint16)
+        synth.fill_layer_blobs(w, d, b, threads=min(32, len(os.sched_getaffinity(0))))
+        blobs.append(b)
+    for l in range(w.n_layers):
+        wr, bias = synth.router_weights(w, l)
+        ora.register_router(l, wr, bias)
+        ora.register_experts(l, blobs[l % distinct_layers])
+    threads = 1
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([int(i.get("num_threads", 1)) for i in threadpool_info()] or [1])
+    except Exception:
+        pass
+    times = []
+    t_start = time.perf_counter()
+    done = False
+    for _, _, h_bits, conf in synth.denoise_inputs(w):
+        x = h_bits
+        for l in range(w.n_layers):
+            t0 = time.perf_counter()
+            res = ora.denoise_step(l, x, conf)
+            times.append(time.perf_counter() - t0)
+            xf = synth.bf16_bits_to_f32(x).astype(np.float64) + res["out"]
+            x = synth.f32_to_bf16_bits(xf.astype(np.float32))
+            if len(times) >= max_steps or time.perf_counter() - t_start > budget_s:
+                done = True
+                break
+        if done:
+            break
+    return sum(times) / len(times), len(times), threads
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle on the host cores; one step = one layer execution, scaled."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = max(1, args.steps + args.warmup)
+    sec, count, threads = oracle_layer_steps(w, budget_s=150.0, max_steps=n)
+    ms_step = sec * w.n_layers * 1e3
+    value = w.tokens / (sec * w.n_layers)
+    sample = (f"{count} layer executions of {w.name} (1 distinct layer of weights aliased across "
+              f"the stack), scaled by {w.n_layers} layers per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, "A"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, variant):
+    return {"workload": w.name, "variant": variant, "layers": w.n_layers, "hidden": w.hidden,
+            "experts": w.n_experts, "top_k": w.top_k, "intermediate": w.intermediate,
+            "tokens_per_step": w.tokens, "iters_per_block": w.iters, "capacity_per_layer": w.capacity,
+            "residency": w.residency, "rho": w.rho,
+            "l2": "inputs larger than L2 (each step streams >= 10 GB of expert weights)"}
+
+
+# ------------------------------------------------------------------------------ GPU legs
+def measure_h2d(torch, device, blob_bytes: int) -> dict:
+    big = 256 << 20
+    src = torch.empty(big, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(big, dtype=torch.uint8, device=device)
+    best = 0.0
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        dst.copy_(src, non_blocking=True)
+        b.record()
+        b.synchronize()
+        best = max(best, big / (a.elapsed_time(b) * 1e-3) / 1e9)
+    n = max(1, min(16, big // blob_bytes))
+    best_train = 0.0
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n):
+            dst[i * blob_bytes:(i + 1) * blob_bytes].copy_(src[i * blob_bytes:(i + 1) * blob_bytes],
+                                                           non_blocking=True)
+        b.record()
+        b.synchronize()
+        best_train = max(best_train, n * blob_bytes / (a.elapsed_time(b) * 1e-3) / 1e9)
+    return {"gbs_256mb": best, "gbs_blob_train": best_train}
+
+
+def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None):
+    """warmup + steps denoising iterations; returns (ms total, launches, stats delta)."""
+    w = run.w
+    n_tok = w.tokens
+    dev_out = torch.empty((n_tok, w.hidden), dtype=torch.bfloat16, device=run.device)
+    if host:
+        hx = [x.cpu().pin_memory() for x in xs]
+        hc = [c.cpu().pin_memory() for c in cs]
+        ho = torch.empty((n_tok, w.hidden), dtype=torch.bfloat16).pin_memory()
+
+    def one(i):
+        if host:
+            run.ctx.denoise_iteration_host(hx[i].data_ptr(), hc[i].data_ptr(), n_tok, ho.data_ptr())
+        else:
+            run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), n_tok, dev_out.data_ptr())
+
+    run.ctx.reset_cache()
+    for i in range(warmup):
+        one(i)
+    run.ctx.synchronize()
+    s0, l0 = run.ctx.stats(), run.ctx.launch_count()
+    from paper_2609_33385_b200 import dist
+    dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(run.stream)
+    for i in range(warmup, warmup + steps):
+        one(i)
+    b.record(run.stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = a.elapsed_time(b)
+    s1, l1 = run.ctx.stats(), run.ctx.launch_count()
+    delta = {k: getattr(s1, k) - getattr(s0, k) for k in
+             ("steps", "hits", "misses", "bytes_moved", "evictions", "active_experts", "assignments")}
+    return ms, l1 - l0, delta, clocks
+
+
+def step_roofline(w, delta, steps, ms_per_step, peaks, h2d_gbs):
+    """Binding roofline of the whole step from the algorithmic work of the timed region."""
+    blob = w.expert_bytes
+    layer_steps = max(1, delta["steps"])
+    b_hbm = (delta["active_experts"] * blob + delta["misses"] * blob +
+             layer_steps * (w.n_experts * w.hidden * 2 + 2 * w.tokens * w.hidden * 2)) / steps
+    b_h2d = delta["bytes_moved"] / steps
+    flops = 6.0 * delta["assignments"] * w.hidden * w.intermediate / steps
+    t_hbm = b_hbm / (peaks["hbm_gbs"] * 1e9) * 1e3
+    t_h2d = b_h2d / (h2d_gbs * 1e9) * 1e3
+    t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+    terms = {"hbm": t_hbm, "host_link": t_h2d, "tensor": t_tc}
+    bound = max(terms, key=terms.get)
+    return {"bound": bound, "t_roof_ms": terms[bound], "t_measured_ms": ms_per_step,
+            "frac": terms[bound] / ms_per_step, "terms_ms": terms,
+            "hbm_bytes_per_step": b_hbm, "h2d_bytes_per_step": b_h2d, "flops_per_step": flops}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="workload configuration index (0..4)")
+    ap.add_argument("--variant", default="A", choices=["A", "B"],
+                    help="A: literal i.i.d. tokens; B: tokens of a block share a direction")
+    ap.add_argument("--residency", type=float, default=None)
+    ap.add_argument("--distinct-layers", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-full-residency", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2609_33385_b200 import synth
+    over = {}
+    if args.residency is not None:
+        over["residency"] = args.residency
+    if args.variant == "B":
+        over["shared_beta"] = 0.9
+        over["rho"] = 0.98
+    w = synth.config(args.config, **over)
+    n_iters = args.warmup + args.steps
+    w = w.replace(blocks=int(math.ceil(n_iters / w.iters)))
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_2609_33385_b200 import build, dist
+    build.build()
+    from paper_2609_33385_b200.binding import OPT_PROFILE
+    from paper_2609_33385_b200.runner import StackRunner, bits_to_dev
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = dist.init("nccl")
+    device = f"cuda:{local_rank}"
+    torch.cuda.set_device(device)
+    peaks = load_peaks()
+    cores = len(os.sched_getaffinity(0))
+    threads = max(1, min(32, cores // max(1, world)))
+
+    t_setup = time.perf_counter()
+    run = StackRunner(w, device=device, gen_threads=threads, distinct_layers=args.distinct_layers)
+    xs, cs = [], []
+    for _, _, h_bits, conf in synth.denoise_inputs(w):
+        xs.append(bits_to_dev(h_bits, device))
+        cs.append(torch.from_numpy(conf).to(device))
+        if len(xs) >= n_iters:
+            break
+    setup_s = time.perf_counter() - t_setup
+    h2d = measure_h2d(torch, device, w.expert_bytes)
+    gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid).replace("GPU-", "")
+
+    # 1. device-resident inputs: the headline value
+    ms, launches, delta, clocks = timed_pass(torch, run, xs, cs, args.warmup, args.steps,
+                                             sampler=ClockSampler(gpu_uuid) if rank == 0 else None)
+    units, ms_max = dist.aggregate(w.tokens * args.steps, ms, device)
+    value = units / (ms_max * 1e-3)
+    ms_per_step = ms_max / args.steps
+
+    # 2. end to end: host buffers through the C ABI, copies inside the timed region
+    ms_e, _, delta_e, _ = timed_pass(torch, run, xs, cs, args.warmup, args.steps, host=True)
+    units_e, ms_e_max = dist.aggregate(w.tokens * args.steps, ms_e, device)
+    in_bytes = w.tokens * w.hidden * 2 + w.tokens * 4
+    ctrl_bytes = w.n_layers * w.n_experts * 12
+    e2e = {"value": units_e / (ms_e_max * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": in_bytes + delta_e["bytes_moved"] / args.steps,
+           "d2h_bytes_per_step": w.tokens * w.hidden * 2 + ctrl_bytes,
+           "input_h2d_bytes_per_step": in_bytes,
+           "expert_fill_h2d_bytes_per_step": delta_e["bytes_moved"] / args.steps,
+           "ms_per_step": ms_e_max / args.steps}
+
+    # 3. per-kernel CUDA-event timing of the same region (separate pass: events add overhead)
+    run.ctx.set_option(OPT_PROFILE, 0)
+    run.ctx.reset_cache()
+    out_dev = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=device)
+    for i in range(args.warmup):
+        run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out_dev.data_ptr())
+    run.ctx.synchronize()
+    run.ctx.set_option(OPT_PROFILE, 1)
+    for i in range(args.warmup, n_iters):
+        run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out_dev.data_ptr())
+    prof = run.ctx.profile_read(reset=True)
+    run.ctx.set_option(OPT_PROFILE, 0)
+    top = max(prof, key=lambda k: prof[k]["ms"])
+    kp = prof[top]
+    ach = kp["bytes"] / max(kp["ms"], 1e-9) / 1e6          # GB/s
+    roofline = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                "traffic": None, "launches": kp["launches"],
+                "avg_launch_us": kp["ms"] * 1e3 / max(1, kp["launches"]),
+                "algorithmic_bytes_per_launch": kp["bytes"] / max(1, kp["launches"])}
+    kernels = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                   "gbs": (v["bytes"] / v["ms"] / 1e6) if v["ms"] > 0 else None}
+               for k, v in prof.items()}
+
+    step_roof = step_roofline(w, delta, args.steps, ms_per_step, peaks, h2d["gbs_blob_train"])
+    extra = {"tpot_ms": ms_per_step * w.iters / w.tokens,
+             "hits": delta["hits"], "misses": delta["misses"],
+             "cache_utilisation": delta["hits"] / max(1, delta["steps"] * w.capacity),
+             "active_experts_per_layer_step": delta["active_experts"] / max(1, delta["steps"]),
+             "h2d_link": {"achieved_gbs": delta["bytes_moved"] / (ms * 1e-3) / 1e9, **h2d},
+             "setup_s": setup_s}
+
+    # 4. full residency on the same workload (C = E): the HBM-bound regime and the TPOT ratio
+    if not args.no_full_residency:
+        full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run)
+        ms_f, _, delta_f, _ = timed_pass(torch, full, xs, cs, args.warmup, args.steps)
+        _, ms_f_max = dist.aggregate(0, ms_f, device)
+        msf = ms_f_max / args.steps
+        rf = step_roofline(w.replace(residency=1.0), delta_f, args.steps, msf, peaks, h2d["gbs_blob_train"])
+        full.ctx.reset_cache()
+        for i in range(args.warmup):
+            full.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out_dev.data_ptr())
+        full.ctx.synchronize()
+        full.ctx.set_option(OPT_PROFILE, 1)
+        for i in range(args.warmup, n_iters):
+            full.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out_dev.data_ptr())
+        pf = full.ctx.profile_read(reset=True)
+        extra["full_residency"] = {
+            "ms_per_step": msf, "tokens_per_s": w.tokens / (msf * 1e-3),
+            "tpot_ms": msf * w.iters / w.tokens, "misses": delta_f["misses"], "roofline_step": rf,
+            "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                            "gbs": (v["bytes"] / v["ms"] / 1e6) if v["ms"] > 0 else None}
+                        for k, v in pf.items()}}
+        extra["tpot_ratio_vs_full_residency"] = ms_per_step / msf
+        # lower bound of that ratio given the measured link: the fills that cannot hide
+        extra["tpot_ratio_min_from_link"] = max(1.0, step_roof["terms_ms"]["host_link"] / msf)
+        full.close()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec, count, thr = oracle_layer_steps(w, budget_s=args.cpu_budget_s, max_steps=64)
+        cpu = {"value": w.tokens / (sec * w.n_layers), "unit": UNIT, "cores": thr, "kind": "oracle",
+               "sample": f"{count} layer executions of {w.name} ({sec:.3f} s each; 1 distinct layer of "
+                         f"weights), scaled by {w.n_layers} layers per step",
+               "host_cores_available": cores}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(w, args.variant), "clocks": clocks, "e2e": e2e,
+                "gpu_launches": launches, "roofline": roofline, "roofline_step": step_roof,
+                "kernels": kernels, "cpu_baseline": cpu, **extra}
+        print(json.dumps(line))
+    run.close()
+    dist.shutdown()
+
+
+if __name__ == "__main__":
+    main()

@@ -117,6 +117,19 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
 int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden,
                            const float* host_confidences, int32_t n_tokens, void* host_out);
 
+/* One denoising iteration of the whole stack (Sec. 2.1: one iteration = one forward over the
+ * block): layers 0..L-1 in order, x_{l+1} = bf16(x_l + out_l).  hidden / hidden_out are device
+ * [n_tokens,H] bf16 (hidden_out may not alias hidden), confidences device fp32[n_tokens] and are
+ * used for every layer of the iteration.  Errors as oled_denoise_step(). */
+int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confidences,
+                           int32_t n_tokens, void* hidden_out);
+
+/* The same with HOST buffers (copied in and out on the context's stream; returns after
+ * hidden_out has arrived). */
+int oled_denoise_iteration_host(oled_ctx* ctx, const void* host_hidden,
+                                const float* host_confidences, int32_t n_tokens,
+                                void* host_hidden_out);
+
 /* Counters of one layer, or summed over layers for layer = -1.  Synchronises the stream. */
 int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out);
 
@@ -139,10 +152,33 @@ int oled_reset_cache(oled_ctx* ctx);
 int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size_t n);
 
 /* Options.  OLED_OPT_FFN_IMPL: 0 = tcgen05 tensor-core kernels (default), 1 = plain-FMA
- * bring-up kernels.  OLED_OPT_MISS_CHUNK: experts per fill group (default 4). */
+ * bring-up kernels.  OLED_OPT_MISS_CHUNK: experts per fill group (default 4).
+ * OLED_OPT_PROFILE: 1 = bracket every kernel launch with CUDA events on the context's stream
+ * (adds two event records per launch; off by default). */
 #define OLED_OPT_FFN_IMPL 1
 #define OLED_OPT_MISS_CHUNK 2
+#define OLED_OPT_PROFILE 3
 int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value);
+
+/* Per-kernel timing collected while OLED_OPT_PROFILE is on.  bytes / flops are the ALGORITHMIC
+ * figures of the launches (weights of each expert once, token rows in, result rows out), not
+ * measured traffic. */
+#define OLED_KERNEL_ROUTE 0
+#define OLED_KERNEL_PERMUTE 1
+#define OLED_KERNEL_GATHER 2
+#define OLED_KERNEL_FFN_GATE_UP 3
+#define OLED_KERNEL_FFN_DOWN 4
+#define OLED_KERNEL_COMBINE 5
+#define OLED_N_KERNELS 6
+typedef struct {
+  uint64_t launches;
+  double ms;       /* sum of CUDA-event durations */
+  uint64_t bytes;
+  uint64_t flops;
+} oled_kernel_profile;
+/* Synchronises, folds pending event pairs into the totals and returns those of `kernel`;
+ * reset != 0 clears them afterwards. */
+int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_profile* out);
 
 /* Number of kernels the library has launched on this context so far. */
 int oled_launch_count(oled_ctx* ctx, uint64_t* out);

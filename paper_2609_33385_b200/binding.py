@@ -22,12 +22,13 @@ LIB_PATH = os.path.join(_HERE, "liboled.so")
 OLED_OK = 0
 ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -2, -3, -4
 ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -9
-OPT_FFN_IMPL, OPT_MISS_CHUNK = 1, 2
+OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE = 1, 2, 3
+KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
 
 EXPORTS = [
     "oled_create", "oled_register_router", "oled_register_experts", "oled_denoise_step",
-    "oled_denoise_step_host", "oled_stats", "oled_debug_last", "oled_debug_logits",
-    "oled_reset_cache", "oled_residual_add", "oled_set_option", "oled_launch_count",
+    "oled_denoise_step_host", "oled_denoise_iteration", "oled_denoise_iteration_host", "oled_stats", "oled_debug_last", "oled_debug_logits",
+    "oled_reset_cache", "oled_residual_add", "oled_set_option", "oled_profile_read", "oled_launch_count",
     "oled_synchronize", "oled_destroy", "oled_strerror", "oled_last_cuda_error",
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy",
 ]
@@ -37,6 +38,11 @@ class ModelShape(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_experts", C.c_int32),
                 ("top_k", C.c_int32), ("intermediate", C.c_int32), ("max_tokens", C.c_int32),
                 ("has_router_bias", C.c_int32), ("staging_slots", C.c_int32)]
+
+
+class KernelProfile(C.Structure):
+    _fields_ = [("launches", C.c_uint64), ("ms", C.c_double), ("bytes", C.c_uint64),
+                ("flops", C.c_uint64)]
 
 
 class StatsStruct(C.Structure):
@@ -84,12 +90,15 @@ def load() -> C.CDLL:
     lib.oled_register_experts.argtypes = [vp, i32, vp, C.c_size_t]
     lib.oled_denoise_step.argtypes = [vp, i32, vp, vp, i32, vp]
     lib.oled_denoise_step_host.argtypes = [vp, i32, vp, vp, i32, vp]
+    lib.oled_denoise_iteration.argtypes = [vp, vp, vp, i32, vp]
+    lib.oled_denoise_iteration_host.argtypes = [vp, vp, vp, i32, vp]
     lib.oled_stats.argtypes = [vp, i32, C.POINTER(StatsStruct)]
     lib.oled_debug_last.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.oled_debug_logits.argtypes = [vp, i32, vp]
     lib.oled_reset_cache.argtypes = [vp]
     lib.oled_residual_add.argtypes = [vp, vp, vp, vp, C.c_size_t]
     lib.oled_set_option.argtypes = [vp, i32, C.c_int64]
+    lib.oled_profile_read.argtypes = [vp, i32, i32, C.POINTER(KernelProfile)]
     lib.oled_launch_count.argtypes = [vp, u64p]
     lib.oled_synchronize.argtypes = [vp]
     lib.oled_destroy.argtypes = [vp]
@@ -159,6 +168,14 @@ class OledContext:
         self._check(self._lib.oled_denoise_step_host(self._h, layer, hidden_ptr, conf_ptr,
                                                      n_tokens, out_ptr), "oled_denoise_step_host")
 
+    def denoise_iteration(self, hidden_ptr: int, conf_ptr: int, n_tokens: int, out_ptr: int) -> None:
+        self._check(self._lib.oled_denoise_iteration(self._h, hidden_ptr, conf_ptr, n_tokens, out_ptr),
+                    "oled_denoise_iteration")
+
+    def denoise_iteration_host(self, hidden_ptr: int, conf_ptr: int, n_tokens: int, out_ptr: int) -> None:
+        self._check(self._lib.oled_denoise_iteration_host(self._h, hidden_ptr, conf_ptr, n_tokens,
+                                                          out_ptr), "oled_denoise_iteration_host")
+
     def stats(self, layer: int = -1) -> Stats:
         s = StatsStruct()
         self._check(self._lib.oled_stats(self._h, layer, C.byref(s)), "oled_stats")
@@ -189,6 +206,17 @@ class OledContext:
 
     def set_option(self, option: int, value: int) -> None:
         self._check(self._lib.oled_set_option(self._h, option, value), "oled_set_option")
+
+    def profile_read(self, reset: bool = True) -> dict:
+        """Per-kernel {launches, ms, bytes, flops} collected while OPT_PROFILE was on."""
+        out = {}
+        for k, name in enumerate(KERNEL_NAMES):
+            p = KernelProfile()
+            self._check(self._lib.oled_profile_read(self._h, k, 1 if reset else 0, C.byref(p)),
+                        "oled_profile_read")
+            out[name] = dict(launches=int(p.launches), ms=float(p.ms), bytes=int(p.bytes),
+                             flops=int(p.flops))
+        return out
 
     def launch_count(self) -> int:
         v = C.c_uint64()

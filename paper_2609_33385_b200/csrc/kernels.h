@@ -55,8 +55,8 @@ struct FfnTcMaps {
 // Builds the tensor maps; returns 0 or a negative oled_status.
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
-// Two launches: gate/up + SwiGLU into hbuf, then down projection into y.
-int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count,
+// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
+int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
                   const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
                   uint32_t* status);
 

@@ -58,11 +58,18 @@ struct oled_ctx {
   uint16_t* d_hidden_stage = nullptr;  // for the host-buffer entry point
   float* d_conf_stage = nullptr;
   uint16_t* d_out_stage = nullptr;
+  uint16_t* d_iter[2] = {nullptr, nullptr};  // ping-pong hidden states of the stack iteration
   // pinned host mirror of the control block
   uint8_t* h_ctrl = nullptr;
   uint32_t* h_status = nullptr;
 
   FfnTcMaps maps;
+  // optional per-kernel timing with CUDA events on the context's stream
+  bool profile = false;
+  struct ProfRec { int kernel; cudaEvent_t a, b; };
+  std::vector<ProfRec> prof_pending;
+  std::vector<cudaEvent_t> prof_free;
+  oled_kernel_profile prof_acc[OLED_N_KERNELS] = {};
   int ffn_impl = 0;
   int miss_chunk = 4;
   uint64_t launches = 0;
@@ -131,13 +138,69 @@ void free_ctx(oled_ctx* ctx) {
   cudaFree(ctx->d_hidden_stage);
   cudaFree(ctx->d_conf_stage);
   cudaFree(ctx->d_out_stage);
+  cudaFree(ctx->d_iter[0]);
+  cudaFree(ctx->d_iter[1]);
   if (ctx->h_ctrl) cudaFreeHost(ctx->h_ctrl);
   if (ctx->h_status) cudaFreeHost(ctx->h_status);
   for (auto ev : ctx->fill_events) cudaEventDestroy(ev);
+  for (auto& r : ctx->prof_pending) {
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  for (auto ev : ctx->prof_free) cudaEventDestroy(ev);
   if (ctx->gate_event) cudaEventDestroy(ctx->gate_event);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   cudaGetLastError();
   delete ctx;
+}
+
+cudaEvent_t prof_event(oled_ctx* ctx) {
+  if (!ctx->prof_free.empty()) {
+    cudaEvent_t e = ctx->prof_free.back();
+    ctx->prof_free.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return e;
+}
+
+// Brackets one kernel launch with events when profiling is on.
+struct ProfScope {
+  oled_ctx* ctx;
+  cudaEvent_t a = nullptr, b = nullptr;
+  int kernel;
+  ProfScope(oled_ctx* c, int k, uint64_t bytes, uint64_t flops) : ctx(c), kernel(k) {
+    if (!ctx->profile) return;
+    a = prof_event(ctx);
+    b = prof_event(ctx);
+    if (a && b) {
+      cudaEventRecord(a, ctx->stream);
+      ctx->prof_acc[k].launches += 1;
+      ctx->prof_acc[k].bytes += bytes;
+      ctx->prof_acc[k].flops += flops;
+    }
+  }
+  ~ProfScope() {
+    if (a && b) {
+      cudaEventRecord(b, ctx->stream);
+      ctx->prof_pending.push_back({kernel, a, b});
+    }
+  }
+};
+
+void prof_resolve(oled_ctx* ctx) {
+  for (auto& r : ctx->prof_pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) ctx->prof_acc[r.kernel].ms += ms;
+    ctx->prof_free.push_back(r.a);
+    ctx->prof_free.push_back(r.b);
+  }
+  ctx->prof_pending.clear();
+  cudaGetLastError();
 }
 
 // One FFN launch pair over `experts` (ids), weights through the layer's slot table.
@@ -159,9 +222,19 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
                       ctx->d_y, H, I);
   } else {
-    const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, ctx->d_offsets, ctx->d_hbuf, ctx->d_y,
-                                 H, I, ctx->n_sms, ctx->d_status);
-    if (rc != OLED_OK) return rc;
+    uint64_t rows = 0;
+    for (size_t i = begin; i < end; ++i) rows += (uint64_t)counts[experts[i]];
+    const uint64_t hi = (uint64_t)H * I, n = (uint64_t)grp.n;
+    for (int kind = 1; kind <= 2; ++kind) {
+      // algorithmic bytes: each expert's weights once, the token rows in, the result rows out
+      const uint64_t bytes = kind == 1 ? n * 2 * hi * 2 + rows * H * 2 + rows * I * 2
+                                       : n * hi * 2 + rows * I * 2 + rows * H * 4;
+      const uint64_t flops = (kind == 1 ? 4 : 2) * rows * hi;
+      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, bytes, flops);
+      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, ctx->d_offsets, ctx->d_hbuf,
+                                   ctx->d_y, H, I, ctx->n_sms, ctx->d_status);
+      if (rc != OLED_OK) return rc;
+    }
   }
   ctx->launches += 2;
   OLED_CUDA(ctx, cudaGetLastError());
@@ -261,6 +334,8 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   if ((rc = dev_alloc(ctx, &ctx->d_hidden_stage, T * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_conf_stage, T)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_out_stage, T * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_iter[0], T * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_iter[1], T * H)) != OLED_OK) return fail(rc);
   for (int l = 0; l < s.n_layers; ++l) {
     if ((rc = dev_alloc(ctx, &ctx->layers[l].w_router, E * H)) != OLED_OK) return fail(rc);
     if (s.has_router_bias && (rc = dev_alloc(ctx, &ctx->layers[l].bias, E)) != OLED_OK) return fail(rc);
@@ -351,12 +426,22 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
 
   // 1. gate, counts and reuse-score numerators; read them back while the permutation runs
   OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
-  launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
-               ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores);
+  {
+    ProfScope ps(ctx, OLED_KERNEL_ROUTE, ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * 8,
+                 2ull * T * H * E);
+    launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
+                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores);
+  }
   OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_ctrl, ctx->d_scores, ctx->ctrl_bytes, cudaMemcpyDeviceToHost, st));
   OLED_CUDA(ctx, cudaEventRecord(ctx->gate_event, st));
-  launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos);
-  launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
+  {
+    ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12, 0);
+    launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos);
+  }
+  {
+    ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
+    launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
+  }
   ctx->launches += 3;
   OLED_CUDA(ctx, cudaGetLastError());
   OLED_CUDA(ctx, cudaEventSynchronize(ctx->gate_event));
@@ -395,7 +480,10 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
   }
 
   // 5. combine
-  launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out));
+  {
+    ProfScope ps(ctx, OLED_KERNEL_COMBINE, (uint64_t)T * K * H * 4 + (uint64_t)T * H * 2, 2ull * T * K * H);
+    launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out));
+  }
   ctx->launches += 1;
   OLED_CUDA(ctx, cudaGetLastError());
 
@@ -427,6 +515,48 @@ int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden
     OLED_CUDA(ctx, cudaMemcpyAsync(host_out, ctx->d_out_stage, bytes, cudaMemcpyDeviceToHost, ctx->stream));
     OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
   }
+  return OLED_OK;
+}
+
+int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confidences, int32_t n_tokens,
+                           void* hidden_out) {
+  if (!ctx || n_tokens < 0) return OLED_ERR_INVALID_ARG;
+  if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
+  if (n_tokens > 0 && (!hidden || !confidences || !hidden_out)) return OLED_ERR_INVALID_ARG;
+  const size_t n = (size_t)n_tokens * ctx->shape.hidden;
+  const void* x = hidden;
+  for (int l = 0; l < ctx->shape.n_layers; ++l) {
+    const int rc = oled_denoise_step(ctx, l, x, confidences, n_tokens, ctx->d_out_stage);
+    if (rc != OLED_OK) return rc;
+    void* nxt = (l + 1 == ctx->shape.n_layers) ? hidden_out : (void*)ctx->d_iter[l & 1];
+    if (n > 0) {
+      launch_residual_add(ctx->stream, static_cast<const uint16_t*>(x), ctx->d_out_stage,
+                          static_cast<uint16_t*>(nxt), n);
+      ctx->launches += 1;
+      OLED_CUDA(ctx, cudaGetLastError());
+    }
+    x = nxt;
+  }
+  return OLED_OK;
+}
+
+int oled_denoise_iteration_host(oled_ctx* ctx, const void* host_hidden, const float* host_confidences,
+                                int32_t n_tokens, void* host_hidden_out) {
+  if (!ctx || n_tokens < 0) return OLED_ERR_INVALID_ARG;
+  if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
+  if (n_tokens == 0) return oled_denoise_iteration(ctx, nullptr, nullptr, 0, nullptr);
+  if (!host_hidden || !host_confidences || !host_hidden_out) return OLED_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)n_tokens * ctx->shape.hidden * 2;
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->d_hidden_stage, host_hidden, bytes, cudaMemcpyHostToDevice, ctx->stream));
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->d_conf_stage, host_confidences, (size_t)n_tokens * sizeof(float),
+                                 cudaMemcpyHostToDevice, ctx->stream));
+  // the last layer's residual writes into the staging buffer the input came from: by then the
+  // input has been consumed (layer 0 reads it; later layers read the ping-pong buffers)
+  uint16_t* final_dev = ctx->shape.n_layers > 1 ? ctx->d_hidden_stage : ctx->d_iter[0];
+  const int rc = oled_denoise_iteration(ctx, ctx->d_hidden_stage, ctx->d_conf_stage, n_tokens, final_dev);
+  if (rc != OLED_OK) return rc;
+  OLED_CUDA(ctx, cudaMemcpyAsync(host_hidden_out, final_dev, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
   return OLED_OK;
 }
 
@@ -509,6 +639,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       if (value != 0 && value != 1) return OLED_ERR_INVALID_ARG;
       ctx->ffn_impl = (int)value;
       return OLED_OK;
+    case OLED_OPT_PROFILE:
+      ctx->profile = value != 0;
+      return OLED_OK;
     case OLED_OPT_MISS_CHUNK:
       if (value < 1) return OLED_ERR_INVALID_ARG;
       ctx->miss_chunk = (int)std::min<int64_t>(value, OLED_MAX_EXPERTS);
@@ -516,6 +649,15 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
     default:
       return OLED_ERR_INVALID_ARG;
   }
+}
+
+int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_profile* out) {
+  if (!ctx || !out || kernel < 0 || kernel >= OLED_N_KERNELS) return OLED_ERR_INVALID_ARG;
+  const int rc = sync_all(ctx);
+  prof_resolve(ctx);
+  *out = ctx->prof_acc[kernel];
+  if (reset) ctx->prof_acc[kernel] = oled_kernel_profile{};
+  return rc;
 }
 
 int oled_launch_count(oled_ctx* ctx, uint64_t* out) {

@@ -35,7 +35,7 @@ class StackRunner:
                  device: str = "cuda:0", distinct_layers: Optional[int] = None,
                  gen_threads: Optional[int] = None, ffn_impl: Optional[int] = None,
                  miss_chunk: Optional[int] = None, max_tokens: Optional[int] = None,
-                 staging_slots: int = 0):
+                 staging_slots: int = 0, share_store_of: Optional["StackRunner"] = None):
         self.w = w
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -56,7 +56,11 @@ class StackRunner:
         # host expert store: pinned, one [E, 3*H*I] block of bf16 bits per distinct layer
         self._host_t: List[torch.Tensor] = []
         self.blobs: List[np.ndarray] = []
-        for d in range(n_distinct):
+        if share_store_of is not None:         # same pinned host expert store, another context
+            self.n_distinct = n_distinct = share_store_of.n_distinct
+            self._host_t = share_store_of._host_t
+            self.blobs = share_store_of.blobs
+        for d in range(0 if share_store_of is not None else n_distinct):
             t = torch.empty((w.n_experts, w.expert_elems), dtype=torch.int16, pin_memory=True)
             a = t.numpy().view(np.uint16)
             synth.fill_layer_blobs(w, d, a, threads=threads)
