@@ -264,6 +264,7 @@ def main():
                     help="A: literal i.i.d. tokens; B: tokens of a block share a direction")
     ap.add_argument("--residency", type=float, default=None)
     ap.add_argument("--distinct-layers", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-residency", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
@@ -274,6 +275,8 @@ def main():
     over = {}
     if args.residency is not None:
         over["residency"] = args.residency
+    if args.layers is not None:
+        over["n_layers"] = args.layers
     if args.variant == "B":
         over["shared_beta"] = 0.9
         over["rho"] = 0.98

@@ -19,6 +19,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "kernels.h"
 
@@ -390,15 +391,27 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint32_t estr[3] = {1, 1, 1};
+  CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+  if (const char* env = getenv("OLED_FFN_L2PROMO")) {
+    const int v = atoi(env);
+    promo = v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+                   : v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
+                             : v == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+  }
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides,
             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int stages_for(int kind, int n_box) {
+  static int cap = -1;  // tuning aid: OLED_FFN_STAGES caps the pipeline depth
+  if (cap < 0) {
+    const char* env = getenv("OLED_FFN_STAGES");
+    cap = env ? std::max(1, atoi(env)) : kMaxStages;
+  }
   const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
-  return (int)std::min<uint32_t>(kMaxStages, avail / stage);
+  return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage);
 }
 uint32_t smem_for(int kind, int n_box, int stages) {
   const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
@@ -447,8 +460,13 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
 }
 
 static int box_index(int max_count, int cap) {
+  static int min_box = -1;  // tuning aid: OLED_FFN_MIN_NBOX forces wider token tiles
+  if (min_box < 0) {
+    const char* env = getenv("OLED_FFN_MIN_NBOX");
+    min_box = env ? atoi(env) : 0;
+  }
   int i = 0;
-  while ((16 << i) < max_count && (16 << i) < cap) ++i;
+  while (((16 << i) < max_count || (16 << i) < min_box) && (16 << i) < cap) ++i;
   return i;
 }
 
