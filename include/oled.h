@@ -193,6 +193,30 @@ const char* oled_strerror(int code);
 /* The CUDA error code of the last OLED_ERR_CUDA on this context (cudaError_t as int). */
 int oled_last_cuda_error(oled_ctx* ctx);
 
+/* Routing of one step without any allocation.  The paper has no counterpart: this exists for
+ * hosts that cannot let a library allocate device memory - a server that gives all of it to its
+ * own arena at start-up, or a decode loop that cannot afford the device-wide synchronisation
+ * hidden in cudaMalloc/cudaFree.  It runs the same gate, top-k, gate-score and permutation
+ * kernels as oled_denoise_step(), needs no context, and keeps its scratch (gate logits, inverse
+ * permutation, reuse-score accumulators; about 0.55 MB) in a fixed array inside the library
+ * image, which every GPU that loads the library holds until the process exits.
+ *   hidden [n_tokens,hidden_dim] bf16, w_router [n_experts,hidden_dim] bf16, bias fp32[n_experts]
+ *   or NULL, confidences fp32[n_tokens]: device, read only.
+ *   ids int32[n_tokens*top_k], gate fp32[n_tokens*top_k], counts int32[n_experts],
+ *   offsets int32[n_experts+1], perm int32[n_tokens*top_k]: device, written; caller-owned.
+ *   n_tokens <= OLED_NOALLOC_MAX_TOKENS, else OLED_ERR_TOO_MANY_TOKENS; other limits as above.
+ * The work is enqueued on cuda_stream.  The first call on a device looks up the array's device
+ * address (one-time set-up under a lock); make that first call before any stream capture.
+ * All calls share the one array, which still holds the previous call's data: the accumulators
+ * are cleared on the stream at the start of every call, and two calls whose work overlaps on
+ * the GPU (different streams, no ordering between them) race on it.  Calls cudaMemsetAsync and
+ * kernel launches only: no cudaMalloc, cudaFree or allocating library routine. */
+#define OLED_NOALLOC_MAX_TOKENS 256
+int oled_route_noalloc(const void* hidden, const void* w_router, const float* bias,
+                       const float* confidences, int32_t n_tokens, int32_t hidden_dim,
+                       int32_t n_experts, int32_t top_k, void* cuda_stream, int32_t* ids,
+                       float* gate, int32_t* counts, int32_t* offsets, int32_t* perm);
+
 /* ---- host-only policy simulator (no GPU needed): the same C++ policy code the step uses,
  * driven by recorded counts and integer scores.  For tests of the host logic. ---- */
 typedef struct oled_policy oled_policy;

@@ -30,8 +30,9 @@ EXPORTS = [
     "oled_denoise_step_host", "oled_denoise_iteration", "oled_denoise_iteration_host", "oled_stats", "oled_debug_last", "oled_debug_logits",
     "oled_reset_cache", "oled_residual_add", "oled_set_option", "oled_profile_read", "oled_launch_count",
     "oled_synchronize", "oled_destroy", "oled_strerror", "oled_last_cuda_error",
-    "oled_policy_create", "oled_policy_step", "oled_policy_destroy",
+    "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
 ]
+NOALLOC_MAX_TOKENS = 256
 
 
 class ModelShape(C.Structure):
@@ -111,6 +112,7 @@ def load() -> C.CDLL:
                                      C.POINTER(i32)]
     lib.oled_policy_destroy.argtypes = [vp]
     lib.oled_policy_destroy.restype = None
+    lib.oled_route_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -236,6 +238,16 @@ class OledContext:
             self.destroy()
         except Exception:
             pass
+
+
+def route_noalloc(hidden_ptr, w_router_ptr, bias_ptr, conf_ptr, n_tokens: int, hidden: int,
+                  n_experts: int, top_k: int, cuda_stream: int, ids_ptr, gate_ptr, counts_ptr,
+                  offsets_ptr, perm_ptr) -> int:
+    """``oled_route_noalloc``: routing of one step with library-internal static scratch; the
+    library allocates nothing.  All pointers are device pointers; returns the status code."""
+    return load().oled_route_noalloc(hidden_ptr, w_router_ptr, bias_ptr, conf_ptr, n_tokens, hidden,
+                                     n_experts, top_k, C.c_void_p(cuda_stream), ids_ptr, gate_ptr,
+                                     counts_ptr, offsets_ptr, perm_ptr)
 
 
 class PolicySim:

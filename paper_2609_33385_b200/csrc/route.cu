@@ -12,6 +12,7 @@
 //   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
 // The router stays off the tensor cores on purpose: their accumulation order is unspecified.
 #include <algorithm>
+#include <mutex>
 
 #include "kernels.h"
 
@@ -267,3 +268,81 @@ void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int 
 }
 
 }  // namespace oled
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free routing entry point (no counterpart in the paper).
+//
+// Some hosts cannot let a library allocate: an inference server that hands every byte of
+// device memory to its own arena at start-up, or a latency-critical decode loop in which the
+// implicit device-wide synchronisation of cudaMalloc / cudaFree is not acceptable.  For them
+// this entry point runs the gate, top-k, gate scores and the token->expert permutation of one
+// step with its scratch (gate logits, inverse permutation, reuse-score accumulators) in a
+// fixed array that is part of the loaded module, so nothing is allocated or freed.
+namespace oled {
+namespace {
+
+constexpr size_t kNaScoreBytes = (size_t)OLED_MAX_EXPERTS * sizeof(unsigned long long);
+constexpr size_t kNaPosBytes = (size_t)OLED_NOALLOC_MAX_TOKENS * OLED_MAX_TOPK * sizeof(int32_t);
+constexpr size_t kNaLogitBytes = (size_t)OLED_NOALLOC_MAX_TOKENS * OLED_MAX_EXPERTS * sizeof(float);
+constexpr size_t kNaScratchBytes = kNaScoreBytes + kNaPosBytes + kNaLogitBytes;
+
+// Lives in every GPU that loads the library until the process exits (about 0.55 MB).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaScratchBytes];
+
+constexpr int kNaMaxDevices = 64;
+std::mutex g_na_mutex;
+void* g_na_ptr[kNaMaxDevices] = {};
+
+// In host code g_noalloc_scratch is only a handle for the symbol, not an address a kernel can
+// use: the device address is looked up once per device, with that device current.
+int noalloc_scratch_ptr(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return OLED_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_na_mutex);
+  if (g_na_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return OLED_ERR_CUDA;
+    }
+    g_na_ptr[dev] = p;
+  }
+  *out = static_cast<unsigned char*>(g_na_ptr[dev]);
+  return OLED_OK;
+}
+
+}  // namespace
+}  // namespace oled
+
+extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, const float* bias,
+                                  const float* confidences, int32_t n_tokens, int32_t hidden_dim,
+                                  int32_t n_experts, int32_t top_k, void* cuda_stream, int32_t* ids,
+                                  float* gate, int32_t* counts, int32_t* offsets, int32_t* perm) {
+  using namespace oled;
+  if (n_tokens < 0 || hidden_dim <= 0 || hidden_dim % 256 != 0 || n_experts <= 0 ||
+      n_experts > OLED_MAX_EXPERTS || top_k <= 0 || top_k > OLED_MAX_TOPK || top_k > n_experts ||
+      !counts || !offsets)
+    return OLED_ERR_INVALID_ARG;
+  if (n_tokens > OLED_NOALLOC_MAX_TOKENS) return OLED_ERR_TOO_MANY_TOKENS;
+  if (n_tokens > 0 && (!hidden || !w_router || !confidences || !ids || !gate || !perm))
+    return OLED_ERR_INVALID_ARG;
+  unsigned char* scratch = nullptr;
+  const int rc = noalloc_scratch_ptr(&scratch);
+  if (rc != OLED_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long* scores = reinterpret_cast<unsigned long long*>(scratch);
+  int32_t* pos = reinterpret_cast<int32_t*>(scratch + kNaScoreBytes);
+  float* logits = reinterpret_cast<float*>(scratch + kNaScoreBytes + kNaPosBytes);
+  // the array keeps the previous call's contents: the accumulators must start at zero
+  if (cudaMemsetAsync(scores, 0, (size_t)n_experts * sizeof(unsigned long long), st) != cudaSuccess ||
+      cudaMemsetAsync(counts, 0, (size_t)n_experts * sizeof(int32_t), st) != cudaSuccess ||
+      cudaMemsetAsync(offsets, 0, (size_t)(n_experts + 1) * sizeof(int32_t), st) != cudaSuccess) {
+    cudaGetLastError();
+    return OLED_ERR_CUDA;
+  }
+  if (n_tokens == 0) return OLED_OK;
+  launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
+               confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores);
+  launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos);
+  return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
+}
