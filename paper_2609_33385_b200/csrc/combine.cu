@@ -12,7 +12,8 @@ namespace {
 
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
-               const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out) {
+               const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next) {
   const int t = blockIdx.x;
   __shared__ float s_g[OLED_MAX_TOPK];
   __shared__ int s_r[OLED_MAX_TOPK];
@@ -37,6 +38,18 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
     pk.x = *reinterpret_cast<uint32_t*>(&lo);
     pk.y = *reinterpret_cast<uint32_t*>(&hi);
     *reinterpret_cast<uint2*>(out + (size_t)t * H + h) = pk;
+    if (x_next != nullptr) {  // residual on the rounded output: bf16(x + bf16(out))
+      const uint2 xv = *reinterpret_cast<const uint2*>(x + (size_t)t * H + h);
+      const float2 o0 = __bfloat1622float2(lo), o1 = __bfloat1622float2(hi);
+      __nv_bfloat162 r0 = __floats2bfloat162_rn(__uint_as_float(xv.x << 16) + o0.x,
+                                                __uint_as_float(xv.x & 0xffff0000u) + o0.y);
+      __nv_bfloat162 r1 = __floats2bfloat162_rn(__uint_as_float(xv.y << 16) + o1.x,
+                                                __uint_as_float(xv.y & 0xffff0000u) + o1.y);
+      uint2 rk;
+      rk.x = *reinterpret_cast<uint32_t*>(&r0);
+      rk.y = *reinterpret_cast<uint32_t*>(&r1);
+      *reinterpret_cast<uint2*>(x_next + (size_t)t * H + h) = rk;
+    }
   }
 }
 
@@ -55,8 +68,8 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 }  // namespace
 
 void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
-                    int H, int K, uint16_t* out) {
-  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out);
+                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next) {
+  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out, x, x_next);
 }
 
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {

@@ -471,21 +471,27 @@ static int box_index(int max_count, int cap) {
 }
 
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
-                  const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
                   uint32_t* status) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   // KIND 1 holds two accumulators per tile: N <= 128 keeps them double-buffered in TMEM.
   const int i1 = box_index(max_count, 128), i2 = box_index(max_count, 256);
+  // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
+  auto grid_for = [&](int n_box, int m_tiles) {
+    long long tiles = 0;
+    for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + n_box - 1) / n_box;
+    return (int)std::max<long long>(1, std::min<long long>(n_sms, tiles * m_tiles));
+  };
   if (kind == 1) {
     grp.n_box = 16 << i1;
     const int stages = stages_for(1, grp.n_box);
-    ffn_tc_kernel<1><<<n_sms, kThreads, smem_for(1, grp.n_box, stages), st>>>(
+    ffn_tc_kernel<1><<<grid_for(grp.n_box, I / kBlockM), kThreads, smem_for(1, grp.n_box, stages), st>>>(
         maps.w13, maps.xp[i1], grp, offsets, hbuf, H, I, stages, status);
   } else {
     grp.n_box = 16 << i2;
     const int stages = stages_for(2, grp.n_box);
-    ffn_tc_kernel<2><<<n_sms, kThreads, smem_for(2, grp.n_box, stages), st>>>(
+    ffn_tc_kernel<2><<<grid_for(grp.n_box, H / kBlockM), kThreads, smem_for(2, grp.n_box, stages), st>>>(
         maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;

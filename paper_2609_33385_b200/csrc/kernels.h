@@ -27,17 +27,20 @@ enum : uint32_t { kStatusOk = 0, kStatusWaitTimeout = 1 };
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores);
-// Offsets (exclusive scan), stable permutation by expert and its inverse.
+// Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
+// kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
-                    int32_t* offsets, int32_t* perm, int32_t* pos);
+                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp,
+                    int H);
 // xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);
 
 // ---- combine.cu -----------------------------------------------------------------------
-// out[t,:] = bf16( sum_j gate[t,j] * y[pos[t*K+j],:] ), j ascending, fp32 accumulation.
+// out[t,:] = bf16( sum_j gate[t,j] * y[pos[t*K+j],:] ), j ascending, fp32 accumulation.  With
+// x_next != nullptr also x_next[t,:] = bf16(x[t,:] + out[t,:]) (the residual between layers).
 void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
-                    int H, int K, uint16_t* out);
+                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next);
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n);
 
 // ---- ffn_simple.cu (bring-up path, plain FMA) ---------------------------------------------
@@ -57,7 +60,7 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
-                  const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
                   uint32_t* status);
 
 }  // namespace oled

@@ -231,7 +231,7 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
                                        : n * hi * 2 + rows * I * 2 + rows * H * 4;
       const uint64_t flops = (kind == 1 ? 4 : 2) * rows * hi;
       ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, bytes, flops);
-      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, ctx->d_offsets, ctx->d_hbuf,
+      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, counts, ctx->d_offsets, ctx->d_hbuf,
                                    ctx->d_y, H, I, ctx->n_sms, ctx->d_status);
       if (rc != OLED_OK) return rc;
     }
@@ -400,8 +400,9 @@ int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob, s
   return OLED_OK;
 }
 
-int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
-                      int32_t n_tokens, void* out) {
+// x_next != nullptr: also write x_next = bf16(hidden + out), the residual between layers.
+static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
+                     int32_t n_tokens, void* out, void* x_next) {
   if (!ctx || layer < 0 || layer >= ctx->shape.n_layers || n_tokens < 0) return OLED_ERR_INVALID_ARG;
   if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
   LayerData& L = ctx->layers[layer];
@@ -434,15 +435,17 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
   }
   OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_ctrl, ctx->d_scores, ctx->ctrl_bytes, cudaMemcpyDeviceToHost, st));
   OLED_CUDA(ctx, cudaEventRecord(ctx->gate_event, st));
+  const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
   {
-    ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12, 0);
-    launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos);
+    ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
+    launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
+                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H);
   }
-  {
+  if (!fuse_gather) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
   }
-  ctx->launches += 3;
+  ctx->launches += fuse_gather ? 2 : 3;
   OLED_CUDA(ctx, cudaGetLastError());
   OLED_CUDA(ctx, cudaEventSynchronize(ctx->gate_event));
   // Everything enqueued before this step has completed, so slots released earlier are free to
@@ -482,7 +485,8 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
   // 5. combine
   {
     ProfScope ps(ctx, OLED_KERNEL_COMBINE, (uint64_t)T * K * H * 4 + (uint64_t)T * H * 2, 2ull * T * K * H);
-    launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out));
+    launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out),
+                   static_cast<const uint16_t*>(hidden), static_cast<uint16_t*>(x_next));
   }
   ctx->launches += 1;
   OLED_CUDA(ctx, cudaGetLastError());
@@ -496,6 +500,11 @@ int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const fl
   L.stats.active_experts += (uint64_t)plan.n_active;
   L.stats.assignments += (uint64_t)T * K;
   return OLED_OK;
+}
+
+int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
+                      int32_t n_tokens, void* out) {
+  return step_impl(ctx, layer, hidden, confidences, n_tokens, out, nullptr);
 }
 
 int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden,
@@ -523,18 +532,11 @@ int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confi
   if (!ctx || n_tokens < 0) return OLED_ERR_INVALID_ARG;
   if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
   if (n_tokens > 0 && (!hidden || !confidences || !hidden_out)) return OLED_ERR_INVALID_ARG;
-  const size_t n = (size_t)n_tokens * ctx->shape.hidden;
   const void* x = hidden;
   for (int l = 0; l < ctx->shape.n_layers; ++l) {
-    const int rc = oled_denoise_step(ctx, l, x, confidences, n_tokens, ctx->d_out_stage);
-    if (rc != OLED_OK) return rc;
     void* nxt = (l + 1 == ctx->shape.n_layers) ? hidden_out : (void*)ctx->d_iter[l & 1];
-    if (n > 0) {
-      launch_residual_add(ctx->stream, static_cast<const uint16_t*>(x), ctx->d_out_stage,
-                          static_cast<uint16_t*>(nxt), n);
-      ctx->launches += 1;
-      OLED_CUDA(ctx, cudaGetLastError());
-    }
+    const int rc = step_impl(ctx, l, x, confidences, n_tokens, ctx->d_out_stage, nxt);
+    if (rc != OLED_OK) return rc;
     x = nxt;
   }
   return OLED_OK;

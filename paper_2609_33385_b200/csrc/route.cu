@@ -42,13 +42,14 @@ __device__ __forceinline__ float exp_spec(float x) {
   return __fmul_rn(p, scale);
 }
 
-constexpr int kRouteThreads = 256;
-constexpr int kRouteWarps = kRouteThreads / 32;
 constexpr int kEPerWarp = 4;                   // experts per warp per pass
 constexpr int kMaxEPerLane = OLED_MAX_EXPERTS / 32;
 
-template <int TT>
-__global__ void __launch_bounds__(kRouteThreads)
+// TT tokens per CTA, WARPS warps; each warp owns 4 experts per pass and all TT tokens.  Small
+// blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
+// chunks of loads in flight; the chain order of every logit is the same in all variants.
+template <int TT, int WARPS, int UNROLL>
+__global__ void __launch_bounds__(WARPS * 32)
 route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
              const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
              int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
@@ -58,6 +59,7 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
 
+  constexpr int kRouteWarps = WARPS;
   for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
     float acc[TT][kEPerWarp];
 #pragma unroll
@@ -65,6 +67,7 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 #pragma unroll
       for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = 0.0f;
 
+#pragma unroll UNROLL
     for (int hc = 0; hc < H; hc += 256) {
       const int h = hc + lane * 8;
       uint4 xv[TT], wv[kEPerWarp];
@@ -178,9 +181,12 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 
 // One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
 // assignment list (ascending t*K+j) hands out consecutive sorted rows.
+// If xp != nullptr the CTA also copies the token rows of its expert into sorted order
+// (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
 __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
-               int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos) {
+               int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K) {
   __shared__ int s_red[8];
   __shared__ int s_base;
   const int e = blockIdx.x;
@@ -222,6 +228,15 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     }
     base += total;
   }
+  if (xp == nullptr) return;
+  __syncthreads();  // this CTA's perm entries are visible to all of its threads
+  const int vec_per_row = H / 8, first = s_base, rows = counts[e];
+  for (int i = threadIdx.x; i < rows * vec_per_row; i += blockDim.x) {
+    const int r = first + i / vec_per_row, c = i % vec_per_row;
+    const int t = perm[r] / K;
+    reinterpret_cast<uint4*>(xp)[(size_t)r * vec_per_row + c] =
+        reinterpret_cast<const uint4*>(x)[(size_t)t * vec_per_row + c];
+  }
 }
 
 __global__ void __launch_bounds__(256)
@@ -244,20 +259,25 @@ gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, 
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores) {
-  if (T <= 512) {
-    constexpr int TT = 2;
-    route_kernel<TT><<<(T + TT - 1) / TT, kRouteThreads, TT * E * sizeof(float), st>>>(
+  if (T <= 128) {
+    constexpr int TT = 1, W = 16;
+    route_kernel<TT, W, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+  } else if (T <= 1024) {
+    constexpr int TT = 2, W = 8;
+    route_kernel<TT, W, 2><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
         x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
   } else {
-    constexpr int TT = 8;
-    route_kernel<TT><<<(T + TT - 1) / TT, kRouteThreads, TT * E * sizeof(float), st>>>(
+    constexpr int TT = 8, W = 8;
+    route_kernel<TT, W, 1><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
         x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
   }
 }
 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
-                    int32_t* offsets, int32_t* perm, int32_t* pos) {
-  permute_kernel<<<E, 256, 0, st>>>(ids, counts, T * K, E, offsets, perm, pos);
+                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp,
+                    int H) {
+  permute_kernel<<<E, 256, 0, st>>>(ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K);
 }
 
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
@@ -343,6 +363,7 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   if (n_tokens == 0) return OLED_OK;
   launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
                confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores);
-  launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos);
+  launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
+                 hidden_dim);
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

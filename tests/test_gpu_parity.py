@@ -137,11 +137,12 @@ def test_ragged_token_counts(n_tokens):
         run.close()
 
 
-def test_many_tokens_per_expert_multi_tile():
-    """More than 256 rows for one expert: several N tiles per expert in both FFN kernels."""
+@pytest.mark.parametrize("n", [700, 2100])
+def test_many_tokens_per_expert_multi_tile(n):
+    """More than 256 rows for one expert: several N tiles per expert in both FFN kernels; the
+    larger case also takes the many-token variants of the gate and gather kernels."""
     from paper_2609_33385_b200.runner import bits_to_dev
     w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=256, intermediate=128)
-    n = 700                                     # ~350 rows per expert on average
     run = _runner(w, capacity=[4], max_tokens=n)
     ora = _oracle_for(run, [4])
     try:
@@ -178,6 +179,33 @@ def test_output_bit_identical_at_every_capacity():
         for (o0, i0), (o1, i1) in zip(outs[0], res):
             assert np.array_equal(i0, i1) and np.array_equal(o0, o1)
     assert miss[0] >= miss[1] >= miss[2]
+
+
+def test_iteration_entry_points_match_layer_by_layer_steps():
+    """oled_denoise_iteration (device and host buffers) == steps + residual adds, bit for bit."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=3, n_experts=8, top_k=2)
+    runs = [_runner(w, capacity=[3, 4, 2]) for _ in range(3)]
+    try:
+        dev = runs[0].device
+        out = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=dev)
+        bufs = [torch.empty_like(out), torch.empty_like(out)]
+        for _, _, h_bits, conf in synth.denoise_inputs(w):
+            x, c = bits_to_dev(h_bits, dev), torch.from_numpy(conf).to(dev)
+            ref = dev_to_bits(runs[0].iteration(x, c, bufs, out)).copy()
+            y = torch.empty_like(out)
+            runs[1].ctx.denoise_iteration(x.data_ptr(), c.data_ptr(), w.tokens, y.data_ptr())
+            assert np.array_equal(dev_to_bits(y), ref)
+            hx = torch.from_numpy(h_bits.view(np.int16)).pin_memory()
+            hc = torch.from_numpy(conf).pin_memory()
+            hy = torch.empty((w.tokens, w.hidden), dtype=torch.int16).pin_memory()
+            runs[2].ctx.denoise_iteration_host(hx.data_ptr(), hc.data_ptr(), w.tokens, hy.data_ptr())
+            assert np.array_equal(hy.numpy().view(np.uint16), ref)
+        assert runs[0].ctx.stats() == runs[1].ctx.stats() == runs[2].ctx.stats()
+        assert runs[0].ctx.stats().steps == 3 * w.iters * w.blocks
+    finally:
+        for r in runs:
+            r.close()
 
 
 def test_host_buffer_entry_point_matches_device_entry_point():
