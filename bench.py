@@ -349,14 +349,24 @@ def main():
     top = max(prof, key=lambda k: prof[k]["ms"])
     kp = prof[top]
     ach = kp["bytes"] / max(kp["ms"], 1e-9) / 1e6          # GB/s
-    roofline = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"],
+    ach_tf = kp["flops"] / max(kp["ms"], 1e-9) / 1e9       # TFLOP/s
+    tensor_bound = ach_tf / peaks["bf16_tflops_sustained"] > ach / peaks["hbm_gbs"]
+    roofline = {"kernel": top, "bound": "tensor" if tensor_bound else "hbm",
+                "achieved": ach_tf if tensor_bound else ach,
+                "peak": peaks["bf16_tflops_sustained"] if tensor_bound else peaks["hbm_gbs"],
+                "unit": "TFLOP/s" if tensor_bound else "GB/s",
+                "frac": (ach_tf / peaks["bf16_tflops_sustained"]) if tensor_bound else ach / peaks["hbm_gbs"],
+                "peak_source": peaks["source"] + (" (sustained bf16 matmul)" if tensor_bound else " (copy)"),
                 "traffic": None, "launches": kp["launches"],
                 "avg_launch_us": kp["ms"] * 1e3 / max(1, kp["launches"]),
-                "algorithmic_bytes_per_launch": kp["bytes"] / max(1, kp["launches"])}
+                "algorithmic_bytes_per_launch": kp["bytes"] / max(1, kp["launches"]),
+                "algorithmic_flops_per_launch": kp["flops"] / max(1, kp["launches"]),
+                "achieved_gbs": ach, "achieved_tflops": ach_tf}
     kernels = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
                    "gbs": (v["bytes"] / v["ms"] / 1e6) if v["ms"] > 0 else None}
                for k, v in prof.items()}
+    for k, v in prof.items():
+        kernels[k]["tflops"] = (v["flops"] / v["ms"] / 1e9) if v["ms"] > 0 else None
 
     step_roof = step_roofline(w, delta, args.steps, ms_per_step, peaks, h2d["gbs_blob_train"])
     extra = {"tpot_ms": ms_per_step * w.iters / w.tokens,
@@ -367,7 +377,7 @@ def main():
              "setup_s": setup_s}
 
     # 4. full residency on the same workload (C = E): the HBM-bound regime and the TPOT ratio
-    if not args.no_full_residency:
+    if not args.no_full_residency and w.residency < 1.0:
         full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run)
         ms_f, _, delta_f, _ = timed_pass(torch, full, xs, cs, args.warmup, args.steps)
         _, ms_f_max = dist.aggregate(0, ms_f, device)

@@ -25,7 +25,7 @@
  *     to oled_create(); oled_denoise_step() blocks the host until the gate results of the step
  *     are known (a few hundred bytes are read back to plan the copies), not until the step ends.
  *   - Shape limits: hidden a multiple of 256; intermediate a multiple of 128;
- *     1 <= top_k <= 32, top_k <= n_experts <= OLED_MAX_EXPERTS.
+ *     1 <= top_k <= 32, top_k <= n_experts <= OLED_MAX_EXPERTS, max_tokens <= 65535.
  */
 #ifndef OLED_H_
 #define OLED_H_

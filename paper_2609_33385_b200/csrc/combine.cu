@@ -13,8 +13,11 @@ namespace {
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
-               const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next) {
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next,
+               uint32_t* __restrict__ zero_words, int n_zero_words) {
   const int t = blockIdx.x;
+  if (t == 0 && zero_words != nullptr)
+    for (int i = threadIdx.x; i < n_zero_words; i += blockDim.x) zero_words[i] = 0u;
   __shared__ float s_g[OLED_MAX_TOPK];
   __shared__ int s_r[OLED_MAX_TOPK];
   if (threadIdx.x < K) {
@@ -68,8 +71,9 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 }  // namespace
 
 void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
-                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next) {
-  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out, x, x_next);
+                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
+                    uint32_t* zero_words, int n_zero_words) {
+  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out, x, x_next, zero_words, n_zero_words);
 }
 
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {

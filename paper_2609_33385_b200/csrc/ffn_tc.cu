@@ -479,6 +479,7 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   const int i1 = box_index(max_count, 128), i2 = box_index(max_count, 256);
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int n_box, int m_tiles) {
+    if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
     long long tiles = 0;
     for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + n_box - 1) / n_box;
     return (int)std::max<long long>(1, std::min<long long>(n_sms, tiles * m_tiles));

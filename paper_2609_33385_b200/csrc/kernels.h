@@ -21,12 +21,22 @@ struct FfnGroup {
 // Device status word values (0 = ok).
 enum : uint32_t { kStatusOk = 0, kStatusWaitTimeout = 1 };
 
+// Where the gate kernel's last CTA publishes the step's counts and scores for the host: mapped
+// pinned host memory, one 8-byte word per value with the step's sequence number in the upper
+// bits (scores: seq & 0xffff in bits 48..63; counts: seq in bits 32..63).  All-null = no report.
+struct RouteReport {
+  unsigned int* ticket = nullptr;               // device, zero before the launch
+  unsigned long long* host_scores = nullptr;    // mapped host [E]
+  unsigned long long* host_counts = nullptr;    // mapped host [E]
+  unsigned int seq = 0;
+};
+
 // ---- route.cu -------------------------------------------------------------------------
 // Gate logits in the contract order, top-k (ties to the lower index), softmax over the selected
 // logits, per-expert counts and integer reuse-score numerators (atomics on zeroed arrays).
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores);
+                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep);
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
 // kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
@@ -39,8 +49,11 @@ void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int 
 // ---- combine.cu -----------------------------------------------------------------------
 // out[t,:] = bf16( sum_j gate[t,j] * y[pos[t*K+j],:] ), j ascending, fp32 accumulation.  With
 // x_next != nullptr also x_next[t,:] = bf16(x[t,:] + out[t,:]) (the residual between layers).
+// zero_words != nullptr: CTA 0 also clears n_zero_words 32-bit words there (the step's control
+// block, ready for the next step's atomics).
 void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
-                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next);
+                    int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
+                    uint32_t* zero_words, int n_zero_words);
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n);
 
 // ---- ffn_simple.cu (bring-up path, plain FMA) ---------------------------------------------

@@ -2,6 +2,8 @@
 // orchestration (gate -> policy -> fills on a side stream -> grouped FFN -> combine) and the
 // counters.  The flow follows the paper's per-layer order (Sec. 4.1) with the sets of Sec. 4.2
 // and the retention rule of Sec. 4.2/4.3; every missed expert is fetched (no CPU execution).
+#include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -55,6 +57,12 @@ struct oled_ctx {
   uint16_t* d_hbuf = nullptr;  // [T*k,I]
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
+  unsigned int* d_ticket = nullptr;   // last word of the control block
+  bool ctrl_dirty = true;             // control block must be cleared before the next gate launch
+  unsigned int seq = 0;               // step sequence number echoed by the gate kernel
+  volatile unsigned long long* h_report = nullptr;  // pinned, mapped: tagged scores [E] | tagged counts [E]
+  std::vector<unsigned long long> host_scores;       // decoded copy of the last report
+  std::vector<int32_t> host_counts;
   uint16_t* d_hidden_stage = nullptr;  // for the host-buffer entry point
   float* d_conf_stage = nullptr;
   uint16_t* d_out_stage = nullptr;
@@ -203,7 +211,42 @@ void prof_resolve(oled_ctx* ctx) {
   cudaGetLastError();
 }
 
-// One FFN launch pair over `experts` (ids), weights through the layer's slot table.
+void prof_add(oled_ctx* ctx, int kernel, uint64_t bytes, uint64_t flops) {
+  if (!ctx->profile) return;
+  ctx->prof_acc[kernel].bytes += bytes;
+  ctx->prof_acc[kernel].flops += flops;
+}
+
+// Algorithmic bytes / flops of the two FFN kernels for n experts with `rows` token rows in total:
+// each expert's weights once, the token rows in, the result rows out.
+void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
+  const uint64_t H = ctx->shape.hidden, I = ctx->shape.intermediate, hi = H * I;
+  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * 2 * hi * 2 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
+  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * hi * 2 + rows * I * 2 + rows * H * 4, 2 * rows * hi);
+}
+
+// The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
+// known on the host yet (the group is the resident set and experts without tokens cost nothing).
+int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts) {
+  if (grp.n <= 0) return OLED_OK;
+  const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
+  if (ctx->ffn_impl == 1) {
+    launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
+                      ctx->d_y, H, I);
+  } else {
+    for (int kind = 1; kind <= 2; ++kind) {
+      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
+      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
+                                   ctx->d_hbuf, ctx->d_y, H, I, ctx->n_sms, ctx->d_status);
+      if (rc != OLED_OK) return rc;
+    }
+  }
+  ctx->launches += 2;
+  OLED_CUDA(ctx, cudaGetLastError());
+  return OLED_OK;
+}
+
+// FFN over experts[begin, end) (ids) with known counts, weights through the layer's slot table.
 int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& experts, size_t begin, size_t end,
                   const int32_t* counts) {
   if (begin >= end) return OLED_OK;
@@ -211,33 +254,44 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
   grp.n = (int32_t)(end - begin);
   grp.n_box = 16;
   int max_count = 0;
+  uint64_t rows = 0;
   for (size_t i = begin; i < end; ++i) {
     const int32_t e = experts[i];
     grp.expert[i - begin] = (uint16_t)e;
     grp.slot[i - begin] = (uint16_t)L.cache.slot_of[e];
     max_count = std::max(max_count, counts[e]);
+    rows += (uint64_t)counts[e];
   }
-  const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
-  if (ctx->ffn_impl == 1) {
-    launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
-                      ctx->d_y, H, I);
-  } else {
-    uint64_t rows = 0;
-    for (size_t i = begin; i < end; ++i) rows += (uint64_t)counts[experts[i]];
-    const uint64_t hi = (uint64_t)H * I, n = (uint64_t)grp.n;
-    for (int kind = 1; kind <= 2; ++kind) {
-      // algorithmic bytes: each expert's weights once, the token rows in, the result rows out
-      const uint64_t bytes = kind == 1 ? n * 2 * hi * 2 + rows * H * 2 + rows * I * 2
-                                       : n * hi * 2 + rows * I * 2 + rows * H * 4;
-      const uint64_t flops = (kind == 1 ? 4 : 2) * rows * hi;
-      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, bytes, flops);
-      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, counts, ctx->d_offsets, ctx->d_hbuf,
-                                   ctx->d_y, H, I, ctx->n_sms, ctx->d_status);
-      if (rc != OLED_OK) return rc;
+  prof_add_ffn(ctx, (uint64_t)grp.n, rows);
+  return run_ffn_launches(ctx, grp, max_count, counts);
+}
+
+// Blocks until the gate kernel of step `seq` has published counts and scores, and decodes them.
+int wait_gate_report(oled_ctx* ctx) {
+  const size_t E = (size_t)ctx->shape.n_experts;
+  const unsigned long long tag16 = (unsigned long long)(ctx->seq & 0xffffu);
+  const unsigned long long tag32 = (unsigned long long)ctx->seq;
+  const auto t0 = std::chrono::steady_clock::now();
+  bool synced = false;
+  for (size_t i = 0; i < 2 * E; ++i) {
+    for (uint64_t spin = 0;; ++spin) {
+      const unsigned long long v = ctx->h_report[i];
+      if (i < E ? (v >> 48) == tag16 : (v >> 32) == tag32) {
+        if (i < E) ctx->host_scores[i] = v & 0xffffffffffffull;
+        else ctx->host_counts[i - E] = (int32_t)(uint32_t)v;
+        break;
+      }
+      if ((spin & 0xFFFF) == 0xFFFF) {
+        const double s = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+        if (s > 20.0) {  // the kernel did not report: find out why instead of spinning for ever
+          if (synced) return OLED_ERR_TIMEOUT;
+          OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+          synced = true;
+        }
+      }
     }
   }
-  ctx->launches += 2;
-  OLED_CUDA(ctx, cudaGetLastError());
+  std::atomic_thread_fence(std::memory_order_acquire);
   return OLED_OK;
 }
 
@@ -268,7 +322,8 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   const oled_model_shape& s = *shape;
   if (s.n_layers <= 0 || s.hidden <= 0 || s.hidden % 256 != 0 || s.intermediate <= 0 ||
       s.intermediate % 128 != 0 || s.n_experts <= 0 || s.n_experts > OLED_MAX_EXPERTS || s.top_k <= 0 ||
-      s.top_k > OLED_MAX_TOPK || s.top_k > s.n_experts || s.max_tokens <= 0 || s.staging_slots < 0)
+      s.top_k > OLED_MAX_TOPK || s.top_k > s.n_experts || s.max_tokens <= 0 || s.max_tokens > 65535 ||
+      s.staging_slots < 0)
     return OLED_ERR_INVALID_ARG;
   int min_cap = s.n_experts;
   long long total_cap = 0;
@@ -315,12 +370,13 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
-  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t));
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + 2 * sizeof(uint32_t);
   uint8_t* ctrl = nullptr;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctrl, ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
   ctx->d_scores = reinterpret_cast<unsigned long long*>(ctrl);
   ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
+  ctx->d_ticket = reinterpret_cast<unsigned int*>(ctrl + E * (sizeof(unsigned long long) + sizeof(int32_t)));
   if ((rc = dev_alloc(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
@@ -340,10 +396,14 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
     if ((rc = dev_alloc(ctx, &ctx->layers[l].w_router, E * H)) != OLED_OK) return fail(rc);
     if (s.has_router_bias && (rc = dev_alloc(ctx, &ctx->layers[l].bias, E)) != OLED_OK) return fail(rc);
   }
-  if (cudaMallocHost(reinterpret_cast<void**>(&ctx->h_ctrl), ctx->ctrl_bytes) != cudaSuccess ||
+  if (cudaMallocHost(reinterpret_cast<void**>(&ctx->h_ctrl), 2 * E * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMallocHost(reinterpret_cast<void**>(&ctx->h_status), sizeof(uint32_t)) != cudaSuccess)
     return fail(OLED_ERR_OOM);
   *ctx->h_status = kStatusOk;
+  memset(ctx->h_ctrl, 0, 2 * E * sizeof(unsigned long long));
+  ctx->h_report = reinterpret_cast<volatile unsigned long long*>(ctx->h_ctrl);
+  ctx->host_scores.assign(E, 0);
+  ctx->host_counts.assign(E, 0);
   if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess ||
       cudaMemset(ctx->d_xp, 0, T * K * H * 2) != cudaSuccess ||
       cudaMemset(ctx->d_hbuf, 0, T * K * I * 2) != cudaSuccess ||
@@ -425,16 +485,21 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     return OLED_OK;
   }
 
-  // 1. gate, counts and reuse-score numerators; read them back while the permutation runs
-  OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
+  // 1. gate, counts and reuse-score numerators; the kernel's last CTA reports them to the host
+  if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
+  ctx->ctrl_dirty = true;
+  ctx->seq += 1;
+  RouteReport rep;
+  rep.ticket = ctx->d_ticket;
+  rep.host_scores = reinterpret_cast<unsigned long long*>(ctx->h_ctrl);
+  rep.host_counts = reinterpret_cast<unsigned long long*>(ctx->h_ctrl) + E;
+  rep.seq = ctx->seq;
   {
     ProfScope ps(ctx, OLED_KERNEL_ROUTE, ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * 8,
                  2ull * T * H * E);
     launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
-                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores);
+                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, rep);
   }
-  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_ctrl, ctx->d_scores, ctx->ctrl_bytes, cudaMemcpyDeviceToHost, st));
-  OLED_CUDA(ctx, cudaEventRecord(ctx->gate_event, st));
   const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
@@ -447,11 +512,32 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   }
   ctx->launches += fuse_gather ? 2 : 3;
   OLED_CUDA(ctx, cudaGetLastError());
-  OLED_CUDA(ctx, cudaEventSynchronize(ctx->gate_event));
-  // Everything enqueued before this step has completed, so slots released earlier are free to
-  // be overwritten by the side stream.
-  const unsigned long long* scores = reinterpret_cast<const unsigned long long*>(ctx->h_ctrl);
-  const int32_t* counts = reinterpret_cast<const int32_t*>(ctx->h_ctrl + (size_t)E * sizeof(unsigned long long));
+
+  // 1b. cache hits need no decision: the FFN over the experts resident BEFORE the step is
+  // enqueued at once (experts that received no token contribute no tile), so the GPU does not
+  // wait for the host's round trip below.
+  {
+    FfnGroup grp;
+    grp.n = 0;
+    grp.n_box = 16;
+    for (int32_t e = 0; e < E; ++e)
+      if (L.cache.resident[e] && L.cache.slot_of[e] >= 0) {
+        grp.expert[grp.n] = (uint16_t)e;
+        grp.slot[grp.n] = (uint16_t)L.cache.slot_of[e];
+        ++grp.n;
+      }
+    const int rc0 = run_ffn_launches(ctx, grp, T, nullptr);
+    if (rc0 != OLED_OK) return rc0;
+  }
+
+  // The report implies that everything enqueued before this step has completed, so slots
+  // released earlier are free to be overwritten by the side stream.
+  {
+    const int rcw = wait_gate_report(ctx);
+    if (rcw != OLED_OK) return rcw;
+  }
+  const unsigned long long* scores = ctx->host_scores.data();
+  const int32_t* counts = ctx->host_counts.data();
 
   // 2. hits / misses against the pre-step resident set, Top-C retention, slot plan
   StepPlan& plan = ctx->plan;
@@ -473,9 +559,13 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
       OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[n_chunks++], ctx->copy_stream));
   }
 
-  // 4. grouped FFN: hits at once, misses chunk by chunk as their weights land
-  int rc = run_ffn_group(ctx, L, plan.hits, 0, plan.hits.size(), counts);
-  if (rc != OLED_OK) return rc;
+  // 4. grouped FFN over the misses, chunk by chunk as their weights land (hits: step 1b)
+  {
+    uint64_t hit_rows = 0;
+    for (int32_t e : plan.hits) hit_rows += (uint64_t)counts[e];
+    prof_add_ffn(ctx, plan.hits.size(), hit_rows);
+  }
+  int rc = OLED_OK;
   for (size_t c = 0; c < n_chunks; ++c) {
     OLED_CUDA(ctx, cudaStreamWaitEvent(st, ctx->fill_events[c], 0));
     rc = run_ffn_group(ctx, L, plan.misses, c * chunk, std::min(n_miss, (c + 1) * chunk), counts);
@@ -486,10 +576,12 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   {
     ProfScope ps(ctx, OLED_KERNEL_COMBINE, (uint64_t)T * K * H * 4 + (uint64_t)T * H * 2, 2ull * T * K * H);
     launch_combine(st, ctx->d_y, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out),
-                   static_cast<const uint16_t*>(hidden), static_cast<uint16_t*>(x_next));
+                   static_cast<const uint16_t*>(hidden), static_cast<uint16_t*>(x_next),
+                   reinterpret_cast<uint32_t*>(ctx->d_scores), (int)(ctx->ctrl_bytes / 4));
   }
   ctx->launches += 1;
   OLED_CUDA(ctx, cudaGetLastError());
+  ctx->ctrl_dirty = false;  // combine's CTA 0 cleared the control block for the next step
 
   finish_step(L.cache, ctx->slots, plan);
   L.stats.steps += 1;
@@ -592,8 +684,8 @@ int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int
     if (ids) OLED_CUDA(ctx, cudaMemcpy(ids, ctx->d_ids, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
     if (gate) OLED_CUDA(ctx, cudaMemcpy(gate, ctx->d_gate, n * sizeof(float), cudaMemcpyDeviceToHost));
     if (perm) OLED_CUDA(ctx, cudaMemcpy(perm, ctx->d_perm, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
-    if (counts) OLED_CUDA(ctx, cudaMemcpy(counts, ctx->d_counts, E * sizeof(int32_t), cudaMemcpyDeviceToHost));
-    if (scores) OLED_CUDA(ctx, cudaMemcpy(scores, ctx->d_scores, E * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    if (counts) memcpy(counts, ctx->host_counts.data(), E * sizeof(int32_t));
+    if (scores) memcpy(scores, ctx->host_scores.data(), E * sizeof(uint64_t));
   } else {
     if (counts) memset(counts, 0, E * sizeof(int32_t));
     if (scores) memset(scores, 0, E * sizeof(uint64_t));

@@ -54,8 +54,9 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
              const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
              int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
              float* __restrict__ gate, int32_t* __restrict__ counts,
-             unsigned long long* __restrict__ scores) {
+             unsigned long long* __restrict__ scores, RouteReport rep) {
   extern __shared__ float s_logits[];  // [TT][E]
+  __shared__ int s_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
 
@@ -177,6 +178,25 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
       atomicAdd(&scores[my_id], q);
     }
   }
+
+  // The last CTA to finish publishes counts and scores to the host (mapped pinned memory).
+  // Every 8-byte word carries the step's sequence tag in its upper bits, so the host can tell
+  // word by word that the data is there: no ordering fence, no copy operation, no event.
+  if (rep.host_scores == nullptr) return;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
+  const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    rep.host_scores[e] = tag16 | __ldcg(&scores[e]);                               // score < 2^48
+    rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
+  }
 }
 
 // One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
@@ -258,19 +278,19 @@ gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, 
 
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores) {
+                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep) {
   if (T <= 128) {
     constexpr int TT = 1, W = 16;
     route_kernel<TT, W, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else if (T <= 1024) {
     constexpr int TT = 2, W = 8;
     route_kernel<TT, W, 2><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else {
     constexpr int TT = 8, W = 8;
     route_kernel<TT, W, 1><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores);
+        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   }
 }
 
@@ -362,7 +382,8 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   }
   if (n_tokens == 0) return OLED_OK;
   launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
-               confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores);
+               confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores,
+               RouteReport{});
   launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
                  hidden_dim);
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
