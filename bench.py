@@ -194,7 +194,7 @@ def measure_h2d(torch, device, blob_bytes: int) -> dict:
     return {"gbs_256mb": best, "gbs_blob_train": best_train}
 
 
-def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None):
+def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None, dummy=None):
     """warmup + steps denoising iterations; returns (ms total, launches, stats delta)."""
     w = run.w
     n_tok = w.tokens
@@ -211,6 +211,9 @@ def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None):
             run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), n_tok, dev_out.data_ptr())
 
     run.ctx.reset_cache()
+    if dummy is not None:          # warm the cache with dummy requests before the warm-up steps
+        for dx, dc in dummy:
+            run.ctx.denoise_iteration(dx.data_ptr(), dc.data_ptr(), n_tok, dev_out.data_ptr())
     for i in range(warmup):
         one(i)
     run.ctx.synchronize()
@@ -379,11 +382,19 @@ def main():
     # 4. full residency on the same workload (C = E): the HBM-bound regime and the TPOT ratio
     if not args.no_full_residency and w.residency < 1.0:
         full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run)
-        ms_f, _, delta_f, _ = timed_pass(torch, full, xs, cs, args.warmup, args.steps)
+        # dummy requests (i.i.d. tokens activate nearly every expert) so that no cold miss is left
+        dummy = []
+        for j, (_, _, h_bits, conf) in enumerate(synth.denoise_inputs(w.replace(shared_beta=0.0, seed=w.seed + 1))):
+            dummy.append((bits_to_dev(h_bits, device), torch.from_numpy(conf).to(device)))
+            if j >= 3:
+                break
+        ms_f, _, delta_f, _ = timed_pass(torch, full, xs, cs, args.warmup, args.steps, dummy=dummy)
         _, ms_f_max = dist.aggregate(0, ms_f, device)
         msf = ms_f_max / args.steps
         rf = step_roofline(w.replace(residency=1.0), delta_f, args.steps, msf, peaks, h2d["gbs_blob_train"])
         full.ctx.reset_cache()
+        for dx, dc in dummy:
+            full.ctx.denoise_iteration(dx.data_ptr(), dc.data_ptr(), w.tokens, out_dev.data_ptr())
         for i in range(args.warmup):
             full.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out_dev.data_ptr())
         full.ctx.synchronize()

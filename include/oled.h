@@ -152,7 +152,8 @@ int oled_reset_cache(oled_ctx* ctx);
 int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size_t n);
 
 /* Options.  OLED_OPT_FFN_IMPL: 0 = tcgen05 tensor-core kernels (default), 1 = plain-FMA
- * bring-up kernels.  OLED_OPT_MISS_CHUNK: experts per fill group (default 4).
+ * bring-up kernels.  OLED_OPT_MISS_CHUNK: size of the last fill group of a step, the only one whose
+ * FFN runs after all copies have landed (default 4).
  * OLED_OPT_PROFILE: 1 = bracket every kernel launch with CUDA events on the context's stream
  * (adds two event records per launch; off by default). */
 #define OLED_OPT_FFN_IMPL 1

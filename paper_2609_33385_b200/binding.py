@@ -17,7 +17,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liboled.so")
+LIB_PATH = os.environ.get("OLED_LIB_PATH") or os.path.join(_HERE, "liboled.so")
 
 OLED_OK = 0
 ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -2, -3, -4

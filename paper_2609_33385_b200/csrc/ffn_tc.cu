@@ -11,8 +11,13 @@
 // 256.  Weights are addressed through the expert->slot table: one 3-D tensor map covers the
 // whole slot pool and the slot number is a TMA coordinate.
 //
-// Warp roles (192 threads): warps 0-3 epilogue (TMEM lane quarter = warp id), warp 4 lane 0 TMA
-// producer, warp 5 lane 0 MMA issuer (warp 5 also owns the TMEM allocation).  Every mbarrier
+// In the many-token regime (N tile 256) both kernels work on two 128-row weight tiles that share
+// one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
+// which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
+//
+// Warp roles (320 threads): warps 0-7 epilogue (TMEM lane quarter = warp id mod 4, the two warps
+// of a quarter alternate 16-column chunks), warp 8 lane 0 TMA producer, warp 9 lane 0 MMA issuer
+// (warp 9 also owns the TMEM allocation).  Every mbarrier
 // wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
 // copies time to land, frees its TMEM and returns.
 #include <cuda.h>
@@ -26,7 +31,13 @@
 namespace oled {
 namespace {
 
-constexpr int kThreads = 192;
+#ifndef OLED_EPI_WARPS
+#define OLED_EPI_WARPS 8
+#endif
+constexpr int kEpiWarps = OLED_EPI_WARPS;                 // two warps per TMEM lane quarter, alternating 16-column chunks
+constexpr int kProducerWarp = kEpiWarps;
+constexpr int kMmaWarp = kEpiWarps + 1;
+constexpr int kThreads = (kEpiWarps + 2) * 32;
 constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
 constexpr uint32_t kATile = kBlockM * kBlockK * 2;
@@ -163,18 +174,20 @@ struct Item {
   int slot, m0, row0, valid;
 };
 __device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int m_tiles,
-                                            int n_box, int& g, Item& it) {
+                                            int m_rows, int n_box, int& g, Item& it) {
   const int q = item / m_tiles;
   const int m = item - q * m_tiles;
   while (ctl->tile_prefix[g + 1] <= q) ++g;
   const int nt = q - ctl->tile_prefix[g];
   it.slot = grp.slot[g];
-  it.m0 = m * kBlockM;
+  it.m0 = m * m_rows;
   it.row0 = ctl->row_start[g] + nt * n_box;
   it.valid = min(n_box, ctl->count[g] - nt * n_box);
 }
 
-template <int KIND>
+// DUAL: two accumulators per item - gate and up (KIND 1, always), or two row blocks of Wd
+// (KIND 2 with the 256-token tile).
+template <int KIND, bool DUAL>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
@@ -185,11 +198,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_box = grp.n_box;
-  constexpr uint32_t a_bytes = (KIND == 1 ? 2u : 1u) * kATile;
+  constexpr bool dual = DUAL;
+  constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t stage_bytes = a_bytes + (uint32_t)n_box * 128u;
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
-  const int m_tiles = (KIND == 1 ? I : H) / kBlockM;
-  const int acc_cols = (KIND == 1 ? 2 : 1) * n_box;
+  constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : kBlockM;  // output features per item
+  const int m_tiles = (KIND == 1 ? I : H) / m_rows;
+  const int acc_cols = (dual ? 2 : 1) * n_box;
   const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
@@ -208,7 +223,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[a]), 128);
+      mbar_init(smem_u32(&ctl->tmem_empty[a]), (n_box > 16 ? kEpiWarps : 4) * 32);
     }
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -224,7 +239,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     ctl->tile_prefix[grp.n] = acc;
     ctl->n_tiles_total = acc;
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&ctl->tmem_base)),
                  "r"(tmem_cols)
@@ -239,14 +254,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int total_items = ctl->n_tiles_total * m_tiles;
   volatile int* abort_flag = &ctl->abort;
 
-  if (warp == 4 && lane == 0) {
+  if (warp == kProducerWarp && lane == 0) {
     // ------------------------------------------------------------ TMA producer
     int stage = 0, g = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
       Item it;
-      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       for (int kb = 0; kb < k_blocks; ++kb) {
         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status)) {
           ok = false;
@@ -260,6 +275,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
         } else {
           tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // down rows
+          if (dual) tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
         }
         tma_load_2d(&tm_act, a_addr + a_bytes, bar, kb * kBlockK, it.row0);
         if (++stage == n_stages) {
@@ -273,14 +289,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       while (globaltimer() - t0 < 2000000ull) {
       }
     }
-  } else if (warp == 5 && lane == 0) {
+  } else if (warp == kMmaWarp && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
     int stage = 0, g = 0, local = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
       Item it;
-      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
       if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
@@ -301,7 +317,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           const uint64_t db = make_smem_desc(b_addr + k * 32);
           const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
           tc_mma(d0, make_smem_desc(a_addr + k * 32), db, idesc, accum);
-          if (KIND == 1) tc_mma(d0 + (uint32_t)n_box, make_smem_desc(a_addr + kATile + k * 32), db, idesc, accum);
+#ifndef OLED_DBG_SKIP_SECOND_MMA  // timing experiment only: results are wrong when defined
+          if (dual) tc_mma(d0 + (uint32_t)n_box, make_smem_desc(a_addr + kATile + k * 32), db, idesc, accum);
+#endif
         }
         tc_commit(smem_u32(&ctl->empty[stage]));
         if (++stage == n_stages) {
@@ -311,22 +329,27 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
-  } else if (warp < 4) {
+  } else if (warp < (n_box > 16 ? kEpiWarps : 4)) {
     // ------------------------------------------------------------ epilogue
+    // (a 16-column accumulator is one chunk: the second warp of each quarter has nothing to do)
     int g = 0, local = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
       Item it;
-      decode_item(ctl, grp, item, m_tiles, n_box, g, it);
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
-      // warp-uniform outcome: tcgen05.ld below is warp-collective
-      const bool ready = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, status);
-      if (!__all_sync(0xffffffffu, ready)) break;
+      // one lane polls (keeps issue slots free for the producer and MMA threads); the outcome is
+      // warp-uniform because tcgen05.ld below is warp-collective
+      int ready = 0;
+      if (lane == 0) ready = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, status) ? 1 : 0;
+      ready = __shfl_sync(0xffffffffu, ready, 0);
+      if (!ready) break;
       tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * acc_cols);
+      const int quarter = warp & 3, half = warp >> 2;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * acc_cols);
       const int n_mma = max(16, (it.valid + 15) & ~15);
-      const int col = it.m0 + warp * 32 + lane;  // output feature owned by this thread
-      for (int c = 0; c < n_mma; c += 16) {
+      const int col = it.m0 + quarter * 32 + lane;  // output feature owned by this thread
+      for (int c = half * 16; c < n_mma; c += 32) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
         if (KIND == 1) {
@@ -345,11 +368,23 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
           }
         } else {
-          tmem_ld_wait();
           float* y = reinterpret_cast<float*>(out_ptr);
+          if (dual) {
+            uint32_t rb[16];
+            tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
+            tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (c + j < it.valid) y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
+            for (int j = 0; j < 16; ++j)
+              if (c + j < it.valid) {
+                y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
+                y[(size_t)(it.row0 + c + j) * H + col + kBlockM] = __uint_as_float(rb[j]);
+              }
+          } else {
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (c + j < it.valid) y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
+          }
         }
       }
       tc_fence_before();
@@ -360,7 +395,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // ---- teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
@@ -409,12 +444,12 @@ int stages_for(int kind, int n_box) {
     const char* env = getenv("OLED_FFN_STAGES");
     cap = env ? std::max(1, atoi(env)) : kMaxStages;
   }
-  const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+  const uint32_t stage = ((kind == 1 || n_box == 256) ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
   return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage);
 }
 uint32_t smem_for(int kind, int n_box, int stages) {
-  const uint32_t stage = (kind == 1 ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+  const uint32_t stage = ((kind == 1 || n_box == 256) ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   return kCtlBytes + 1024u + (uint32_t)stages * stage;
 }
 
@@ -449,10 +484,12 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   }
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(ffn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) !=
-            cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemMax) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemMax) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemMax) != cudaSuccess)
       return OLED_ERR_CUDA;
     attr_done = true;
   }
@@ -475,8 +512,9 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
                   uint32_t* status) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
-  // KIND 1 holds two accumulators per tile: N <= 128 keeps them double-buffered in TMEM.
-  const int i1 = box_index(max_count, 128), i2 = box_index(max_count, 256);
+  // N <= 128 keeps the accumulators double-buffered in TMEM; more tokens per expert than that
+  // take N = 256 with two weight tiles per item (all 512 TMEM columns, one accumulator stage).
+  const int i1 = box_index(max_count, 256), i2 = box_index(max_count, 256);
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int n_box, int m_tiles) {
     if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
@@ -487,13 +525,17 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   if (kind == 1) {
     grp.n_box = 16 << i1;
     const int stages = stages_for(1, grp.n_box);
-    ffn_tc_kernel<1><<<grid_for(grp.n_box, I / kBlockM), kThreads, smem_for(1, grp.n_box, stages), st>>>(
+    ffn_tc_kernel<1, true><<<grid_for(grp.n_box, I / kBlockM), kThreads, smem_for(1, grp.n_box, stages), st>>>(
         maps.w13, maps.xp[i1], grp, offsets, hbuf, H, I, stages, status);
   } else {
     grp.n_box = 16 << i2;
     const int stages = stages_for(2, grp.n_box);
-    ffn_tc_kernel<2><<<grid_for(grp.n_box, H / kBlockM), kThreads, smem_for(2, grp.n_box, stages), st>>>(
-        maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
+    if (grp.n_box == 256)
+      ffn_tc_kernel<2, true><<<grid_for(256, H / (2 * kBlockM)), kThreads, smem_for(2, 256, stages), st>>>(
+          maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
+    else
+      ffn_tc_kernel<2, false><<<grid_for(grp.n_box, H / kBlockM), kThreads, smem_for(2, grp.n_box, stages), st>>>(
+          maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

@@ -526,7 +526,9 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
         grp.slot[grp.n] = (uint16_t)L.cache.slot_of[e];
         ++grp.n;
       }
-    const int rc0 = run_ffn_launches(ctx, grp, T, nullptr);
+    // token tile of this launch: twice the mean load per expert (a fuller expert takes more tiles)
+    const int mean_load = (int)(((size_t)T * K + E - 1) / E);
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr);
     if (rc0 != OLED_OK) return rc0;
   }
 
@@ -546,29 +548,39 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   ctx->last_before = plan.before;
   ctx->last_after = plan.after;
 
-  // 3. fills: one pinned-host -> HBM copy per miss on the side stream, an event per chunk
+  // 3. fills: one pinned-host -> HBM copy per miss on the side stream.  The misses form two
+  // groups: everything but the last `miss_chunk` experts, then those last few.  The first group's
+  // FFN is one large launch that runs under the copies of the second; only the small second
+  // group's FFN is exposed after the last byte has arrived.
   const size_t n_miss = plan.misses.size();
-  const size_t chunk = (size_t)ctx->miss_chunk;
-  size_t n_chunks = 0;
-  for (size_t i = 0; i < n_miss; ++i) {
-    const int32_t e = plan.misses[i];
-    OLED_CUDA(ctx, cudaMemcpyAsync(ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes,
-                                   L.host_blob + (size_t)e * L.host_stride, ctx->slot_bytes,
-                                   cudaMemcpyHostToDevice, ctx->copy_stream));
-    if ((i + 1) % chunk == 0 || i + 1 == n_miss)
-      OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[n_chunks++], ctx->copy_stream));
+  const size_t tail = std::min(n_miss, (size_t)ctx->miss_chunk);
+  const size_t bounds[3] = {0, n_miss - tail, n_miss};
+  size_t n_groups = 0;
+  size_t group_begin[2], group_end[2];
+  for (int gi = 0; gi < 2; ++gi) {
+    if (bounds[gi] == bounds[gi + 1]) continue;
+    for (size_t i = bounds[gi]; i < bounds[gi + 1]; ++i) {
+      const int32_t e = plan.misses[i];
+      OLED_CUDA(ctx, cudaMemcpyAsync(ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes,
+                                     L.host_blob + (size_t)e * L.host_stride, ctx->slot_bytes,
+                                     cudaMemcpyHostToDevice, ctx->copy_stream));
+    }
+    OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[n_groups], ctx->copy_stream));
+    group_begin[n_groups] = bounds[gi];
+    group_end[n_groups] = bounds[gi + 1];
+    ++n_groups;
   }
 
-  // 4. grouped FFN over the misses, chunk by chunk as their weights land (hits: step 1b)
+  // 4. grouped FFN over the misses as their weights land (hits: step 1b)
   {
     uint64_t hit_rows = 0;
     for (int32_t e : plan.hits) hit_rows += (uint64_t)counts[e];
     prof_add_ffn(ctx, plan.hits.size(), hit_rows);
   }
   int rc = OLED_OK;
-  for (size_t c = 0; c < n_chunks; ++c) {
+  for (size_t c = 0; c < n_groups; ++c) {
     OLED_CUDA(ctx, cudaStreamWaitEvent(st, ctx->fill_events[c], 0));
-    rc = run_ffn_group(ctx, L, plan.misses, c * chunk, std::min(n_miss, (c + 1) * chunk), counts);
+    rc = run_ffn_group(ctx, L, plan.misses, group_begin[c], group_end[c], counts);
     if (rc != OLED_OK) return rc;
   }
 

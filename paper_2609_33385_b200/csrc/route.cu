@@ -42,13 +42,12 @@ __device__ __forceinline__ float exp_spec(float x) {
   return __fmul_rn(p, scale);
 }
 
-constexpr int kEPerWarp = 4;                   // experts per warp per pass
 constexpr int kMaxEPerLane = OLED_MAX_EXPERTS / 32;
 
-// TT tokens per CTA, WARPS warps; each warp owns 4 experts per pass and all TT tokens.  Small
+// TT tokens per CTA, WARPS warps; each warp owns kEPerWarp experts per pass and all TT tokens.  Small
 // blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
 // chunks of loads in flight; the chain order of every logit is the same in all variants.
-template <int TT, int WARPS, int UNROLL>
+template <int TT, int WARPS, int UNROLL, int kEPerWarp>
 __global__ void __launch_bounds__(WARPS * 32)
 route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
              const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
@@ -227,25 +226,47 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   __syncthreads();
   if (counts[e] == 0) return;
   int base = s_base;
-  for (int a0 = 0; a0 < n; a0 += blockDim.x) {
-    const int a = a0 + threadIdx.x;
-    const bool match = a < n && ids[a] == e;
-    const uint32_t bal = __ballot_sync(0xffffffffu, match);
+  // stable scan, 8 consecutive assignments per thread and 2048 per round
+  for (int a0 = 0; a0 < n; a0 += 8 * blockDim.x) {
+    const int first = a0 + threadIdx.x * 8;
+    int v[8];
+    if (first + 8 <= n) {
+      const int4 lo = *reinterpret_cast<const int4*>(ids + first);
+      const int4 hi = *reinterpret_cast<const int4*>(ids + first + 4);
+      v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w;
+      v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = first + i < n ? ids[first + i] : -1;
+    }
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m |= (v[i] == e ? 1u : 0u) << i;
+    const int c = __popc(m);
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
+    }
     __syncthreads();  // previous round's s_red fully consumed
-    if (lane == 0) s_red[warp] = __popc(bal);
+    if (lane == 31) s_red[warp] = incl;
     __syncthreads();
     int before = 0, total = 0;
 #pragma unroll
     for (int w = 0; w < 8; ++w) {
-      const int c = s_red[w];
-      if (w < warp) before += c;
-      total += c;
+      const int cw = s_red[w];
+      if (w < warp) before += cw;
+      total += cw;
     }
-    if (match) {
-      const int r = base + before + __popc(bal & ((1u << lane) - 1u));
-      perm[r] = a;
-      pos[a] = r;
-    }
+    int r = base + before + incl - c;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if ((m >> i) & 1u) {
+        perm[r] = first + i;
+        pos[first + i] = r;
+        ++r;
+      }
     base += total;
   }
   if (xp == nullptr) return;
@@ -281,15 +302,15 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
                   float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep) {
   if (T <= 128) {
     constexpr int TT = 1, W = 16;
-    route_kernel<TT, W, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
+    route_kernel<TT, W, 4, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
         x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else if (T <= 1024) {
     constexpr int TT = 2, W = 8;
-    route_kernel<TT, W, 2><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
+    route_kernel<TT, W, 2, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
         x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else {
     constexpr int TT = 8, W = 8;
-    route_kernel<TT, W, 1><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
+    route_kernel<TT, W, 1, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
         x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   }
 }
