@@ -15,7 +15,7 @@ from typing import Callable, List, Optional, Sequence
 import numpy as np
 
 from .cache_policy import LayerCache, LayerStats
-from .moe_layer import moe_layer_forward
+from .moe_layer import bf16_to_f32, gate_logits, moe_layer_forward, permutation, topk_route
 
 
 class OracleStack:
@@ -55,6 +55,23 @@ class OracleStack:
                         self.top_k)
         res.update(self.caches[layer].step(res["ids"], res["gate"], conf))
         return res
+
+    def route_step(self, layer: int, hidden_bits: np.ndarray, conf: np.ndarray) -> dict:
+        """Gate, permutation and cache policy of one layer execution, without the expert FFNs
+        (for large shapes, where outputs are checked on sampled tokens with ``token_outputs``)."""
+        x = bf16_to_f32(hidden_bits)
+        logits = gate_logits(x, bf16_to_f32(self.router[layer]), self.bias[layer])
+        ids, g = topk_route(logits, self.top_k)
+        counts, offsets, perm, pos = permutation(ids, self.n_experts)
+        res = dict(logits=logits, ids=ids, gate=g, counts=counts, offsets=offsets, perm=perm, pos=pos)
+        res.update(self.caches[layer].step(ids, g, conf))
+        return res
+
+    def token_outputs(self, layer: int, hidden_bits: np.ndarray, tokens) -> np.ndarray:
+        """Layer output rows of the given tokens only (each token's output depends on no other)."""
+        sel = np.asarray(hidden_bits)[list(tokens)]
+        return moe_layer_forward(sel, self.router[layer], self.bias[layer], self.experts[layer],
+                                 self.top_k)["out"]
 
     def policy_step(self, layer: int, ids: np.ndarray, gate: np.ndarray, conf: np.ndarray) -> dict:
         """Cache simulation alone, from recorded routing."""
