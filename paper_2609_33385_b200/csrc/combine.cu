@@ -16,6 +16,8 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next,
                uint32_t* __restrict__ zero_words, int n_zero_words) {
   const int t = blockIdx.x;
+  griddep_launch_dependents();
+  griddep_wait();
   if (t == 0 && zero_words != nullptr)
     for (int i = threadIdx.x; i < n_zero_words; i += blockDim.x) zero_words[i] = 0u;
   __shared__ float s_g[OLED_MAX_TOPK];
@@ -59,6 +61,8 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
 __global__ void __launch_bounds__(256)
 residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ r,
                     uint16_t* __restrict__ y, size_t n) {
+  griddep_launch_dependents();
+  griddep_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
        i += (size_t)gridDim.x * blockDim.x) {
     const float a = __uint_as_float((uint32_t)x[i] << 16);
@@ -73,12 +77,13 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
                     uint32_t* zero_words, int n_zero_words) {
-  combine_kernel<<<T, 256, 0, st>>>(y, gate, pos, H, K, out, x, x_next, zero_words, n_zero_words);
+  launch_pdl(combine_kernel, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+             n_zero_words);
 }
 
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {
   const int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-  residual_add_kernel<<<blocks, 256, 0, st>>>(x, r, y, n);
+  launch_pdl(residual_add_kernel, dim3(blocks), dim3(256), 0, st, x, r, y, n);
 }
 
 }  // namespace oled

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(256)
 ffn1_simple_kernel(const __grid_constant__ FfnGroup grp, const uint8_t* __restrict__ pool,
                    size_t slot_bytes, const int32_t* __restrict__ offsets,
                    const uint16_t* __restrict__ xp, uint16_t* __restrict__ hbuf, int H, int I) {
+  griddep_wait();
   const int e = grp.expert[blockIdx.y];
   const uint16_t* w = reinterpret_cast<const uint16_t*>(pool + (size_t)grp.slot[blockIdx.y] * slot_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -60,6 +61,7 @@ __global__ void __launch_bounds__(256)
 ffn2_simple_kernel(const __grid_constant__ FfnGroup grp, const uint8_t* __restrict__ pool,
                    size_t slot_bytes, const int32_t* __restrict__ offsets,
                    const uint16_t* __restrict__ hbuf, float* __restrict__ y, int H, int I) {
+  griddep_wait();
   const int e = grp.expert[blockIdx.y];
   const uint16_t* w = reinterpret_cast<const uint16_t*>(pool + (size_t)grp.slot[blockIdx.y] * slot_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -209,13 +209,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
 
-  // ---- set-up: work table, barriers, TMEM
-  for (int g = threadIdx.x; g < grp.n; g += kThreads) {
-    const int e = grp.expert[g];
-    const int s = offsets[e];
-    ctl->row_start[g] = s;
-    ctl->count[g] = offsets[e + 1] - s;
-  }
+  // ---- set-up that depends on no earlier kernel: barriers, TMEM (overlaps the predecessor's tail)
+  griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(smem_u32(&ctl->full[s]), 1);
@@ -229,6 +224,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (warp == kMmaWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&ctl->tmem_base)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // ---- from here on the step's earlier kernels must have completed: work table from offsets
+  griddep_wait();
+  for (int g = threadIdx.x; g < grp.n; g += kThreads) {
+    const int e = grp.expert[g];
+    const int s = offsets[e];
+    ctl->row_start[g] = s;
+    ctl->count[g] = offsets[e + 1] - s;
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     int acc = 0;
@@ -238,13 +248,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
     ctl->tile_prefix[grp.n] = acc;
     ctl->n_tiles_total = acc;
-  }
-  if (warp == kMmaWarp) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&ctl->tmem_base)),
-                 "r"(tmem_cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -525,17 +528,19 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   if (kind == 1) {
     grp.n_box = 16 << i1;
     const int stages = stages_for(1, grp.n_box);
-    ffn_tc_kernel<1, true><<<grid_for(grp.n_box, I / kBlockM), kThreads, smem_for(1, grp.n_box, stages), st>>>(
-        maps.w13, maps.xp[i1], grp, offsets, hbuf, H, I, stages, status);
+    launch_pdl(ffn_tc_kernel<1, true>, dim3(grid_for(grp.n_box, I / kBlockM)), dim3(kThreads),
+               smem_for(1, grp.n_box, stages), st, maps.w13, maps.xp[i1], grp, offsets, (void*)hbuf, H, I, stages,
+               status);
   } else {
     grp.n_box = 16 << i2;
     const int stages = stages_for(2, grp.n_box);
     if (grp.n_box == 256)
-      ffn_tc_kernel<2, true><<<grid_for(256, H / (2 * kBlockM)), kThreads, smem_for(2, 256, stages), st>>>(
-          maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
+      launch_pdl(ffn_tc_kernel<2, true>, dim3(grid_for(256, H / (2 * kBlockM))), dim3(kThreads),
+                 smem_for(2, 256, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, status);
     else
-      ffn_tc_kernel<2, false><<<grid_for(grp.n_box, H / kBlockM), kThreads, smem_for(2, grp.n_box, stages), st>>>(
-          maps.w2, maps.hbuf[i2], grp, offsets, y, H, I, stages, status);
+      launch_pdl(ffn_tc_kernel<2, false>, dim3(grid_for(grp.n_box, H / kBlockM)), dim3(kThreads),
+                 smem_for(2, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages,
+                 status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

@@ -4,10 +4,41 @@
 #include <cuda_runtime.h>
 #include <cstddef>
 #include <cstdint>
+#include <utility>
 
 #include "../../include/oled.h"
 
 namespace oled {
+
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Every kernel of a step is launched with programmatic stream serialization: it may be scheduled
+// while its predecessor drains, does its data-independent prologue, then blocks in
+// griddep_wait() until the predecessor has completed and its writes are visible.  Every kernel
+// executes griddep_wait() before touching global data, so dependencies hold transitively.
+#ifdef __CUDACC__
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+bool pdl_enabled();            // attribute on? (OLED_PDL=0 turns it off for good)
+void pdl_set_step(bool on);    // per step: used for small steps only (it costs ~2 % on many-token steps)
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // The experts one FFN launch works on and the slot each one's weights sit in: the per-launch
 // image of the expert->slot indirection table, passed by value in kernel-parameter space.

@@ -485,6 +485,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     return OLED_OK;
   }
 
+  pdl_set_step((size_t)T * K <= 4096);
   // 1. gate, counts and reuse-score numerators; the kernel's last CTA reports them to the host
   if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
   ctx->ctrl_dirty = true;

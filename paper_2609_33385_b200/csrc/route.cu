@@ -12,6 +12,7 @@
 //   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
 // The router stays off the tensor cores on purpose: their accumulation order is unspecified.
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "kernels.h"
@@ -58,6 +59,8 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   __shared__ int s_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
+  griddep_launch_dependents();
+  griddep_wait();
 
   constexpr int kRouteWarps = WARPS;
   for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
@@ -210,6 +213,8 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   __shared__ int s_base;
   const int e = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  griddep_launch_dependents();
+  griddep_wait();
   int part = 0;
   for (int i = threadIdx.x; i < e; i += blockDim.x) part += counts[i];
 #pragma unroll
@@ -285,6 +290,8 @@ gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, 
               int K, uint16_t* __restrict__ xp) {
   const int vec_per_row = H / 8;
   const size_t total = (size_t)n_rows * vec_per_row;
+  griddep_launch_dependents();
+  griddep_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(i / vec_per_row);
@@ -297,35 +304,46 @@ gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, 
 
 }  // namespace
 
+static thread_local bool g_pdl_step = true;
+void pdl_set_step(bool on) { g_pdl_step = on; }
+bool pdl_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char* env = getenv("OLED_PDL");
+    on = (env && atoi(env) == 0) ? 0 : 1;
+  }
+  return on == 1 && g_pdl_step;
+}
+
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep) {
   if (T <= 128) {
     constexpr int TT = 1, W = 16;
-    route_kernel<TT, W, 4, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
+    launch_pdl(route_kernel<TT, W, 4, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
+               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else if (T <= 1024) {
     constexpr int TT = 2, W = 8;
-    route_kernel<TT, W, 2, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
+    launch_pdl(route_kernel<TT, W, 2, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
+               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else {
     constexpr int TT = 8, W = 8;
-    route_kernel<TT, W, 1, 4><<<(T + TT - 1) / TT, W * 32, TT * E * sizeof(float), st>>>(
-        x, w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
+    launch_pdl(route_kernel<TT, W, 1, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
+               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   }
 }
 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp,
                     int H) {
-  permute_kernel<<<E, 256, 0, st>>>(ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K);
+  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K);
 }
 
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp) {
   const size_t total = (size_t)T * K * (H / 8);
   const int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-  gather_kernel<<<blocks, 256, 0, st>>>(x, perm, T * K, H, K, xp);
+  launch_pdl(gather_kernel, dim3(blocks), dim3(256), 0, st, x, perm, T * K, H, K, xp);
 }
 
 }  // namespace oled

@@ -1,0 +1,102 @@
+"""Cache-capacity x hidden-state-correlation sweep on the 64-expert / top-8 / hidden-2048 shape.
+
+The synthetic analogue of the paper's cache-capacity sensitivity study (Sec. 5.4): for every
+(residency, rho) point it reports hits, misses, host->HBM bytes and TPOT of a MoE-only stack,
+next to the full-residency TPOT and the lower bound the measured host link puts on the step.
+
+    python -m paper_2609_33385_b200.sweep [--layers 16] [--variant A|B] [--out file.md]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+import torch
+
+from . import build, synth
+from .runner import StackRunner, bits_to_dev
+
+
+def run_point(run: StackRunner, xs, cs, warmup: int, steps: int):
+    w = run.w
+    out = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=run.device)
+    run.ctx.reset_cache()
+    for i in range(warmup):
+        run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out.data_ptr())
+    run.ctx.synchronize()
+    s0 = run.ctx.stats()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(run.stream)
+    for i in range(warmup, warmup + steps):
+        run.ctx.denoise_iteration(xs[i].data_ptr(), cs[i].data_ptr(), w.tokens, out.data_ptr())
+    b.record(run.stream)
+    torch.cuda.synchronize()
+    s1 = run.ctx.stats()
+    ms = a.elapsed_time(b) / steps
+    d = {k: getattr(s1, k) - getattr(s0, k) for k in ("steps", "hits", "misses", "bytes_moved",
+                                                     "active_experts")}
+    return ms, d
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--layers", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--variant", default="A", choices=["A", "B"])
+    ap.add_argument("--h2d-gbs", type=float, default=54.5, help="measured host-link bandwidth")
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args()
+    build.build()
+    device = "cuda:0"
+    rows = []
+    base_store = None
+    for rho in (0.5, 0.9, 0.98):
+        over = dict(n_layers=args.layers, rho=rho)
+        if args.variant == "B":
+            over["shared_beta"] = 0.9
+        w0 = synth.config(3, **over)
+        n_it = args.warmup + args.steps
+        w0 = w0.replace(blocks=-(-n_it // w0.iters))
+        xs, cs = [], []
+        for _, _, h_bits, conf in synth.denoise_inputs(w0):
+            xs.append(bits_to_dev(h_bits, device))
+            cs.append(torch.from_numpy(conf).to(device))
+        full_ms = None
+        for res in (1.0, 0.6, 0.4, 0.2, 0.1):
+            w = w0.replace(residency=res)
+            run = StackRunner(w, device=device, share_store_of=base_store)
+            if base_store is None:
+                base_store = run
+            ms, d = run_point(run, xs, cs, args.warmup, args.steps)
+            if res == 1.0:
+                full_ms = ms
+            link_ms = d["bytes_moved"] / args.steps / (args.h2d_gbs * 1e9) * 1e3
+            rows.append(dict(rho=rho, residency=res, capacity=w.capacity, ms_per_step=ms,
+                             tpot_ms=ms * w.iters / w.tokens, hits=d["hits"], misses=d["misses"],
+                             h2d_gb_per_step=d["bytes_moved"] / args.steps / 1e9,
+                             utilisation=d["hits"] / max(1, d["steps"] * w.capacity),
+                             active=d["active_experts"] / max(1, d["steps"]),
+                             ratio_vs_full=ms / full_ms, link_bound_ms=link_ms,
+                             frac_of_link=(link_ms / ms) if link_ms > 0 else None))
+            if run is not base_store:
+                run.close()
+    lines = ["| rho | residency | C | hits | misses | H2D GB/step | ms/step | TPOT ms | utilisation | "
+             "active/layer | x full | link bound ms | link frac |", "|" + "---|" * 13]
+    for r in rows:
+        lf = "-" if r["frac_of_link"] is None else f"{r['frac_of_link']:.2f}"
+        lines.append(f"| {r['rho']} | {r['residency']:.0%} | {r['capacity']} | {r['hits']} | {r['misses']} | "
+                     f"{r['h2d_gb_per_step']:.3f} | {r['ms_per_step']:.3f} | {r['tpot_ms']:.3f} | "
+                     f"{r['utilisation']:.3f} | {r['active']:.1f} | {r['ratio_vs_full']:.2f} | "
+                     f"{r['link_bound_ms']:.2f} | {lf} |")
+    text = "\n".join(lines)
+    print(text)
+    if args.out:
+        with open(args.out, "w") as f:
+            f.write(text + "\n")
+            f.write("\n" + json.dumps(rows) + "\n")
+
+
+if __name__ == "__main__":
+    sys.exit(main())
