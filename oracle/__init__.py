@@ -7,6 +7,6 @@ reference legs import this package.
 """
 from .moe_layer import (bf16_to_f32, gate_logits, exp_spec, topk_route, permutation,  # noqa: F401
                         expert_ffn, moe_layer_forward)
-from .cache_policy import (psi, reuse_scores, priorities, retain_top_c, LayerCache,  # noqa: F401
-                           LayerStats)
+from .cache_policy import (psi, reuse_scores, priorities, retain_top_c, retain_by_value,  # noqa: F401
+                           ideal_hits, apportion, AdaptiveSizer, LayerCache, LayerStats)
 from .denoise import OracleStack  # noqa: F401

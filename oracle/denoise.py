@@ -14,7 +14,7 @@ from typing import Callable, List, Optional, Sequence
 
 import numpy as np
 
-from .cache_policy import LayerCache, LayerStats
+from .cache_policy import AdaptiveSizer, LayerCache, LayerStats
 from .moe_layer import bf16_to_f32, gate_logits, moe_layer_forward, permutation, topk_route
 
 
@@ -22,13 +22,15 @@ class OracleStack:
     """Weights, per-layer cache state and counters of an L-layer MoE stack."""
 
     def __init__(self, n_layers: int, hidden: int, n_experts: int, top_k: int, intermediate: int,
-                 capacity: Sequence[int]):
+                 capacity: Sequence[int], policy: str = "priority"):
         assert len(capacity) == n_layers
         self.n_layers, self.hidden, self.n_experts = n_layers, hidden, n_experts
         self.top_k, self.intermediate = top_k, intermediate
         self.expert_bytes = 3 * hidden * intermediate * 2
-        self.caches: List[LayerCache] = [LayerCache(n_experts, int(c), self.expert_bytes)
+        self.caches: List[LayerCache] = [LayerCache(n_experts, int(c), self.expert_bytes, policy=policy)
                                          for c in capacity]
+        self.total_capacity = sum(int(c) for c in capacity)
+        self.sizer = AdaptiveSizer(n_layers, n_experts)
         self.router: List[Optional[np.ndarray]] = [None] * n_layers
         self.bias: List[Optional[np.ndarray]] = [None] * n_layers
         self.experts: List[Optional[Callable[[int], tuple]]] = [None] * n_layers
@@ -77,6 +79,14 @@ class OracleStack:
         """Cache simulation alone, from recorded routing."""
         return self.caches[layer].step(ids, gate, conf)
 
+    def adapt_capacity(self) -> List[int]:
+        """Layer-adaptive sizing (Sec. 4.3): new C_l from the statistics of the period that just
+        ended; a layer left with more residents than slots drops its lowest-valued ones at once."""
+        caps = self.sizer.refresh(self.caches, self.total_capacity)
+        for c, cap in zip(self.caches, caps):
+            c.shrink_to(cap)
+        return caps
+
     def stats(self, layer: int = -1) -> LayerStats:
         if layer >= 0:
             return self.caches[layer].stats
@@ -88,3 +98,4 @@ class OracleStack:
     def reset_cache(self) -> None:
         for c in self.caches:
             c.reset()
+        self.sizer = AdaptiveSizer(self.n_layers, self.n_experts)
