@@ -75,6 +75,9 @@ typedef struct {
   uint64_t evictions;      /* sum of #(R \ R')                                   */
   uint64_t active_experts; /* sum of #A                                          */
   uint64_t assignments;    /* sum of n_tokens * k                                */
+  uint64_t fills_reused;   /* fetched experts that were retained and activated again at the
+                              layer's next execution (Sec. 5.3 effective transfer ratio =
+                              fills_reused / misses)                               */
 } oled_stats_t;
 
 /* Create a context on the current CUDA device.
@@ -155,11 +158,30 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * bring-up kernels.  OLED_OPT_MISS_CHUNK: size of the last fill group of a step, the only one whose
  * FFN runs after all copies have landed (default 4).
  * OLED_OPT_PROFILE: 1 = bracket every kernel launch with CUDA events on the context's stream
- * (adds two event records per launch; off by default). */
+ * (adds two event records per launch; off by default).
+ * OLED_OPT_POLICY: retention value used by the cache update of every layer (OLED_POLICY_*).
+ * OLED_OPT_ADAPT_PERIOD: n > 0 makes oled_denoise_iteration() call oled_adapt_capacity() after
+ * every n-th iteration (the paper refreshes every five); 0 = fixed capacities (default). */
 #define OLED_OPT_FFN_IMPL 1
 #define OLED_OPT_MISS_CHUNK 2
 #define OLED_OPT_PROFILE 3
+#define OLED_OPT_POLICY 4
+#define OLED_OPT_ADAPT_PERIOD 5
+#define OLED_POLICY_PRIORITY 0 /* confidence- and gate-guided priority, Sec. 4.3 (default) */
+#define OLED_POLICY_LRU 1      /* comparison point: least recently used (Sec. 5.1 Naive-LRU)  */
+#define OLED_POLICY_LFU 2      /* comparison point: least frequently used (Sec. 5.3)          */
 int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value);
+
+/* Layer-adaptive cache sizing (Sec. 4.3): w_l = a_l * u_l with a_l the activation ratio and u_l
+ * the cache utilisation of layer l over the layer executions since the previous call (smoothed
+ * over calls by halving), C_l = C_total * w_l / sum_j w_j with C_total the sum of the capacities
+ * given to oled_create(), every C_l in [1, E].  A layer left with more residents than slots
+ * evicts its lowest-valued ones at once (a table update).  new_capacity: host int32[n_layers]
+ * or NULL.  Host-side only; no GPU work. */
+int oled_adapt_capacity(oled_ctx* ctx, int32_t* new_capacity);
+
+/* Current per-layer capacities (host int32[n_layers]). */
+int oled_get_capacity(oled_ctx* ctx, int32_t* capacity);
 
 /* Per-kernel timing collected while OLED_OPT_PROFILE is on.  bytes / flops are the ALGORITHMIC
  * figures of the launches (weights of each expert once, token rows in, result rows out), not
@@ -228,6 +250,13 @@ int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scor
                      uint8_t* resident_before, uint8_t* resident_after, int32_t* slot_of,
                      int32_t* n_hits, int32_t* n_misses, int32_t* n_evictions);
 void oled_policy_destroy(oled_policy* p);
+/* Retention value of the simulator's layer (OLED_POLICY_*). */
+int oled_policy_set_policy(oled_policy* p, int32_t policy);
+/* fills_reused counter of the simulator's layer. */
+int oled_policy_fills_reused(oled_policy* p, uint64_t* out);
+/* Layer-adaptive sizing over n simulated layers (one oled_policy each): as oled_adapt_capacity(). */
+int oled_policy_adapt(oled_policy** layers, int32_t n_layers, int32_t total_capacity,
+                      int32_t* new_capacity);
 
 #ifdef __cplusplus
 }

@@ -22,7 +22,9 @@ LIB_PATH = os.environ.get("OLED_LIB_PATH") or os.path.join(_HERE, "liboled.so")
 OLED_OK = 0
 ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -2, -3, -4
 ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -9
-OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE = 1, 2, 3
+OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE, OPT_POLICY, OPT_ADAPT_PERIOD = 1, 2, 3, 4, 5
+POLICY_PRIORITY, POLICY_LRU, POLICY_LFU = 0, 1, 2
+POLICY_IDS = {"priority": 0, "lru": 1, "lfu": 2}
 KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
 
 EXPORTS = [
@@ -31,6 +33,8 @@ EXPORTS = [
     "oled_reset_cache", "oled_residual_add", "oled_set_option", "oled_profile_read", "oled_launch_count",
     "oled_synchronize", "oled_destroy", "oled_strerror", "oled_last_cuda_error",
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
+    "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
+    "oled_policy_adapt",
 ]
 NOALLOC_MAX_TOKENS = 256
 
@@ -48,7 +52,7 @@ class KernelProfile(C.Structure):
 
 class StatsStruct(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("steps", "hits", "misses", "bytes_moved", "evictions",
-                                          "active_experts", "assignments")]
+                                          "active_experts", "assignments", "fills_reused")]
 
 
 @dataclass
@@ -60,6 +64,7 @@ class Stats:
     evictions: int = 0
     active_experts: int = 0
     assignments: int = 0
+    fills_reused: int = 0
 
 
 class OledError(RuntimeError):
@@ -112,6 +117,11 @@ def load() -> C.CDLL:
                                      C.POINTER(i32)]
     lib.oled_policy_destroy.argtypes = [vp]
     lib.oled_policy_destroy.restype = None
+    lib.oled_adapt_capacity.argtypes = [vp, vp]
+    lib.oled_get_capacity.argtypes = [vp, vp]
+    lib.oled_policy_set_policy.argtypes = [vp, i32]
+    lib.oled_policy_fills_reused.argtypes = [vp, u64p]
+    lib.oled_policy_adapt.argtypes = [C.POINTER(vp), i32, i32, vp]
     lib.oled_route_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
@@ -200,6 +210,16 @@ class OledContext:
         self._check(self._lib.oled_debug_logits(self._h, layer, _np_ptr(out)), "oled_debug_logits")
         return out
 
+    def adapt_capacity(self) -> list:
+        caps = np.zeros(self.shape.n_layers, np.int32)
+        self._check(self._lib.oled_adapt_capacity(self._h, _np_ptr(caps)), "oled_adapt_capacity")
+        return caps.tolist()
+
+    def get_capacity(self) -> list:
+        caps = np.zeros(self.shape.n_layers, np.int32)
+        self._check(self._lib.oled_get_capacity(self._h, _np_ptr(caps)), "oled_get_capacity")
+        return caps.tolist()
+
     def reset_cache(self) -> None:
         self._check(self._lib.oled_reset_cache(self._h), "oled_reset_cache")
 
@@ -253,7 +273,7 @@ def route_noalloc(hidden_ptr, w_router_ptr, bias_ptr, conf_ptr, n_tokens: int, h
 class PolicySim:
     """Host-only policy simulator (``oled_policy_*``): the library's C++ policy code, no GPU."""
 
-    def __init__(self, n_experts: int, capacity: int, pool_slots: int):
+    def __init__(self, n_experts: int, capacity: int, pool_slots: int, policy: str = "priority"):
         self._lib = load()
         self.n_experts = n_experts
         h = C.c_void_p()
@@ -261,6 +281,24 @@ class PolicySim:
         if rc != OLED_OK:
             raise OledError(rc, "oled_policy_create")
         self._h = h
+        rc = self._lib.oled_policy_set_policy(self._h, POLICY_IDS[policy])
+        if rc != OLED_OK:
+            raise OledError(rc, "oled_policy_set_policy")
+
+    def fills_reused(self) -> int:
+        v = C.c_uint64()
+        self._lib.oled_policy_fills_reused(self._h, C.byref(v))
+        return int(v.value)
+
+    @staticmethod
+    def adapt(sims, total_capacity: int) -> list:
+        """Layer-adaptive sizing over simulated layers (``oled_policy_adapt``)."""
+        arr = (C.c_void_p * len(sims))(*[s._h for s in sims])
+        caps = np.zeros(len(sims), np.int32)
+        rc = load().oled_policy_adapt(arr, len(sims), total_capacity, _np_ptr(caps))
+        if rc != OLED_OK:
+            raise OledError(rc, "oled_policy_adapt")
+        return caps.tolist()
 
     def step(self, counts: np.ndarray, scores: np.ndarray) -> dict:
         e = self.n_experts

@@ -80,6 +80,9 @@ struct oled_ctx {
   oled_kernel_profile prof_acc[OLED_N_KERNELS] = {};
   int ffn_impl = 0;
   int miss_chunk = 4;
+  long long total_capacity = 0;
+  int adapt_period = 0;        // iterations between automatic capacity refreshes (0 = off)
+  uint64_t iterations = 0;     // oled_denoise_iteration() calls so far
   uint64_t launches = 0;
   int last_cuda_error = 0;
   int last_layer = -1;
@@ -365,6 +368,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   ctx->n_slots = (int)std::min<long long>(total_cap + staging, 65535);
   if (total_cap + staging > 65535) return fail(OLED_ERR_INVALID_ARG);
   ctx->slots.init(ctx->n_slots);
+  ctx->total_capacity = total_cap;
   ctx->layers.resize(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) ctx->layers[l].cache.init(s.n_experts, cache_capacity[l]);
 
@@ -604,6 +608,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.stats.evictions += (uint64_t)plan.n_evictions;
   L.stats.active_experts += (uint64_t)plan.n_active;
   L.stats.assignments += (uint64_t)T * K;
+  L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
   return OLED_OK;
 }
 
@@ -644,6 +649,29 @@ int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confi
     if (rc != OLED_OK) return rc;
     x = nxt;
   }
+  ctx->iterations += 1;
+  if (ctx->adapt_period > 0 && ctx->iterations % (uint64_t)ctx->adapt_period == 0)
+    return oled_adapt_capacity(ctx, nullptr);
+  return OLED_OK;
+}
+
+int oled_adapt_capacity(oled_ctx* ctx, int32_t* new_capacity) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  std::vector<LayerCacheState*> layers;
+  for (auto& L : ctx->layers) layers.push_back(&L.cache);
+  const std::vector<int32_t> caps = adaptive_capacities(layers, ctx->total_capacity);
+  // Slots of residents evicted here may still be read by kernels already enqueued; they are
+  // reused only after the next step's gate report, which those kernels precede in stream order.
+  for (size_t l = 0; l < layers.size(); ++l)
+    ctx->layers[l].stats.evictions += (uint64_t)shrink_to(*layers[l], ctx->slots, caps[l]);
+  if (new_capacity)
+    for (size_t l = 0; l < caps.size(); ++l) new_capacity[l] = caps[l];
+  return OLED_OK;
+}
+
+int oled_get_capacity(oled_ctx* ctx, int32_t* capacity) {
+  if (!ctx || !capacity) return OLED_ERR_INVALID_ARG;
+  for (size_t l = 0; l < ctx->layers.size(); ++l) capacity[l] = ctx->layers[l].cache.capacity;
   return OLED_OK;
 }
 
@@ -681,6 +709,7 @@ int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out) {
     acc.evictions += s.evictions;
     acc.active_experts += s.active_experts;
     acc.assignments += s.assignments;
+    acc.fills_reused += s.fills_reused;
   }
   *out = acc;
   return rc;
@@ -725,6 +754,7 @@ int oled_reset_cache(oled_ctx* ctx) {
     drop_all(L.cache, ctx->slots);
     L.stats = oled_stats_t{};
   }
+  ctx->iterations = 0;
   ctx->last_layer = -1;
   return rc;
 }
@@ -748,6 +778,14 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       return OLED_OK;
     case OLED_OPT_PROFILE:
       ctx->profile = value != 0;
+      return OLED_OK;
+    case OLED_OPT_POLICY:
+      if (value < OLED_POLICY_PRIORITY || value > OLED_POLICY_LFU) return OLED_ERR_INVALID_ARG;
+      for (auto& L : ctx->layers) L.cache.policy = (int32_t)value;
+      return OLED_OK;
+    case OLED_OPT_ADAPT_PERIOD:
+      if (value < 0) return OLED_ERR_INVALID_ARG;
+      ctx->adapt_period = (int)value;
       return OLED_OK;
     case OLED_OPT_MISS_CHUNK:
       if (value < 1) return OLED_ERR_INVALID_ARG;
@@ -787,6 +825,7 @@ struct oled_policy {
   LayerCacheState cache;
   SlotPool pool;
   StepPlan plan;
+  uint64_t fills_reused = 0;
 };
 
 int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, oled_policy** out) {
@@ -814,10 +853,40 @@ int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scor
   if (n_hits) *n_hits = (int32_t)p->plan.hits.size();
   if (n_misses) *n_misses = (int32_t)p->plan.misses.size();
   if (n_evictions) *n_evictions = p->plan.n_evictions;
+  p->fills_reused += (uint64_t)p->plan.n_fills_reused;
   finish_step(p->cache, p->pool, p->plan);
   return OLED_OK;
 }
 
 void oled_policy_destroy(oled_policy* p) { delete p; }
+
+int oled_policy_set_policy(oled_policy* p, int32_t policy) {
+  if (!p || policy < OLED_POLICY_PRIORITY || policy > OLED_POLICY_LFU) return OLED_ERR_INVALID_ARG;
+  p->cache.policy = policy;
+  return OLED_OK;
+}
+
+int oled_policy_fills_reused(oled_policy* p, uint64_t* out) {
+  if (!p || !out) return OLED_ERR_INVALID_ARG;
+  *out = p->fills_reused;
+  return OLED_OK;
+}
+
+int oled_policy_adapt(oled_policy** layers, int32_t n_layers, int32_t total_capacity, int32_t* new_capacity) {
+  if (!layers || n_layers <= 0 || !new_capacity) return OLED_ERR_INVALID_ARG;
+  std::vector<LayerCacheState*> ls;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    if (!layers[l]) return OLED_ERR_INVALID_ARG;
+    ls.push_back(&layers[l]->cache);
+  }
+  if (total_capacity < n_layers || total_capacity > (int64_t)n_layers * ls[0]->n_experts)
+    return OLED_ERR_INVALID_ARG;
+  const std::vector<int32_t> caps = adaptive_capacities(ls, total_capacity);
+  for (int32_t l = 0; l < n_layers; ++l) {
+    shrink_to(*ls[l], layers[l]->pool, caps[l]);
+    new_capacity[l] = caps[l];
+  }
+  return OLED_OK;
+}
 
 }  // extern "C"

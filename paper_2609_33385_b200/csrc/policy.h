@@ -29,16 +29,39 @@ struct SlotPool {
   void release(int32_t s) { free_.push_back(s); }
 };
 
+// Retention value of a candidate: the paper's confidence- and gate-guided priority (Sec. 4.3),
+// or the recency / frequency values of the LRU and LFU comparison policies (Sec. 5.1, 5.3).
+enum Policy : int32_t { kPolicyPriority = 0, kPolicyLru = 1, kPolicyLfu = 2 };
+
 struct LayerCacheState {
   int32_t n_experts = 0;
   int32_t capacity = 0;
+  int32_t policy = kPolicyPriority;
   std::vector<int32_t> slot_of;   // expert -> slot, -1 = weights not in HBM
   std::vector<uint8_t> resident;  // R: the policy's resident set
+  uint64_t executions = 0;        // layer executions so far
+  std::vector<uint64_t> last_used;    // LRU: last execution that activated the expert
+  std::vector<uint64_t> frequency;    // LFU: executions that activated the expert
+  std::vector<uint64_t> last_value;   // value of every expert at the last update
+  std::vector<uint8_t> pending_fill;  // fetched and retained at the last execution
+  // statistics of the current sizing period and their smoothed Q16 values (Sec. 4.3)
+  uint64_t period_steps = 0, period_active = 0, period_hits = 0, period_capacity = 0;
+  int64_t a_q16 = -1, u_q16 = -1;     // -1: no period observed yet
   void init(int32_t e, int32_t c) {
     n_experts = e;
     capacity = c;
     slot_of.assign(e, -1);
     resident.assign(e, 0);
+    clear_history();
+  }
+  void clear_history() {
+    executions = 0;
+    last_used.assign(n_experts, 0);
+    frequency.assign(n_experts, 0);
+    last_value.assign(n_experts, 0);
+    pending_fill.assign(n_experts, 0);
+    period_steps = period_active = period_hits = period_capacity = 0;
+    a_q16 = u_q16 = -1;
   }
 };
 
@@ -49,6 +72,7 @@ struct StepPlan {
   std::vector<int32_t> release_after;  // activated experts that are not retained
   int32_t n_evictions = 0;             // #(R \ R')
   int32_t n_active = 0;
+  int32_t n_fills_reused = 0;          // fetched at the last execution, retained, activated again now
 };
 
 // Decide the step.  Returns false (and changes nothing) if the pool cannot hold the misses.
@@ -72,7 +96,16 @@ inline bool plan_step(LayerCacheState& L, SlotPool& pool, const int32_t* counts,
   }
   plan.n_active = (int32_t)(plan.hits.size() + plan.misses.size());
 
-  auto value = [&](int32_t e) -> uint64_t { return counts[e] > 0 ? scores[e] : 0ull; };
+  // values under the layer's policy (history is advanced on a copy: a failed plan changes nothing)
+  const uint64_t now = L.executions + 1;
+  std::vector<uint64_t> val(E);
+  for (int32_t e = 0; e < E; ++e) {
+    const bool act = counts[e] > 0;
+    if (L.policy == kPolicyPriority) val[e] = act ? scores[e] : 0ull;   // stale residents: priority 0
+    else if (L.policy == kPolicyLru) val[e] = act ? now : L.last_used[e];
+    else val[e] = L.frequency[e] + (act ? 1 : 0);
+  }
+  auto value = [&](int32_t e) -> uint64_t { return val[e]; };
   std::stable_sort(cand.begin(), cand.end(), [&](int32_t a, int32_t b) {
     const uint64_t va = value(a), vb = value(b);
     if (va != vb) return va > vb;
@@ -101,6 +134,23 @@ inline bool plan_step(LayerCacheState& L, SlotPool& pool, const int32_t* counts,
   for (int32_t e : plan.misses) L.slot_of[e] = pool.alloc();
   for (int32_t e = 0; e < E; ++e)
     if (counts[e] > 0 && !plan.after[e]) plan.release_after.push_back(e);
+  // history, effective-transfer bookkeeping (Sec. 5.3) and sizing statistics (Sec. 4.3)
+  plan.n_fills_reused = 0;
+  for (int32_t e = 0; e < E; ++e) {
+    const bool act = counts[e] > 0;
+    if (act) {
+      L.last_used[e] = now;
+      L.frequency[e] += 1;
+      if (L.pending_fill[e]) ++plan.n_fills_reused;
+    }
+    L.pending_fill[e] = (act && !plan.before[e] && plan.after[e]) ? 1 : 0;
+  }
+  L.last_value = val;
+  L.executions = now;
+  L.period_steps += 1;
+  L.period_active += (uint64_t)plan.n_active;
+  L.period_hits += plan.hits.size();
+  L.period_capacity += (uint64_t)L.capacity;
   L.resident = plan.after;
   return true;
 }
@@ -121,6 +171,85 @@ inline void drop_all(LayerCacheState& L, SlotPool& pool) {
     L.slot_of[e] = -1;
     L.resident[e] = 0;
   }
+  L.clear_history();
+}
+
+// New capacity for a layer.  If fewer slots than residents remain, the residents with the highest
+// value at the last update stay (ties to the lower id); the others are evicted at once, which is a
+// table update only.  Returns the number of evictions.
+inline int32_t shrink_to(LayerCacheState& L, SlotPool& pool, int32_t capacity) {
+  L.capacity = capacity;
+  std::vector<int32_t> res;
+  for (int32_t e = 0; e < L.n_experts; ++e)
+    if (L.resident[e]) res.push_back(e);
+  if ((int32_t)res.size() <= capacity) return 0;
+  std::stable_sort(res.begin(), res.end(), [&](int32_t a, int32_t b) {
+    if (L.last_value[a] != L.last_value[b]) return L.last_value[a] > L.last_value[b];
+    return a < b;
+  });
+  for (size_t i = (size_t)capacity; i < res.size(); ++i) {
+    const int32_t e = res[i];
+    L.resident[e] = 0;
+    L.pending_fill[e] = 0;
+    if (L.slot_of[e] >= 0) pool.release(L.slot_of[e]);
+    L.slot_of[e] = -1;
+  }
+  return (int32_t)res.size() - capacity;
+}
+
+// C_l = total * w_l / sum_j w_j in integers (Sec. 4.3 proportional allocation): floor of the quota
+// clamped to [lo, hi]; spare units go one by one to the layer furthest below its quota (ties to the
+// lower index), surplus units are taken from the layer furthest above it (ties to the higher index).
+inline std::vector<int32_t> apportion(std::vector<uint64_t> w, int64_t total, int32_t lo, int32_t hi) {
+  const size_t n = w.size();
+  unsigned __int128 sw = 0;
+  for (uint64_t x : w) sw += x;
+  if (sw == 0) {
+    w.assign(n, 1);
+    sw = n;
+  }
+  std::vector<int32_t> c(n);
+  int64_t sum = 0;
+  for (size_t l = 0; l < n; ++l) {
+    const int64_t q = (int64_t)(((unsigned __int128)total * w[l]) / sw);
+    c[l] = (int32_t)std::min<int64_t>(hi, std::max<int64_t>(lo, q));
+    sum += c[l];
+  }
+  auto deficit = [&](size_t l) -> __int128 {
+    return (__int128)((unsigned __int128)total * w[l]) - (__int128)c[l] * (__int128)sw;
+  };
+  while (sum < total) {
+    long best = -1;
+    for (size_t l = 0; l < n; ++l)
+      if (c[l] < hi && (best < 0 || deficit(l) > deficit((size_t)best))) best = (long)l;
+    c[(size_t)best] += 1;
+    ++sum;
+  }
+  while (sum > total) {
+    long best = -1;
+    for (size_t l = 0; l < n; ++l)
+      if (c[l] > lo && (best < 0 || deficit(l) <= deficit((size_t)best))) best = (long)l;
+    c[(size_t)best] -= 1;
+    --sum;
+  }
+  return c;
+}
+
+// Layer-adaptive sizing (Sec. 4.3): w_l = a_l * u_l from the statistics of the period that just
+// ended, smoothed over periods by s <- (s + new) / 2 in Q16; returns the new capacities.
+inline std::vector<int32_t> adaptive_capacities(std::vector<LayerCacheState*>& layers, int64_t total) {
+  std::vector<uint64_t> w;
+  for (LayerCacheState* L : layers) {
+    if (L->period_steps > 0) {
+      const int64_t a_new = (int64_t)(L->period_active * 65536ull / (L->period_steps * (uint64_t)L->n_experts));
+      const int64_t u_new = (int64_t)(L->period_hits * 65536ull / std::max<uint64_t>(1, L->period_capacity));
+      L->a_q16 = L->a_q16 < 0 ? a_new : (L->a_q16 + a_new) / 2;
+      L->u_q16 = L->u_q16 < 0 ? u_new : (L->u_q16 + u_new) / 2;
+      L->period_steps = L->period_active = L->period_hits = L->period_capacity = 0;
+    }
+    w.push_back((uint64_t)std::max<int64_t>(0, L->a_q16) * (uint64_t)std::max<int64_t>(0, L->u_q16));
+  }
+  return apportion(w, total, 1, layers.empty() ? 1 : layers[0]->n_experts);
 }
 
 }  // namespace oled

@@ -16,7 +16,8 @@ import numpy as np
 import torch
 
 from . import synth
-from .binding import OPT_FFN_IMPL, OPT_MISS_CHUNK, OledContext
+from .binding import (OPT_ADAPT_PERIOD, OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_POLICY, POLICY_IDS,
+                      OledContext)
 
 
 def bits_to_dev(bits: np.ndarray, device) -> torch.Tensor:
@@ -35,7 +36,8 @@ class StackRunner:
                  device: str = "cuda:0", distinct_layers: Optional[int] = None,
                  gen_threads: Optional[int] = None, ffn_impl: Optional[int] = None,
                  miss_chunk: Optional[int] = None, max_tokens: Optional[int] = None,
-                 staging_slots: int = 0, share_store_of: Optional["StackRunner"] = None):
+                 staging_slots: int = 0, share_store_of: Optional["StackRunner"] = None,
+                 policy: Optional[str] = None, adapt_period: Optional[int] = None):
         self.w = w
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -50,6 +52,10 @@ class StackRunner:
             self.ctx.set_option(OPT_FFN_IMPL, ffn_impl)
         if miss_chunk is not None:
             self.ctx.set_option(OPT_MISS_CHUNK, miss_chunk)
+        if policy is not None:
+            self.ctx.set_option(OPT_POLICY, POLICY_IDS[policy])
+        if adapt_period is not None:
+            self.ctx.set_option(OPT_ADAPT_PERIOD, adapt_period)
         threads = gen_threads or min(32, len(os.sched_getaffinity(0)))
         n_distinct = w.n_layers if distinct_layers is None else max(1, min(distinct_layers, w.n_layers))
         self.n_distinct = n_distinct

@@ -25,9 +25,9 @@ def _runner(w, **kw):
     return StackRunner(w, **kw)
 
 
-def _oracle_for(run, caps):
+def _oracle_for(run, caps, policy="priority"):
     w = run.w
-    st = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, caps)
+    st = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, caps, policy=policy)
     for l in range(w.n_layers):
         st.register_router(l, run.router_bits[l], run.bias[l])
         st.register_experts(l, run.layer_blobs(l))
@@ -64,8 +64,10 @@ def _check_step(run, layer, n_tokens, out_t, ref, check_out=True):
 def _check_stats(run, ora):
     for l in range(run.w.n_layers):
         a, b = run.ctx.stats(l), ora.stats(l)
-        assert (a.steps, a.hits, a.misses, a.bytes_moved, a.evictions, a.active_experts, a.assignments) == \
-               (b.steps, b.hits, b.misses, b.bytes_moved, b.evictions, b.active_experts, b.assignments)
+        assert (a.steps, a.hits, a.misses, a.bytes_moved, a.evictions, a.active_experts, a.assignments,
+                a.fills_reused) == \
+               (b.steps, b.hits, b.misses, b.bytes_moved, b.evictions, b.active_experts, b.assignments,
+                b.fills_reused)
     a, b = run.ctx.stats(-1), ora.stats(-1)
     assert (a.hits, a.misses, a.bytes_moved) == (b.hits, b.misses, b.bytes_moved)
 
@@ -281,5 +283,57 @@ def test_reset_cache_returns_to_cold_state():
         assert run.ctx.stats().steps == 0
         run.step(0, x, c, out)
         assert run.ctx.stats().misses == m1
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("policy", ["lru", "lfu"])
+def test_comparison_policies_match_oracle(policy):
+    """LRU / LFU retention through the real step: resident sets, counters and outputs."""
+    w = synth.tiny(n_layers=2, blocks=2, iters=4, n_experts=8, top_k=2)
+    run = _runner(w, capacity=[3, 2], policy=policy)
+    try:
+        _run_stack(run, _oracle_for(run, [3, 2], policy=policy))
+    finally:
+        run.close()
+
+
+def test_layer_adaptive_sizing_through_the_iteration_entry_point():
+    """oled_denoise_iteration with a refresh period of 2: capacities, resident sets and counters
+    follow the oracle's layer-adaptive sizing; outputs stay within tolerance."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=3, blocks=3, iters=3, n_experts=8, top_k=2)
+    caps = [3, 3, 3]
+    run = _runner(w, capacity=caps, adapt_period=2, staging_slots=8)
+    ora = _oracle_for(run, caps)
+    try:
+        dev = run.device
+        y = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=dev)
+        out = torch.empty_like(y)
+        bufs = [torch.empty_like(y), torch.empty_like(y)]
+        shadow = _runner(w, capacity=caps, staging_slots=8)       # same inputs, step by step, for replay
+        changed = False
+        for it, (_, _, h_bits, conf) in enumerate(synth.denoise_inputs(w)):
+            x, c = bits_to_dev(h_bits, dev), torch.from_numpy(conf).to(dev)
+            run.ctx.denoise_iteration(x.data_ptr(), c.data_ptr(), w.tokens, y.data_ptr())
+            # replay the same iteration layer by layer on the shadow context to feed the oracle
+            xs = x
+            for l in range(w.n_layers):
+                shadow.step(l, xs, c, out)
+                ora.denoise_step(l, dev_to_bits(xs), conf)
+                nxt = bufs[l & 1]
+                shadow.ctx.residual_add(xs.data_ptr(), out.data_ptr(), nxt.data_ptr(), xs.numel())
+                xs = nxt
+            assert np.array_equal(dev_to_bits(y), dev_to_bits(xs))   # capacity never changes outputs
+            if (it + 1) % 2 == 0:
+                want = ora.adapt_capacity()
+                assert run.ctx.get_capacity() == want and sum(want) == sum(caps)
+                changed = changed or want != caps
+            for l in range(w.n_layers):
+                a, b = run.ctx.stats(l), ora.stats(l)
+                assert (a.hits, a.misses, a.evictions, a.fills_reused) == \
+                       (b.hits, b.misses, b.evictions, b.fills_reused), (it, l)
+        assert changed, "the allocation never moved: the test exercises nothing"
+        shadow.close()
     finally:
         run.close()

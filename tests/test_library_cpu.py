@@ -81,3 +81,46 @@ def test_host_policy_pool_exhaustion_is_an_error_not_a_crash(binding):
     counts[[3, 4, 5]] = 1                                   # the failed step changed nothing
     got = sim.step(counts, np.arange(8, dtype=np.uint64) + 1)
     assert got["misses"] == 3
+
+
+@pytest.mark.parametrize("policy", ["priority", "lru", "lfu"])
+def test_host_policy_variants_match_oracle(binding, policy):
+    rng = np.random.default_rng(11)
+    e, cap = 24, 7
+    sim = binding.PolicySim(e, cap, e, policy=policy)
+    ref = cp.LayerCache(e, cap, 100, policy=policy)
+    for step in range(80):
+        t, k = int(rng.integers(1, 8)), 2
+        ids = np.stack([rng.permutation(e)[:k] for _ in range(t)]).astype(np.int32)
+        gate = rng.dirichlet(np.ones(k), size=t).astype(np.float32)
+        conf = rng.choice([0.0, 0.3, 1.0], size=t).astype(np.float32)
+        r = ref.step(ids, gate, conf)
+        counts = np.bincount(ids.reshape(-1), minlength=e).astype(np.int32)
+        got = sim.step(counts, np.array(r["scores"], dtype=np.uint64))
+        assert set(np.flatnonzero(got["resident_after"])) == r["resident_after"]
+        assert got["misses"] == len(r["misses"])
+    assert sim.fills_reused() == ref.stats.fills_reused
+
+
+def test_host_adaptive_sizing_matches_oracle(binding):
+    from oracle import OracleStack
+    rng = np.random.default_rng(12)
+    n_layers, e, caps = 5, 16, [4, 4, 4, 4, 4]
+    sims = [binding.PolicySim(e, c, e) for c in caps]
+    ora = OracleStack(n_layers, 256, e, 2, 128, caps)
+    width = [2, 4, 8, 12, 16]                       # layer l draws its experts from the first width[l]
+    for it in range(23):
+        for l in range(n_layers):
+            t = 6
+            ids = np.stack([rng.permutation(width[l])[:2] for _ in range(t)]).astype(np.int32)
+            gate = rng.dirichlet(np.ones(2), size=t).astype(np.float32)
+            conf = rng.uniform(0, 1, size=t).astype(np.float32)
+            r = ora.policy_step(l, ids, gate, conf)
+            counts = np.bincount(ids.reshape(-1), minlength=e).astype(np.int32)
+            got = sims[l].step(counts, np.array(r["scores"], dtype=np.uint64))
+            assert set(np.flatnonzero(got["resident_after"])) == r["resident_after"], (it, l)
+        if it % 5 == 4:                              # the paper's refresh period
+            want = ora.adapt_capacity()
+            assert binding.PolicySim.adapt(sims, sum(caps)) == want
+            assert sum(want) == sum(caps)
+    assert want[0] < want[-1]                        # slots moved to the layers with the larger working sets
