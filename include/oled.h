@@ -78,6 +78,8 @@ typedef struct {
   uint64_t fills_reused;   /* fetched experts that were retained and activated again at the
                               layer's next execution (Sec. 5.3 effective transfer ratio =
                               fills_reused / misses)                               */
+  uint64_t ideal_hits;     /* sum of min(C_l, #A): hits of the clairvoyant cache bound of
+                              Sec. 5.1 under the same capacity                     */
 } oled_stats_t;
 
 /* Create a context on the current CUDA device.

@@ -112,10 +112,11 @@ class LayerStats:
     active_experts: int = 0
     assignments: int = 0
     fills_reused: int = 0      # fetched, retained and activated again at the next execution
+    ideal_hits: int = 0        # hits of the clairvoyant bound under the same capacity
 
     def add(self, o: "LayerStats") -> None:
         for f in ("steps", "hits", "misses", "bytes_moved", "evictions", "active_experts",
-                  "assignments", "fills_reused"):
+                  "assignments", "fills_reused", "ideal_hits"):
             setattr(self, f, getattr(self, f) + getattr(o, f))
 
 
@@ -163,6 +164,7 @@ class LayerCache:
             after = retain_by_value(before, misses, value, self.capacity)
         self.last_value = value
         self.stats.fills_reused += len(self.pending_fills & activated)
+        self.stats.ideal_hits += ideal_hits(len(activated), self.capacity)
         self.pending_fills = misses & after
         self.period_steps += 1
         self.period_active += len(activated)

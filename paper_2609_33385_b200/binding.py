@@ -52,7 +52,7 @@ class KernelProfile(C.Structure):
 
 class StatsStruct(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("steps", "hits", "misses", "bytes_moved", "evictions",
-                                          "active_experts", "assignments", "fills_reused")]
+                                          "active_experts", "assignments", "fills_reused", "ideal_hits")]
 
 
 @dataclass
@@ -65,6 +65,7 @@ class Stats:
     active_experts: int = 0
     assignments: int = 0
     fills_reused: int = 0
+    ideal_hits: int = 0
 
 
 class OledError(RuntimeError):

@@ -609,6 +609,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.stats.active_experts += (uint64_t)plan.n_active;
   L.stats.assignments += (uint64_t)T * K;
   L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
+  L.stats.ideal_hits += (uint64_t)std::min<int64_t>(plan.n_active, plan.capacity_used);
   return OLED_OK;
 }
 
@@ -710,6 +711,7 @@ int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out) {
     acc.active_experts += s.active_experts;
     acc.assignments += s.assignments;
     acc.fills_reused += s.fills_reused;
+    acc.ideal_hits += s.ideal_hits;
   }
   *out = acc;
   return rc;

@@ -73,6 +73,7 @@ struct StepPlan {
   int32_t n_evictions = 0;             // #(R \ R')
   int32_t n_active = 0;
   int32_t n_fills_reused = 0;          // fetched at the last execution, retained, activated again now
+  int32_t capacity_used = 0;           // the layer's capacity at this execution
 };
 
 // Decide the step.  Returns false (and changes nothing) if the pool cannot hold the misses.
@@ -95,6 +96,7 @@ inline bool plan_step(LayerCacheState& L, SlotPool& pool, const int32_t* counts,
     if (act || L.resident[e]) cand.push_back(e);
   }
   plan.n_active = (int32_t)(plan.hits.size() + plan.misses.size());
+  plan.capacity_used = L.capacity;
 
   // values under the layer's policy (history is advanced on a copy: a failed plan changes nothing)
   const uint64_t now = L.executions + 1;

@@ -47,7 +47,7 @@ class StackRunner:
         self.stream = torch.cuda.current_stream(self.device)
         self.ctx = OledContext(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate,
                                self.max_tokens, caps, self.stream.cuda_stream,
-                               has_router_bias=w.zipf_bias > 0.0, staging_slots=staging_slots)
+                               has_router_bias=w.has_bias, staging_slots=staging_slots)
         if ffn_impl is not None:
             self.ctx.set_option(OPT_FFN_IMPL, ffn_impl)
         if miss_chunk is not None:

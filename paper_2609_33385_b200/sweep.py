@@ -35,8 +35,51 @@ def run_point(run: StackRunner, xs, cs, warmup: int, steps: int):
     s1 = run.ctx.stats()
     ms = a.elapsed_time(b) / steps
     d = {k: getattr(s1, k) - getattr(s0, k) for k in ("steps", "hits", "misses", "bytes_moved",
-                                                     "active_experts")}
+                                                     "active_experts", "fills_reused", "ideal_hits",
+                                                     "evictions")}
     return ms, d
+
+
+def policy_mode(args, device):
+    """Priority vs LRU vs LFU (uniform allocation) and Priority with layer-adaptive sizing, on a
+    workload whose confidences carry routing-stability information and whose layers differ in
+    activation footprint (the regime Sec. 4.3 describes)."""
+    rows = []
+    base = None
+    w0 = synth.config(3, n_layers=args.layers, rho=0.9, shared_beta=0.9, conf_coupling=0.6,
+                      layer_zipf=3.0)
+    n_it = args.warmup + args.steps
+    w0 = w0.replace(blocks=-(-n_it // w0.iters))
+    xs, cs = [], []
+    for _, _, h_bits, conf in synth.denoise_inputs(w0):
+        xs.append(bits_to_dev(h_bits, device))
+        cs.append(torch.from_numpy(conf).to(device))
+    for res in (0.1, 0.2, 0.4, 0.6):
+        for policy, period in (("priority", 0), ("lru", 0), ("lfu", 0), ("priority", 5)):
+            w = w0.replace(residency=res)
+            run = StackRunner(w, device=device, share_store_of=base, distinct_layers=args.distinct_layers,
+                              policy=policy, adapt_period=period, staging_slots=w.n_experts)
+            if base is None:
+                base = run
+            ms, d = run_point(run, xs, cs, args.warmup, args.steps)
+            slots = d["steps"] * w.capacity
+            rows.append(dict(residency=res, capacity=w.capacity, policy=policy, adaptive=bool(period),
+                             ms_per_step=ms, hits=d["hits"], misses=d["misses"],
+                             ideal_hits=d["ideal_hits"], utilisation=d["hits"] / max(1, slots),
+                             ideal_utilisation=d["ideal_hits"] / max(1, slots),
+                             transfer_ratio=d["fills_reused"] / max(1, d["misses"]),
+                             active=d["active_experts"] / max(1, d["steps"]),
+                             final_capacity=run.ctx.get_capacity()))
+            if run is not base:
+                run.close()
+    lines = ["| residency | C/layer | policy | sizing | hits | misses | ideal hits | utilisation | ideal util. | "
+             "eff. transfer | active/layer | ms/step |", "|" + "---|" * 12]
+    for r in rows:
+        lines.append(f"| {r['residency']:.0%} | {r['capacity']} | {r['policy']} | "
+                     f"{'adaptive' if r['adaptive'] else 'uniform'} | {r['hits']} | {r['misses']} | "
+                     f"{r['ideal_hits']} | {r['utilisation']:.3f} | {r['ideal_utilisation']:.3f} | "
+                     f"{r['transfer_ratio']:.3f} | {r['active']:.1f} | {r['ms_per_step']:.2f} |")
+    return rows, "\n".join(lines)
 
 
 def main():
@@ -47,9 +90,18 @@ def main():
     ap.add_argument("--variant", default="A", choices=["A", "B"])
     ap.add_argument("--h2d-gbs", type=float, default=54.5, help="measured host-link bandwidth")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--mode", default="capacity", choices=["capacity", "policy"])
+    ap.add_argument("--distinct-layers", type=int, default=None)
     args = ap.parse_args()
     build.build()
     device = "cuda:0"
+    if args.mode == "policy":
+        rows, text = policy_mode(args, device)
+        print(text)
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text + "\n\n" + json.dumps(rows) + "\n")
+        return 0
     rows = []
     base_store = None
     for rho in (0.5, 0.9, 0.98):

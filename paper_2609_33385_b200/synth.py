@@ -70,7 +70,13 @@ class Workload:
     zipf_bias: float = 0.0     # >0: per-expert bias b_e = -zipf_bias*ln(1+pi(e))
     finalize_threshold: float = 0.9
     shared_beta: float = 0.0   # >0: "dLLM-shaped" variant, tokens share a block direction
+    conf_coupling: float = 0.0 # >0: a confident token's hidden state changes less (Sec. 4.3)
+    layer_zipf: float = 0.0    # >0: per-layer gate bias of growing strength (layers differ in footprint)
     seed: int = 0
+
+    @property
+    def has_bias(self) -> bool:
+        return self.zipf_bias > 0.0 or self.layer_zipf > 0.0
 
     @property
     def tokens(self) -> int:
@@ -142,9 +148,10 @@ def router_weights(w: Workload, layer: int) -> Tuple[np.ndarray, Optional[np.nda
     g = _rng(w, _STREAM_ROUTER, layer)
     wr = g.standard_normal((w.n_experts, w.hidden), dtype=np.float32) * np.float32(w.router_std)
     bias = None
-    if w.zipf_bias > 0.0:
+    if w.has_bias:
+        strength = w.zipf_bias + w.layer_zipf * (layer / max(1, w.n_layers - 1))
         perm = _rng(w, _STREAM_BIAS, layer).permutation(w.n_experts)
-        bias = (-w.zipf_bias * np.log1p(perm.astype(np.float64))).astype(np.float32)
+        bias = (-strength * np.log1p(perm.astype(np.float64))).astype(np.float32)
     return f32_to_bf16_bits(wr), bias
 
 
@@ -212,11 +219,17 @@ def denoise_inputs(w: Workload) -> Iterator[Tuple[int, int, np.ndarray, np.ndarr
         gc = _rng(w, _STREAM_CONF, b)
         h = _noise(w, gh)
         final = np.zeros(t, dtype=bool)
+        c = None
         for i in range(w.iters):
             if i > 0:
                 eps = _noise(w, gh)
                 if w.literal_mix:
                     nh = np.float32(w.rho) * h + np.float32(1.0 - w.rho) * eps
+                elif w.conf_coupling > 0.0:
+                    # per-token correlation: the previous iteration's confidence decides how far a
+                    # token moves (high confidence => stable hidden state => stable routing)
+                    rt = np.clip(w.rho + w.conf_coupling * (c.astype(np.float64) - 0.5), 0.0, 0.999)
+                    nh = (rt[:, None] * h + np.sqrt(1.0 - rt * rt)[:, None] * eps).astype(np.float32)
                 else:
                     nh = np.float32(w.rho) * h + np.float32(math.sqrt(1.0 - w.rho * w.rho)) * eps
                 h = np.where(final[:, None], h, nh).astype(np.float32)

@@ -65,9 +65,9 @@ def _check_stats(run, ora):
     for l in range(run.w.n_layers):
         a, b = run.ctx.stats(l), ora.stats(l)
         assert (a.steps, a.hits, a.misses, a.bytes_moved, a.evictions, a.active_experts, a.assignments,
-                a.fills_reused) == \
+                a.fills_reused, a.ideal_hits) == \
                (b.steps, b.hits, b.misses, b.bytes_moved, b.evictions, b.active_experts, b.assignments,
-                b.fills_reused)
+                b.fills_reused, b.ideal_hits)
     a, b = run.ctx.stats(-1), ora.stats(-1)
     assert (a.hits, a.misses, a.bytes_moved) == (b.hits, b.misses, b.bytes_moved)
 
