@@ -15,9 +15,9 @@
 // one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
 // which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
 //
-// Warp roles (320 threads): warps 0-7 epilogue (TMEM lane quarter = warp id mod 4, the two warps
-// of a quarter alternate 16-column chunks), warp 8 lane 0 TMA producer, warp 9 lane 0 MMA issuer
-// (warp 9 also owns the TMEM allocation).  Every mbarrier
+// Warp roles (576 threads): warps 0-15 epilogue (TMEM lane quarter = warp id mod 4, the warps of
+// a quarter interleave 16-column chunks; only as many as the token tile has chunks are active),
+// warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation).  Every mbarrier
 // wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
 // copies time to land, frees its TMEM and returns.
 #include <cuda.h>
@@ -32,9 +32,9 @@ namespace oled {
 namespace {
 
 #ifndef OLED_EPI_WARPS
-#define OLED_EPI_WARPS 8
+#define OLED_EPI_WARPS 16
 #endif
-constexpr int kEpiWarps = OLED_EPI_WARPS;                 // two warps per TMEM lane quarter, alternating 16-column chunks
+constexpr int kEpiWarps = OLED_EPI_WARPS;  // up to four warps per TMEM lane quarter, interleaving 16-column chunks
 constexpr int kProducerWarp = kEpiWarps;
 constexpr int kMmaWarp = kEpiWarps + 1;
 constexpr int kThreads = (kEpiWarps + 2) * 32;
@@ -206,6 +206,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
   const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
+  // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
+  // plain store epilogue of KIND 2 runs best with 8
+  const int epi_warps = min(KIND == 1 ? kEpiWarps : 8, 4 * (n_box / 16));
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
 
@@ -218,7 +221,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[a]), (n_box > 16 ? kEpiWarps : 4) * 32);
+      mbar_init(smem_u32(&ctl->tmem_empty[a]), (uint32_t)epi_warps * 32u);
     }
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -332,9 +335,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
-  } else if (warp < (n_box > 16 ? kEpiWarps : 4)) {
+  } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
-    // (a 16-column accumulator is one chunk: the second warp of each quarter has nothing to do)
+    // (only as many warps per quarter as the token tile has 16-column chunks)
     int g = 0, local = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
       Item it;
@@ -348,11 +351,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) break;
       tc_fence_after();
-      const int quarter = warp & 3, half = warp >> 2;
+      const int quarter = warp & 3, half = warp >> 2;  // `half`: which 16-column chunks this warp takes
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * acc_cols);
       const int n_mma = max(16, (it.valid + 15) & ~15);
       const int col = it.m0 + quarter * 32 + lane;  // output feature owned by this thread
-      for (int c = half * 16; c < n_mma; c += 32) {
+      for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
         if (KIND == 1) {

@@ -82,6 +82,43 @@ def policy_mode(args, device):
     return rows, "\n".join(lines)
 
 
+def shape_mode(args, device):
+    """Block length x capacity and batch-size sweeps (the paper's sensitivity studies, Sec. 5.4):
+    tokens per step from 1 to 1024 on the same stack, crossing from the few-tokens-per-expert
+    regime (weight streaming) towards the many-token regime (tensor bound)."""
+    rows = []
+    base = None
+    points = [(1, bl) for bl in (1, 4, 16, 32, 64)] + [(b, 32) for b in (2, 4, 8, 16, 32)]
+    for batch, block_len in points:
+        for res in (1.0, 0.4):
+            w = synth.config(3, n_layers=args.layers, batch=batch, block_len=block_len, residency=res,
+                             shared_beta=0.9 if args.variant == "B" else 0.0)
+            n_it = args.warmup + args.steps
+            w = w.replace(blocks=-(-n_it // w.iters))
+            xs, cs = [], []
+            for _, _, h_bits, conf in synth.denoise_inputs(w):
+                xs.append(bits_to_dev(h_bits, device))
+                cs.append(torch.from_numpy(conf).to(device))
+            run = StackRunner(w, device=device, share_store_of=base, distinct_layers=args.distinct_layers)
+            if base is None:
+                base = run
+            ms, d = run_point(run, xs, cs, args.warmup, args.steps)
+            rows.append(dict(batch=batch, block_len=block_len, tokens=w.tokens, residency=res,
+                             capacity=w.capacity, ms_per_step=ms, tokens_per_s=w.tokens / (ms * 1e-3),
+                             tpot_ms=ms * w.iters / w.tokens, misses=d["misses"], hits=d["hits"],
+                             active=d["active_experts"] / max(1, d["steps"]),
+                             h2d_gb_per_step=d["bytes_moved"] / args.steps / 1e9))
+            if run is not base:
+                run.close()
+    lines = ["| batch | block | tokens/step | residency | active/layer | misses | H2D GB/step | ms/step | "
+             "tokens/s | TPOT ms |", "|" + "---|" * 10]
+    for r in rows:
+        lines.append(f"| {r['batch']} | {r['block_len']} | {r['tokens']} | {r['residency']:.0%} | "
+                     f"{r['active']:.1f} | {r['misses']} | {r['h2d_gb_per_step']:.3f} | {r['ms_per_step']:.3f} | "
+                     f"{r['tokens_per_s']:.0f} | {r['tpot_ms']:.4f} |")
+    return rows, "\n".join(lines)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--layers", type=int, default=16)
@@ -90,13 +127,13 @@ def main():
     ap.add_argument("--variant", default="A", choices=["A", "B"])
     ap.add_argument("--h2d-gbs", type=float, default=54.5, help="measured host-link bandwidth")
     ap.add_argument("--out", default=None)
-    ap.add_argument("--mode", default="capacity", choices=["capacity", "policy"])
+    ap.add_argument("--mode", default="capacity", choices=["capacity", "policy", "shape"])
     ap.add_argument("--distinct-layers", type=int, default=None)
     args = ap.parse_args()
     build.build()
     device = "cuda:0"
-    if args.mode == "policy":
-        rows, text = policy_mode(args, device)
+    if args.mode in ("policy", "shape"):
+        rows, text = (policy_mode if args.mode == "policy" else shape_mode)(args, device)
         print(text)
         if args.out:
             with open(args.out, "w") as f:
