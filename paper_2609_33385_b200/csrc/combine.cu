@@ -10,6 +10,7 @@
 namespace oled {
 namespace {
 
+template <bool Y_BF16>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
@@ -30,7 +31,15 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
   for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j = 0; j < K; ++j) {
-      const float4 v = *reinterpret_cast<const float4*>(y + (size_t)s_r[j] * H + h);
+      float4 v;
+      if (Y_BF16) {
+        const uint2 p = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(y) +
+                                                        (size_t)s_r[j] * H + h);
+        v = make_float4(__uint_as_float(p.x << 16), __uint_as_float(p.x & 0xffff0000u),
+                        __uint_as_float(p.y << 16), __uint_as_float(p.y & 0xffff0000u));
+      } else {
+        v = *reinterpret_cast<const float4*>(y + (size_t)s_r[j] * H + h);
+      }
       const float g = s_g[j];
       acc.x = fmaf(g, v.x, acc.x);
       acc.y = fmaf(g, v.y, acc.y);
@@ -74,11 +83,15 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 
 }  // namespace
 
-void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
+void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
                     uint32_t* zero_words, int n_zero_words) {
-  launch_pdl(combine_kernel, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
-             n_zero_words);
+  if (y_bf16)
+    launch_pdl(combine_kernel<true>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+               n_zero_words);
+  else
+    launch_pdl(combine_kernel<false>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+               n_zero_words);
 }
 
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {

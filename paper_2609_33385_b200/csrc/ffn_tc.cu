@@ -191,7 +191,8 @@ template <int KIND, bool DUAL>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
-              void* __restrict__ out_ptr, int H, int I, int n_stages, uint32_t* __restrict__ status) {
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
+              uint32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
@@ -208,7 +209,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
-  const int epi_warps = min(KIND == 1 ? kEpiWarps : 8, 4 * (n_box / 16));
+  const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
 
@@ -375,22 +376,26 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           }
         } else {
           float* y = reinterpret_cast<float*>(out_ptr);
-          if (dual) {
-            uint32_t rb[16];
-            tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
-            tmem_ld_wait();
+          uint16_t* yb = reinterpret_cast<uint16_t*>(out_ptr);  // many-token steps keep y in bf16
+          uint32_t rb[16];
+          if (dual) tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
+          tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (c + j < it.valid) {
-                y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
-                y[(size_t)(it.row0 + c + j) * H + col + kBlockM] = __uint_as_float(rb[j]);
+          for (int j = 0; j < 16; ++j)
+            if (c + j < it.valid) {
+              const size_t o = (size_t)(it.row0 + c + j) * H + col;
+              if (out_bf16) {
+                const __nv_bfloat16 b0 = __float2bfloat16_rn(__uint_as_float(ra[j]));
+                yb[o] = *reinterpret_cast<const uint16_t*>(&b0);
+                if (dual) {
+                  const __nv_bfloat16 b1 = __float2bfloat16_rn(__uint_as_float(rb[j]));
+                  yb[o + kBlockM] = *reinterpret_cast<const uint16_t*>(&b1);
+                }
+              } else {
+                y[o] = __uint_as_float(ra[j]);
+                if (dual) y[o + kBlockM] = __uint_as_float(rb[j]);
               }
-          } else {
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (c + j < it.valid) y[(size_t)(it.row0 + c + j) * H + col] = __uint_as_float(ra[j]);
-          }
+            }
         }
       }
       tc_fence_before();
@@ -514,8 +519,8 @@ static int box_index(int max_count, int cap) {
 }
 
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
-                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
-                  uint32_t* status) {
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
+                  int n_sms, uint32_t* status) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   // N <= 128 keeps the accumulators double-buffered in TMEM; more tokens per expert than that
@@ -533,17 +538,18 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     const int stages = stages_for(1, grp.n_box);
     launch_pdl(ffn_tc_kernel<1, true>, dim3(grid_for(grp.n_box, I / kBlockM)), dim3(kThreads),
                smem_for(1, grp.n_box, stages), st, maps.w13, maps.xp[i1], grp, offsets, (void*)hbuf, H, I, stages,
-               status);
+               0, status);
   } else {
     grp.n_box = 16 << i2;
     const int stages = stages_for(2, grp.n_box);
     if (grp.n_box == 256)
       launch_pdl(ffn_tc_kernel<2, true>, dim3(grid_for(256, H / (2 * kBlockM))), dim3(kThreads),
-                 smem_for(2, 256, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, status);
+                 smem_for(2, 256, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, y_bf16,
+                 status);
     else
       launch_pdl(ffn_tc_kernel<2, false>, dim3(grid_for(grp.n_box, H / kBlockM)), dim3(kThreads),
                  smem_for(2, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages,
-                 status);
+                 y_bf16, status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

@@ -82,7 +82,8 @@ void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int 
 // x_next != nullptr also x_next[t,:] = bf16(x[t,:] + out[t,:]) (the residual between layers).
 // zero_words != nullptr: CTA 0 also clears n_zero_words 32-bit words there (the step's control
 // block, ready for the next step's atomics).
-void launch_combine(cudaStream_t st, const float* y, const float* gate, const int32_t* pos, int T,
+// y_bf16 != 0: y holds bf16 rows (many-token steps) instead of fp32.
+void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
                     uint32_t* zero_words, int n_zero_words);
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n);
@@ -104,7 +105,7 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
-                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int H, int I, int n_sms,
-                  uint32_t* status);
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
+                  int I, int n_sms, uint32_t* status);
 
 }  // namespace oled

@@ -45,91 +45,17 @@ __device__ __forceinline__ float exp_spec(float x) {
 
 constexpr int kMaxEPerLane = OLED_MAX_EXPERTS / 32;
 
-// TT tokens per CTA, WARPS warps; each warp owns kEPerWarp experts per pass and all TT tokens.  Small
-// blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
-// chunks of loads in flight; the chain order of every logit is the same in all variants.
-template <int TT, int WARPS, int UNROLL, int kEPerWarp>
-__global__ void __launch_bounds__(WARPS * 32)
-route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
-             const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
-             int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
-             float* __restrict__ gate, int32_t* __restrict__ counts,
-             unsigned long long* __restrict__ scores, RouteReport rep) {
-  extern __shared__ float s_logits[];  // [TT][E]
-  __shared__ int s_last;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t0 = blockIdx.x * TT;
-  griddep_launch_dependents();
-  griddep_wait();
-
-  constexpr int kRouteWarps = WARPS;
-  for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
-    float acc[TT][kEPerWarp];
-#pragma unroll
-    for (int a = 0; a < TT; ++a)
-#pragma unroll
-      for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = 0.0f;
-
-#pragma unroll UNROLL
-    for (int hc = 0; hc < H; hc += 256) {
-      const int h = hc + lane * 8;
-      uint4 xv[TT], wv[kEPerWarp];
-#pragma unroll
-      for (int a = 0; a < TT; ++a) {
-        const int t = min(t0 + a, T - 1);
-        xv[a] = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
-      }
-#pragma unroll
-      for (int b = 0; b < kEPerWarp; ++b) {
-        const int e = min(eb + b, E - 1);
-        wv[b] = *reinterpret_cast<const uint4*>(wr + (size_t)e * H + h);
-      }
-      // elements j = 0..7 in ascending h: word0.lo, word0.hi, word1.lo, ...
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float wf[kEPerWarp];
-#pragma unroll
-        for (int b = 0; b < kEPerWarp; ++b) {
-          const uint32_t w32 = (j >> 1) == 0 ? wv[b].x : (j >> 1) == 1 ? wv[b].y
-                               : (j >> 1) == 2 ? wv[b].z : wv[b].w;
-          wf[b] = (j & 1) ? bf16_hi(w32) : bf16_lo(w32);
-        }
-#pragma unroll
-        for (int a = 0; a < TT; ++a) {
-          const uint32_t x32 = (j >> 1) == 0 ? xv[a].x : (j >> 1) == 1 ? xv[a].y
-                               : (j >> 1) == 2 ? xv[a].z : xv[a].w;
-          const float xf = (j & 1) ? bf16_hi(x32) : bf16_lo(x32);
-#pragma unroll
-          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf, wf[b], acc[a][b]);
-        }
-      }
-    }
-#pragma unroll
-    for (int a = 0; a < TT; ++a)
-#pragma unroll
-      for (int b = 0; b < kEPerWarp; ++b) {
-        float v = acc[a][b];
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, d));
-        const int e = eb + b;
-        if (lane == 0 && e < E && t0 + a < T) {
-          if (bias != nullptr) v = __fadd_rn(v, bias[e]);
-          s_logits[a * E + e] = v;
-          if (logits_out != nullptr) logits_out[(size_t)(t0 + a) * E + e] = v;
-        }
-      }
-  }
-  __syncthreads();
-
-  // top-k, gate scores, counts and reuse-score numerators: one warp per token
-  for (int a = warp; a < TT; a += kRouteWarps) {
-    const int t = t0 + a;
-    if (t >= T) continue;
+// Top-k (ties to the lower index), gate scores over the selected logits, counts and integer
+// reuse-score numerators of one token; executed by one warp.  row: the token's E logits.
+__device__ __forceinline__ void route_token_tail(const float* row, int t, int lane, int E, int K,
+                                                 const float* __restrict__ conf, int32_t* __restrict__ ids,
+                                                 float* __restrict__ gate, int32_t* __restrict__ counts,
+                                                 unsigned long long* __restrict__ scores) {
     float v[kMaxEPerLane];
 #pragma unroll
     for (int i = 0; i < kMaxEPerLane; ++i) {
       const int e = lane + 32 * i;
-      v[i] = e < E ? s_logits[a * E + e] : 0.0f;
+      v[i] = e < E ? row[e] : 0.0f;
     }
     uint32_t used = 0;
     int my_id = 0;
@@ -181,17 +107,19 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
     }
   }
 
-  // The last CTA to finish publishes counts and scores to the host (mapped pinned memory).
-  // Every 8-byte word carries the step's sequence tag in its upper bits, so the host can tell
-  // word by word that the data is there: no ordering fence, no copy operation, no event.
+// The last CTA to finish publishes counts and scores to the host (mapped pinned memory).
+// Every 8-byte word carries the step's sequence tag in its upper bits, so the host can tell
+// word by word that the data is there: no ordering fence, no copy operation, no event.
+__device__ __forceinline__ void route_publish(const RouteReport& rep, const int32_t* counts,
+                                              const unsigned long long* scores, int E, int* s_last) {
   if (rep.host_scores == nullptr) return;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
-    s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+    *s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
   }
   __syncthreads();
-  if (!s_last) return;
+  if (!*s_last) return;
   __threadfence();
   const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
   const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
@@ -199,6 +127,96 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
     rep.host_scores[e] = tag16 | __ldcg(&scores[e]);                               // score < 2^48
     rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
   }
+}
+
+// TT tokens per CTA, WARPS warps; each warp owns kEPerWarp experts per pass and all TT tokens.  Small
+// blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
+// chunks of loads in flight; the chain order of every logit is the same in all variants.
+template <int TT, int WARPS, int UNROLL, int kEPerWarp>
+__global__ void __launch_bounds__(WARPS * 32)
+route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
+             const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
+             int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
+             float* __restrict__ gate, int32_t* __restrict__ counts,
+             unsigned long long* __restrict__ scores, RouteReport rep) {
+  extern __shared__ float s_logits[];  // [TT][E]
+  __shared__ int s_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = blockIdx.x * TT;
+  griddep_launch_dependents();
+  griddep_wait();
+
+  constexpr int kRouteWarps = WARPS;
+  for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
+    float acc[TT][kEPerWarp];
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = 0.0f;
+
+#pragma unroll UNROLL
+    for (int hc = 0; hc < H; hc += 256) {
+      const int h = hc + lane * 8;
+      uint32_t xw[TT][4], ww[kEPerWarp][4];
+#pragma unroll
+      for (int a = 0; a < TT; ++a) {
+        const int t = min(t0 + a, T - 1);
+        const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+        xw[a][0] = v.x; xw[a][1] = v.y; xw[a][2] = v.z; xw[a][3] = v.w;
+      }
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        const int e = min(eb + b, E - 1);
+        const uint4 v = *reinterpret_cast<const uint4*>(wr + (size_t)e * H + h);
+        ww[b][0] = v.x; ww[b][1] = v.y; ww[b][2] = v.z; ww[b][3] = v.w;
+      }
+      // elements in ascending h: word 0 low half, word 0 high half, word 1 low half, ...
+#pragma unroll
+      for (int wi = 0; wi < 4; ++wi) {
+        float xf[TT], wf[kEPerWarp];
+#pragma unroll
+        for (int a = 0; a < TT; ++a) xf[a] = bf16_lo(xw[a][wi]);
+#pragma unroll
+        for (int b = 0; b < kEPerWarp; ++b) wf[b] = bf16_lo(ww[b][wi]);
+#pragma unroll
+        for (int a = 0; a < TT; ++a)
+#pragma unroll
+          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf[a], wf[b], acc[a][b]);
+#pragma unroll
+        for (int a = 0; a < TT; ++a) xf[a] = bf16_hi(xw[a][wi]);
+#pragma unroll
+        for (int b = 0; b < kEPerWarp; ++b) wf[b] = bf16_hi(ww[b][wi]);
+#pragma unroll
+        for (int a = 0; a < TT; ++a)
+#pragma unroll
+          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf[a], wf[b], acc[a][b]);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        float v = acc[a][b];
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, d));
+        const int e = eb + b;
+        if (lane == 0 && e < E && t0 + a < T) {
+          if (bias != nullptr) v = __fadd_rn(v, bias[e]);
+          s_logits[a * E + e] = v;
+          if (logits_out != nullptr) logits_out[(size_t)(t0 + a) * E + e] = v;
+        }
+      }
+  }
+  __syncthreads();
+
+  // top-k, gate scores, counts and reuse-score numerators: one warp per token
+  for (int a = warp; a < TT; a += kRouteWarps) {
+    const int t = t0 + a;
+    if (t >= T) continue;
+    route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores);
+  }
+
+  route_publish(rep, counts, scores, E, &s_last);
 }
 
 // One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
