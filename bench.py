@@ -218,6 +218,7 @@ def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None, dumm
         one(i)
     run.ctx.synchronize()
     s0, l0 = run.ctx.stats(), run.ctx.launch_count()
+    p0 = run.ctx.policy_time()
     from paper_2609_33385_b200 import dist
     dist.barrier()
     torch.cuda.synchronize()
@@ -234,7 +235,10 @@ def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None, dumm
     ms = a.elapsed_time(b)
     s1, l1 = run.ctx.stats(), run.ctx.launch_count()
     delta = {k: getattr(s1, k) - getattr(s0, k) for k in
-             ("steps", "hits", "misses", "bytes_moved", "evictions", "active_experts", "assignments")}
+             ("steps", "hits", "misses", "bytes_moved", "evictions", "active_experts", "assignments",
+              "fills_reused", "ideal_hits")}
+    p1 = run.ctx.policy_time()
+    delta["policy_us_per_layer_step"] = (p1[0] - p0[0]) / max(1, p1[1] - p0[1]) / 1e3
     return ms, l1 - l0, delta, clocks
 
 
@@ -378,6 +382,9 @@ def main():
     extra = {"tpot_ms": ms_per_step * w.iters / w.tokens,
              "hits": delta["hits"], "misses": delta["misses"],
              "cache_utilisation": delta["hits"] / max(1, delta["steps"] * w.capacity),
+             "ideal_cache_utilisation": delta["ideal_hits"] / max(1, delta["steps"] * w.capacity),
+             "effective_transfer_ratio": delta["fills_reused"] / max(1, delta["misses"]),
+             "policy_overhead_us_per_layer_step": delta["policy_us_per_layer_step"],
              "active_experts_per_layer_step": delta["active_experts"] / max(1, delta["steps"]),
              "h2d_link": {"achieved_gbs": delta["bytes_moved"] / (ms * 1e-3) / 1e9, **h2d},
              "setup_s": setup_s}

@@ -163,12 +163,17 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * (adds two event records per launch; off by default).
  * OLED_OPT_POLICY: retention value used by the cache update of every layer (OLED_POLICY_*).
  * OLED_OPT_ADAPT_PERIOD: n > 0 makes oled_denoise_iteration() call oled_adapt_capacity() after
- * every n-th iteration (the paper refreshes every five); 0 = fixed capacities (default). */
+ * every n-th iteration (the paper refreshes every five); 0 = fixed capacities (default).
+ * OLED_OPT_TEST_WITHHOLD_LOADS: test aid for the failure path.  1 = the tensor-core FFN kernels'
+ * load producers issue nothing, so the consumers' bounded waits (2 s) run out: the kernels set
+ * the status word, free their TMEM and return, and the next synchronising call reports
+ * OLED_ERR_TIMEOUT.  The context stays usable; oled_clear_status() re-arms it. */
 #define OLED_OPT_FFN_IMPL 1
 #define OLED_OPT_MISS_CHUNK 2
 #define OLED_OPT_PROFILE 3
 #define OLED_OPT_POLICY 4
 #define OLED_OPT_ADAPT_PERIOD 5
+#define OLED_OPT_TEST_WITHHOLD_LOADS 6
 #define OLED_POLICY_PRIORITY 0 /* confidence- and gate-guided priority, Sec. 4.3 (default) */
 #define OLED_POLICY_LRU 1      /* comparison point: least recently used (Sec. 5.1 Naive-LRU)  */
 #define OLED_POLICY_LFU 2      /* comparison point: least frequently used (Sec. 5.3)          */
@@ -204,6 +209,13 @@ typedef struct {
 /* Synchronises, folds pending event pairs into the totals and returns those of `kernel`;
  * reset != 0 clears them afterwards. */
 int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_profile* out);
+
+/* Clears a recorded device-side time-out (OLED_ERR_TIMEOUT is sticky until then).  Synchronises. */
+int oled_clear_status(oled_ctx* ctx);
+
+/* Host time spent in the cache policy (hit/miss resolution, Top-C retention, slot plan) so far, in
+ * nanoseconds, and the number of policy runs - the "policy overhead" of Sec. 5.4. */
+int oled_policy_time(oled_ctx* ctx, uint64_t* nanoseconds, uint64_t* runs);
 
 /* Number of kernels the library has launched on this context so far. */
 int oled_launch_count(oled_ctx* ctx, uint64_t* out);

@@ -23,6 +23,7 @@ OLED_OK = 0
 ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -2, -3, -4
 ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -9
 OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE, OPT_POLICY, OPT_ADAPT_PERIOD = 1, 2, 3, 4, 5
+OPT_TEST_WITHHOLD_LOADS = 6
 POLICY_PRIORITY, POLICY_LRU, POLICY_LFU = 0, 1, 2
 POLICY_IDS = {"priority": 0, "lru": 1, "lfu": 2}
 KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
@@ -34,7 +35,7 @@ EXPORTS = [
     "oled_synchronize", "oled_destroy", "oled_strerror", "oled_last_cuda_error",
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
     "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
-    "oled_policy_adapt",
+    "oled_policy_adapt", "oled_clear_status", "oled_policy_time",
 ]
 NOALLOC_MAX_TOKENS = 256
 
@@ -118,6 +119,8 @@ def load() -> C.CDLL:
                                      C.POINTER(i32)]
     lib.oled_policy_destroy.argtypes = [vp]
     lib.oled_policy_destroy.restype = None
+    lib.oled_clear_status.argtypes = [vp]
+    lib.oled_policy_time.argtypes = [vp, u64p, u64p]
     lib.oled_adapt_capacity.argtypes = [vp, vp]
     lib.oled_get_capacity.argtypes = [vp, vp]
     lib.oled_policy_set_policy.argtypes = [vp, i32]
@@ -248,6 +251,18 @@ class OledContext:
 
     def synchronize(self) -> None:
         self._check(self._lib.oled_synchronize(self._h), "oled_synchronize")
+
+    def synchronize_rc(self) -> int:
+        return self._lib.oled_synchronize(self._h)
+
+    def clear_status(self) -> None:
+        self._check(self._lib.oled_clear_status(self._h), "oled_clear_status")
+
+    def policy_time(self):
+        """(nanoseconds spent in the host cache policy, number of policy runs)."""
+        ns, runs = C.c_uint64(), C.c_uint64()
+        self._check(self._lib.oled_policy_time(self._h, C.byref(ns), C.byref(runs)), "oled_policy_time")
+        return int(ns.value), int(runs.value)
 
     def destroy(self) -> None:
         if self._h is not None:

@@ -266,7 +266,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     int stage = 0, g = 0;
     uint32_t phase = 0;
     bool ok = true;
-    for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+    for (int item = blockIdx.x; ok && !grp.withhold_loads && item < total_items; item += gridDim.x) {
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       for (int kb = 0; kb < k_blocks; ++kb) {

@@ -45,6 +45,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 struct FfnGroup {
   int32_t n;
   int32_t n_box;  // token rows per TMA box / MMA N tile of this launch
+  int32_t withhold_loads;  // test aid: the producer issues nothing, the consumers' waits run out
+  int32_t pad;
   uint16_t expert[OLED_MAX_EXPERTS];
   uint16_t slot[OLED_MAX_EXPERTS];
 };

@@ -81,6 +81,8 @@ struct oled_ctx {
   int ffn_impl = 0;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
   int miss_chunk = 4;
+  int withhold_loads = 0;      // test aid, see OLED_OPT_TEST_WITHHOLD_LOADS
+  uint64_t policy_ns = 0, policy_runs = 0;
   long long total_capacity = 0;
   int adapt_period = 0;        // iterations between automatic capacity refreshes (0 = off)
   uint64_t iterations = 0;     // oled_denoise_iteration() calls so far
@@ -257,6 +259,8 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
   FfnGroup grp;
   grp.n = (int32_t)(end - begin);
   grp.n_box = 16;
+  grp.withhold_loads = ctx->withhold_loads;
+  grp.pad = 0;
   int max_count = 0;
   uint64_t rows = 0;
   for (size_t i = begin; i < end; ++i) {
@@ -529,6 +533,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     FfnGroup grp;
     grp.n = 0;
     grp.n_box = 16;
+    grp.withhold_loads = ctx->withhold_loads;
+    grp.pad = 0;
     for (int32_t e = 0; e < E; ++e)
       if (L.cache.resident[e] && L.cache.slot_of[e] >= 0) {
         grp.expert[grp.n] = (uint16_t)e;
@@ -552,8 +558,14 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
 
   // 2. hits / misses against the pre-step resident set, Top-C retention, slot plan
   StepPlan& plan = ctx->plan;
-  if (!plan_step(L.cache, ctx->slots, counts, reinterpret_cast<const uint64_t*>(scores), plan))
-    return OLED_ERR_NO_SLOT;
+  {
+    const auto p0 = std::chrono::steady_clock::now();
+    const bool ok = plan_step(L.cache, ctx->slots, counts, reinterpret_cast<const uint64_t*>(scores), plan);
+    ctx->policy_ns += (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(
+                          std::chrono::steady_clock::now() - p0).count();
+    ctx->policy_runs += 1;
+    if (!ok) return OLED_ERR_NO_SLOT;
+  }
   ctx->last_before = plan.before;
   ctx->last_after = plan.after;
 
@@ -794,6 +806,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       if (value < 0) return OLED_ERR_INVALID_ARG;
       ctx->adapt_period = (int)value;
       return OLED_OK;
+    case OLED_OPT_TEST_WITHHOLD_LOADS:
+      ctx->withhold_loads = value != 0 ? 1 : 0;
+      return OLED_OK;
     case OLED_OPT_MISS_CHUNK:
       if (value < 1) return OLED_ERR_INVALID_ARG;
       ctx->miss_chunk = (int)std::min<int64_t>(value, OLED_MAX_EXPERTS);
@@ -810,6 +825,22 @@ int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_
   *out = ctx->prof_acc[kernel];
   if (reset) ctx->prof_acc[kernel] = oled_kernel_profile{};
   return rc;
+}
+
+int oled_clear_status(oled_ctx* ctx) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
+  OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), ctx->stream));
+  OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  *ctx->h_status = kStatusOk;
+  return OLED_OK;
+}
+
+int oled_policy_time(oled_ctx* ctx, uint64_t* nanoseconds, uint64_t* runs) {
+  if (!ctx || !nanoseconds || !runs) return OLED_ERR_INVALID_ARG;
+  *nanoseconds = ctx->policy_ns;
+  *runs = ctx->policy_runs;
+  return OLED_OK;
 }
 
 int oled_launch_count(oled_ctx* ctx, uint64_t* out) {

@@ -337,3 +337,35 @@ def test_layer_adaptive_sizing_through_the_iteration_entry_point():
         shadow.close()
     finally:
         run.close()
+
+
+def test_bounded_device_wait_reports_timeout_and_context_survives():
+    """Failure path without a fault: the FFN kernels' load producers are told to issue nothing, so
+    the consumers' bounded waits run out; the kernels flag it and return, the host reads
+    OLED_ERR_TIMEOUT, and after oled_clear_status() the same context computes correct results."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1)
+    run = _runner(w, capacity=[w.n_experts])
+    ora = _oracle_for(run, [w.n_experts])
+    try:
+        h_bits, conf = synth.flat_tokens(w, 5)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((5, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)                                   # warm: everything resident
+        ref = ora.denoise_step(0, h_bits, conf)
+        run.ctx.synchronize()
+        run.ctx.set_option(binding.OPT_TEST_WITHHOLD_LOADS, 1)
+        run.step(0, x, c, out)                                   # hits only: one FFN launch pair
+        assert run.ctx.synchronize_rc() == binding.ERR_TIMEOUT
+        assert run.ctx.synchronize_rc() == binding.ERR_TIMEOUT   # sticky until cleared
+        run.ctx.set_option(binding.OPT_TEST_WITHHOLD_LOADS, 0)
+        run.ctx.clear_status()
+        assert run.ctx.synchronize_rc() == binding.OLED_OK
+        ora.denoise_step(0, h_bits, conf)                        # keep the oracle's counters in step
+        run.step(0, x, c, out)
+        _check_out(dev_to_bits(out), ora.denoise_step(0, h_bits, conf)["out"])
+        ns, runs = run.ctx.policy_time()
+        assert runs == 3 and ns > 0
+    finally:
+        run.close()
