@@ -449,18 +449,18 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
             promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int stages_for(int kind, int n_box) {
+int stages_for(bool dual, int n_box) {
   static int cap = -1;  // tuning aid: OLED_FFN_STAGES caps the pipeline depth
   if (cap < 0) {
     const char* env = getenv("OLED_FFN_STAGES");
     cap = env ? std::max(1, atoi(env)) : kMaxStages;
   }
-  const uint32_t stage = ((kind == 1 || n_box == 256) ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+  const uint32_t stage = (dual ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
   return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage);
 }
-uint32_t smem_for(int kind, int n_box, int stages) {
-  const uint32_t stage = ((kind == 1 || n_box == 256) ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
+uint32_t smem_for(bool dual, int n_box, int stages) {
+  const uint32_t stage = (dual ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   return kCtlBytes + 1024u + (uint32_t)stages * stage;
 }
 
@@ -535,20 +535,26 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   };
   if (kind == 1) {
     grp.n_box = 16 << i1;
-    const int stages = stages_for(1, grp.n_box);
+    const int stages = stages_for(true, grp.n_box);
     launch_pdl(ffn_tc_kernel<1, true>, dim3(grid_for(grp.n_box, I / kBlockM)), dim3(kThreads),
-               smem_for(1, grp.n_box, stages), st, maps.w13, maps.xp[i1], grp, offsets, (void*)hbuf, H, I, stages,
+               smem_for(true, grp.n_box, stages), st, maps.w13, maps.xp[i1], grp, offsets, (void*)hbuf, H, I, stages,
                0, status);
   } else {
     grp.n_box = 16 << i2;
-    const int stages = stages_for(2, grp.n_box);
-    if (grp.n_box == 256)
-      launch_pdl(ffn_tc_kernel<2, true>, dim3(grid_for(256, H / (2 * kBlockM))), dim3(kThreads),
-                 smem_for(2, 256, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, y_bf16,
+    static int force_dual = -1;  // tuning aid: OLED_FFN2_DUAL=1 pairs Wd row blocks at every token tile
+    if (force_dual < 0) {
+      const char* env = getenv("OLED_FFN2_DUAL");
+      force_dual = env ? atoi(env) : 0;
+    }
+    const bool dual = grp.n_box == 256 || force_dual == 1;
+    const int stages = stages_for(dual, grp.n_box);
+    if (dual)
+      launch_pdl(ffn_tc_kernel<2, true>, dim3(grid_for(grp.n_box, H / (2 * kBlockM))), dim3(kThreads),
+                 smem_for(true, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, y_bf16,
                  status);
     else
       launch_pdl(ffn_tc_kernel<2, false>, dim3(grid_for(grp.n_box, H / kBlockM)), dim3(kThreads),
-                 smem_for(2, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages,
+                 smem_for(false, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages,
                  y_bf16, status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
