@@ -336,20 +336,14 @@ bool pdl_enabled() {
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep) {
-  static int small_max = -1, mid_max = -1;  // tuning aids: token-count thresholds of the variants
+  static int small_max = -1;  // tuning aid: largest step that takes the one-token-per-CTA variant
   if (small_max < 0) {
     const char* a = getenv("OLED_ROUTE_SMALL_MAX");
-    const char* b = getenv("OLED_ROUTE_MID_MAX");
     small_max = a ? atoi(a) : 1024;
-    mid_max = b ? atoi(b) : 1024;
   }
   if (T <= small_max) {
     constexpr int TT = 1, W = 16;
     launch_pdl(route_kernel<TT, W, 4, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
-               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
-  } else if (T <= mid_max) {
-    constexpr int TT = 2, W = 8;
-    launch_pdl(route_kernel<TT, W, 2, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
                w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
   } else {
     constexpr int TT = 8, W = 8;

@@ -369,3 +369,59 @@ def test_bounded_device_wait_reports_timeout_and_context_survives():
         assert runs == 3 and ns > 0
     finally:
         run.close()
+
+
+def test_maximum_expert_count_and_top_k():
+    """512 experts (OLED_MAX_EXPERTS) with top-32 (OLED_MAX_TOPK): the widest gate the ABI allows."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=512, top_k=32, hidden=256, intermediate=128)
+    run = _runner(w, capacity=[40], max_tokens=8)
+    ora = _oracle_for(run, [40])
+    try:
+        for rep, n in enumerate((3, 8)):
+            h_bits, conf = synth.flat_tokens(w, n, 20 + rep)
+            x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, x, c, out)
+            _check_step(run, 0, n, out, ora.denoise_step(0, h_bits, conf))
+        _check_stats(run, ora)
+    finally:
+        run.close()
+
+
+def test_degenerate_routing_cases():
+    """Identical tokens (one expert set takes every token), zero confidences (all reuse scores
+    zero: retention falls back to the id order) and top-k equal to the number of experts."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=4, hidden=256, intermediate=128)
+    run = _runner(w, capacity=[2], max_tokens=40)
+    ora = _oracle_for(run, [2])
+    try:
+        h_bits, conf = synth.flat_tokens(w, 40, 30)
+        same = np.repeat(h_bits[:1], 40, axis=0)                       # every token identical
+        zero_c = np.zeros(40, np.float32)
+        for hb, cf in ((same, conf), (h_bits, zero_c), (same, zero_c)):
+            x, c = bits_to_dev(hb, run.device), torch.from_numpy(cf).to(run.device)
+            out = torch.empty((40, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, x, c, out)
+            ref = ora.denoise_step(0, hb, cf)
+            _check_step(run, 0, 40, out, ref)
+            assert ref["counts"].tolist() == [40, 40, 40, 40]           # k = E: every expert, every token
+        _check_stats(run, ora)
+    finally:
+        run.close()
+    # a single expert set for all tokens with k < E: two experts hold all 2*T assignments
+    w2 = synth.tiny(n_layers=1, n_experts=8, top_k=2, hidden=256, intermediate=128)
+    run = _runner(w2, capacity=[3], max_tokens=300)
+    ora = _oracle_for(run, [3])
+    try:
+        h_bits, conf = synth.flat_tokens(w2, 300, 31)
+        same = np.repeat(h_bits[:1], 300, axis=0)
+        x, c = bits_to_dev(same, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((300, w2.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        ref = ora.denoise_step(0, same, conf)
+        assert sorted(ref["counts"].tolist())[-2:] == [300, 300] and ref["counts"].sum() == 600
+        _check_step(run, 0, 300, out, ref)
+    finally:
+        run.close()
