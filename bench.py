@@ -32,6 +32,20 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# DRAM traffic per algorithmic byte of the FFN kernels, from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the
+# captured launch).  Traffic grows in proportion to the experts (few-token regime) or token rows
+# (many-token regime) a launch processes, so the ratio scales a capture to any launch.
+NCU_TRAFFIC_RATIO = {
+    # profiles/ffn_tc_kernel_cfg2_full_residency.md: 63 experts x 4 tokens, H 2048, I 1024
+    ("ffn_gate_up", "few_tokens"): (521.34 + 3.96) / 530.1,
+    ("ffn_down", "few_tokens"): (260.61 + 5.42) / 267.0,
+    # profiles/ffn_tc_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
+    ("ffn_gate_up", "many_tokens"): (2091.3 + 102.3) / 1979.7,
+    ("ffn_down", "many_tokens"): (973.8 + 524.4) / 1442.0,
+}
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -367,11 +381,17 @@ def main():
                 "unit": "TFLOP/s" if tensor_bound else "GB/s",
                 "frac": (ach_tf / peaks["bf16_tflops_sustained"]) if tensor_bound else ach / peaks["hbm_gbs"],
                 "peak_source": peaks["source"] + (" (sustained bf16 matmul)" if tensor_bound else " (copy)"),
-                "traffic": None, "launches": kp["launches"],
+                "traffic": None, "traffic_source": None, "launches": kp["launches"],
                 "avg_launch_us": kp["ms"] * 1e3 / max(1, kp["launches"]),
                 "algorithmic_bytes_per_launch": kp["bytes"] / max(1, kp["launches"]),
                 "algorithmic_flops_per_launch": kp["flops"] / max(1, kp["launches"]),
                 "achieved_gbs": ach, "achieved_tflops": ach_tf}
+    regime = "many_tokens" if w.tokens * w.top_k > 4096 else "few_tokens"
+    ratio = NCU_TRAFFIC_RATIO.get((top, regime))
+    if ratio is not None:
+        roofline["traffic"] = ratio * roofline["algorithmic_bytes_per_launch"]
+        roofline["traffic_source"] = (f"ncu capture of the {regime.replace('_', '-')} regime (profiles/), scaled by "
+                                      "the algorithmic bytes of the average launch")
     kernels = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
                    "gbs": (v["bytes"] / v["ms"] / 1e6) if v["ms"] > 0 else None}
                for k, v in prof.items()}
