@@ -11,6 +11,12 @@
 // 256.  Weights are addressed through the expert->slot table: one 3-D tensor map covers the
 // whole slot pool and the slot number is a TMA coordinate.
 //
+// KIND 1 has a second form for small token tiles (N <= 32), "stacked": 64 gate rows and the 64 up
+// rows of the same intermediate features share ONE 128-row MMA tile (lanes 0-63 gate, 64-127 up),
+// so an item is half as large and twice as many items exist - with ~4 tokens per expert the
+// kernel is a weight stream, and finer items are what keeps all 148 SMs streaming to the end of
+// the launch.  The up values cross to the gate rows' warps through shared memory.
+//
 // In the many-token regime (N tile 256) both kernels work on two 128-row weight tiles that share
 // one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
 // which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
@@ -24,6 +30,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstddef>
 #include <cstdlib>
 
 #include "kernels.h"
@@ -50,6 +57,8 @@ struct __align__(16) SharedCtl {
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
+  unsigned long long x_full[2][2];   // stacked gate/up mode: [buffer][chunk group], up rows -> gate rows
+  unsigned long long x_empty[2][2];
   uint32_t tmem_base;
   int abort;
   int n_tiles_total;
@@ -57,7 +66,11 @@ struct __align__(16) SharedCtl {
   int tile_prefix[OLED_MAX_EXPERTS + 1];
   int row_start[OLED_MAX_EXPERTS];
   int count[OLED_MAX_EXPERTS];
+  // [buffer][chunk group][row][column]: up values of one 16-column chunk; read and written with
+  // 16-byte vector accesses, hence the alignment
+  __align__(16) float xchg[2][2][64][16];
 };
+static_assert(offsetof(SharedCtl, xchg) % 16 == 0, "xchg must be 16-byte aligned");
 constexpr uint32_t kCtlBytes = (sizeof(SharedCtl) + 1023u) & ~1023u;
 
 // ---------------------------------------------------------------- PTX helpers
@@ -200,10 +213,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_box = grp.n_box;
   constexpr bool dual = DUAL;
+  constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t stage_bytes = a_bytes + (uint32_t)n_box * 128u;
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
-  constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : kBlockM;  // output features per item
+  constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
   const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
@@ -223,6 +237,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[a]), (uint32_t)epi_warps * 32u);
+      for (int hgrp = 0; hgrp < 2; ++hgrp) {
+        mbar_init(smem_u32(&ctl->x_full[a][hgrp]), 64);
+        mbar_init(smem_u32(&ctl->x_empty[a][hgrp]), 64);
+      }
     }
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -277,7 +295,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         const uint32_t bar = smem_u32(&ctl->full[stage]);
         const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
         mbar_expect_tx(bar, stage_bytes);
-        if (KIND == 1) {
+        if (stacked) {  // tm_w has 64-row boxes here
+          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);                   // 64 gate rows
+          tma_load_3d(&tm_w, a_addr + kATile / 2, bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
+        } else if (KIND == 1) {
           tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // gate rows
           tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
         } else {
@@ -340,7 +361,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
     int g = 0, local = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
+    uint32_t xn = 0;  // stacked mode: 16-column chunks this warp's chunk group has exchanged so far
+    bool alive = true;
+    for (int item = blockIdx.x; alive && item < total_items; item += gridDim.x, ++local) {
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
@@ -359,7 +382,53 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
-        if (KIND == 1) {
+        if (stacked) {
+          // lanes 0-63 hold silu's argument (gate rows), lanes 64-127 the up rows of the same
+          // features: warps 2,3 hand their chunk to warps 0,1 through a double-buffered slot
+          tmem_ld_wait();
+          const uint32_t buf = xn & 1u, ph = (xn >> 1) & 1u;
+          ++xn;
+          const int xrow = (quarter & 1) * 32 + lane;
+          float* slot = &ctl->xchg[buf][half][xrow][0];
+          int ok = 0;
+          if (quarter >= 2) {
+            if (lane == 0) ok = mbar_wait(smem_u32(&ctl->x_empty[buf][half]), ph ^ 1u, abort_flag, status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) {
+              alive = false;
+              break;
+            }
+#pragma unroll
+            for (int j = 0; j < 16; j += 4)
+              *reinterpret_cast<uint4*>(slot + j) = make_uint4(ra[j], ra[j + 1], ra[j + 2], ra[j + 3]);
+            mbar_arrive(smem_u32(&ctl->x_full[buf][half]));
+          } else {
+            if (lane == 0) ok = mbar_wait(smem_u32(&ctl->x_full[buf][half]), ph, abort_flag, status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) {
+              alive = false;
+              break;
+            }
+            __syncwarp();  // lane 0's acquire orders the whole warp's reads of the slot
+            float u[16];
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) {
+              const float4 v = *reinterpret_cast<const float4*>(slot + j);
+              u[j] = v.x; u[j + 1] = v.y; u[j + 2] = v.z; u[j + 3] = v.w;
+            }
+            mbar_arrive(smem_u32(&ctl->x_empty[buf][half]));
+            uint16_t* hb = reinterpret_cast<uint16_t*>(out_ptr);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (c + j < it.valid) {
+                const float a = __uint_as_float(ra[j]);
+                const float hm = __fdividef(a, 1.0f + __expf(-a)) * u[j];
+                const __nv_bfloat16 b = __float2bfloat16_rn(hm);
+                hb[(size_t)(it.row0 + c + j) * I + it.m0 + xrow] = *reinterpret_cast<const uint16_t*>(&b);
+              }
+            }
+          }
+        } else if (KIND == 1) {
           uint32_t rb[16];
           tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
           tmem_ld_wait();
@@ -398,6 +467,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
         }
       }
+      if (!alive) break;
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
     }
@@ -474,6 +544,12 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
     const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
     if (!encode(&maps->w13, 3, pool, dims, strides, box)) return OLED_ERR_CUDA;
   }
+  {  // the same matrix with 64-row boxes (stacked gate/up tiles)
+    const cuuint64_t dims[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
+    const cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)slot_bytes};
+    const cuuint32_t box[3] = {kBlockK, kBlockM / 2, 1};
+    if (!encode(&maps->w13_half, 3, pool, dims, strides, box)) return OLED_ERR_CUDA;
+  }
   {
     const cuuint64_t dims[3] = {(cuuint64_t)I, (cuuint64_t)H, (cuuint64_t)n_slots};
     const cuuint64_t strides[2] = {(cuuint64_t)I * 2, (cuuint64_t)slot_bytes};
@@ -496,6 +572,8 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(ffn_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemMax) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSmemMax) != cudaSuccess ||
         cudaFuncSetAttribute(ffn_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSmemMax) != cudaSuccess ||
@@ -533,7 +611,18 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + n_box - 1) / n_box;
     return (int)std::max<long long>(1, std::min<long long>(n_sms, tiles * m_tiles));
   };
-  if (kind == 1) {
+  static int use_stacked = -1;  // tuning aid: OLED_FFN1_STACKED=0 keeps the two-accumulator form
+  if (use_stacked < 0) {
+    const char* env = getenv("OLED_FFN1_STACKED");
+    use_stacked = env ? atoi(env) : 1;
+  }
+  if (kind == 1 && (16 << i1) <= 32 && use_stacked == 1) {
+    grp.n_box = 16 << i1;
+    const int stages = stages_for(false, grp.n_box);
+    launch_pdl(ffn_tc_kernel<1, false>, dim3(grid_for(grp.n_box, I / (kBlockM / 2))), dim3(kThreads),
+               smem_for(false, grp.n_box, stages), st, maps.w13_half, maps.xp[i1], grp, offsets, (void*)hbuf, H, I,
+               stages, 0, status);
+  } else if (kind == 1) {
     grp.n_box = 16 << i1;
     const int stages = stages_for(true, grp.n_box);
     launch_pdl(ffn_tc_kernel<1, true>, dim3(grid_for(grp.n_box, I / kBlockM)), dim3(kThreads),

@@ -98,6 +98,7 @@ void launch_ffn_simple(cudaStream_t st, const FfnGroup& grp, const uint8_t* pool
 // ---- ffn_tc.cu (tcgen05 / TMEM / TMA) ------------------------------------------------------
 struct FfnTcMaps {
   CUtensorMap w13;       // [slots][2I][H] bf16, box {64,128,1}
+  CUtensorMap w13_half;  // the same, box {64,64,1}
   CUtensorMap w2;        // [slots][H][I]  bf16, box {64,128,1}
   CUtensorMap xp[5];     // [rows][H] bf16, box {64, 16<<i}
   CUtensorMap hbuf[5];   // [rows][I] bf16, box {64, 16<<i}
