@@ -15,7 +15,8 @@ from typing import Callable, List, Optional, Sequence
 import numpy as np
 
 from .cache_policy import AdaptiveSizer, LayerCache, LayerStats
-from .moe_layer import bf16_to_f32, gate_logits, moe_layer_forward, permutation, topk_route
+from .moe_layer import (bf16_to_f32, fp8_expert_weights, gate_logits, moe_layer_forward, permutation,
+                        topk_route)
 
 
 class OracleStack:
@@ -50,6 +51,15 @@ class OracleStack:
             return (b[:h * i].reshape(i, h), b[h * i:2 * h * i].reshape(i, h),
                     b[2 * h * i:].reshape(h, i))
         self.experts[layer] = get
+
+    def register_experts_fp8(self, layer: int, blobs: np.ndarray) -> None:
+        """blobs: uint8 [E, blob_bytes], each row an fp8 expert blob (codes, then row scales)."""
+        h, i = self.hidden, self.intermediate
+        assert blobs.shape[0] == self.n_experts and blobs.shape[1] >= 3 * h * i + 4 * (2 * i + h)
+        self.experts[layer] = lambda e: fp8_expert_weights(blobs[e], h, i)
+        self.expert_bytes = int(blobs.shape[1])
+        for c in self.caches:
+            c.expert_bytes = self.expert_bytes
 
     def denoise_step(self, layer: int, hidden_bits: np.ndarray, conf: np.ndarray) -> dict:
         """One layer execution of one denoising iteration; returns every intermediate."""

@@ -33,6 +33,30 @@ def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
     return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def fp8_e4m3_to_f32(codes: np.ndarray) -> np.ndarray:
+    """Decode fp8 e4m3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities,
+    0x7F / 0xFF are NaN; exponent field 0 is subnormal: m * 2^-9)."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int32)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e, m = (c >> 3) & 0xF, c & 7
+    mag = np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return (sign * mag).astype(np.float32)
+
+
+def fp8_expert_weights(blob: np.ndarray, hidden: int, intermediate: int):
+    """Dequantised (gate[I,H], up[I,H], down[H,I]) in fp64 from an fp8 expert blob: e4m3 codes of
+    the three matrices followed by fp32 scales s_gate[I] | s_up[I] | s_down[H], one per row."""
+    h, i = hidden, intermediate
+    n = 3 * h * i
+    sc = np.asarray(blob[n:n + 4 * (2 * i + h)], dtype=np.uint8).view(np.float32).astype(np.float64)
+    vals = fp8_e4m3_to_f32(blob[:n]).astype(np.float64)
+    gate = vals[:h * i].reshape(i, h) * sc[:i, None]
+    up = vals[h * i:2 * h * i].reshape(i, h) * sc[i:2 * i, None]
+    down = vals[2 * h * i:].reshape(h, i) * sc[2 * i:, None]
+    return gate, up, down
+
+
 # --------------------------------------------------------------------------
 # Gate logits, fixed reduction order
 # --------------------------------------------------------------------------
@@ -199,8 +223,9 @@ def moe_layer_forward(x_bits, w_router_bits, bias, expert_weights, k: int):
         rows = perm[offsets[ee]:offsets[ee + 1]]
         toks = rows // k
         wg, wu, wd = expert_weights(ee)
-        y[offsets[ee]:offsets[ee + 1]] = expert_ffn(x[toks], bf16_to_f32(wg), bf16_to_f32(wu),
-                                                    bf16_to_f32(wd))
+        if wg.dtype == np.uint16:           # bf16 bit patterns; fp8 stores hand over decoded floats
+            wg, wu, wd = bf16_to_f32(wg), bf16_to_f32(wu), bf16_to_f32(wd)
+        y[offsets[ee]:offsets[ee + 1]] = expert_ffn(x[toks], wg, wu, wd)
     out = np.zeros((t, h), dtype=np.float64)
     for tt in range(t):
         for j in range(k):

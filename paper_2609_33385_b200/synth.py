@@ -245,3 +245,57 @@ def flat_tokens(w: Workload, n_tokens: int, stream_id: int = 0) -> Tuple[np.ndar
     h = g.standard_normal((n_tokens, w.hidden), dtype=np.float32)
     c = g.beta(w.beta_a, w.beta_b, size=n_tokens).astype(np.float32)
     return f32_to_bf16_bits(h), c
+
+
+# --------------------------------------------------------------------------
+# Narrow expert blobs: fp8 (e4m3) weights with one fp32 scale per output row
+# --------------------------------------------------------------------------
+def _e4m3_positive_values() -> np.ndarray:
+    """The 127 finite non-negative e4m3 values in code order (code 0x00..0x7E)."""
+    vals = []
+    for code in range(0x7F):
+        e, m = code >> 3, code & 7
+        vals.append(m * 2.0 ** -9 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals, dtype=np.float64)
+
+
+_E4M3_POS = _e4m3_positive_values()
+
+
+def f32_to_e4m3_codes(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest e4m3 value (ties to the even code), saturating at +-448."""
+    a = np.minimum(np.abs(np.asarray(x, dtype=np.float64)), 448.0)
+    hi = np.clip(np.searchsorted(_E4M3_POS, a, side="left"), 0, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = _E4M3_POS[hi] - a, a - _E4M3_POS[lo]
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return code | (np.signbit(x).astype(np.uint8) << 7)
+
+
+def fp8_blob_bytes(w: Workload) -> int:
+    """Bytes of one fp8 expert blob: gate[I,H] | up[I,H] | down[H,I] codes, then fp32 scales
+    s_gate[I] | s_up[I] | s_down[H]; padded to a multiple of 256."""
+    n = 3 * w.hidden * w.intermediate + 4 * (2 * w.intermediate + w.hidden)
+    return (n + 255) // 256 * 256
+
+
+def quantize_expert_blob(w: Workload, blob_bits: np.ndarray, out: Optional[np.ndarray] = None) -> np.ndarray:
+    """bf16 expert blob -> fp8 blob.  Every row of the three matrices gets the scale
+    max|row| / 448 (1 for an all-zero row) and its elements are rounded to e4m3."""
+    h, i = w.hidden, w.intermediate
+    if out is None:
+        out = np.zeros(fp8_blob_bytes(w), dtype=np.uint8)
+    mats = split_blob(w, blob_bits)
+    off, scales = 0, []
+    for m in mats:
+        f = bf16_bits_to_f32(m)
+        amax = np.abs(f).max(axis=1)
+        sc = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+        q = f32_to_e4m3_codes(f.astype(np.float64) / sc[:, None].astype(np.float64))
+        out[off:off + q.size] = q.reshape(-1)
+        off += q.size
+        scales.append(sc)
+    sc_all = np.concatenate(scales).astype(np.float32)
+    out[off:off + 4 * sc_all.size] = sc_all.view(np.uint8)
+    return out

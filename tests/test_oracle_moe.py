@@ -285,3 +285,72 @@ def test_layer_empty_step():
     x, wr, blobs, get = _layer(rng)
     res = om.moe_layer_forward(x[:0], wr, None, get, 2)
     assert res["out"].shape == (0, 256) and res["counts"].sum() == 0
+
+
+# ------------------------------------------------------------------ fp8 expert blobs
+def test_fp8_decode_against_format_definition_and_torch():
+    codes = np.arange(256, dtype=np.uint8)
+    got = om.fp8_e4m3_to_f32(codes)
+    assert got[0] == 0.0 and got[0x80] == 0.0 and np.signbit(got[0x80])
+    assert got[0x01] == 2.0 ** -9 and got[0x07] == 7 * 2.0 ** -9          # subnormals
+    assert got[0x08] == 2.0 ** -6 and got[0x38] == 1.0 and got[0x3C] == 1.5
+    assert got[0x7E] == 448.0 and got[0xFE] == -448.0                       # largest finite
+    assert np.isnan(got[0x7F]) and np.isnan(got[0xFF])
+    finite = got[:0x7F]
+    assert np.all(np.diff(finite) > 0)                                      # codes are monotone
+    torch = pytest.importorskip("torch")
+    if hasattr(torch, "float8_e4m3fn"):
+        ref = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+        ok = ~np.isnan(ref)
+        assert np.array_equal(got[ok], ref[ok]) and np.array_equal(np.isnan(got), np.isnan(ref))
+
+
+def test_fp8_encode_roundtrip_and_rounding():
+    vals = om.fp8_e4m3_to_f32(np.arange(256, dtype=np.uint8))
+    fin = ~np.isnan(vals)
+    back = synth.f32_to_e4m3_codes(vals[fin])
+    assert np.array_equal(om.fp8_e4m3_to_f32(back), vals[fin])              # every code survives
+    # midpoints go to the even code; anything beyond 448 saturates
+    assert synth.f32_to_e4m3_codes(np.array([1.0625, 1.1875, 1000.0, -1000.0])).tolist() == \
+        [0x38, 0x3A, 0x7E, 0xFE]
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal(20000) * 50
+    q = om.fp8_e4m3_to_f32(synth.f32_to_e4m3_codes(x)).astype(np.float64)
+    pos = np.sort(np.abs(vals[fin]).astype(np.float64))
+    xa = np.minimum(np.abs(x), 448.0)
+    nearest = pos[np.abs(pos[None, :] - xa[:, None]).argmin(axis=1)]
+    assert np.allclose(np.abs(q), nearest)                                   # nearest representable
+
+
+def test_fp8_blob_layout_and_dequantisation_error():
+    w = synth.tiny(n_layers=1)
+    blob = synth.expert_blob_bits(w, 0, 3)
+    q = synth.quantize_expert_blob(w, blob)
+    assert q.size == synth.fp8_blob_bytes(w) and q.size % 256 == 0
+    g, u, d = om.fp8_expert_weights(q, w.hidden, w.intermediate)
+    for deq, ref in zip((g, u, d), synth.split_blob(w, blob)):
+        r = om.bf16_to_f32(ref).astype(np.float64)
+        assert deq.shape == r.shape
+        # per-row scaling: error at most half an e4m3 step of the row maximum (1/16 relative)
+        bound = np.abs(r).max(axis=1, keepdims=True) / 16.0 + 1e-12
+        assert np.all(np.abs(deq - r) <= bound)
+        assert np.allclose(np.abs(deq).max(axis=1), np.abs(r).max(axis=1), rtol=1e-6)
+
+
+def test_fp8_layer_matches_layer_on_dequantised_weights():
+    rng = np.random.default_rng(21)
+    w = synth.tiny(n_layers=1)
+    x, conf = synth.flat_tokens(w, 6)
+    wr, _ = synth.router_weights(w, 0)
+    blobs = np.stack([synth.quantize_expert_blob(w, synth.expert_blob_bits(w, 0, e)) for e in range(w.n_experts)])
+    res = om.moe_layer_forward(x, wr, None, lambda e: om.fp8_expert_weights(blobs[e], w.hidden, w.intermediate),
+                               w.top_k)
+    # the same layer evaluated token by token with explicit fp64 formulas
+    xf = om.bf16_to_f32(x).astype(np.float64)
+    for t in range(6):
+        acc = np.zeros(w.hidden)
+        for j in range(w.top_k):
+            g, u, d = om.fp8_expert_weights(blobs[res["ids"][t, j]], w.hidden, w.intermediate)
+            a = g @ xf[t]
+            acc += float(res["gate"][t, j]) * (d @ (a / (1 + np.exp(-a)) * (u @ xf[t])))
+        assert np.allclose(res["out"][t], acc, rtol=1e-10, atol=1e-13)
