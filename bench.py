@@ -256,9 +256,9 @@ def timed_pass(torch, run, xs, cs, warmup, steps, host=False, sampler=None, dumm
     return ms, l1 - l0, delta, clocks
 
 
-def step_roofline(w, delta, steps, ms_per_step, peaks, h2d_gbs):
+def step_roofline(w, delta, steps, ms_per_step, peaks, h2d_gbs, blob=None):
     """Binding roofline of the whole step from the algorithmic work of the timed region."""
-    blob = w.expert_bytes
+    blob = blob or w.expert_bytes
     layer_steps = max(1, delta["steps"])
     b_hbm = (delta["active_experts"] * blob + delta["misses"] * blob +
              layer_steps * (w.n_experts * w.hidden * 2 + 2 * w.tokens * w.hidden * 2)) / steps
@@ -289,6 +289,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-residency", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    ap.add_argument("--expert-format", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: e4m3 expert blobs with row scales (an extension; the headline is bf16)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -325,7 +327,8 @@ def main():
     threads = max(1, min(32, cores // max(1, world)))
 
     t_setup = time.perf_counter()
-    run = StackRunner(w, device=device, gen_threads=threads, distinct_layers=args.distinct_layers)
+    fp8 = args.expert_format == "fp8"
+    run = StackRunner(w, device=device, gen_threads=threads, distinct_layers=args.distinct_layers, fp8=fp8)
     xs, cs = [], []
     for _, _, h_bits, conf in synth.denoise_inputs(w):
         xs.append(bits_to_dev(h_bits, device))
@@ -333,7 +336,7 @@ def main():
         if len(xs) >= n_iters:
             break
     setup_s = time.perf_counter() - t_setup
-    h2d = measure_h2d(torch, device, w.expert_bytes)
+    h2d = measure_h2d(torch, device, run.ctx.expert_bytes)
     gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid).replace("GPU-", "")
 
     # 1. device-resident inputs: the headline value
@@ -398,7 +401,7 @@ def main():
     for k, v in prof.items():
         kernels[k]["tflops"] = (v["flops"] / v["ms"] / 1e9) if v["ms"] > 0 else None
 
-    step_roof = step_roofline(w, delta, args.steps, ms_per_step, peaks, h2d["gbs_blob_train"])
+    step_roof = step_roofline(w, delta, args.steps, ms_per_step, peaks, h2d["gbs_blob_train"], run.ctx.expert_bytes)
     extra = {"tpot_ms": ms_per_step * w.iters / w.tokens,
              "hits": delta["hits"], "misses": delta["misses"],
              "cache_utilisation": delta["hits"] / max(1, delta["steps"] * w.capacity),
@@ -411,7 +414,7 @@ def main():
 
     # 4. full residency on the same workload (C = E): the HBM-bound regime and the TPOT ratio
     if not args.no_full_residency and w.residency < 1.0:
-        full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run)
+        full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run, fp8=fp8)
         # dummy requests (i.i.d. tokens activate nearly every expert) so that no cold miss is left
         dummy = []
         for j, (_, _, h_bits, conf) in enumerate(synth.denoise_inputs(w.replace(shared_beta=0.0, seed=w.seed + 1))):
@@ -421,7 +424,8 @@ def main():
         ms_f, _, delta_f, _ = timed_pass(torch, full, xs, cs, args.warmup, args.steps, dummy=dummy)
         _, ms_f_max = dist.aggregate(0, ms_f, device)
         msf = ms_f_max / args.steps
-        rf = step_roofline(w.replace(residency=1.0), delta_f, args.steps, msf, peaks, h2d["gbs_blob_train"])
+        rf = step_roofline(w.replace(residency=1.0), delta_f, args.steps, msf, peaks, h2d["gbs_blob_train"],
+                           run.ctx.expert_bytes)
         full.ctx.reset_cache()
         for dx, dc in dummy:
             full.ctx.denoise_iteration(dx.data_ptr(), dc.data_ptr(), w.tokens, out_dev.data_ptr())
@@ -444,7 +448,7 @@ def main():
         full.close()
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not fp8:
         sec, count, thr = oracle_layer_steps(w, budget_s=args.cpu_budget_s, max_steps=64)
         cpu = {"value": w.tokens / (sec * w.n_layers), "unit": UNIT, "cores": thr, "kind": "oracle",
                "sample": f"{count} layer executions of {w.name} ({sec:.3f} s each; 1 distinct layer of "
@@ -455,7 +459,9 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": workload_config(w, args.variant), "clocks": clocks, "e2e": e2e,
+                "config": dict(workload_config(w, args.variant),
+                               expert_format="fp8_e4m3_row_scaled" if fp8 else "bf16"),
+                "clocks": clocks, "e2e": e2e,
                 "gpu_launches": launches, "roofline": roofline, "roofline_step": step_roof,
                 "kernels": kernels, "cpu_baseline": cpu, **extra}
         print(json.dumps(line))

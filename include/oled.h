@@ -64,14 +64,27 @@ typedef struct {
   int32_t max_tokens;      /* upper bound on n_tokens of any step */
   int32_t has_router_bias; /* 1: oled_register_router() takes a per-expert fp32 bias */
   int32_t staging_slots;   /* transient slots for misses beyond capacity; 0 = E - min capacity */
+  int32_t expert_format;   /* OLED_EXPERTS_BF16 (0) or OLED_EXPERTS_FP8 */
 } oled_model_shape;
+
+/* Expert blob formats of the host store and of the HBM slots (a blob is copied as it is).
+ *   OLED_EXPERTS_BF16: gate[I,H] | up[I,H] | down[H,I] in bf16; 3*H*I*2 bytes.
+ *   OLED_EXPERTS_FP8:  the same three matrices as fp8 e4m3 codes (1 byte each), followed by one
+ *     fp32 scale per weight row, s_gate[I] | s_up[I] | s_down[H]; a weight is code * scale of its
+ *     row.  3*H*I + 4*(2*I+H) bytes, padded to a multiple of 256.  Half the host-link and HBM
+ *     traffic per expert (the paper names quantisation as the complementary lever for H2D volume);
+ *     the codes are widened to bf16 on chip (exactly), the arithmetic is the bf16 path's. */
+#define OLED_EXPERTS_BF16 0
+#define OLED_EXPERTS_FP8 1
+/* Bytes of one expert blob in the given format. */
+size_t oled_expert_blob_bytes(int32_t hidden, int32_t intermediate, int32_t expert_format);
 
 /* Cumulative counters (Sec. 5.1 metrics: cache utilisation = hits / capacity per execution). */
 typedef struct {
   uint64_t steps;          /* layer executions                                   */
   uint64_t hits;           /* sum of #(A n R), R taken before execution (Sec. 4.2) */
   uint64_t misses;         /* sum of #(A \ R)                                    */
-  uint64_t bytes_moved;    /* host->HBM bytes: misses * 3*H*I*2                  */
+  uint64_t bytes_moved;    /* host->HBM bytes: misses * blob bytes               */
   uint64_t evictions;      /* sum of #(R \ R')                                   */
   uint64_t active_experts; /* sum of #A                                          */
   uint64_t assignments;    /* sum of n_tokens * k                                */
@@ -87,7 +100,7 @@ typedef struct {
  *   cache_capacity  host int32[n_layers]; slots C_l per layer, 1 <= C_l <= E ("Cache" in Sec. 5.1).
  *   cuda_stream     a cudaStream_t (may be 0) on which every step is enqueued; borrowed.
  *   out_ctx         receives the context; the library owns it until oled_destroy().
- * Allocates the slot pool (sum C_l + staging slots, each 3*H*I*2 bytes), router weights and
+ * Allocates the slot pool (sum C_l + staging slots, each one expert blob), router weights and
  * scratch in device memory.  Errors: INVALID_ARG, OOM, CUDA. */
 int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, void* cuda_stream,
                 oled_ctx** out_ctx);
@@ -99,8 +112,8 @@ int oled_register_router(oled_ctx* ctx, int32_t layer, const void* w_router, con
 
 /* Give a layer its host expert store (Sec. 2.2, Sec. 4.1).  host_blob is PINNED host memory,
  * borrowed until oled_destroy() and never written; expert e starts at
- * host_blob + e*expert_stride_bytes and holds gate[I,H] | up[I,H] | down[H,I] in bf16
- * (3*H*I*2 bytes; stride >= that and a multiple of 16).  Errors: NOT_PINNED, INVALID_ARG. */
+ * host_blob + e*expert_stride_bytes and holds one blob in the context's expert_format
+ * (stride >= oled_expert_blob_bytes() and a multiple of 16).  Errors: NOT_PINNED, INVALID_ARG. */
 int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob,
                           size_t expert_stride_bytes);
 

@@ -35,15 +35,17 @@ EXPORTS = [
     "oled_synchronize", "oled_destroy", "oled_strerror", "oled_last_cuda_error",
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
     "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
-    "oled_policy_adapt", "oled_clear_status", "oled_policy_time",
+    "oled_policy_adapt", "oled_clear_status", "oled_policy_time", "oled_expert_blob_bytes",
 ]
+EXPERTS_BF16, EXPERTS_FP8 = 0, 1
 NOALLOC_MAX_TOKENS = 256
 
 
 class ModelShape(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_experts", C.c_int32),
                 ("top_k", C.c_int32), ("intermediate", C.c_int32), ("max_tokens", C.c_int32),
-                ("has_router_bias", C.c_int32), ("staging_slots", C.c_int32)]
+                ("has_router_bias", C.c_int32), ("staging_slots", C.c_int32),
+                ("expert_format", C.c_int32)]
 
 
 class KernelProfile(C.Structure):
@@ -119,6 +121,8 @@ def load() -> C.CDLL:
                                      C.POINTER(i32)]
     lib.oled_policy_destroy.argtypes = [vp]
     lib.oled_policy_destroy.restype = None
+    lib.oled_expert_blob_bytes.argtypes = [i32, i32, i32]
+    lib.oled_expert_blob_bytes.restype = C.c_size_t
     lib.oled_clear_status.argtypes = [vp]
     lib.oled_policy_time.argtypes = [vp, u64p, u64p]
     lib.oled_adapt_capacity.argtypes = [vp, vp]
@@ -144,17 +148,17 @@ class OledContext:
 
     def __init__(self, n_layers: int, hidden: int, n_experts: int, top_k: int, intermediate: int,
                  max_tokens: int, cache_capacity: Sequence[int], cuda_stream: int = 0,
-                 has_router_bias: bool = False, staging_slots: int = 0):
+                 has_router_bias: bool = False, staging_slots: int = 0, expert_format: int = EXPERTS_BF16):
         self._lib = load()
         self.shape = ModelShape(n_layers, hidden, n_experts, top_k, intermediate, max_tokens,
-                                1 if has_router_bias else 0, staging_slots)
+                                1 if has_router_bias else 0, staging_slots, expert_format)
         caps = (C.c_int32 * n_layers)(*[int(c) for c in cache_capacity])
         h = C.c_void_p()
         rc = self._lib.oled_create(C.byref(self.shape), caps, C.c_void_p(cuda_stream), C.byref(h))
         self._h = h if rc == OLED_OK else None
         if rc != OLED_OK:
             raise OledError(rc, "oled_create")
-        self.expert_bytes = 3 * hidden * intermediate * 2
+        self.expert_bytes = int(self._lib.oled_expert_blob_bytes(hidden, intermediate, expert_format))
 
     # -- helpers
     def _check(self, rc: int, what: str) -> None:

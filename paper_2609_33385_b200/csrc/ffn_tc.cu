@@ -23,11 +23,18 @@
 //
 // Warp roles (576 threads): warps 0-15 epilogue (TMEM lane quarter = warp id mod 4, the warps of
 // a quarter interleave 16-column chunks; only as many as the token tile has chunks are active),
-// warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation).  Every mbarrier
+// warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation),
+// warps 18-21 widen fp8 weight tiles (fp8 expert stores only, idle otherwise).
+//
+// fp8 expert stores (e4m3 codes + one fp32 scale per weight row): TMA brings the raw 64-byte
+// rows into a staging area of the stage, the converter warps write them as bf16 (exact) into the
+// swizzled operand tile, the MMA runs in bf16 as before and the epilogue multiplies each output
+// row by its scale - the rows of a weight tile are the accumulator's lanes.  Every mbarrier
 // wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
 // copies time to land, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <algorithm>
 #include <cstddef>
@@ -44,7 +51,9 @@ namespace {
 constexpr int kEpiWarps = OLED_EPI_WARPS;  // up to four warps per TMEM lane quarter, interleaving 16-column chunks
 constexpr int kProducerWarp = kEpiWarps;
 constexpr int kMmaWarp = kEpiWarps + 1;
-constexpr int kThreads = (kEpiWarps + 2) * 32;
+constexpr int kConvWarp0 = kEpiWarps + 2;     // four warps that widen fp8 weight tiles to bf16 (fp8 stores only)
+constexpr int kConvThreads = 128;
+constexpr int kThreads = (kEpiWarps + 6) * 32;
 constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
 constexpr uint32_t kATile = kBlockM * kBlockK * 2;
@@ -55,6 +64,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 struct __align__(16) SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
+  unsigned long long raw_full[kMaxStages];  // fp8 stores: the raw weight rows of the stage have landed
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long x_full[2][2];   // stacked gate/up mode: [buffer][chunk group], up rows -> gate rows
@@ -183,6 +193,29 @@ __device__ __forceinline__ uint32_t make_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 }
 
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4& v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+// Two e4m3 codes (low byte first) -> two bf16 (exact: e4m3 fits bf16's exponent and mantissa).
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t two_codes) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
+  const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+  const __nv_bfloat162 b = __floats2bfloat162_rn(f.x, f.y);
+  return *reinterpret_cast<const uint32_t*>(&b);
+}
+// Four codes in one 32-bit word -> four bf16 in two words.
+__device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  lo = e4m3x2_to_bf16x2(w & 0xffffu);
+  hi = e4m3x2_to_bf16x2(w >> 16);
+}
+
 struct Item {
   int slot, m0, row0, valid;
 };
@@ -200,11 +233,13 @@ __device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup
 
 // DUAL: two accumulators per item - gate and up (KIND 1, always), or two row blocks of Wd
 // (KIND 2 with the 256-token tile).
-template <int KIND, bool DUAL>
+// FP8: the slot pool holds fp8 expert blobs (tm_w is a byte map over the e4m3 codes).
+template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
               void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
+              const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
@@ -215,7 +250,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr bool dual = DUAL;
   constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
-  const uint32_t stage_bytes = a_bytes + (uint32_t)n_box * 128u;
+  const uint32_t b_bytes = (uint32_t)n_box * 128u;
+  constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;  // staging of the stage's e4m3 rows
+  const uint32_t stage_bytes = a_bytes + b_bytes + raw_bytes;
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
@@ -231,8 +268,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 1u + kConvThreads : 1u);  // token tile (+ converters)
       mbar_init(smem_u32(&ctl->empty[s]), 1);
+      mbar_init(smem_u32(&ctl->raw_full[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
@@ -294,16 +332,25 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
         const uint32_t bar = smem_u32(&ctl->full[stage]);
         const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-        mbar_expect_tx(bar, stage_bytes);
-        if (stacked) {  // tm_w has 64-row boxes here
-          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);                   // 64 gate rows
-          tma_load_3d(&tm_w, a_addr + kATile / 2, bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
-        } else if (KIND == 1) {
-          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // gate rows
-          tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
+        // weight rows: bf16 straight into the operand tile, or e4m3 into the stage's staging area
+        const uint32_t w_addr = FP8 ? a_addr + a_bytes + b_bytes : a_addr;
+        const uint32_t w_bar = FP8 ? smem_u32(&ctl->raw_full[stage]) : bar;
+        constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
+        if (FP8) {
+          mbar_expect_tx(w_bar, raw_bytes);
+          mbar_expect_tx(bar, b_bytes);
         } else {
-          tma_load_3d(&tm_w, a_addr, bar, kb * kBlockK, it.m0, it.slot);               // down rows
-          if (dual) tma_load_3d(&tm_w, a_addr + kATile, bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
+          mbar_expect_tx(bar, stage_bytes);
+        }
+        if (stacked) {  // tm_w has 64-row boxes here
+          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);                  // 64 gate rows
+          tma_load_3d(&tm_w, w_addr + w_tile / 2, w_bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
+        } else if (KIND == 1) {
+          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);               // gate rows
+          tma_load_3d(&tm_w, w_addr + w_tile, w_bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
+        } else {
+          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);               // down rows
+          if (dual) tma_load_3d(&tm_w, w_addr + w_tile, w_bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
         }
         tma_load_2d(&tm_act, a_addr + a_bytes, bar, kb * kBlockK, it.row0);
         if (++stage == n_stages) {
@@ -357,6 +404,47 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
+  } else if (FP8 && warp >= kConvWarp0) {
+    // ------------------------------------------------------------ fp8 -> bf16 converters
+    // Thread ct owns weight rows ct (and ct + 128 when the stage holds 256): 64 codes in, 128
+    // bytes out, written in the 128-byte-swizzled layout the MMA descriptor describes (the
+    // 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
+    const int ct = (int)threadIdx.x - kConvWarp0 * 32;
+    long n_kb = 0;
+    if ((int)blockIdx.x < total_items && !grp.withhold_loads)
+      n_kb = (long)((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
+    int stage = 0;
+    uint32_t phase = 0;
+    for (long i = 0; i < n_kb; ++i) {
+      int ok = 0;
+      if (lane == 0) ok = mbar_wait(smem_u32(&ctl->raw_full[stage]), phase, abort_flag, status) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      __syncwarp();
+      const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
+      const uint32_t raw_addr = a_addr + a_bytes + b_bytes;
+#pragma unroll
+      for (int rr = ct; rr < (int)(a_bytes / 128u); rr += kConvThreads) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 c = lds128(raw_addr + (uint32_t)rr * 64u + (uint32_t)q * 16u);
+          uint4 lo, hi;
+          e4m3x4_to_bf16x4(c.x, lo.x, lo.y);
+          e4m3x4_to_bf16x4(c.y, lo.z, lo.w);
+          e4m3x4_to_bf16x4(c.z, hi.x, hi.y);
+          e4m3x4_to_bf16x4(c.w, hi.z, hi.w);
+          const uint32_t row_addr = a_addr + (uint32_t)rr * 128u;
+          sts128(row_addr + (uint32_t)(((2 * q) ^ (rr & 7)) * 16), lo);
+          sts128(row_addr + (uint32_t)(((2 * q + 1) ^ (rr & 7)) * 16), hi);
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
+      mbar_arrive(smem_u32(&ctl->full[stage]));
+      if (++stage == n_stages) {
+        stage = 0;
+        phase ^= 1u;
+      }
+    }
   } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
@@ -379,6 +467,22 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * acc_cols);
       const int n_mma = max(16, (it.valid + 15) & ~15);
       const int col = it.m0 + quarter * 32 + lane;  // output feature owned by this thread
+      // fp8 stores: one fp32 scale per weight row behind the codes: s_gate[I] | s_up[I] | s_down[H]
+      const float* sc = FP8 ? reinterpret_cast<const float*>(pool + (size_t)it.slot * slot_bytes + (size_t)3 * H * I)
+                            : nullptr;
+      float s0 = 1.0f, s1 = 1.0f;
+      if (FP8) {
+        if (stacked) {
+          const int f = it.m0 + (quarter & 1) * 32 + lane;
+          s0 = quarter >= 2 ? sc[I + f] : sc[f];  // this thread's row: an up row or a gate row
+        } else if (KIND == 1) {
+          s0 = sc[col];
+          s1 = sc[I + col];
+        } else {
+          s0 = sc[2 * I + col];
+          if (dual) s1 = sc[2 * I + col + kBlockM];
+        }
+      }
       for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
@@ -400,7 +504,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
 #pragma unroll
             for (int j = 0; j < 16; j += 4)
-              *reinterpret_cast<uint4*>(slot + j) = make_uint4(ra[j], ra[j + 1], ra[j + 2], ra[j + 3]);
+              *reinterpret_cast<float4*>(slot + j) =
+                  make_float4(__uint_as_float(ra[j]) * s0, __uint_as_float(ra[j + 1]) * s0,
+                              __uint_as_float(ra[j + 2]) * s0, __uint_as_float(ra[j + 3]) * s0);
             mbar_arrive(smem_u32(&ctl->x_full[buf][half]));
           } else {
             if (lane == 0) ok = mbar_wait(smem_u32(&ctl->x_full[buf][half]), ph, abort_flag, status) ? 1 : 0;
@@ -421,7 +527,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               if (c + j < it.valid) {
-                const float a = __uint_as_float(ra[j]);
+                const float a = __uint_as_float(ra[j]) * s0;
                 const float hm = __fdividef(a, 1.0f + __expf(-a)) * u[j];
                 const __nv_bfloat16 b = __float2bfloat16_rn(hm);
                 hb[(size_t)(it.row0 + c + j) * I + it.m0 + xrow] = *reinterpret_cast<const uint16_t*>(&b);
@@ -436,8 +542,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             if (c + j < it.valid) {
-              const float a = __uint_as_float(ra[j]);
-              const float u = __uint_as_float(rb[j]);
+              const float a = __uint_as_float(ra[j]) * s0;
+              const float u = __uint_as_float(rb[j]) * s1;
               const float hm = __fdividef(a, 1.0f + __expf(-a)) * u;
               const __nv_bfloat16 b = __float2bfloat16_rn(hm);
               hb[(size_t)(it.row0 + c + j) * I + col] = *reinterpret_cast<const uint16_t*>(&b);
@@ -454,15 +560,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             if (c + j < it.valid) {
               const size_t o = (size_t)(it.row0 + c + j) * H + col;
               if (out_bf16) {
-                const __nv_bfloat16 b0 = __float2bfloat16_rn(__uint_as_float(ra[j]));
+                const __nv_bfloat16 b0 = __float2bfloat16_rn(__uint_as_float(ra[j]) * s0);
                 yb[o] = *reinterpret_cast<const uint16_t*>(&b0);
                 if (dual) {
-                  const __nv_bfloat16 b1 = __float2bfloat16_rn(__uint_as_float(rb[j]));
+                  const __nv_bfloat16 b1 = __float2bfloat16_rn(__uint_as_float(rb[j]) * s1);
                   yb[o + kBlockM] = *reinterpret_cast<const uint16_t*>(&b1);
                 }
               } else {
-                y[o] = __uint_as_float(ra[j]);
-                if (dual) y[o + kBlockM] = __uint_as_float(rb[j]);
+                y[o] = __uint_as_float(ra[j]) * s0;
+                if (dual) y[o + kBlockM] = __uint_as_float(rb[j]) * s1;
               }
             }
         }
@@ -503,7 +609,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, const cuuint64_t* strides,
-            const cuuint32_t* box) {
+            const cuuint32_t* box, bool bytes = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint32_t estr[3] = {1, 1, 1};
@@ -514,47 +620,70 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
                    : v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
                              : v == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
   }
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides,
-            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; raw e4m3 rows (64 bytes
+  // per k-block) land row-major in the staging area and are re-laid out by the converter warps
+  return fn(m, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            bytes ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, promo,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int stages_for(bool dual, int n_box) {
+uint32_t stage_bytes_for(bool dual, int n_box, bool fp8) {
+  const uint32_t a = (dual ? 2u : 1u) * kATile;
+  return a + (uint32_t)n_box * 128u + (fp8 ? a / 2 : 0u);
+}
+int stages_for(bool dual, int n_box, bool fp8) {
   static int cap = -1;  // tuning aid: OLED_FFN_STAGES caps the pipeline depth
   if (cap < 0) {
     const char* env = getenv("OLED_FFN_STAGES");
     cap = env ? std::max(1, atoi(env)) : kMaxStages;
   }
-  const uint32_t stage = (dual ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
-  return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage);
+  return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage_bytes_for(dual, n_box, fp8));
 }
-uint32_t smem_for(bool dual, int n_box, int stages) {
-  const uint32_t stage = (dual ? 2u : 1u) * kATile + (uint32_t)n_box * 128u;
-  return kCtlBytes + 1024u + (uint32_t)stages * stage;
+uint32_t smem_for(bool dual, int n_box, bool fp8, int stages) {
+  return kCtlBytes + 1024u + (uint32_t)stages * stage_bytes_for(dual, n_box, fp8);
+}
+
+template <int KIND, bool DUAL, bool FP8>
+bool set_smem_attr() {
+  return cudaFuncSetAttribute(ffn_tc_kernel<KIND, DUAL, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)kSmemMax) == cudaSuccess;
+}
+
+template <int KIND, bool DUAL>
+void launch_variant(bool fp8, int grid, uint32_t smem, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
+                    const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int stages, int out_bf16,
+                    const uint8_t* pool, size_t slot_bytes, uint32_t* status) {
+  if (fp8)
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), smem, st, tw, ta, grp, offsets, out, H, I,
+               stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
+  else
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), smem, st, tw, ta, grp, offsets, out, H, I,
+               stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
 }
 
 }  // namespace
 
-int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I,
+int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows) {
+  maps->fp8 = fp8;
+  maps->pool = pool;
+  maps->slot_bytes = slot_bytes;
+  const cuuint64_t esz = fp8 ? 1 : 2;  // bytes per weight element in the slot pool
   {
     const cuuint64_t dims[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
-    const cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)slot_bytes};
+    const cuuint64_t strides[2] = {(cuuint64_t)H * esz, (cuuint64_t)slot_bytes};
     const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
-    if (!encode(&maps->w13, 3, pool, dims, strides, box)) return OLED_ERR_CUDA;
-  }
-  {  // the same matrix with 64-row boxes (stacked gate/up tiles)
-    const cuuint64_t dims[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
-    const cuuint64_t strides[2] = {(cuuint64_t)H * 2, (cuuint64_t)slot_bytes};
-    const cuuint32_t box[3] = {kBlockK, kBlockM / 2, 1};
-    if (!encode(&maps->w13_half, 3, pool, dims, strides, box)) return OLED_ERR_CUDA;
+    const cuuint32_t box_half[3] = {kBlockK, kBlockM / 2, 1};  // stacked gate/up tiles
+    if (!encode(&maps->w13, 3, pool, dims, strides, box, fp8)) return OLED_ERR_CUDA;
+    if (!encode(&maps->w13_half, 3, pool, dims, strides, box_half, fp8)) return OLED_ERR_CUDA;
   }
   {
     const cuuint64_t dims[3] = {(cuuint64_t)I, (cuuint64_t)H, (cuuint64_t)n_slots};
-    const cuuint64_t strides[2] = {(cuuint64_t)I * 2, (cuuint64_t)slot_bytes};
+    const cuuint64_t strides[2] = {(cuuint64_t)I * esz, (cuuint64_t)slot_bytes};
     const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
-    if (!encode(&maps->w2, 3, pool + (size_t)2 * I * H * 2, dims, strides, box)) return OLED_ERR_CUDA;
+    if (!encode(&maps->w2, 3, pool + (size_t)2 * I * H * esz, dims, strides, box, fp8)) return OLED_ERR_CUDA;
   }
   for (int i = 0; i < 5; ++i) {
     const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(16 << i)};
@@ -571,14 +700,9 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   }
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemMax) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemMax) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemMax) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemMax) != cudaSuccess)
+    if (!set_smem_attr<1, true, false>() || !set_smem_attr<1, false, false>() || !set_smem_attr<2, true, false>() ||
+        !set_smem_attr<2, false, false>() || !set_smem_attr<1, true, true>() || !set_smem_attr<1, false, true>() ||
+        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>())
       return OLED_ERR_CUDA;
     attr_done = true;
   }
@@ -601,50 +725,45 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
                   int n_sms, uint32_t* status) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
+  const bool fp8 = maps.fp8;
   // N <= 128 keeps the accumulators double-buffered in TMEM; more tokens per expert than that
   // take N = 256 with two weight tiles per item (all 512 TMEM columns, one accumulator stage).
-  const int i1 = box_index(max_count, 256), i2 = box_index(max_count, 256);
+  const int ib = box_index(max_count, 256);
+  grp.n_box = 16 << ib;
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
-  auto grid_for = [&](int n_box, int m_tiles) {
+  auto grid_for = [&](int m_tiles) {
     if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
     long long tiles = 0;
-    for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + n_box - 1) / n_box;
+    for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + grp.n_box - 1) / grp.n_box;
     return (int)std::max<long long>(1, std::min<long long>(n_sms, tiles * m_tiles));
   };
-  static int use_stacked = -1;  // tuning aid: OLED_FFN1_STACKED=0 keeps the two-accumulator form
+  static int use_stacked = -1, force_dual = -1;  // tuning aids
   if (use_stacked < 0) {
-    const char* env = getenv("OLED_FFN1_STACKED");
-    use_stacked = env ? atoi(env) : 1;
+    const char* a = getenv("OLED_FFN1_STACKED");  // 0 keeps the two-accumulator form for small token tiles
+    const char* b = getenv("OLED_FFN2_DUAL");     // 1 pairs Wd row blocks at every token tile
+    use_stacked = a ? atoi(a) : 1;
+    force_dual = b ? atoi(b) : 0;
   }
-  if (kind == 1 && (16 << i1) <= 32 && use_stacked == 1) {
-    grp.n_box = 16 << i1;
-    const int stages = stages_for(false, grp.n_box);
-    launch_pdl(ffn_tc_kernel<1, false>, dim3(grid_for(grp.n_box, I / (kBlockM / 2))), dim3(kThreads),
-               smem_for(false, grp.n_box, stages), st, maps.w13_half, maps.xp[i1], grp, offsets, (void*)hbuf, H, I,
-               stages, 0, status);
+  if (kind == 1 && grp.n_box <= 32 && use_stacked == 1) {
+    const int stages = stages_for(false, grp.n_box, fp8);
+    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), smem_for(false, grp.n_box, fp8, stages), st,
+                             maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I, stages, 0, maps.pool,
+                             maps.slot_bytes, status);
   } else if (kind == 1) {
-    grp.n_box = 16 << i1;
-    const int stages = stages_for(true, grp.n_box);
-    launch_pdl(ffn_tc_kernel<1, true>, dim3(grid_for(grp.n_box, I / kBlockM)), dim3(kThreads),
-               smem_for(true, grp.n_box, stages), st, maps.w13, maps.xp[i1], grp, offsets, (void*)hbuf, H, I, stages,
-               0, status);
+    const int stages = stages_for(true, grp.n_box, fp8);
+    launch_variant<1, true>(fp8, grid_for(I / kBlockM), smem_for(true, grp.n_box, fp8, stages), st, maps.w13,
+                            maps.xp[ib], grp, offsets, hbuf, H, I, stages, 0, maps.pool, maps.slot_bytes, status);
   } else {
-    grp.n_box = 16 << i2;
-    static int force_dual = -1;  // tuning aid: OLED_FFN2_DUAL=1 pairs Wd row blocks at every token tile
-    if (force_dual < 0) {
-      const char* env = getenv("OLED_FFN2_DUAL");
-      force_dual = env ? atoi(env) : 0;
-    }
     const bool dual = grp.n_box == 256 || force_dual == 1;
-    const int stages = stages_for(dual, grp.n_box);
+    const int stages = stages_for(dual, grp.n_box, fp8);
     if (dual)
-      launch_pdl(ffn_tc_kernel<2, true>, dim3(grid_for(grp.n_box, H / (2 * kBlockM))), dim3(kThreads),
-                 smem_for(true, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages, y_bf16,
-                 status);
+      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), smem_for(true, grp.n_box, fp8, stages), st, maps.w2,
+                              maps.hbuf[ib], grp, offsets, y, H, I, stages, y_bf16, maps.pool, maps.slot_bytes,
+                              status);
     else
-      launch_pdl(ffn_tc_kernel<2, false>, dim3(grid_for(grp.n_box, H / kBlockM)), dim3(kThreads),
-                 smem_for(false, grp.n_box, stages), st, maps.w2, maps.hbuf[i2], grp, offsets, (void*)y, H, I, stages,
-                 y_bf16, status);
+      launch_variant<2, false>(fp8, grid_for(H / kBlockM), smem_for(false, grp.n_box, fp8, stages), st, maps.w2,
+                               maps.hbuf[ib], grp, offsets, y, H, I, stages, y_bf16, maps.pool, maps.slot_bytes,
+                               status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

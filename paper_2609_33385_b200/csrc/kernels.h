@@ -102,9 +102,12 @@ struct FfnTcMaps {
   CUtensorMap w2;        // [slots][H][I]  bf16, box {64,128,1}
   CUtensorMap xp[5];     // [rows][H] bf16, box {64, 16<<i}
   CUtensorMap hbuf[5];   // [rows][I] bf16, box {64, 16<<i}
+  bool fp8 = false;      // slots hold fp8 blobs: the weight maps are byte maps over the e4m3 codes
+  const uint8_t* pool = nullptr;
+  size_t slot_bytes = 0;
 };
 // Builds the tensor maps; returns 0 or a negative oled_status.
-int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I,
+int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,

@@ -307,6 +307,13 @@ int wait_gate_report(oled_ctx* ctx) {
 
 extern "C" {
 
+size_t oled_expert_blob_bytes(int32_t hidden, int32_t intermediate, int32_t expert_format) {
+  const size_t hi = (size_t)hidden * (size_t)intermediate;
+  if (expert_format == OLED_EXPERTS_FP8)
+    return (3 * hi + 4 * (2 * (size_t)intermediate + (size_t)hidden) + 255) / 256 * 256;
+  return 3 * hi * 2;
+}
+
 const char* oled_strerror(int code) {
   switch (code) {
     case OLED_OK: return "ok";
@@ -331,7 +338,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   if (s.n_layers <= 0 || s.hidden <= 0 || s.hidden % 256 != 0 || s.intermediate <= 0 ||
       s.intermediate % 128 != 0 || s.n_experts <= 0 || s.n_experts > OLED_MAX_EXPERTS || s.top_k <= 0 ||
       s.top_k > OLED_MAX_TOPK || s.top_k > s.n_experts || s.max_tokens <= 0 || s.max_tokens > 65535 ||
-      s.staging_slots < 0)
+      s.staging_slots < 0 || (s.expert_format != OLED_EXPERTS_BF16 && s.expert_format != OLED_EXPERTS_FP8))
     return OLED_ERR_INVALID_ARG;
   int min_cap = s.n_experts;
   long long total_cap = 0;
@@ -369,7 +376,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   }
 
   const int staging = s.staging_slots > 0 ? s.staging_slots : (s.n_experts - min_cap);
-  ctx->slot_bytes = (size_t)3 * s.hidden * s.intermediate * 2;
+  ctx->slot_bytes = oled_expert_blob_bytes(s.hidden, s.intermediate, s.expert_format);
   ctx->n_slots = (int)std::min<long long>(total_cap + staging, 65535);
   if (total_cap + staging > 65535) return fail(OLED_ERR_INVALID_ARG);
   ctx->slots.init(ctx->n_slots);
@@ -418,10 +425,12 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
       cudaMemset(ctx->d_hbuf, 0, T * K * I * 2) != cudaSuccess ||
       cudaMemset(ctx->d_y, 0, T * K * H * 4) != cudaSuccess)
     return fail(OLED_ERR_CUDA);
-  rc = ffn_tc_setup(&ctx->maps, ctx->pool, ctx->slot_bytes, ctx->n_slots, s.hidden, s.intermediate, ctx->d_xp,
+  rc = ffn_tc_setup(&ctx->maps, ctx->pool, ctx->slot_bytes, ctx->n_slots, s.hidden, s.intermediate,
+                    s.expert_format == OLED_EXPERTS_FP8, ctx->d_xp,
                     ctx->d_hbuf, (int)(T * K));
   if (rc != OLED_OK) return fail(rc);
-  if (const char* env = getenv("OLED_FFN_IMPL")) ctx->ffn_impl = atoi(env) == 1 ? 1 : 0;
+  if (const char* env = getenv("OLED_FFN_IMPL"))
+    ctx->ffn_impl = (atoi(env) == 1 && s.expert_format == OLED_EXPERTS_BF16) ? 1 : 0;
   if (const char* env = getenv("OLED_MISS_CHUNK")) ctx->miss_chunk = std::max(1, atoi(env));
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(OLED_ERR_CUDA);
   *out_ctx = ctx;
@@ -793,6 +802,7 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
   switch (option) {
     case OLED_OPT_FFN_IMPL:
       if (value != 0 && value != 1) return OLED_ERR_INVALID_ARG;
+      if (value == 1 && ctx->shape.expert_format != OLED_EXPERTS_BF16) return OLED_ERR_INVALID_ARG;
       ctx->ffn_impl = (int)value;
       return OLED_OK;
     case OLED_OPT_PROFILE:

@@ -10,13 +10,14 @@ layers of this MoE-only stack is x_{l+1} = bf16(x_l + out_l).
 from __future__ import annotations
 
 import os
+from concurrent.futures import ThreadPoolExecutor
 from typing import List, Optional, Sequence
 
 import numpy as np
 import torch
 
 from . import synth
-from .binding import (OPT_ADAPT_PERIOD, OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_POLICY, POLICY_IDS,
+from .binding import (EXPERTS_BF16, EXPERTS_FP8, OPT_ADAPT_PERIOD, OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_POLICY, POLICY_IDS,
                       OledContext)
 
 
@@ -37,7 +38,7 @@ class StackRunner:
                  gen_threads: Optional[int] = None, ffn_impl: Optional[int] = None,
                  miss_chunk: Optional[int] = None, max_tokens: Optional[int] = None,
                  staging_slots: int = 0, share_store_of: Optional["StackRunner"] = None,
-                 policy: Optional[str] = None, adapt_period: Optional[int] = None):
+                 policy: Optional[str] = None, adapt_period: Optional[int] = None, fp8: bool = False):
         self.w = w
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -47,7 +48,9 @@ class StackRunner:
         self.stream = torch.cuda.current_stream(self.device)
         self.ctx = OledContext(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate,
                                self.max_tokens, caps, self.stream.cuda_stream,
-                               has_router_bias=w.has_bias, staging_slots=staging_slots)
+                               has_router_bias=w.has_bias, staging_slots=staging_slots,
+                               expert_format=EXPERTS_FP8 if fp8 else EXPERTS_BF16)
+        self.fp8 = fp8
         if ffn_impl is not None:
             self.ctx.set_option(OPT_FFN_IMPL, ffn_impl)
         if miss_chunk is not None:
@@ -67,9 +70,18 @@ class StackRunner:
             self._host_t = share_store_of._host_t
             self.blobs = share_store_of.blobs
         for d in range(0 if share_store_of is not None else n_distinct):
-            t = torch.empty((w.n_experts, w.expert_elems), dtype=torch.int16, pin_memory=True)
-            a = t.numpy().view(np.uint16)
-            synth.fill_layer_blobs(w, d, a, threads=threads)
+            if fp8:   # bf16 weights are generated, then quantised row by row into the pinned fp8 store
+                nb = synth.fp8_blob_bytes(w)
+                t = torch.zeros((w.n_experts, nb), dtype=torch.uint8, pin_memory=True)
+                a = t.numpy()
+                def one(e, d=d, a=a):
+                    synth.quantize_expert_blob(w, synth.expert_blob_bits(w, d, e), a[e])
+                with ThreadPoolExecutor(max_workers=max(1, threads)) as ex:
+                    list(ex.map(one, range(w.n_experts)))
+            else:
+                t = torch.empty((w.n_experts, w.expert_elems), dtype=torch.int16, pin_memory=True)
+                a = t.numpy().view(np.uint16)
+                synth.fill_layer_blobs(w, d, a, threads=threads)
             self._host_t.append(t)
             self.blobs.append(a)
         self.router_bits: List[np.ndarray] = []
@@ -84,7 +96,7 @@ class StackRunner:
             self._router_dev.append((wr_d, b_d))
             self.ctx.register_router(l, wr_d.data_ptr(), None if b_d is None else b_d.data_ptr())
             ht = self._host_t[l % n_distinct]
-            self.ctx.register_experts(l, ht.data_ptr(), w.expert_bytes)
+            self.ctx.register_experts(l, ht.data_ptr(), self.ctx.expert_bytes)
 
     def layer_blobs(self, layer: int) -> np.ndarray:
         return self.blobs[layer % self.n_distinct]

@@ -250,27 +250,19 @@ def flat_tokens(w: Workload, n_tokens: int, stream_id: int = 0) -> Tuple[np.ndar
 # --------------------------------------------------------------------------
 # Narrow expert blobs: fp8 (e4m3) weights with one fp32 scale per output row
 # --------------------------------------------------------------------------
-def _e4m3_positive_values() -> np.ndarray:
-    """The 127 finite non-negative e4m3 values in code order (code 0x00..0x7E)."""
-    vals = []
-    for code in range(0x7F):
-        e, m = code >> 3, code & 7
-        vals.append(m * 2.0 ** -9 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
-    return np.array(vals, dtype=np.float64)
-
-
-_E4M3_POS = _e4m3_positive_values()
-
-
 def f32_to_e4m3_codes(x: np.ndarray) -> np.ndarray:
     """Round to the nearest e4m3 value (ties to the even code), saturating at +-448."""
-    a = np.minimum(np.abs(np.asarray(x, dtype=np.float64)), 448.0)
-    hi = np.clip(np.searchsorted(_E4M3_POS, a, side="left"), 0, 126)
-    lo = np.maximum(hi - 1, 0)
-    d_hi, d_lo = _E4M3_POS[hi] - a, a - _E4M3_POS[lo]
-    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
-    code = np.where(pick_hi, hi, lo).astype(np.uint8)
-    return code | (np.signbit(x).astype(np.uint8) << 7)
+    xf = np.asarray(x, dtype=np.float64)
+    a = np.minimum(np.abs(xf), 448.0)
+    _, ex = np.frexp(a)                                   # a = m * 2^ex, m in [0.5, 1)
+    qe = np.maximum(ex - 1, -6) - 3                       # exponent of the rounding quantum
+    v = np.rint(np.ldexp(a, -qe))                         # 0..16 quanta, ties to even
+    val = np.ldexp(v, qe)                                 # the rounded magnitude (may reach the next binade)
+    _, ex2 = np.frexp(val)
+    e_field = np.where(val < 2.0 ** -6, 0, ex2 - 1 + 7)
+    m_field = np.where(val < 2.0 ** -6, np.ldexp(val, 9), (np.ldexp(val, -(ex2 - 1)) - 1.0) * 8.0)
+    code = (e_field.astype(np.int64) << 3 | m_field.astype(np.int64)).astype(np.uint8)
+    return code | (np.signbit(xf).astype(np.uint8) << 7)
 
 
 def fp8_blob_bytes(w: Workload) -> int:

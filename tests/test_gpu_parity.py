@@ -30,7 +30,10 @@ def _oracle_for(run, caps, policy="priority"):
     st = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, caps, policy=policy)
     for l in range(w.n_layers):
         st.register_router(l, run.router_bits[l], run.bias[l])
-        st.register_experts(l, run.layer_blobs(l))
+        if getattr(run, "fp8", False):
+            st.register_experts_fp8(l, run.layer_blobs(l))
+        else:
+            st.register_experts(l, run.layer_blobs(l))
     return st
 
 
@@ -423,5 +426,38 @@ def test_degenerate_routing_cases():
         ref = ora.denoise_step(0, same, conf)
         assert sorted(ref["counts"].tolist())[-2:] == [300, 300] and ref["counts"].sum() == 600
         _check_step(run, 0, 300, out, ref)
+    finally:
+        run.close()
+
+
+def test_fp8_expert_store_tiny_stack():
+    """fp8 (e4m3 + row scales) expert blobs: same discrete results, outputs within the same
+    tolerance of the oracle evaluated on the dequantised weights, half the bytes moved."""
+    w = synth.tiny(blocks=2, iters=3)
+    run = _runner(w, capacity=[3, 5], fp8=True)
+    try:
+        ora = _oracle_for(run, [3, 5])
+        _run_stack(run, ora)
+        st = run.ctx.stats()
+        assert st.bytes_moved == st.misses * synth.fp8_blob_bytes(w)
+        assert synth.fp8_blob_bytes(w) < 0.55 * w.expert_bytes
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("n", [40, 300, 700])
+def test_fp8_expert_store_token_tile_variants(n):
+    """fp8 blobs through every FFN tile form: stacked (few tokens), two accumulators (up to 128
+    tokens per expert) and the 256-token form with two weight tiles per item."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    run = _runner(w, capacity=[4], max_tokens=n, fp8=True)
+    ora = _oracle_for(run, [4])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 50)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        _check_step(run, 0, n, out, ora.denoise_step(0, h_bits, conf))
     finally:
         run.close()
