@@ -27,8 +27,8 @@
 // warps 18-21 widen fp8 weight tiles (fp8 expert stores only, idle otherwise).
 //
 // fp8 expert stores (e4m3 codes + one fp32 scale per weight row): TMA brings the raw 64-byte
-// rows into a staging area of the stage, the converter warps write them as bf16 (exact) into the
-// swizzled operand tile, the MMA runs in bf16 as before and the epilogue multiplies each output
+// rows into the second half of the stage's operand-tile region, the converter warps rewrite them
+// in place as bf16 (exact) in the swizzled operand layout, the MMA runs in bf16 as before and the epilogue multiplies each output
 // row by its scale - the rows of a weight tile are the accumulator's lanes.  Every mbarrier
 // wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
 // copies time to land, frees its TMEM and returns.
@@ -52,7 +52,6 @@ constexpr int kEpiWarps = OLED_EPI_WARPS;  // up to four warps per TMEM lane qua
 constexpr int kProducerWarp = kEpiWarps;
 constexpr int kMmaWarp = kEpiWarps + 1;
 constexpr int kConvWarp0 = kEpiWarps + 2;     // four warps that widen fp8 weight tiles to bf16 (fp8 stores only)
-constexpr int kConvThreads = 128;
 constexpr int kThreads = (kEpiWarps + 6) * 32;
 constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
@@ -202,18 +201,23 @@ __device__ __forceinline__ void sts128(uint32_t addr, const uint4& v) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                : "memory");
 }
-// Two e4m3 codes (low byte first) -> two bf16 (exact: e4m3 fits bf16's exponent and mantissa).
-__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t two_codes) {
-  uint32_t h2;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)two_codes));
-  const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
-  const __nv_bfloat162 b = __floats2bfloat162_rn(f.x, f.y);
-  return *reinterpret_cast<const uint32_t*>(&b);
+// Two e4m3 codes (low byte first) -> two bf16, exactly, without the conversion unit: the code's
+// exponent and mantissa bits are placed in a bf16 whose exponent field is the code's (bias 7
+// instead of 127, and for exponent field 0 a bf16 subnormal 0.mmm * 2^-126), so multiplying by
+// 2^120 gives the code's value in both cases (2^(e-7) * 1.mmm, or 0.mmm * 2^-6).  Four integer
+// operations and one packed multiply per two codes.
+__device__ __forceinline__ uint32_t e4m3x2_hi_bytes_to_bf16x2(uint32_t a) {
+  // a holds one code in the top byte of each 16-bit half (sign already at bit 15 / 31)
+  const uint32_t bits = (a & 0x80008000u) | ((a >> 4) & 0x07F007F0u);
+  const uint32_t two_pow_120 = 0x7B807B80u;  // bf16 2^120 in both halves
+  const __nv_bfloat162 r = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&bits),
+                                   *reinterpret_cast<const __nv_bfloat162*>(&two_pow_120));
+  return *reinterpret_cast<const uint32_t*>(&r);
 }
-// Four codes in one 32-bit word -> four bf16 in two words.
+// Four codes in one 32-bit word (lowest byte first) -> four bf16 in two words.
 __device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
-  lo = e4m3x2_to_bf16x2(w & 0xffffu);
-  hi = e4m3x2_to_bf16x2(w >> 16);
+  lo = e4m3x2_hi_bytes_to_bf16x2(__byte_perm(w, 0u, 0x1404u));  // (b1 << 24) | (b0 << 8)
+  hi = e4m3x2_hi_bytes_to_bf16x2(__byte_perm(w, 0u, 0x3424u));  // (b3 << 24) | (b2 << 8)
 }
 
 struct Item {
@@ -251,8 +255,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t b_bytes = (uint32_t)n_box * 128u;
-  constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;  // staging of the stage's e4m3 rows
-  const uint32_t stage_bytes = a_bytes + b_bytes + raw_bytes;
+  // fp8 stores: the stage's e4m3 rows land in the SECOND HALF of the operand-tile region and are
+  // widened in place (see the converter warps), so a stage is as large as in the bf16 case
+  constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
@@ -261,6 +267,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
   const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+  // fp8 stores: the four dedicated converter warps plus the epilogue warps this token tile leaves idle
+  // (never more converters than pipeline stages: a converter owns stages)
+  const int n_conv = FP8 ? min(4 + (kEpiWarps - epi_warps), n_stages) : 0;
+  int conv_id = !FP8 ? -1
+                : warp >= kConvWarp0 ? warp - kConvWarp0
+                : (warp >= epi_warps && warp < kEpiWarps) ? 4 + (warp - epi_warps) : -1;
+  if (conv_id >= n_conv) conv_id = -2;  // a spare warp: neither converter nor epilogue
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
 
@@ -268,7 +281,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 1u + kConvThreads : 1u);  // token tile (+ converters)
+      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 1u + 32u : 1u);  // token tile (+ the converting warp)
       mbar_init(smem_u32(&ctl->empty[s]), 1);
       mbar_init(smem_u32(&ctl->raw_full[s]), 1);
     }
@@ -332,8 +345,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
         const uint32_t bar = smem_u32(&ctl->full[stage]);
         const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-        // weight rows: bf16 straight into the operand tile, or e4m3 into the stage's staging area
-        const uint32_t w_addr = FP8 ? a_addr + a_bytes + b_bytes : a_addr;
+        // weight rows: bf16 straight into the operand tile, or e4m3 into its second half
+        const uint32_t w_addr = FP8 ? a_addr + raw_bytes : a_addr;
         const uint32_t w_bar = FP8 ? smem_u32(&ctl->raw_full[stage]) : bar;
         constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
         if (FP8) {
@@ -404,48 +417,55 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
-  } else if (FP8 && warp >= kConvWarp0) {
+  } else if (conv_id >= 0) {
     // ------------------------------------------------------------ fp8 -> bf16 converters
-    // Thread ct owns weight rows ct (and ct + 128 when the stage holds 256): 64 codes in, 128
-    // bytes out, written in the 128-byte-swizzled layout the MMA descriptor describes (the
-    // 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
-    const int ct = (int)threadIdx.x - kConvWarp0 * 32;
+    // Every converter warp widens whole stages, so that several stages are in conversion at once (one stage is a chain of shared
+    // loads, integer work, shared stores and a proxy fence).  Lane l owns weight rows l, l + 32,
+    // ...: 64 codes in, 128 bytes out, written in the 128-byte-swizzled layout the MMA descriptor
+    // describes (the 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
     long n_kb = 0;
     if ((int)blockIdx.x < total_items && !grp.withhold_loads)
       n_kb = (long)((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
-    int stage = 0;
-    uint32_t phase = 0;
+    // A converter warp owns pipeline STAGES (stage s belongs to warp s mod n_conv) and walks its
+    // k-blocks in order: it reaches round r of a stage only after it finished round r-1 of the same
+    // stage, so the parity wait below can never mistake an older phase for the one it wants.
     for (long i = 0; i < n_kb; ++i) {
+      const int stage = (int)(i % n_stages);
+      if (stage % n_conv != conv_id) continue;
+      const uint32_t phase = (uint32_t)(i / n_stages) & 1u;
       int ok = 0;
       if (lane == 0) ok = mbar_wait(smem_u32(&ctl->raw_full[stage]), phase, abort_flag, status) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       __syncwarp();
       const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-      const uint32_t raw_addr = a_addr + a_bytes + b_bytes;
+      const uint32_t raw_addr = a_addr + raw_bytes;
+      // In place: code row r sits at raw_addr + 64 r, its bf16 form goes to a_addr + 128 r.  Rows
+      // are taken in ascending waves of 32 (one per lane); a wave reads its codes into registers
+      // before it writes, and what it overwrites are code rows <= its own, already consumed.
+      for (int r0 = 0; r0 < (int)(a_bytes / 128u); r0 += 32) {
+        const int rr = r0 + lane;
+        uint4 c[4];
 #pragma unroll
-      for (int rr = ct; rr < (int)(a_bytes / 128u); rr += kConvThreads) {
+        for (int q = 0; q < 4; ++q) c[q] = lds128(raw_addr + (uint32_t)rr * 64u + (uint32_t)q * 16u);
+        __syncwarp();
+        const uint32_t row_addr = a_addr + (uint32_t)rr * 128u;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const uint4 c = lds128(raw_addr + (uint32_t)rr * 64u + (uint32_t)q * 16u);
           uint4 lo, hi;
-          e4m3x4_to_bf16x4(c.x, lo.x, lo.y);
-          e4m3x4_to_bf16x4(c.y, lo.z, lo.w);
-          e4m3x4_to_bf16x4(c.z, hi.x, hi.y);
-          e4m3x4_to_bf16x4(c.w, hi.z, hi.w);
-          const uint32_t row_addr = a_addr + (uint32_t)rr * 128u;
+          e4m3x4_to_bf16x4(c[q].x, lo.x, lo.y);
+          e4m3x4_to_bf16x4(c[q].y, lo.z, lo.w);
+          e4m3x4_to_bf16x4(c[q].z, hi.x, hi.y);
+          e4m3x4_to_bf16x4(c[q].w, hi.z, hi.w);
           sts128(row_addr + (uint32_t)(((2 * q) ^ (rr & 7)) * 16), lo);
           sts128(row_addr + (uint32_t)(((2 * q + 1) ^ (rr & 7)) * 16), hi);
         }
+        __syncwarp();
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
       mbar_arrive(smem_u32(&ctl->full[stage]));
-      if (++stage == n_stages) {
-        stage = 0;
-        phase ^= 1u;
-      }
     }
-  } else if (warp < epi_warps) {
+  } else if (warp < epi_warps && conv_id == -1) {
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
     int g = 0, local = 0;
@@ -629,8 +649,9 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
 }
 
 uint32_t stage_bytes_for(bool dual, int n_box, bool fp8) {
+  (void)fp8;  // fp8 rows are widened in place: same stage size as bf16
   const uint32_t a = (dual ? 2u : 1u) * kATile;
-  return a + (uint32_t)n_box * 128u + (fp8 ? a / 2 : 0u);
+  return a + (uint32_t)n_box * 128u;
 }
 int stages_for(bool dual, int n_box, bool fp8) {
   static int cap = -1;  // tuning aid: OLED_FFN_STAGES caps the pipeline depth

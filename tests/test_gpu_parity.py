@@ -461,3 +461,31 @@ def test_fp8_expert_store_token_tile_variants(n):
         _check_step(run, 0, n, out, ora.denoise_step(0, h_bits, conf))
     finally:
         run.close()
+
+
+def test_fp8_subnormal_codes_decode_exactly():
+    """Blobs whose row scales are so large that every code is an e4m3 subnormal (exponent field
+    0): the on-chip widening must reproduce them exactly, not flush them."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=256, intermediate=128)
+    run = _runner(w, capacity=[4], max_tokens=24, fp8=True)
+    try:
+        h, i = w.hidden, w.intermediate
+        rng = np.random.default_rng(77)
+        for e in range(w.n_experts):
+            blob = run.blobs[0][e]
+            codes = (rng.integers(0, 8, size=3 * h * i).astype(np.uint8) |
+                     (rng.integers(0, 2, size=3 * h * i).astype(np.uint8) << 7))     # +-{0..7} * 2^-9
+            blob[:3 * h * i] = codes
+            scales = rng.uniform(2.0, 6.0, size=2 * i + h).astype(np.float32)
+            blob[3 * h * i:3 * h * i + 4 * scales.size] = scales.view(np.uint8)
+        ora = _oracle_for(run, [4])
+        h_bits, conf = synth.flat_tokens(w, 24, 60)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((24, h), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        ref = ora.denoise_step(0, h_bits, conf)
+        assert np.abs(ref["out"]).max() > 1e-3                 # the subnormal codes carry the whole signal
+        _check_step(run, 0, 24, out, ref)
+    finally:
+        run.close()
