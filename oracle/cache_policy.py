@@ -63,7 +63,8 @@ def reuse_scores(ids: np.ndarray, gate: np.ndarray, conf: np.ndarray, n_experts:
     for tt in range(t):
         for j in range(k):
             v = F32(gate[tt, j] * w[tt])                 # one rounded fp32 product
-            q = int(np.floor(np.float64(v) * 4294967296.0))   # exact scaling, then floor
+            # exact scaling, then floor; a NaN product (non-finite activations) adds nothing
+            q = 0 if v != v else int(np.floor(np.float64(v) * 4294967296.0))
             s[int(ids[tt, j])] += q
     return s
 

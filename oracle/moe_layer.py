@@ -131,9 +131,13 @@ def topk_route(logits: np.ndarray, k: int):
     Order: logit descending, ties to the lower expert index; rank 0 is the
     largest.  Scores: z_j = exp_spec(L_j - L_0), S = ((z_0+z_1)+z_2)+...,
     g_j = z_j / S, every operation a rounded fp32 operation.
+    A NaN logit is read as -inf (the paper does not say what a router does
+    with non-finite activations; this keeps the order total, so the k ids of
+    a token stay distinct).
     Returns ids [T,k] int32 and g [T,k] fp32.
     """
     logits = np.asarray(logits, dtype=F32)
+    logits = np.where(np.isnan(logits), F32(-np.inf), logits).astype(F32)
     t, e = logits.shape
     assert 1 <= k <= e
     ids = np.empty((t, k), dtype=np.int32)

@@ -354,3 +354,24 @@ def test_fp8_layer_matches_layer_on_dequantised_weights():
             a = g @ xf[t]
             acc += float(res["gate"][t, j]) * (d @ (a / (1 + np.exp(-a)) * (u @ xf[t])))
         assert np.allclose(res["out"][t], acc, rtol=1e-10, atol=1e-13)
+
+
+def test_nan_logit_ranks_below_every_number_and_ids_stay_distinct():
+    """Non-finite activations: a NaN logit is read as -inf, so the order is total; the ids of a
+    token are distinct, NaN entries come last and among themselves in index order."""
+    logits = np.array([[np.nan, 1.0, np.nan, -3.0, 2.0],
+                       [np.nan, np.nan, np.nan, np.nan, np.nan],
+                       [np.inf, 0.0, -np.inf, np.nan, 5.0]], dtype=np.float32)
+    with np.errstate(all="ignore"):
+        ids, g = om.topk_route(logits, 4)
+    assert ids.tolist() == [[4, 1, 3, 0], [0, 1, 2, 3], [0, 4, 1, 2]]
+    assert g[0, 3] == 0.0 and np.isclose(g[0, :3].sum(), 1.0)       # exp_spec(-inf) is 0
+    assert np.isnan(g[1]).all()                                       # -inf - -inf
+    assert np.isnan(g[2]).all()                                       # inf - inf poisons the sum
+
+
+def test_nan_reuse_score_adds_nothing():
+    from oracle import cache_policy as P
+    ids = np.array([[0, 1]], dtype=np.int32)
+    gate = np.array([[np.nan, 0.5]], dtype=np.float32)
+    assert P.reuse_scores(ids, gate, np.array([1.0], np.float32), 2) == [0, 2 ** 31]
