@@ -21,17 +21,21 @@
 // one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
 // which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
 //
-// Warp roles (576 threads): warps 0-15 epilogue (TMEM lane quarter = warp id mod 4, the warps of
+// Warp roles (704 threads): warps 0-15 epilogue (TMEM lane quarter = warp id mod 4, the warps of
 // a quarter interleave 16-column chunks; only as many as the token tile has chunks are active),
 // warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation),
 // warps 18-21 widen fp8 weight tiles (fp8 expert stores only, idle otherwise).
 //
-// fp8 expert stores (e4m3 codes + one fp32 scale per weight row): TMA brings the raw 64-byte
-// rows into the second half of the stage's operand-tile region, the converter warps rewrite them
-// in place as bf16 (exact) in the swizzled operand layout, the MMA runs in bf16 as before and the epilogue multiplies each output
-// row by its scale - the rows of a weight tile are the accumulator's lanes.  Every mbarrier
-// wait is bounded: on a timeout the CTA raises a flag in the status word, gives in-flight
-// copies time to land, frees its TMEM and returns.
+// fp8 expert stores (e4m3 codes + one fp32 scale per weight row) use TWO rings in shared memory:
+// a deep ring of load slots - the raw code tile of a k-block (64 bytes per weight row) next to
+// its token tile - that the producer keeps full, which is what hides the HBM latency at half the
+// bytes per tile of the bf16 form, and a short ring of bf16 weight-operand stages.  Groups of
+// converter warps widen a slot's codes into a free operand stage (exact, in the swizzled layout
+// the MMA descriptor describes); the MMA reads the weights from the stage and the tokens from the
+// slot, runs in bf16 as before, and its completion frees both; the epilogue multiplies each
+// output row by its scale - the rows of a weight tile are the accumulator's lanes.  Every mbarrier wait is bounded: on a
+// timeout the CTA raises a flag in the status word, gives in-flight copies time to land, frees
+// its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -48,6 +52,15 @@ namespace {
 #ifndef OLED_EPI_WARPS
 #define OLED_EPI_WARPS 16
 #endif
+#ifndef OLED_NAP_EPI  // nanoseconds between polls, fp8 form: epilogue, TMA producers, converters
+#define OLED_NAP_EPI 128
+#endif
+#ifndef OLED_NAP_LOAD
+#define OLED_NAP_LOAD 64
+#endif
+#ifndef OLED_NAP_CONV
+#define OLED_NAP_CONV 32
+#endif
 constexpr int kEpiWarps = OLED_EPI_WARPS;  // up to four warps per TMEM lane quarter, interleaving 16-column chunks
 constexpr int kProducerWarp = kEpiWarps;
 constexpr int kMmaWarp = kEpiWarps + 1;
@@ -57,13 +70,15 @@ constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
 constexpr uint32_t kATile = kBlockM * kBlockK * 2;
 constexpr int kMaxStages = 10;
+constexpr int kMaxRaw = 16;  // fp8 stores: depth limit of the ring of load slots
 constexpr uint32_t kSmemMax = 232448;  // 227 KB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct __align__(16) SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
-  unsigned long long raw_full[kMaxStages];  // fp8 stores: the raw weight rows of the stage have landed
+  unsigned long long slot_full[kMaxRaw];   // fp8 stores: the slot's code tile and token tile have landed
+  unsigned long long slot_empty[kMaxRaw];  // fp8 stores: the MMAs that read the slot's token tile are done
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long x_full[2][2];   // stacked gate/up mode: [buffer][chunk group], up rows -> gate rows
@@ -112,12 +127,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return done != 0;
 }
-// Bounded wait.  Returns false if the CTA is aborting or the time limit ran out.
+// Bounded wait.  Returns false if the CTA is aborting or the time limit ran out.  sleep_ns > 0:
+// the thread sleeps between polls, leaving the issue slots to the warps that have work (the fp8
+// converters share their schedulers with every polling warp).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* status) {
+                                          uint32_t* status, uint32_t sleep_ns = 0) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 1023u) == 1023u) {
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
@@ -242,7 +260,7 @@ template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
-              void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int n_raw, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -255,10 +273,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t b_bytes = (uint32_t)n_box * 128u;
-  // fp8 stores: the stage's e4m3 rows land in the SECOND HALF of the operand-tile region and are
-  // widened in place (see the converter warps), so a stage is as large as in the bf16 case
+  // bf16 stores: a stage holds the weight tile(s) and the token tile of a k-block.  fp8 stores: a
+  // stage holds the widened weight tile(s) only; behind the n_stages stages sits the ring of n_raw
+  // load slots, each the code tile (one byte per element) followed by the token tile.
   constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const uint32_t stage_bytes = FP8 ? a_bytes : a_bytes + b_bytes;
+  const uint32_t slot_ring_bytes = raw_bytes + b_bytes;
+  const uint32_t raw_base = tiles_base + (uint32_t)n_stages * stage_bytes;
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
@@ -267,13 +288,18 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
   const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
-  // fp8 stores: the four dedicated converter warps plus the epilogue warps this token tile leaves idle
-  // (never more converters than pipeline stages: a converter owns stages)
-  const int n_conv = FP8 ? min(4 + (kEpiWarps - epi_warps), n_stages) : 0;
+  // fp8 stores: the four dedicated converter warps plus the epilogue warps this token tile leaves
+  // idle (4, 12 or 16 warps) form conv_groups groups of conv_width warps.  Group g owns the
+  // k-blocks i with i mod conv_groups == g; conv_groups divides both ring depths, so every raw
+  // slot and every operand stage belongs to ONE group, which visits the rounds of its barriers in
+  // order - a parity wait can then never take an older phase for the one it wants.
+  const int n_conv = FP8 ? 4 + (kEpiWarps - epi_warps) : 0;
+  int conv_groups = n_conv >= 16 ? 4 : n_conv >= 12 ? 2 : 1;
+  while (conv_groups > 1 && (n_stages % conv_groups != 0 || n_raw % conv_groups != 0)) conv_groups >>= 1;
+  const int conv_width = FP8 ? n_conv / conv_groups : 1;
   int conv_id = !FP8 ? -1
-                : warp >= kConvWarp0 ? warp - kConvWarp0
+                : (warp >= kConvWarp0 && warp < kConvWarp0 + 4) ? warp - kConvWarp0
                 : (warp >= epi_warps && warp < kEpiWarps) ? 4 + (warp - epi_warps) : -1;
-  if (conv_id >= n_conv) conv_id = -2;  // a spare warp: neither converter nor epilogue
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
 
@@ -281,9 +307,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 1u + 32u : 1u);  // token tile (+ the converting warp)
+      // the stage's TMA transaction, or every lane of the converting group
+      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 32u * (uint32_t)conv_width : 1u);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
-      mbar_init(smem_u32(&ctl->raw_full[s]), 1);
+    }
+    for (int s = 0; s < kMaxRaw; ++s) {
+      mbar_init(smem_u32(&ctl->slot_full[s]), 1);
+      mbar_init(smem_u32(&ctl->slot_empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
@@ -326,47 +356,47 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
 
+  // polling back-off of the fp8 form, by role (the MMA thread never sleeps)
+  constexpr uint32_t nap_epi = FP8 ? OLED_NAP_EPI : 0u, nap_load = FP8 ? OLED_NAP_LOAD : 0u,
+                     nap_conv = FP8 ? OLED_NAP_CONV : 0u;
   const uint32_t tmem_base = ctl->tmem_base;
   const int total_items = ctl->n_tiles_total * m_tiles;
   volatile int* abort_flag = &ctl->abort;
 
   if (warp == kProducerWarp && lane == 0) {
     // ------------------------------------------------------------ TMA producer
+    // bf16 stores: weight rows and token tile of a k-block go to one operand stage; fp8 stores:
+    // code rows and token tile go to one load slot
     int stage = 0, g = 0;
     uint32_t phase = 0;
     bool ok = true;
+    const int ring = FP8 ? n_raw : n_stages;
     for (int item = blockIdx.x; ok && !grp.withhold_loads && item < total_items; item += gridDim.x) {
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status)) {
+        const uint32_t free_bar = smem_u32(FP8 ? &ctl->slot_empty[stage] : &ctl->empty[stage]);
+        if (!mbar_wait(free_bar, phase ^ 1u, abort_flag, status, nap_load)) {
           ok = false;
           break;
         }
-        const uint32_t bar = smem_u32(&ctl->full[stage]);
-        const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-        // weight rows: bf16 straight into the operand tile, or e4m3 into its second half
-        const uint32_t w_addr = FP8 ? a_addr + raw_bytes : a_addr;
-        const uint32_t w_bar = FP8 ? smem_u32(&ctl->raw_full[stage]) : bar;
+        const uint32_t w_addr = FP8 ? raw_base + (uint32_t)stage * slot_ring_bytes
+                                    : tiles_base + (uint32_t)stage * stage_bytes;
+        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[stage] : &ctl->full[stage]);
         constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
-        if (FP8) {
-          mbar_expect_tx(w_bar, raw_bytes);
-          mbar_expect_tx(bar, b_bytes);
-        } else {
-          mbar_expect_tx(bar, stage_bytes);
-        }
+        mbar_expect_tx(bar, (FP8 ? raw_bytes : a_bytes) + b_bytes);
         if (stacked) {  // tm_w has 64-row boxes here
-          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);                  // 64 gate rows
-          tma_load_3d(&tm_w, w_addr + w_tile / 2, w_bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
+          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);                  // 64 gate rows
+          tma_load_3d(&tm_w, w_addr + w_tile / 2, bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
         } else if (KIND == 1) {
-          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);               // gate rows
-          tma_load_3d(&tm_w, w_addr + w_tile, w_bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
+          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);               // gate rows
+          tma_load_3d(&tm_w, w_addr + w_tile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
         } else {
-          tma_load_3d(&tm_w, w_addr, w_bar, kb * kBlockK, it.m0, it.slot);               // down rows
-          if (dual) tma_load_3d(&tm_w, w_addr + w_tile, w_bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
+          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);               // down rows
+          if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
         }
-        tma_load_2d(&tm_act, a_addr + a_bytes, bar, kb * kBlockK, it.row0);
-        if (++stage == n_stages) {
+        tma_load_2d(&tm_act, w_addr + (FP8 ? raw_bytes : a_bytes), bar, kb * kBlockK, it.row0);
+        if (++stage == ring) {
           stage = 0;
           phase ^= 1u;
         }
@@ -380,7 +410,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   } else if (warp == kMmaWarp && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
     int stage = 0, g = 0, local = 0;
-    uint32_t phase = 0;
+    int rs = 0;  // fp8 stores: load slot of the k-block (holds its token tile)
+    uint32_t phase = 0, slot_phase = 0;
     bool ok = true;
     for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
       Item it;
@@ -393,23 +424,31 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const uint32_t idesc = make_idesc(n_mma);
       const uint32_t d0 = tmem_base + (uint32_t)(acc * acc_cols);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, status)) {
+        // fp8 stores: the converters arrive on full[] only after the slot has landed; the wait
+        // on the slot's own barrier (already complete) makes this thread an observer of the copy
+        if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, status) ||
+            (FP8 && !mbar_wait(smem_u32(&ctl->slot_full[rs]), slot_phase, abort_flag, status))) {
           ok = false;
           break;
         }
         tc_fence_after();
         const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-        const uint32_t b_addr = a_addr + a_bytes;
+        const uint32_t b_addr = FP8 ? raw_base + (uint32_t)rs * slot_ring_bytes + raw_bytes : a_addr + a_bytes;
 #pragma unroll
         for (int k = 0; k < kBlockK / 16; ++k) {
           const uint64_t db = make_smem_desc(b_addr + k * 32);
           const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
           tc_mma(d0, make_smem_desc(a_addr + k * 32), db, idesc, accum);
-#ifndef OLED_DBG_SKIP_SECOND_MMA  // timing experiment only: results are wrong when defined
           if (dual) tc_mma(d0 + (uint32_t)n_box, make_smem_desc(a_addr + kATile + k * 32), db, idesc, accum);
-#endif
         }
         tc_commit(smem_u32(&ctl->empty[stage]));
+        if (FP8) {
+          tc_commit(smem_u32(&ctl->slot_empty[rs]));
+          if (++rs == n_raw) {
+            rs = 0;
+            slot_phase ^= 1u;
+          }
+        }
         if (++stage == n_stages) {
           stage = 0;
           phase ^= 1u;
@@ -419,51 +458,65 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
   } else if (conv_id >= 0) {
     // ------------------------------------------------------------ fp8 -> bf16 converters
-    // Every converter warp widens whole stages, so that several stages are in conversion at once (one stage is a chain of shared
-    // loads, integer work, shared stores and a proxy fence).  Lane l owns weight rows l, l + 32,
-    // ...: 64 codes in, 128 bytes out, written in the 128-byte-swizzled layout the MMA descriptor
-    // describes (the 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
-    long n_kb = 0;
+    // A group of conv_width warps widens the code tile of one load slot into the operand stage of
+    // the same k-block, several groups (k-blocks) at a time.  The tile is cut into units of 8 weight rows
+    // (512 bytes of codes); lane l of the warp that takes a unit reads the 16 codes of quarter
+    // l mod 4 of row l / 4 - the warp reads 512 contiguous bytes, free of bank conflicts - and
+    // writes their 32 bytes of bf16 in the 128-byte-swizzled layout the MMA descriptor describes
+    // (the 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
+    const int group = conv_id % conv_groups, member = conv_id / conv_groups;
+    int n_kb = 0;  // k-blocks of this CTA
     if ((int)blockIdx.x < total_items && !grp.withhold_loads)
-      n_kb = (long)((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
-    // A converter warp owns pipeline STAGES (stage s belongs to warp s mod n_conv) and walks its
-    // k-blocks in order: it reaches round r of a stage only after it finished round r-1 of the same
-    // stage, so the parity wait below can never mistake an older phase for the one it wants.
-    for (long i = 0; i < n_kb; ++i) {
-      const int stage = (int)(i % n_stages);
-      if (stage % n_conv != conv_id) continue;
-      const uint32_t phase = (uint32_t)(i / n_stages) & 1u;
+      n_kb = ((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
+    constexpr int units = (int)(a_bytes / 128u) / 8;  // 16, or 32 with two weight tiles per stage
+    const uint32_t r8 = (uint32_t)(lane >> 2), cq = (uint32_t)(lane & 3);
+    const uint32_t out_lo = r8 * 128u + (((2u * cq) ^ r8) << 4), out_hi = r8 * 128u + (((2u * cq + 1u) ^ r8) << 4);
+    // ring positions of k-block i = group, group + conv_groups, ... (conv_groups divides both depths)
+    int rs = group, stage = group;
+    uint32_t raw_phase = 0, phase = 0;
+    for (int i = group; i < n_kb; i += conv_groups) {
       int ok = 0;
-      if (lane == 0) ok = mbar_wait(smem_u32(&ctl->raw_full[stage]), phase, abort_flag, status) ? 1 : 0;
+      if (lane == 0)
+        ok = (mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_conv) &&
+              mbar_wait(smem_u32(&ctl->slot_full[rs]), raw_phase, abort_flag, status, nap_conv))
+                 ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       __syncwarp();
       const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-      const uint32_t raw_addr = a_addr + raw_bytes;
-      // In place: code row r sits at raw_addr + 64 r, its bf16 form goes to a_addr + 128 r.  Rows
-      // are taken in ascending waves of 32 (one per lane); a wave reads its codes into registers
-      // before it writes, and what it overwrites are code rows <= its own, already consumed.
-      for (int r0 = 0; r0 < (int)(a_bytes / 128u); r0 += 32) {
-        const int rr = r0 + lane;
+      const uint32_t raw_addr = raw_base + (uint32_t)rs * slot_ring_bytes + (uint32_t)lane * 16u;
+      for (int u0 = member; u0 < units; u0 += 4 * conv_width) {
         uint4 c[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) c[q] = lds128(raw_addr + (uint32_t)rr * 64u + (uint32_t)q * 16u);
-        __syncwarp();
-        const uint32_t row_addr = a_addr + (uint32_t)rr * 128u;
+        for (int q = 0; q < 4; ++q) {
+          const int u = u0 + q * conv_width;
+          if (u < units) c[q] = lds128(raw_addr + (uint32_t)u * 512u);
+        }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          uint4 lo, hi;
-          e4m3x4_to_bf16x4(c[q].x, lo.x, lo.y);
-          e4m3x4_to_bf16x4(c[q].y, lo.z, lo.w);
-          e4m3x4_to_bf16x4(c[q].z, hi.x, hi.y);
-          e4m3x4_to_bf16x4(c[q].w, hi.z, hi.w);
-          sts128(row_addr + (uint32_t)(((2 * q) ^ (rr & 7)) * 16), lo);
-          sts128(row_addr + (uint32_t)(((2 * q + 1) ^ (rr & 7)) * 16), hi);
+          const int u = u0 + q * conv_width;
+          if (u < units) {
+            uint4 lo, hi;
+            e4m3x4_to_bf16x4(c[q].x, lo.x, lo.y);
+            e4m3x4_to_bf16x4(c[q].y, lo.z, lo.w);
+            e4m3x4_to_bf16x4(c[q].z, hi.x, hi.y);
+            e4m3x4_to_bf16x4(c[q].w, hi.z, hi.w);
+            const uint32_t row_addr = a_addr + (uint32_t)u * 1024u;
+            sts128(row_addr + out_lo, lo);
+            sts128(row_addr + out_hi, hi);
+          }
         }
-        __syncwarp();
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
-      mbar_arrive(smem_u32(&ctl->full[stage]));
+      mbar_arrive(smem_u32(&ctl->full[stage]));  // (the slot itself is released by the MMA's completion)
+      if ((rs += conv_groups) >= n_raw) {
+        rs -= n_raw;
+        raw_phase ^= 1u;
+      }
+      if ((stage += conv_groups) >= n_stages) {
+        stage -= n_stages;
+        phase ^= 1u;
+      }
     }
   } else if (warp < epi_warps && conv_id == -1) {
     // ------------------------------------------------------------ epilogue
@@ -479,7 +532,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       // one lane polls (keeps issue slots free for the producer and MMA threads); the outcome is
       // warp-uniform because tcgen05.ld below is warp-collective
       int ready = 0;
-      if (lane == 0) ready = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, status) ? 1 : 0;
+      if (lane == 0) ready = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, status, nap_epi) ? 1 : 0;
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) break;
       tc_fence_after();
@@ -648,22 +701,41 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-uint32_t stage_bytes_for(bool dual, int n_box, bool fp8) {
-  (void)fp8;  // fp8 rows are widened in place: same stage size as bf16
-  const uint32_t a = (dual ? 2u : 1u) * kATile;
-  return a + (uint32_t)n_box * 128u;
-}
-int stages_for(bool dual, int n_box, bool fp8) {
-  static int cap = -1;  // tuning aid: OLED_FFN_STAGES caps the pipeline depth
-  if (cap < 0) {
+struct Rings {
+  int stages;     // operand stages
+  int raw;        // fp8 stores: load slots (code tile + token tile) behind them
+  uint32_t smem;  // dynamic shared memory of the launch
+};
+// bf16 stores: as many operand stages (weight tile(s) + token tile) as fit.  fp8 stores: a short
+// ring of widened weight tiles (the converters and the MMA hand stages over within a few hundred
+// cycles) and the rest of shared memory as load slots in flight; both depths even, multiples of
+// four where the tiles are small, so that the converter groups (see the kernel) divide them.
+Rings rings_for(bool dual, int n_box, bool fp8) {
+  static int cap = -1, op_cap = -1;  // tuning aids: OLED_FFN_STAGES caps the (load) ring depth,
+  if (cap < 0) {                     // OLED_FFN_OP_STAGES sets the fp8 operand ring depth
     const char* env = getenv("OLED_FFN_STAGES");
-    cap = env ? std::max(1, atoi(env)) : kMaxStages;
+    cap = env ? std::max(1, atoi(env)) : 64;
+    const char* env2 = getenv("OLED_FFN_OP_STAGES");
+    op_cap = env2 ? std::max(1, atoi(env2)) : 0;
   }
+  const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
-  return (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / stage_bytes_for(dual, n_box, fp8));
-}
-uint32_t smem_for(bool dual, int n_box, bool fp8, int stages) {
-  return kCtlBytes + 1024u + (uint32_t)stages * stage_bytes_for(dual, n_box, fp8);
+  Rings r;
+  if (!fp8) {
+    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / (a + b));
+    r.raw = 0;
+    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * (a + b);
+  } else {
+    const uint32_t slot = a / 2 + b;
+    r.stages = op_cap > 0 ? std::min(op_cap, kMaxStages) : !dual ? 6 : 2;
+    while (r.stages > 1 && (uint32_t)r.stages * a + 2 * slot > avail) --r.stages;
+    const uint32_t left = avail - (uint32_t)r.stages * a;
+    r.raw = (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxRaw), left / slot);
+    if (r.raw >= 4 && r.stages % 4 == 0) r.raw &= ~3;
+    else if (r.raw >= 2) r.raw &= ~1;
+    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * a + (uint32_t)r.raw * slot;
+  }
+  return r;
 }
 
 template <int KIND, bool DUAL, bool FP8>
@@ -673,15 +745,16 @@ bool set_smem_attr() {
 }
 
 template <int KIND, bool DUAL>
-void launch_variant(bool fp8, int grid, uint32_t smem, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
-                    const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int stages, int out_bf16,
+void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
+                    const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status) {
+  const Rings r = rings_for(DUAL, grp.n_box, fp8);
   if (fp8)
-    launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), smem, st, tw, ta, grp, offsets, out, H, I,
-               stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+               I, r.stages, r.raw, out_bf16, pool, (unsigned long long)slot_bytes, status);
   else
-    launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), smem, st, tw, ta, grp, offsets, out, H, I,
-               stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+               I, r.stages, r.raw, out_bf16, pool, (unsigned long long)slot_bytes, status);
 }
 
 }  // namespace
@@ -766,25 +839,19 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     force_dual = b ? atoi(b) : 0;
   }
   if (kind == 1 && grp.n_box <= 32 && use_stacked == 1) {
-    const int stages = stages_for(false, grp.n_box, fp8);
-    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), smem_for(false, grp.n_box, fp8, stages), st,
-                             maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I, stages, 0, maps.pool,
-                             maps.slot_bytes, status);
+    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
+                             0, maps.pool, maps.slot_bytes, status);
   } else if (kind == 1) {
-    const int stages = stages_for(true, grp.n_box, fp8);
-    launch_variant<1, true>(fp8, grid_for(I / kBlockM), smem_for(true, grp.n_box, fp8, stages), st, maps.w13,
-                            maps.xp[ib], grp, offsets, hbuf, H, I, stages, 0, maps.pool, maps.slot_bytes, status);
+    launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
+                            maps.pool, maps.slot_bytes, status);
   } else {
     const bool dual = grp.n_box == 256 || force_dual == 1;
-    const int stages = stages_for(dual, grp.n_box, fp8);
     if (dual)
-      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), smem_for(true, grp.n_box, fp8, stages), st, maps.w2,
-                              maps.hbuf[ib], grp, offsets, y, H, I, stages, y_bf16, maps.pool, maps.slot_bytes,
-                              status);
+      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
+                              y_bf16, maps.pool, maps.slot_bytes, status);
     else
-      launch_variant<2, false>(fp8, grid_for(H / kBlockM), smem_for(false, grp.n_box, fp8, stages), st, maps.w2,
-                               maps.hbuf[ib], grp, offsets, y, H, I, stages, y_bf16, maps.pool, maps.slot_bytes,
-                               status);
+      launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
+                               maps.pool, maps.slot_bytes, status);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

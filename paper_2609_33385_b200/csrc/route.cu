@@ -7,7 +7,7 @@
 //   * logit(t,e): 32 chains, lane q owns h with (h/8) mod 32 == q, ascending h, one fused
 //     multiply-add per term (bf16*bf16 is exact in fp32, so the fma rounds once, like a plain
 //     add of the exact product); butterfly over xor distances 16,8,4,2,1; bias one rounded add.
-//   * top-k: logit descending, ties to the lower expert index.
+//   * top-k: logit descending, ties to the lower expert index (a NaN logit counts as -inf).
 //   * gate scores: z_j = exp_spec(L_j - L_0); S = ((z_0+z_1)+z_2)...; g_j = z_j / S.
 //   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
 // The router stays off the tensor cores on purpose: their accumulation order is unspecified.
@@ -55,7 +55,8 @@ __device__ __forceinline__ void route_token_tail(const float* row, int t, int la
 #pragma unroll
     for (int i = 0; i < kMaxEPerLane; ++i) {
       const int e = lane + 32 * i;
-      v[i] = e < E ? row[e] : 0.0f;
+      const float x = e < E ? row[e] : 0.0f;
+      v[i] = (x == x) ? x : __int_as_float(0xff800000);  // a NaN logit is read as -inf: the order stays total
     }
     uint32_t used = 0;
     int my_id = 0;
@@ -101,7 +102,9 @@ __device__ __forceinline__ void route_token_tail(const float* row, int t, int la
       float c = conf[t];
       c = (c != c) ? 0.0f : fminf(fmaxf(c, 0.0f), 1.0f);  // psi(c) = c, clamped; NaN -> 0
       const float pv = __fmul_rn(g, c);
-      const unsigned long long q = __float2ull_rz(__fmul_rn(pv, 4294967296.0f));
+      // a NaN product (non-finite activations) adds nothing; the 64-bit conversion of a NaN
+      // would return 2^63
+      const unsigned long long q = (pv == pv) ? __float2ull_rz(__fmul_rn(pv, 4294967296.0f)) : 0ull;
       atomicAdd(&counts[my_id], 1);
       atomicAdd(&scores[my_id], q);
     }
@@ -124,7 +127,8 @@ __device__ __forceinline__ void route_publish(const RouteReport& rep, const int3
   const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
   const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    rep.host_scores[e] = tag16 | __ldcg(&scores[e]);                               // score < 2^48
+    // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
+    rep.host_scores[e] = tag16 | (__ldcg(&scores[e]) & 0xffffffffffffull);
     rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
   }
 }

@@ -430,6 +430,45 @@ def test_degenerate_routing_cases():
         run.close()
 
 
+def test_non_finite_activations_keep_routing_defined_and_the_context_usable():
+    """NaN and Inf in the hidden states: a NaN logit ranks as -inf, so the k ids of every token
+    stay distinct and all discrete results still match the oracle; rows of clean tokens are
+    unaffected; the next clean step is in full parity."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1)
+    run = _runner(w, capacity=[3], max_tokens=40)
+    ora = _oracle_for(run, [3])
+    try:
+        h_bits, conf = synth.flat_tokens(w, 40, 77)
+        bad = h_bits.copy()
+        bad[3, :] = 0x7FC0      # a whole NaN row
+        bad[5, 17] = 0x7FC0     # one NaN element
+        bad[7, 1] = 0x7F80      # +Inf
+        bad[9, 2] = 0xFF80      # -Inf
+        x, c = bits_to_dev(bad, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((40, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)
+        with np.errstate(all="ignore"):
+            ref = ora.denoise_step(0, bad, conf)
+        dbg = run.ctx.debug_last(0, 40)
+        assert np.array_equal(dbg["ids"], ref["ids"])
+        assert all(len(set(row)) == w.top_k for row in dbg["ids"].tolist())
+        assert np.array_equal(np.isnan(dbg["gate"]), np.isnan(ref["gate"]))
+        ok = ~np.isnan(ref["gate"])
+        assert np.array_equal(dbg["gate"][ok].view(np.uint32), ref["gate"][ok].view(np.uint32))
+        assert np.array_equal(dbg["counts"], ref["counts"]) and np.array_equal(dbg["perm"], ref["perm"])
+        assert [int(v) for v in dbg["scores"]] == list(ref["scores"])
+        assert set(np.flatnonzero(dbg["resident_after"])) == ref["resident_after"]
+        clean = [t for t in range(40) if t not in (3, 5, 7, 9)]
+        _check_out(dev_to_bits(out)[clean], ref["out"][clean], "clean rows")
+        x2 = bits_to_dev(h_bits, run.device)
+        run.step(0, x2, c, out)
+        _check_step(run, 0, 40, out, ora.denoise_step(0, h_bits, conf))
+        _check_stats(run, ora)
+    finally:
+        run.close()
+
+
 def test_fp8_expert_store_tiny_stack():
     """fp8 (e4m3 + row scales) expert blobs: same discrete results, outputs within the same
     tolerance of the oracle evaluated on the dequantised weights, half the bytes moved."""
