@@ -26,16 +26,19 @@
 // warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation),
 // warps 18-21 widen fp8 weight tiles (fp8 expert stores only, idle otherwise).
 //
-// fp8 expert stores (e4m3 codes + one fp32 scale per weight row) use TWO rings in shared memory:
-// a deep ring of load slots - the raw code tile of a k-block (64 bytes per weight row) next to
-// its token tile - that the producer keeps full, which is what hides the HBM latency at half the
-// bytes per tile of the bf16 form, and a short ring of bf16 weight-operand stages.  Groups of
-// converter warps widen a slot's codes into a free operand stage (exact, in the swizzled layout
-// the MMA descriptor describes); the MMA reads the weights from the stage and the tokens from the
-// slot, runs in bf16 as before, and its completion frees both; the epilogue multiplies each
-// output row by its scale - the rows of a weight tile are the accumulator's lanes.  Every mbarrier wait is bounded: on a
-// timeout the CTA raises a flag in the status word, gives in-flight copies time to land, frees
-// its TMEM and returns.
+// fp8 expert stores (e4m3 codes + one fp32 scale per weight row): a pipeline stage is a load
+// slot in shared memory - the code tile of a k-block (64 bytes per weight row, half the bytes in
+// flight of the bf16 form) next to its token tile - plus 32 (64) columns of TENSOR memory.
+// Groups of four converter warps, one per TMEM lane quarter, read the codes, widen them to bf16
+// (exact) and write them with tcgen05.st as the MMA's A operand: lane = weight row, two
+// consecutive k per 32-bit column.  The MMA takes the weights from tensor memory and the tokens
+// from the slot, runs in bf16 as before, and its completion frees the stage; the widened weights
+// never touch shared memory.  The accumulators keep their place in front of the weight stages,
+// which is why the fp8 form stops at token tiles of 128.  The epilogue multiplies each output
+// row by its scale - the rows of a weight tile are the accumulator's lanes.
+//
+// Every mbarrier wait is bounded: on a timeout the CTA raises a flag in the status word, gives
+// in-flight copies time to land, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -69,16 +72,14 @@ constexpr int kThreads = (kEpiWarps + 6) * 32;
 constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
 constexpr uint32_t kATile = kBlockM * kBlockK * 2;
-constexpr int kMaxStages = 10;
-constexpr int kMaxRaw = 16;  // fp8 stores: depth limit of the ring of load slots
+constexpr int kMaxStages = 12;
 constexpr uint32_t kSmemMax = 232448;  // 227 KB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct __align__(16) SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
-  unsigned long long slot_full[kMaxRaw];   // fp8 stores: the slot's code tile and token tile have landed
-  unsigned long long slot_empty[kMaxRaw];  // fp8 stores: the MMAs that read the slot's token tile are done
+  unsigned long long slot_full[kMaxStages];  // fp8 stores: the stage's code tile and token tile have landed
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long x_full[2][2];   // stacked gate/up mode: [buffer][chunk group], up rows -> gate rows
@@ -172,14 +173,30 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128.
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                       uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128.  The descriptors are
+// given as (low word, shared high word): the low word carries the address in 16-byte units, so
+// stepping along K or to the next stage is one 32-bit add.
+__device__ __forceinline__ void tc_mma_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same with the weight operand in tensor memory (lane = row, two bf16 of consecutive k per
+// 32-bit column).
+__device__ __forceinline__ void tc_mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -191,6 +208,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[15])
       : "r"(taddr)
       : "memory");
+}
+// 32 consecutive 32-bit columns of the calling thread's TMEM lane (lane quarter = warp id mod 4)
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -260,7 +292,7 @@ template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
-              void* __restrict__ out_ptr, int H, int I, int n_stages, int n_raw, int out_bf16,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -273,48 +305,48 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t b_bytes = (uint32_t)n_box * 128u;
-  // bf16 stores: a stage holds the weight tile(s) and the token tile of a k-block.  fp8 stores: a
-  // stage holds the widened weight tile(s) only; behind the n_stages stages sits the ring of n_raw
-  // load slots, each the code tile (one byte per element) followed by the token tile.
+  // bf16 stores: a stage (shared memory) holds the weight tile(s) and the token tile of a k-block.
+  // fp8 stores: a stage is a load slot in shared memory - the code tile (one byte per element)
+  // followed by the token tile - plus a_cols columns of TENSOR memory, behind the accumulators,
+  // for the widened weights.
   constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;
-  const uint32_t stage_bytes = FP8 ? a_bytes : a_bytes + b_bytes;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
   const uint32_t slot_ring_bytes = raw_bytes + b_bytes;
-  const uint32_t raw_base = tiles_base + (uint32_t)n_stages * stage_bytes;
+  constexpr uint32_t a_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
   const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
-  const int acc_stages = (2 * acc_cols <= 512) ? 2 : 1;
+  const int a_total = FP8 ? n_stages * (int)a_cols : 0;
+  const int acc_stages = (2 * acc_cols + a_total <= 512) ? 2 : 1;
+  const uint32_t a_col0 = (uint32_t)(acc_stages * acc_cols);  // first column of the weight stages
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
   const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
   // fp8 stores: the four dedicated converter warps plus the epilogue warps this token tile leaves
-  // idle (4, 12 or 16 warps) form conv_groups groups of conv_width warps.  Group g owns the
-  // k-blocks i with i mod conv_groups == g; conv_groups divides both ring depths, so every raw
-  // slot and every operand stage belongs to ONE group, which visits the rounds of its barriers in
-  // order - a parity wait can then never take an older phase for the one it wants.
-  const int n_conv = FP8 ? 4 + (kEpiWarps - epi_warps) : 0;
-  int conv_groups = n_conv >= 16 ? 4 : n_conv >= 12 ? 2 : 1;
-  while (conv_groups > 1 && (n_stages % conv_groups != 0 || n_raw % conv_groups != 0)) conv_groups >>= 1;
-  const int conv_width = FP8 ? n_conv / conv_groups : 1;
-  int conv_id = !FP8 ? -1
-                : (warp >= kConvWarp0 && warp < kConvWarp0 + 4) ? warp - kConvWarp0
-                : (warp >= epi_warps && warp < kEpiWarps) ? 4 + (warp - epi_warps) : -1;
+  // idle form conv_groups (1, 3 or 4) groups of four warps, one warp per TMEM lane quarter.
+  // Group g owns the k-blocks i with i mod conv_groups == g; conv_groups divides both ring
+  // depths, so every load slot and every weight stage belongs to ONE group, which visits the
+  // rounds of its barriers in order - a parity wait can then never take an older phase for the
+  // one it wants.
+  int conv_groups = FP8 ? 1 + (kEpiWarps - epi_warps) / 4 : 0;
+  if (conv_groups > 1 && n_stages % conv_groups != 0) conv_groups = 1;
+  const int conv_group = !FP8 ? -1
+                         : (warp >= kConvWarp0 && warp < kConvWarp0 + 4) ? 0
+                         : (warp >= epi_warps && warp < kEpiWarps) ? 1 + (warp - epi_warps) / 4 : -1;
+  const bool is_conv = FP8 && conv_group >= 0 && conv_group < conv_groups;
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < acc_stages * acc_cols) tmem_cols <<= 1;
+  while ((int)tmem_cols < acc_stages * acc_cols + a_total) tmem_cols <<= 1;
 
   // ---- set-up that depends on no earlier kernel: barriers, TMEM (overlaps the predecessor's tail)
   griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      // the stage's TMA transaction, or every lane of the converting group
-      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 32u * (uint32_t)conv_width : 1u);
+      // the stage's TMA transaction, or every lane of the four converting warps
+      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 128u : 1u);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
-    for (int s = 0; s < kMaxRaw; ++s) {
-      mbar_init(smem_u32(&ctl->slot_full[s]), 1);
-      mbar_init(smem_u32(&ctl->slot_empty[s]), 1);
-    }
+    for (int s = 0; s < kMaxStages; ++s) mbar_init(smem_u32(&ctl->slot_full[s]), 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[a]), (uint32_t)epi_warps * 32u);
@@ -370,18 +402,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     int stage = 0, g = 0;
     uint32_t phase = 0;
     bool ok = true;
-    const int ring = FP8 ? n_raw : n_stages;
+    const int ring = n_stages;
     for (int item = blockIdx.x; ok && !grp.withhold_loads && item < total_items; item += gridDim.x) {
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        const uint32_t free_bar = smem_u32(FP8 ? &ctl->slot_empty[stage] : &ctl->empty[stage]);
+        const uint32_t free_bar = smem_u32(&ctl->empty[stage]);
         if (!mbar_wait(free_bar, phase ^ 1u, abort_flag, status, nap_load)) {
           ok = false;
           break;
         }
-        const uint32_t w_addr = FP8 ? raw_base + (uint32_t)stage * slot_ring_bytes
-                                    : tiles_base + (uint32_t)stage * stage_bytes;
+        const uint32_t w_addr = tiles_base + (uint32_t)stage * (FP8 ? slot_ring_bytes : stage_bytes);
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[stage] : &ctl->full[stage]);
         constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
         mbar_expect_tx(bar, (FP8 ? raw_bytes : a_bytes) + b_bytes);
@@ -410,9 +441,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   } else if (warp == kMmaWarp && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
     int stage = 0, g = 0, local = 0;
-    int rs = 0;  // fp8 stores: load slot of the k-block (holds its token tile)
-    uint32_t phase = 0, slot_phase = 0;
+    uint32_t phase = 0;
     bool ok = true;
+    // Descriptor words of stage 0 (K-major, 128-byte swizzle, 8-row groups 1024 bytes apart); the
+    // low word holds the address in 16-byte units, the high word is the same for every operand.
+    const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
+    const uint32_t ring_step = (FP8 ? slot_ring_bytes : stage_bytes) >> 4;
+    const uint32_t a_lo0 = (uint32_t)make_smem_desc(tiles_base);
+    const uint32_t b_lo0 = (uint32_t)make_smem_desc(tiles_base + (FP8 ? raw_bytes : a_bytes));
+    const uint32_t a_tmem0 = tmem_base + a_col0;  // fp8 stores: weights come from tensor memory
+    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+    uint32_t a_lo = a_lo0, b_lo = b_lo0, a_tmem = a_tmem0;
     for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
@@ -424,101 +463,91 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const uint32_t idesc = make_idesc(n_mma);
       const uint32_t d0 = tmem_base + (uint32_t)(acc * acc_cols);
       for (int kb = 0; kb < k_blocks; ++kb) {
-        // fp8 stores: the converters arrive on full[] only after the slot has landed; the wait
-        // on the slot's own barrier (already complete) makes this thread an observer of the copy
-        if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, status) ||
-            (FP8 && !mbar_wait(smem_u32(&ctl->slot_full[rs]), slot_phase, abort_flag, status))) {
+        // (fp8 stores: the converters arrive on full[] only after the stage's slot has landed)
+        if (!mbar_wait(full0 + (uint32_t)stage * 8u, phase, abort_flag, status)) {
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-        const uint32_t b_addr = FP8 ? raw_base + (uint32_t)rs * slot_ring_bytes + raw_bytes : a_addr + a_bytes;
+        const uint32_t first = kb != 0 ? 1u : 0u;
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k) {
-          const uint64_t db = make_smem_desc(b_addr + k * 32);
-          const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-          tc_mma(d0, make_smem_desc(a_addr + k * 32), db, idesc, accum);
-          if (dual) tc_mma(d0 + (uint32_t)n_box, make_smem_desc(a_addr + kATile + k * 32), db, idesc, accum);
-        }
-        tc_commit(smem_u32(&ctl->empty[stage]));
-        if (FP8) {
-          tc_commit(smem_u32(&ctl->slot_empty[rs]));
-          if (++rs == n_raw) {
-            rs = 0;
-            slot_phase ^= 1u;
+        for (int k = 0; k < kBlockK / 16; ++k) {  // 32 bytes along K = 2 address units
+          const uint32_t accum = k != 0 ? 1u : first;
+          if (FP8) {
+            tc_mma_ts_lo(d0, a_tmem + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
+            if (dual) tc_mma_ts_lo(d0 + (uint32_t)n_box, a_tmem + 32 + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
+          } else {
+            tc_mma_lo(d0, a_lo + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
+            if (dual) tc_mma_lo(d0 + (uint32_t)n_box, a_lo + (kATile >> 4) + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
           }
         }
+        tc_commit(empty0 + (uint32_t)stage * 8u);
+        a_lo += ring_step;
+        b_lo += ring_step;
+        a_tmem += a_cols;
         if (++stage == n_stages) {
           stage = 0;
           phase ^= 1u;
+          a_lo = a_lo0;
+          b_lo = b_lo0;
+          a_tmem = a_tmem0;
         }
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
-  } else if (conv_id >= 0) {
+  } else if (is_conv) {
     // ------------------------------------------------------------ fp8 -> bf16 converters
-    // A group of conv_width warps widens the code tile of one load slot into the operand stage of
-    // the same k-block, several groups (k-blocks) at a time.  The tile is cut into units of 8 weight rows
-    // (512 bytes of codes); lane l of the warp that takes a unit reads the 16 codes of quarter
-    // l mod 4 of row l / 4 - the warp reads 512 contiguous bytes, free of bank conflicts - and
-    // writes their 32 bytes of bf16 in the 128-byte-swizzled layout the MMA descriptor describes
-    // (the 16-byte chunk j of row r sits at chunk j xor (r mod 8)).
-    const int group = conv_id % conv_groups, member = conv_id / conv_groups;
+    // The four warps of a group widen the code tile of one load slot into the weight stage (tensor
+    // memory) of the same k-block, several groups (k-blocks) at a time.  A warp can write only
+    // the TMEM lanes of its quarter (warp id mod 4): lane l of the warp owns weight row
+    // 32 * quarter + l, reads its 64 codes (the TMA laid the 64-byte rows out with the 64-byte
+    // swizzle, so that the 32 rows of a quarter spread over all banks), widens them and stores
+    // 32 columns of packed bf16 pairs with one tcgen05.st.
+    const int group = conv_group, quarter = warp & 3;
     int n_kb = 0;  // k-blocks of this CTA
     if ((int)blockIdx.x < total_items && !grp.withhold_loads)
       n_kb = ((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
-    constexpr int units = (int)(a_bytes / 128u) / 8;  // 16, or 32 with two weight tiles per stage
-    const uint32_t r8 = (uint32_t)(lane >> 2), cq = (uint32_t)(lane & 3);
-    const uint32_t out_lo = r8 * 128u + (((2u * cq) ^ r8) << 4), out_hi = r8 * 128u + (((2u * cq + 1u) ^ r8) << 4);
+    const uint32_t row = (uint32_t)(quarter * 32 + lane);
+    const uint32_t sw = (row >> 1) & 3u;  // SWIZZLE_64B: 16-byte chunk index xor address bits 7-8
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + a_col0;
     // ring positions of k-block i = group, group + conv_groups, ... (conv_groups divides both depths)
-    int rs = group, stage = group;
-    uint32_t raw_phase = 0, phase = 0;
+    int stage = group;
+    uint32_t phase = 0;
     for (int i = group; i < n_kb; i += conv_groups) {
       int ok = 0;
       if (lane == 0)
         ok = (mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_conv) &&
-              mbar_wait(smem_u32(&ctl->slot_full[rs]), raw_phase, abort_flag, status, nap_conv))
+              mbar_wait(smem_u32(&ctl->slot_full[stage]), phase, abort_flag, status, nap_conv))
                  ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       __syncwarp();
-      const uint32_t a_addr = tiles_base + (uint32_t)stage * stage_bytes;
-      const uint32_t raw_addr = raw_base + (uint32_t)rs * slot_ring_bytes + (uint32_t)lane * 16u;
-      for (int u0 = member; u0 < units; u0 += 4 * conv_width) {
+      tc_fence_after();  // the stage was released by the completion of the MMAs that read it
+      const uint32_t src = tiles_base + (uint32_t)stage * slot_ring_bytes + row * 64u;
+#pragma unroll
+      for (int tile = 0; tile < (dual ? 2 : 1); ++tile) {
         uint4 c[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int u = u0 + q * conv_width;
-          if (u < units) c[q] = lds128(raw_addr + (uint32_t)u * 512u);
-        }
+        for (int j = 0; j < 4; ++j) c[j] = lds128(src + (uint32_t)tile * (kATile / 2) + (((uint32_t)j ^ sw) << 4));
+        uint32_t r[32];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int u = u0 + q * conv_width;
-          if (u < units) {
-            uint4 lo, hi;
-            e4m3x4_to_bf16x4(c[q].x, lo.x, lo.y);
-            e4m3x4_to_bf16x4(c[q].y, lo.z, lo.w);
-            e4m3x4_to_bf16x4(c[q].z, hi.x, hi.y);
-            e4m3x4_to_bf16x4(c[q].w, hi.z, hi.w);
-            const uint32_t row_addr = a_addr + (uint32_t)u * 1024u;
-            sts128(row_addr + out_lo, lo);
-            sts128(row_addr + out_hi, hi);
-          }
+        for (int j = 0; j < 4; ++j) {
+          e4m3x4_to_bf16x4(c[j].x, r[8 * j], r[8 * j + 1]);
+          e4m3x4_to_bf16x4(c[j].y, r[8 * j + 2], r[8 * j + 3]);
+          e4m3x4_to_bf16x4(c[j].z, r[8 * j + 4], r[8 * j + 5]);
+          e4m3x4_to_bf16x4(c[j].w, r[8 * j + 6], r[8 * j + 7]);
         }
+        tmem_st32(t_lane + (uint32_t)stage * a_cols + (uint32_t)tile * 32u, r);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> tensor-core reads
-      mbar_arrive(smem_u32(&ctl->full[stage]));  // (the slot itself is released by the MMA's completion)
-      if ((rs += conv_groups) >= n_raw) {
-        rs -= n_raw;
-        raw_phase ^= 1u;
-      }
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->full[stage]));  // (the slot itself is released by the MMAs' completion)
       if ((stage += conv_groups) >= n_stages) {
         stage -= n_stages;
         phase ^= 1u;
       }
     }
-  } else if (warp < epi_warps && conv_id == -1) {
+  } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
     int g = 0, local = 0;
@@ -693,47 +722,49 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
                    : v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
                              : v == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
   }
-  // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; raw e4m3 rows (64 bytes
-  // per k-block) land row-major in the staging area and are re-laid out by the converter warps
+  // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; e4m3 rows (64 bytes per
+  // k-block) land with the 64-byte swizzle, which lets 32 lanes read 32 rows free of bank conflicts
   return fn(m, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
             const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            bytes ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, promo,
+            bytes ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, promo,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct Rings {
-  int stages;     // operand stages
-  int raw;        // fp8 stores: load slots (code tile + token tile) behind them
+  int stages;     // weight stages: shared memory (bf16 stores) or tensor memory (fp8 stores)
   uint32_t smem;  // dynamic shared memory of the launch
 };
-// bf16 stores: as many operand stages (weight tile(s) + token tile) as fit.  fp8 stores: a short
-// ring of widened weight tiles (the converters and the MMA hand stages over within a few hundred
-// cycles) and the rest of shared memory as load slots in flight; both depths even, multiples of
-// four where the tiles are small, so that the converter groups (see the kernel) divide them.
-Rings rings_for(bool dual, int n_box, bool fp8) {
-  static int cap = -1, op_cap = -1;  // tuning aids: OLED_FFN_STAGES caps the (load) ring depth,
-  if (cap < 0) {                     // OLED_FFN_OP_STAGES sets the fp8 operand ring depth
+// Epilogue warps the kernel activates for a token tile (the others widen fp8 weights).
+int epi_warps_for(int kind, int out_bf16, int n_box) {
+  return std::min((kind == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+}
+// bf16 stores: as many stages (weight tile(s) + token tile) as fit in shared memory.  fp8 stores:
+// the weight stages take the tensor-memory columns the accumulators leave (two accumulator
+// stages if at least two weight stages still fit), all of shared memory is load slots; both
+// depths are multiples of the number of converter groups (see the kernel).
+Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8) {
+  static int cap = -1, op_cap = -1;  // tuning aids: OLED_FFN_STAGES caps the shared-memory ring depth,
+  if (cap < 0) {                     // OLED_FFN_OP_STAGES the fp8 weight ring in tensor memory
     const char* env = getenv("OLED_FFN_STAGES");
     cap = env ? std::max(1, atoi(env)) : 64;
     const char* env2 = getenv("OLED_FFN_OP_STAGES");
-    op_cap = env2 ? std::max(1, atoi(env2)) : 0;
+    op_cap = env2 ? std::max(1, atoi(env2)) : kMaxStages;
   }
   const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
   Rings r;
   if (!fp8) {
-    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxStages), avail / (a + b));
-    r.raw = 0;
+    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(cap, 10), avail / (a + b));  // (11 measured slower)
     r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * (a + b);
   } else {
+    const int groups = 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4;
+    const int acc_cols = (dual ? 2 : 1) * n_box, a_cols = dual ? 64 : 32;
+    const int free_cols = 512 - 2 * acc_cols >= 2 * a_cols ? 512 - 2 * acc_cols : 512 - acc_cols;
+    r.stages = std::min(std::min(op_cap, kMaxStages), free_cols / a_cols);
     const uint32_t slot = a / 2 + b;
-    r.stages = op_cap > 0 ? std::min(op_cap, kMaxStages) : !dual ? 6 : 2;
-    while (r.stages > 1 && (uint32_t)r.stages * a + 2 * slot > avail) --r.stages;
-    const uint32_t left = avail - (uint32_t)r.stages * a;
-    r.raw = (int)std::min<uint32_t>((uint32_t)std::min(cap, kMaxRaw), left / slot);
-    if (r.raw >= 4 && r.stages % 4 == 0) r.raw &= ~3;
-    else if (r.raw >= 2) r.raw &= ~1;
-    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * a + (uint32_t)r.raw * slot;
+    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(r.stages, cap), avail / slot);
+    if (r.stages >= groups) r.stages -= r.stages % groups;
+    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * slot;
   }
   return r;
 }
@@ -748,13 +779,13 @@ template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status) {
-  const Rings r = rings_for(DUAL, grp.n_box, fp8);
+  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8);
   if (fp8)
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, r.raw, out_bf16, pool, (unsigned long long)slot_bytes, status);
+               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
   else
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, r.raw, out_bf16, pool, (unsigned long long)slot_bytes, status);
+               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
 }
 
 }  // namespace
@@ -822,7 +853,8 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   const bool fp8 = maps.fp8;
   // N <= 128 keeps the accumulators double-buffered in TMEM; more tokens per expert than that
   // take N = 256 with two weight tiles per item (all 512 TMEM columns, one accumulator stage).
-  const int ib = box_index(max_count, 256);
+  // (fp8 stores stop at N = 128: the widened weights need tensor-memory columns of their own)
+  const int ib = box_index(max_count, fp8 ? 128 : 256);
   grp.n_box = 16 << ib;
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int m_tiles) {
