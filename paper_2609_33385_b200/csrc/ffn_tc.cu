@@ -73,6 +73,7 @@ constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // one 128-byte swizzle atom of bf16
 constexpr uint32_t kATile = kBlockM * kBlockK * 2;
 constexpr int kMaxStages = 12;
+constexpr int kItemRing = 8;  // items the producer may publish ahead of the slowest consumer
 constexpr uint32_t kSmemMax = 232448;  // 227 KB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -80,6 +81,8 @@ struct __align__(16) SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
   unsigned long long slot_full[kMaxStages];  // fp8 stores: the stage's code tile and token tile have landed
+  unsigned long long item_full[kItemRing];   // the producer published the CTA's next item
+  unsigned long long item_empty[kItemRing];  // every consumer role has read it
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long x_full[2][2];   // stacked gate/up mode: [buffer][chunk group], up rows -> gate rows
@@ -88,6 +91,7 @@ struct __align__(16) SharedCtl {
   int abort;
   int n_tiles_total;
   int pad;
+  int item_ring[kItemRing];  // item numbers handed out by the producer; -1 = no more work
   int tile_prefix[OLED_MAX_EXPERTS + 1];
   int row_start[OLED_MAX_EXPERTS];
   int count[OLED_MAX_EXPERTS];
@@ -273,6 +277,22 @@ __device__ __forceinline__ void e4m3x4_to_bf16x4(uint32_t w, uint32_t& lo, uint3
 struct Item {
   int slot, m0, row0, valid;
 };
+// Items (expert, token tile, weight tile) are handed out DYNAMICALLY: the producer thread of a
+// CTA draws item numbers from a counter in global memory (one atomic per item, fetched one item
+// ahead) and publishes them to the other roles of its CTA through a small ring in shared
+// memory.  SMs that stream faster take more items, so the launch ends when the work does, not
+// when the slowest SM has finished a fixed share.  Which CTA computes an item does not change
+// its arithmetic.
+// Consumer side: the seq-th item of this CTA, -1 when there is no more work, -2 on an abort.
+__device__ __forceinline__ int take_item(SharedCtl* ctl, int seq, volatile int* abort_flag, uint32_t* status,
+                                         uint32_t nap) {
+  const int slot = seq % kItemRing;
+  const uint32_t ph = (uint32_t)(seq / kItemRing) & 1u;
+  if (!mbar_wait(smem_u32(&ctl->item_full[slot]), ph, abort_flag, status, nap)) return -2;
+  const int item = *reinterpret_cast<volatile int*>(&ctl->item_ring[slot]);
+  mbar_arrive(smem_u32(&ctl->item_empty[slot]));
+  return item;
+}
 __device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int m_tiles,
                                             int m_rows, int n_box, int& g, Item& it) {
   const int q = item / m_tiles;
@@ -294,7 +314,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
               void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
-              uint32_t* __restrict__ status) {
+              uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
@@ -347,6 +367,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int s = 0; s < kMaxStages; ++s) mbar_init(smem_u32(&ctl->slot_full[s]), 1);
+    for (int s = 0; s < kItemRing; ++s) {
+      mbar_init(smem_u32(&ctl->item_full[s]), 1);
+      // consumers: the MMA thread, one lane of every epilogue warp and of every converter warp
+      mbar_init(smem_u32(&ctl->item_empty[s]), 1u + (uint32_t)epi_warps + (FP8 ? 4u * (uint32_t)conv_groups : 0u));
+    }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[a]), (uint32_t)epi_warps * 32u);
@@ -403,9 +428,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     uint32_t phase = 0;
     bool ok = true;
     const int ring = n_stages;
-    for (int item = blockIdx.x; ok && !grp.withhold_loads && item < total_items; item += gridDim.x) {
+    // (with loads withheld - the test of the bounded waits - nothing is published either)
+    int item = grp.withhold_loads ? 0 : (int)atomicAdd(work_counter, 1u);
+    for (int seq = 0; ok && !grp.withhold_loads; ++seq) {
+      const bool none = item >= total_items;
+      // the next item's number is fetched now: the atomic's latency lies under this item's loads
+      const int next = none ? item : (int)atomicAdd(work_counter, 1u);
+      const int ring_slot = seq % kItemRing;
+      if (!mbar_wait(smem_u32(&ctl->item_empty[ring_slot]), ((uint32_t)(seq / kItemRing) & 1u) ^ 1u, abort_flag, status,
+                     nap_load)) {
+        ok = false;
+        break;
+      }
+      *reinterpret_cast<volatile int*>(&ctl->item_ring[ring_slot]) = none ? -1 : item;
+      mbar_arrive(smem_u32(&ctl->item_full[ring_slot]));
+      if (none) break;
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
+      item = next;
       for (int kb = 0; kb < k_blocks; ++kb) {
         const uint32_t free_bar = smem_u32(&ctl->empty[stage]);
         if (!mbar_wait(free_bar, phase ^ 1u, abort_flag, status, nap_load)) {
@@ -452,7 +492,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     const uint32_t a_tmem0 = tmem_base + a_col0;  // fp8 stores: weights come from tensor memory
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     uint32_t a_lo = a_lo0, b_lo = b_lo0, a_tmem = a_tmem0;
-    for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
+    for (; ok; ++local) {
+      const int item = take_item(ctl, local, abort_flag, status, 0u);
+      if (item < 0) break;
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
@@ -504,48 +546,58 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     // swizzle, so that the 32 rows of a quarter spread over all banks), widens them and stores
     // 32 columns of packed bf16 pairs with one tcgen05.st.
     const int group = conv_group, quarter = warp & 3;
-    int n_kb = 0;  // k-blocks of this CTA
-    if ((int)blockIdx.x < total_items && !grp.withhold_loads)
-      n_kb = ((total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * k_blocks;
     const uint32_t row = (uint32_t)(quarter * 32 + lane);
     const uint32_t sw = (row >> 1) & 3u;  // SWIZZLE_64B: 16-byte chunk index xor address bits 7-8
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + a_col0;
-    // ring positions of k-block i = group, group + conv_groups, ... (conv_groups divides both depths)
-    int stage = group;
+    // The CTA's k-blocks form one sequence across its items; this group takes every
+    // conv_groups-th of them (conv_groups divides the ring depth, so the group always meets the
+    // same stages).  `mine`: the group's next k-block, counted from the current item's first.
+    int stage = group, mine = group;
     uint32_t phase = 0;
-    for (int i = group; i < n_kb; i += conv_groups) {
-      int ok = 0;
-      if (lane == 0)
-        ok = (mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_conv) &&
-              mbar_wait(smem_u32(&ctl->slot_full[stage]), phase, abort_flag, status, nap_conv))
-                 ? 1 : 0;
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      __syncwarp();
-      tc_fence_after();  // the stage was released by the completion of the MMAs that read it
-      const uint32_t src = tiles_base + (uint32_t)stage * slot_ring_bytes + row * 64u;
-#pragma unroll
-      for (int tile = 0; tile < (dual ? 2 : 1); ++tile) {
-        uint4 c[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) c[j] = lds128(src + (uint32_t)tile * (kATile / 2) + (((uint32_t)j ^ sw) << 4));
-        uint32_t r[32];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          e4m3x4_to_bf16x4(c[j].x, r[8 * j], r[8 * j + 1]);
-          e4m3x4_to_bf16x4(c[j].y, r[8 * j + 2], r[8 * j + 3]);
-          e4m3x4_to_bf16x4(c[j].z, r[8 * j + 4], r[8 * j + 5]);
-          e4m3x4_to_bf16x4(c[j].w, r[8 * j + 6], r[8 * j + 7]);
+    bool live = true;
+    for (int seq = 0; live; ++seq) {
+      int item = 0;
+      if (lane == 0) item = take_item(ctl, seq, abort_flag, status, nap_conv);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item < 0) break;  // (the converters need the item's length only: every item has k_blocks k-blocks)
+      for (; mine < k_blocks; mine += conv_groups) {
+        int ok = 0;
+        if (lane == 0)
+          ok = (mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_conv) &&
+                mbar_wait(smem_u32(&ctl->slot_full[stage]), phase, abort_flag, status, nap_conv))
+                   ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+          live = false;
+          break;
         }
-        tmem_st32(t_lane + (uint32_t)stage * a_cols + (uint32_t)tile * 32u, r);
+        __syncwarp();
+        tc_fence_after();  // the stage was released by the completion of the MMAs that read it
+        const uint32_t src = tiles_base + (uint32_t)stage * slot_ring_bytes + row * 64u;
+#pragma unroll
+        for (int tile = 0; tile < (dual ? 2 : 1); ++tile) {
+          uint4 c[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) c[j] = lds128(src + (uint32_t)tile * (kATile / 2) + (((uint32_t)j ^ sw) << 4));
+          uint32_t r[32];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            e4m3x4_to_bf16x4(c[j].x, r[8 * j], r[8 * j + 1]);
+            e4m3x4_to_bf16x4(c[j].y, r[8 * j + 2], r[8 * j + 3]);
+            e4m3x4_to_bf16x4(c[j].z, r[8 * j + 4], r[8 * j + 5]);
+            e4m3x4_to_bf16x4(c[j].w, r[8 * j + 6], r[8 * j + 7]);
+          }
+          tmem_st32(t_lane + (uint32_t)stage * a_cols + (uint32_t)tile * 32u, r);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctl->full[stage]));  // (the slot itself is released by the MMAs' completion)
+        if ((stage += conv_groups) >= n_stages) {
+          stage -= n_stages;
+          phase ^= 1u;
+        }
       }
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->full[stage]));  // (the slot itself is released by the MMAs' completion)
-      if ((stage += conv_groups) >= n_stages) {
-        stage -= n_stages;
-        phase ^= 1u;
-      }
+      mine -= k_blocks;
     }
   } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
@@ -553,7 +605,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     int g = 0, local = 0;
     uint32_t xn = 0;  // stacked mode: 16-column chunks this warp's chunk group has exchanged so far
     bool alive = true;
-    for (int item = blockIdx.x; alive && item < total_items; item += gridDim.x, ++local) {
+    for (; alive; ++local) {
+      int item = 0;
+      if (lane == 0) item = take_item(ctl, local, abort_flag, status, nap_epi);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item < 0) break;
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
@@ -778,14 +834,14 @@ bool set_smem_attr() {
 template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
-                    const uint8_t* pool, size_t slot_bytes, uint32_t* status) {
+                    const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter) {
   const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8);
   if (fp8)
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
+               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
   else
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status);
+               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
 }
 
 }  // namespace
@@ -847,7 +903,7 @@ static int box_index(int max_count, int cap) {
 
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
-                  int n_sms, uint32_t* status) {
+                  int n_sms, uint32_t* status, uint32_t* work_counter) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   const bool fp8 = maps.fp8;
@@ -872,18 +928,18 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   }
   if (kind == 1 && grp.n_box <= 32 && use_stacked == 1) {
     launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
-                             0, maps.pool, maps.slot_bytes, status);
+                             0, maps.pool, maps.slot_bytes, status, work_counter);
   } else if (kind == 1) {
     launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
-                            maps.pool, maps.slot_bytes, status);
+                            maps.pool, maps.slot_bytes, status, work_counter);
   } else {
     const bool dual = grp.n_box == 256 || force_dual == 1;
     if (dual)
       launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
-                              y_bf16, maps.pool, maps.slot_bytes, status);
+                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter);
     else
       launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
-                               maps.pool, maps.slot_bytes, status);
+                               maps.pool, maps.slot_bytes, status, work_counter);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

@@ -110,8 +110,11 @@ struct FfnTcMaps {
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
+// work_counter: a device word that is ZERO when the kernel starts; its CTAs draw their work items
+// from it (every launch that can be in flight at the same time needs a word of its own).
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
-                  int I, int n_sms, uint32_t* status);
+                  int I, int n_sms, uint32_t* status, uint32_t* work_counter);
+constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 }  // namespace oled

@@ -57,7 +57,9 @@ struct oled_ctx {
   uint16_t* d_hbuf = nullptr;  // [T*k,I]
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
-  unsigned int* d_ticket = nullptr;   // last word of the control block
+  unsigned int* d_ticket = nullptr;   // control block, after the counts
+  uint32_t* d_work = nullptr;         // control block, last: work-item counters of the step's FFN launches
+  int work_next = 0;                  // next unused counter of the current layer execution
   bool ctrl_dirty = true;             // control block must be cleared before the next gate launch
   unsigned int seq = 0;               // step sequence number echoed by the gate kernel
   volatile unsigned long long* h_report = nullptr;  // pinned, mapped: tagged scores [E] | tagged counts [E]
@@ -242,8 +244,13 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
   } else {
     for (int kind = 1; kind <= 2; ++kind) {
       ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
+      // a fresh (zero) work counter per launch; a layer execution has at most three launch pairs,
+      // should there ever be more, a used word is cleared in stream order and taken again
+      uint32_t* work = ctx->d_work + ctx->work_next % kFfnWorkCounters;
+      if (ctx->work_next >= kFfnWorkCounters) OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
+      ctx->work_next += 1;
       const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
-                                   ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status);
+                                   ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work);
       if (rc != OLED_OK) return rc;
     }
   }
@@ -386,13 +393,14 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
-  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + 2 * sizeof(uint32_t);
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + (2 + kFfnWorkCounters) * sizeof(uint32_t);
   uint8_t* ctrl = nullptr;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctrl, ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
   ctx->d_scores = reinterpret_cast<unsigned long long*>(ctrl);
   ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
   ctx->d_ticket = reinterpret_cast<unsigned int*>(ctrl + E * (sizeof(unsigned long long) + sizeof(int32_t)));
+  ctx->d_work = reinterpret_cast<uint32_t*>(ctx->d_ticket) + 2;
   if ((rc = dev_alloc(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
@@ -510,6 +518,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   // 1. gate, counts and reuse-score numerators; the kernel's last CTA reports them to the host
   if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
   ctx->ctrl_dirty = true;
+  ctx->work_next = 0;
   ctx->seq += 1;
   RouteReport rep;
   rep.ticket = ctx->d_ticket;
