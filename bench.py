@@ -38,8 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # (many-token regime) a launch processes, so the ratio scales a capture to any launch.
 NCU_TRAFFIC_RATIO = {
     # profiles/ffn_tc_kernel_cfg2_full_residency.md: 63 experts x 4 tokens, H 2048, I 1024
-    ("ffn_gate_up", "few_tokens"): (521.34 + 3.96) / 530.1,
-    ("ffn_down", "few_tokens"): (260.61 + 5.42) / 267.0,
+    ("ffn_gate_up", "few_tokens"): (529.63 + 5.88) / 530.1,
+    ("ffn_down", "few_tokens"): (264.83 + 5.29) / 267.0,
+    # profiles/ffn_tc_kernel_fp8_cfg2_full_residency.md: the same launch with fp8 stores
+    ("ffn_gate_up", "few_tokens", "fp8"): (265.88 + 4.06) / 266.6,
+    ("ffn_down", "few_tokens", "fp8"): (133.23 + 4.07) / 135.2,
     # profiles/ffn_tc_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
     ("ffn_gate_up", "many_tokens"): (2091.3 + 102.3) / 1979.7,
     ("ffn_down", "many_tokens"): (973.8 + 524.4) / 1442.0,
@@ -390,7 +393,7 @@ def main():
                 "algorithmic_flops_per_launch": kp["flops"] / max(1, kp["launches"]),
                 "achieved_gbs": ach, "achieved_tflops": ach_tf}
     regime = "many_tokens" if w.tokens * w.top_k > 4096 else "few_tokens"
-    ratio = NCU_TRAFFIC_RATIO.get((top, regime))
+    ratio = NCU_TRAFFIC_RATIO.get((top, regime, "fp8") if fp8 else (top, regime))
     if ratio is not None:
         roofline["traffic"] = ratio * roofline["algorithmic_bytes_per_launch"]
         roofline["traffic_source"] = (f"ncu capture of the {regime.replace('_', '-')} regime (profiles/), scaled by "

@@ -229,8 +229,11 @@ void prof_add(oled_ctx* ctx, int kernel, uint64_t bytes, uint64_t flops) {
 // each expert's weights once, the token rows in, the result rows out.
 void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
   const uint64_t H = ctx->shape.hidden, I = ctx->shape.intermediate, hi = H * I;
-  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * 2 * hi * 2 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
-  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * hi * 2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4), 2 * rows * hi);
+  const bool fp8 = ctx->shape.expert_format == OLED_EXPERTS_FP8;
+  // weight bytes of one expert per kernel: bf16 elements, or e4m3 codes plus the fp32 row scales
+  const uint64_t w13 = fp8 ? 2 * hi + 2 * I * 4 : 2 * hi * 2, w2 = fp8 ? hi + H * 4 : hi * 2;
+  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * w13 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
+  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4), 2 * rows * hi);
 }
 
 // The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
