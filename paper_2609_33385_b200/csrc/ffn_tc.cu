@@ -343,13 +343,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
   const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
-  // fp8 stores: the four dedicated converter warps plus the epilogue warps this token tile leaves
-  // idle form conv_groups (1, 3 or 4) groups of four warps, one warp per TMEM lane quarter.
+  // fp8 stores: the four dedicated converter warps plus epilogue warps this token tile leaves
+  // idle form conv_groups (at most two: more of them take issue slots from the MMA thread and
+  // measured slower) groups of four warps, one warp per TMEM lane quarter.
   // Group g owns the k-blocks i with i mod conv_groups == g; conv_groups divides both ring
   // depths, so every load slot and every weight stage belongs to ONE group, which visits the
   // rounds of its barriers in order - a parity wait can then never take an older phase for the
   // one it wants.
   int conv_groups = FP8 ? 1 + (kEpiWarps - epi_warps) / 4 : 0;
+  if (conv_groups > (grp.pad > 0 ? grp.pad : 2)) conv_groups = grp.pad > 0 ? grp.pad : 2;  // (pad: tuning aid)
   if (conv_groups > 1 && n_stages % conv_groups != 0) conv_groups = 1;
   const int conv_group = !FP8 ? -1
                          : (warp >= kConvWarp0 && warp < kConvWarp0 + 4) ? 0
@@ -813,7 +815,7 @@ Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8) {
     r.stages = (int)std::min<uint32_t>((uint32_t)std::min(cap, 10), avail / (a + b));  // (11 measured slower)
     r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * (a + b);
   } else {
-    const int groups = 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4;
+    const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
     const int acc_cols = (dual ? 2 : 1) * n_box, a_cols = dual ? 64 : 32;
     const int free_cols = 512 - 2 * acc_cols >= 2 * a_cols ? 512 - 2 * acc_cols : 512 - acc_cols;
     r.stages = std::min(std::min(op_cap, kMaxStages), free_cols / a_cols);
@@ -907,6 +909,14 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   const bool fp8 = maps.fp8;
+  {
+    static int conv_cap = -1;  // tuning aid: OLED_FFN_CONV_GROUPS caps the fp8 converter groups
+    if (conv_cap < 0) {
+      const char* env = getenv("OLED_FFN_CONV_GROUPS");
+      conv_cap = env ? std::max(0, atoi(env)) : 0;
+    }
+    grp.pad = conv_cap;
+  }
   // N <= 128 keeps the accumulators double-buffered in TMEM; more tokens per expert than that
   // take N = 256 with two weight tiles per item (all 512 TMEM columns, one accumulator stage).
   // (fp8 stores stop at N = 128: the widened weights need tensor-memory columns of their own)
