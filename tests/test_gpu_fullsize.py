@@ -28,7 +28,10 @@ def _setup(w, **kw):
     ora = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, run.capacity)
     for l in range(w.n_layers):
         ora.register_router(l, run.router_bits[l], run.bias[l])
-        ora.register_experts(l, run.layer_blobs(l))
+        if kw.get("fp8"):
+            ora.register_experts_fp8(l, run.layer_blobs(l))
+        else:
+            ora.register_experts(l, run.layer_blobs(l))
     return run, ora
 
 
@@ -90,6 +93,21 @@ def test_config2_variant_b_block_shared_direction():
     run, ora = _setup(w, distinct_layers=2)
     try:
         _replay(run, ora, 6, sample_layers={1}, n_sample_tokens=2, rng=np.random.default_rng(2))
+    finally:
+        run.close()
+
+
+def test_config2_shape_fp8_expert_stores():
+    """The same layer shape with e4m3 + row-scale expert blobs (half the bytes per fill): the
+    router is not quantised, so every discrete result is that of the bf16 run; outputs are
+    compared with the oracle on the dequantised weights."""
+    w = synth.config(1, blocks=1, iters=3, n_layers=4)
+    run, ora = _setup(w, distinct_layers=1, fp8=True)
+    try:
+        _replay(run, ora, 3, sample_layers={0, 3}, n_sample_tokens=2, rng=np.random.default_rng(5))
+        st = run.ctx.stats()
+        assert st.bytes_moved == st.misses * run.ctx.expert_bytes
+        assert run.ctx.expert_bytes < 0.51 * w.expert_bytes
     finally:
         run.close()
 
