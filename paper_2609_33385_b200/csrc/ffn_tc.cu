@@ -312,7 +312,7 @@ template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
-              void* __restrict__ out_ptr, int H, int I, int n_stages, int out_bf16,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -329,11 +329,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // fp8 stores: a stage is a load slot in shared memory - the code tile (one byte per element)
   // followed by the token tile - plus a_cols columns of TENSOR memory, behind the accumulators,
   // for the widened weights.
+  // A stage spans k_atoms (1 or 2) k-blocks of 64, laid out one after the other, each as
+  // described above: small token tiles take two, which halves the waits and commits per byte on
+  // the serial path of the MMA thread.
   constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
-  const uint32_t slot_ring_bytes = raw_bytes + b_bytes;
-  constexpr uint32_t a_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
-  const int k_blocks = (KIND == 1 ? H : I) / kBlockK;
+  const uint32_t atom_bytes = FP8 ? raw_bytes + b_bytes : a_bytes + b_bytes;  // one k-block in shared memory
+  const uint32_t stage_bytes = (uint32_t)k_atoms * atom_bytes;
+  constexpr uint32_t atom_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
+  const uint32_t a_cols = (uint32_t)k_atoms * atom_cols;
+  const int k_blocks = (KIND == 1 ? H : I) / (kBlockK * k_atoms);  // stages per item
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (KIND == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
@@ -454,21 +458,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           ok = false;
           break;
         }
-        const uint32_t w_addr = tiles_base + (uint32_t)stage * (FP8 ? slot_ring_bytes : stage_bytes);
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[stage] : &ctl->full[stage]);
         constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
-        mbar_expect_tx(bar, (FP8 ? raw_bytes : a_bytes) + b_bytes);
-        if (stacked) {  // tm_w has 64-row boxes here
-          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);                  // 64 gate rows
-          tma_load_3d(&tm_w, w_addr + w_tile / 2, bar, kb * kBlockK, I + it.m0, it.slot);  // 64 up rows
-        } else if (KIND == 1) {
-          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);               // gate rows
-          tma_load_3d(&tm_w, w_addr + w_tile, bar, kb * kBlockK, I + it.m0, it.slot);  // up rows
-        } else {
-          tma_load_3d(&tm_w, w_addr, bar, kb * kBlockK, it.m0, it.slot);               // down rows
-          if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, kb * kBlockK, it.m0 + kBlockM, it.slot);
+        mbar_expect_tx(bar, stage_bytes);
+        for (int atom = 0; atom < k_atoms; ++atom) {
+          const uint32_t w_addr = tiles_base + (uint32_t)stage * stage_bytes + (uint32_t)atom * atom_bytes;
+          const int k0 = (kb * k_atoms + atom) * kBlockK;
+          if (stacked) {  // tm_w has 64-row boxes here
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
+            tma_load_3d(&tm_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
+          } else if (KIND == 1) {
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // gate rows
+            tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, I + it.m0, it.slot);  // up rows
+          } else {
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
+            if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
+          }
+          tma_load_2d(&tm_act, w_addr + (FP8 ? raw_bytes : a_bytes), bar, k0, it.row0);
         }
-        tma_load_2d(&tm_act, w_addr + (FP8 ? raw_bytes : a_bytes), bar, kb * kBlockK, it.row0);
         if (++stage == ring) {
           stage = 0;
           phase ^= 1u;
@@ -488,7 +495,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     // Descriptor words of stage 0 (K-major, 128-byte swizzle, 8-row groups 1024 bytes apart); the
     // low word holds the address in 16-byte units, the high word is the same for every operand.
     const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
-    const uint32_t ring_step = (FP8 ? slot_ring_bytes : stage_bytes) >> 4;
+    const uint32_t ring_step = atom_bytes >> 4;  // one k-block further in shared memory
     const uint32_t a_lo0 = (uint32_t)make_smem_desc(tiles_base);
     const uint32_t b_lo0 = (uint32_t)make_smem_desc(tiles_base + (FP8 ? raw_bytes : a_bytes));
     const uint32_t a_tmem0 = tmem_base + a_col0;  // fp8 stores: weights come from tensor memory
@@ -513,22 +520,25 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           break;
         }
         tc_fence_after();
-        const uint32_t first = kb != 0 ? 1u : 0u;
+        for (int atom = 0; atom < k_atoms; ++atom) {
+          const uint32_t first = (kb | atom) != 0 ? 1u : 0u;
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k) {  // 32 bytes along K = 2 address units
-          const uint32_t accum = k != 0 ? 1u : first;
-          if (FP8) {
-            tc_mma_ts_lo(d0, a_tmem + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
-            if (dual) tc_mma_ts_lo(d0 + (uint32_t)n_box, a_tmem + 32 + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
-          } else {
-            tc_mma_lo(d0, a_lo + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
-            if (dual) tc_mma_lo(d0 + (uint32_t)n_box, a_lo + (kATile >> 4) + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
+          for (int k = 0; k < kBlockK / 16; ++k) {  // 32 bytes along K = 2 address units
+            const uint32_t accum = k != 0 ? 1u : first;
+            if (FP8) {
+              tc_mma_ts_lo(d0, a_tmem + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
+              if (dual) tc_mma_ts_lo(d0 + (uint32_t)n_box, a_tmem + 32 + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
+            } else {
+              tc_mma_lo(d0, a_lo + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
+              if (dual)
+                tc_mma_lo(d0 + (uint32_t)n_box, a_lo + (kATile >> 4) + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
+            }
           }
+          a_lo += ring_step;
+          b_lo += ring_step;
+          a_tmem += atom_cols;
         }
         tc_commit(empty0 + (uint32_t)stage * 8u);
-        a_lo += ring_step;
-        b_lo += ring_step;
-        a_tmem += a_cols;
         if (++stage == n_stages) {
           stage = 0;
           phase ^= 1u;
@@ -575,21 +585,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
         __syncwarp();
         tc_fence_after();  // the stage was released by the completion of the MMAs that read it
-        const uint32_t src = tiles_base + (uint32_t)stage * slot_ring_bytes + row * 64u;
+        for (int atom = 0; atom < k_atoms; ++atom) {
+          const uint32_t src = tiles_base + (uint32_t)stage * stage_bytes + (uint32_t)atom * atom_bytes + row * 64u;
 #pragma unroll
-        for (int tile = 0; tile < (dual ? 2 : 1); ++tile) {
-          uint4 c[4];
+          for (int tile = 0; tile < (dual ? 2 : 1); ++tile) {
+            uint4 c[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) c[j] = lds128(src + (uint32_t)tile * (kATile / 2) + (((uint32_t)j ^ sw) << 4));
-          uint32_t r[32];
+            for (int j = 0; j < 4; ++j)
+              c[j] = lds128(src + (uint32_t)tile * (kATile / 2) + (((uint32_t)j ^ sw) << 4));
+            uint32_t r[32];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            e4m3x4_to_bf16x4(c[j].x, r[8 * j], r[8 * j + 1]);
-            e4m3x4_to_bf16x4(c[j].y, r[8 * j + 2], r[8 * j + 3]);
-            e4m3x4_to_bf16x4(c[j].z, r[8 * j + 4], r[8 * j + 5]);
-            e4m3x4_to_bf16x4(c[j].w, r[8 * j + 6], r[8 * j + 7]);
+            for (int j = 0; j < 4; ++j) {
+              e4m3x4_to_bf16x4(c[j].x, r[8 * j], r[8 * j + 1]);
+              e4m3x4_to_bf16x4(c[j].y, r[8 * j + 2], r[8 * j + 3]);
+              e4m3x4_to_bf16x4(c[j].z, r[8 * j + 4], r[8 * j + 5]);
+              e4m3x4_to_bf16x4(c[j].w, r[8 * j + 6], r[8 * j + 7]);
+            }
+            tmem_st32(t_lane + (uint32_t)stage * a_cols + (uint32_t)atom * atom_cols + (uint32_t)tile * 32u, r);
           }
-          tmem_st32(t_lane + (uint32_t)stage * a_cols + (uint32_t)tile * 32u, r);
         }
         tmem_st_wait();
         tc_fence_before();
@@ -789,41 +802,45 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
 }
 
 struct Rings {
-  int stages;     // weight stages: shared memory (bf16 stores) or tensor memory (fp8 stores)
+  int stages;     // pipeline stages
+  int k_atoms;    // k-blocks of 64 per stage
   uint32_t smem;  // dynamic shared memory of the launch
 };
 // Epilogue warps the kernel activates for a token tile (the others widen fp8 weights).
 int epi_warps_for(int kind, int out_bf16, int n_box) {
   return std::min((kind == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
 }
-// bf16 stores: as many stages (weight tile(s) + token tile) as fit in shared memory.  fp8 stores:
-// the weight stages take the tensor-memory columns the accumulators leave (two accumulator
-// stages if at least two weight stages still fit), all of shared memory is load slots; both
-// depths are multiples of the number of converter groups (see the kernel).
-Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8) {
-  static int cap = -1, op_cap = -1;  // tuning aids: OLED_FFN_STAGES caps the shared-memory ring depth,
-  if (cap < 0) {                     // OLED_FFN_OP_STAGES the fp8 weight ring in tensor memory
+// Stage shape and count.  A stage holds two k-blocks where at least four such stages fit (small
+// token tiles, one weight tile) and the contraction has an even number of k-blocks.  bf16 stores:
+// as many stages (weight tile(s) + token tile) as fit in shared memory, ten k-blocks at most
+// (eleven measured slower).  fp8 stores: a stage is a load slot in shared memory plus columns of
+// tensor memory behind the accumulators (two accumulator stages if at least two weight stages
+// still fit); the depth is a multiple of the number of converter groups (see the kernel).
+Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim) {
+  static int cap = -1, atoms_cap = -1;  // tuning aids: OLED_FFN_STAGES caps the ring depth (in
+  if (cap < 0) {                        // k-blocks), OLED_FFN_K_ATOMS the k-blocks per stage
     const char* env = getenv("OLED_FFN_STAGES");
     cap = env ? std::max(1, atoi(env)) : 64;
-    const char* env2 = getenv("OLED_FFN_OP_STAGES");
-    op_cap = env2 ? std::max(1, atoi(env2)) : kMaxStages;
+    const char* env2 = getenv("OLED_FFN_K_ATOMS");
+    atoms_cap = env2 ? std::max(1, std::min(2, atoi(env2))) : 2;
   }
   const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
-  Rings r;
-  if (!fp8) {
-    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(cap, 10), avail / (a + b));  // (11 measured slower)
-    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * (a + b);
-  } else {
-    const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
+  const uint32_t atom = fp8 ? a / 2 + b : a + b;  // one k-block in shared memory
+  int kblocks = (int)std::min<uint32_t>((uint32_t)std::min(cap, fp8 ? 2 * kMaxStages : 10), avail / atom);
+  if (fp8) {
     const int acc_cols = (dual ? 2 : 1) * n_box, a_cols = dual ? 64 : 32;
     const int free_cols = 512 - 2 * acc_cols >= 2 * a_cols ? 512 - 2 * acc_cols : 512 - acc_cols;
-    r.stages = std::min(std::min(op_cap, kMaxStages), free_cols / a_cols);
-    const uint32_t slot = a / 2 + b;
-    r.stages = (int)std::min<uint32_t>((uint32_t)std::min(r.stages, cap), avail / slot);
-    if (r.stages >= groups) r.stages -= r.stages % groups;
-    r.smem = kCtlBytes + 1024u + (uint32_t)r.stages * slot;
+    kblocks = std::min(kblocks, free_cols / a_cols);
   }
+  Rings r;
+  r.k_atoms = (atoms_cap >= 2 && !dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0) ? 2 : 1;
+  r.stages = std::min(kblocks / r.k_atoms, kMaxStages);
+  if (fp8) {
+    const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
+    if (r.stages >= groups) r.stages -= r.stages % groups;
+  }
+  r.smem = kCtlBytes + 1024u + (uint32_t)(r.stages * r.k_atoms) * atom;
   return r;
 }
 
@@ -837,13 +854,13 @@ template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter) {
-  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8);
+  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 1 ? H : I);
   if (fp8)
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
+               I, r.stages, r.k_atoms, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
   else
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
+               I, r.stages, r.k_atoms, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
 }
 
 }  // namespace
