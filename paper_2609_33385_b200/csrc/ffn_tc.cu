@@ -397,8 +397,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // ---- from here on the step's earlier kernels must have completed: work table from offsets
-  griddep_wait();
+  // ---- from here on the step's earlier kernels must have completed: work table from offsets.
+  // KIND 1 follows the permutation, whose products it reads from the first instruction on.  KIND 2
+  // follows KIND 1 of the same expert group: the offsets and the expert weights are older than
+  // that kernel, only the token tiles (hbuf) are its product - so a KIND 2 CTA, which gets its SM
+  // when a KIND 1 CTA leaves it, sets up and streams its first weight tiles while the slower SMs
+  // still finish KIND 1; its producer waits for the predecessor before the first token-tile load.
+  if (KIND == 1) griddep_wait();
   for (int g = threadIdx.x; g < grp.n; g += kThreads) {
     const int e = grp.expert[g];
     const int s = offsets[e];
@@ -452,17 +457,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       Item it;
       decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       item = next;
-      for (int kb = 0; kb < k_blocks; ++kb) {
-        const uint32_t free_bar = smem_u32(&ctl->empty[stage]);
-        if (!mbar_wait(free_bar, phase ^ 1u, abort_flag, status, nap_load)) {
-          ok = false;
-          break;
-        }
-        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[stage] : &ctl->full[stage]);
-        constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
+      constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
+      auto load_weights = [&](int st, int kb) {
+        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
         mbar_expect_tx(bar, stage_bytes);
         for (int atom = 0; atom < k_atoms; ++atom) {
-          const uint32_t w_addr = tiles_base + (uint32_t)stage * stage_bytes + (uint32_t)atom * atom_bytes;
+          const uint32_t w_addr = tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes;
           const int k0 = (kb * k_atoms + atom) * kBlockK;
           if (stacked) {  // tm_w has 64-row boxes here
             tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
@@ -474,8 +474,33 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
             if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
           }
-          tma_load_2d(&tm_act, w_addr + (FP8 ? raw_bytes : a_bytes), bar, k0, it.row0);
         }
+      };
+      auto load_tokens = [&](int st, int kb) {
+        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
+        for (int atom = 0; atom < k_atoms; ++atom)
+          tma_load_2d(&tm_act,
+                      tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (FP8 ? raw_bytes : a_bytes),
+                      bar, (kb * k_atoms + atom) * kBlockK, it.row0);
+      };
+      int kb = 0;
+      if (KIND == 2 && seq == 0) {
+        // the CTA's first stages (all free): weights now, token tiles once the predecessor is done
+        const int pre = min(n_stages, k_blocks);
+        for (int i = 0; i < pre; ++i) load_weights(i, i);
+        griddep_wait();
+        for (int i = 0; i < pre; ++i) load_tokens(i, i);
+        kb = pre;
+        if (pre == n_stages) phase ^= 1u;
+        else stage = pre;
+      }
+      for (; kb < k_blocks; ++kb) {
+        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_load)) {
+          ok = false;
+          break;
+        }
+        load_weights(stage, kb);
+        load_tokens(stage, kb);
         if (++stage == ring) {
           stage = 0;
           phase ^= 1u;
