@@ -148,9 +148,21 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
   griddep_launch_dependents();
+  constexpr int kRouteWarps = WARPS;
+  if (TT == 1) {
+    // Small steps: the router weights do not depend on the predecessor (the previous layer's
+    // combine), but the expert weights streamed since their last use have pushed them out of
+    // L2 - so they are called back in while this kernel still waits for its input.
+    for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        const int e = min(eb + b, E - 1);
+        for (int off = lane * 64; off < H; off += 32 * 64)  // 128-byte lines of the row
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(wr + (size_t)e * H + off));
+      }
+  }
   griddep_wait();
 
-  constexpr int kRouteWarps = WARPS;
   for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
     float acc[TT][kEPerWarp];
 #pragma unroll
