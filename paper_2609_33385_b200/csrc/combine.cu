@@ -10,7 +10,9 @@
 namespace oled {
 namespace {
 
-template <bool Y_BF16>
+// BATCH: the number of assignment rows whose loads are issued together.  Small steps (a few CTAs,
+// latency-bound) take 8; large steps keep 1, where the extra registers cost occupancy.
+template <bool Y_BF16, int BATCH>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
@@ -30,21 +32,35 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
   __syncthreads();
   for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j = 0; j < K; ++j) {
-      float4 v;
-      if (Y_BF16) {
-        const uint2 p = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(y) +
-                                                        (size_t)s_r[j] * H + h);
-        v = make_float4(__uint_as_float(p.x << 16), __uint_as_float(p.x & 0xffff0000u),
-                        __uint_as_float(p.y << 16), __uint_as_float(p.y & 0xffff0000u));
-      } else {
-        v = *reinterpret_cast<const float4*>(y + (size_t)s_r[j] * H + h);
+    // the rows of BATCH assignments are loaded together (independent requests in flight), then
+    // accumulated in rank order
+    for (int j0 = 0; j0 < K; j0 += BATCH) {
+      float4 v[BATCH];
+#pragma unroll
+      for (int jj = 0; jj < BATCH; ++jj) {
+        const int j = j0 + jj;
+        if (j < K) {
+          if (Y_BF16) {
+            const uint2 p = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(y) +
+                                                            (size_t)s_r[j] * H + h);
+            v[jj] = make_float4(__uint_as_float(p.x << 16), __uint_as_float(p.x & 0xffff0000u),
+                                __uint_as_float(p.y << 16), __uint_as_float(p.y & 0xffff0000u));
+          } else {
+            v[jj] = *reinterpret_cast<const float4*>(y + (size_t)s_r[j] * H + h);
+          }
+        }
       }
-      const float g = s_g[j];
-      acc.x = fmaf(g, v.x, acc.x);
-      acc.y = fmaf(g, v.y, acc.y);
-      acc.z = fmaf(g, v.z, acc.z);
-      acc.w = fmaf(g, v.w, acc.w);
+#pragma unroll
+      for (int jj = 0; jj < BATCH; ++jj) {
+        const int j = j0 + jj;
+        if (j < K) {
+          const float g = s_g[j];
+          acc.x = fmaf(g, v[jj].x, acc.x);
+          acc.y = fmaf(g, v[jj].y, acc.y);
+          acc.z = fmaf(g, v[jj].z, acc.z);
+          acc.w = fmaf(g, v[jj].w, acc.w);
+        }
+      }
     }
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
     __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
@@ -86,11 +102,18 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
                     uint32_t* zero_words, int n_zero_words) {
-  if (y_bf16)
-    launch_pdl(combine_kernel<true>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+  const bool small = (size_t)T * K <= 4096;
+  if (y_bf16 && small)
+    launch_pdl(combine_kernel<true, 8>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+               n_zero_words);
+  else if (y_bf16)
+    launch_pdl(combine_kernel<true, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+               n_zero_words);
+  else if (small)
+    launch_pdl(combine_kernel<false, 8>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
   else
-    launch_pdl(combine_kernel<false>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+    launch_pdl(combine_kernel<false, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
 }
 

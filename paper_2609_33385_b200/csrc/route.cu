@@ -310,12 +310,24 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   }
   if (xp == nullptr) return;
   __syncthreads();  // this CTA's perm entries are visible to all of its threads
+  // eight rows at a time: their token numbers, then their loads, are independent memory
+  // operations in flight together (a row-by-row loop is a chain of dependent round trips)
   const int vec_per_row = H / 8, first = s_base, rows = counts[e];
-  for (int i = threadIdx.x; i < rows * vec_per_row; i += blockDim.x) {
-    const int r = first + i / vec_per_row, c = i % vec_per_row;
-    const int t = perm[r] / K;
-    reinterpret_cast<uint4*>(xp)[(size_t)r * vec_per_row + c] =
-        reinterpret_cast<const uint4*>(x)[(size_t)t * vec_per_row + c];
+  const uint4* src = reinterpret_cast<const uint4*>(x);
+  uint4* dst = reinterpret_cast<uint4*>(xp);
+  for (int r0 = 0; r0 < rows; r0 += 8) {
+    int tok[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tok[j] = r0 + j < rows ? perm[first + r0 + j] / K : -1;
+    for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
+      uint4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (tok[j] >= 0) v[j] = src[(size_t)tok[j] * vec_per_row + c];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (tok[j] >= 0) dst[(size_t)(first + r0 + j) * vec_per_row + c] = v[j];
+    }
   }
 }
 
