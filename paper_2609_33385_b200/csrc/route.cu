@@ -43,11 +43,11 @@ __device__ __forceinline__ float exp_spec(float x) {
   return __fmul_rn(p, scale);
 }
 
-constexpr int kMaxEPerLane = OLED_MAX_EXPERTS / 32;
 
 // Top-k (ties to the lower index), gate scores over the selected logits, counts and integer
 // reuse-score numerators of one token; executed by one warp.  row: the token's E logits.
-__device__ __forceinline__ void route_token_tail(const float* row, int t, int lane, int E, int K,
+template <int kMaxEPerLane>  // E <= 32 * kMaxEPerLane: bounds the per-lane candidate scan
+__device__ __forceinline__ void route_token_tail_n(const float* row, int t, int lane, int E, int K,
                                                  const float* __restrict__ conf, int32_t* __restrict__ ids,
                                                  float* __restrict__ gate, int32_t* __restrict__ counts,
                                                  unsigned long long* __restrict__ scores) {
@@ -109,6 +109,16 @@ __device__ __forceinline__ void route_token_tail(const float* row, int t, int la
       atomicAdd(&scores[my_id], q);
     }
   }
+
+// The same selection whatever the bound: a tighter bound only drops candidates that do not exist.
+__device__ __forceinline__ void route_token_tail(const float* row, int t, int lane, int E, int K,
+                                                 const float* __restrict__ conf, int32_t* __restrict__ ids,
+                                                 float* __restrict__ gate, int32_t* __restrict__ counts,
+                                                 unsigned long long* __restrict__ scores) {
+  if (E <= 64) route_token_tail_n<2>(row, t, lane, E, K, conf, ids, gate, counts, scores);
+  else if (E <= 128) route_token_tail_n<4>(row, t, lane, E, K, conf, ids, gate, counts, scores);
+  else route_token_tail_n<OLED_MAX_EXPERTS / 32>(row, t, lane, E, K, conf, ids, gate, counts, scores);
+}
 
 // The last CTA to finish publishes counts and scores to the host (mapped pinned memory).
 // Every 8-byte word carries the step's sequence tag in its upper bits, so the host can tell
