@@ -21,6 +21,11 @@
 // one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
 // which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
 //
+// Work items (expert, token tile, weight tile) are drawn from a global counter by each CTA's
+// producer and handed to its other roles through a ring in shared memory (see take_item); a
+// pipeline stage holds one k-block of 64, or two for small token tiles; KIND 2 starts its weight
+// stream before its predecessor KIND 1 has finished (see the set-up in the kernel).
+//
 // Warp roles (704 threads): warps 0-15 epilogue (TMEM lane quarter = warp id mod 4, the warps of
 // a quarter interleave 16-column chunks; only as many as the token tile has chunks are active),
 // warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation),
