@@ -159,7 +159,7 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   const int t0 = blockIdx.x * TT;
   griddep_launch_dependents();
   constexpr int kRouteWarps = WARPS;
-  if (TT == 1) {
+  if (TT == 1 && gridDim.x <= 128) {
     // Small steps: the router weights do not depend on the predecessor (the previous layer's
     // combine), but the expert weights streamed since their last use have pushed them out of
     // L2 - so they are called back in while this kernel still waits for its input.
