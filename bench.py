@@ -44,8 +44,8 @@ NCU_TRAFFIC_RATIO = {
     ("ffn_gate_up", "few_tokens", "fp8"): (265.88 + 4.06) / 266.6,
     ("ffn_down", "few_tokens", "fp8"): (133.23 + 4.07) / 135.2,
     # profiles/ffn_tc_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
-    ("ffn_gate_up", "many_tokens"): (2091.3 + 102.3) / 1979.7,
-    ("ffn_down", "many_tokens"): (973.8 + 524.4) / 1442.0,
+    ("ffn_gate_up", "many_tokens"): (1916.5 + 102.1) / 1979.7,
+    ("ffn_down", "many_tokens"): (911.8 + 264.5) / 1174.4,
 }
 
 
