@@ -445,6 +445,16 @@ def main():
             "kernels": {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
                             "gbs": (v["bytes"] / v["ms"] / 1e6) if v["ms"] > 0 else None}
                         for k, v in pf.items()}}
+        # the dominant kernel without expert fills in flight (they slow an overlapping launch)
+        kf = pf.get(top)
+        if kf and kf["ms"] > 0 and not tensor_bound:
+            ach_f = kf["bytes"] / kf["ms"] / 1e6
+            extra["full_residency"]["roofline"] = {
+                "kernel": top, "bound": "hbm", "achieved": ach_f, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach_f / peaks["hbm_gbs"], "launches": kf["launches"],
+                "avg_launch_us": kf["ms"] * 1e3 / max(1, kf["launches"])}
+            roofline["note"] = ("launches that overlap the expert fills run slower than alone; "
+                                "full_residency.roofline is the same kernel with no fill in flight")
         extra["tpot_ratio_vs_full_residency"] = ms_per_step / msf
         # lower bound of that ratio given the measured link: the fills that cannot hide
         extra["tpot_ratio_min_from_link"] = max(1.0, step_roof["terms_ms"]["host_link"] / msf)
