@@ -49,6 +49,10 @@ NCU_TRAFFIC_RATIO = {
 }
 
 
+# nominal figures of a B200 (HGX) and of its PCIe Gen5 x16 host link, per direction
+NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "h2d_gbs": 63.0}
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -272,8 +276,12 @@ def step_roofline(w, delta, steps, ms_per_step, peaks, h2d_gbs, blob=None):
     t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
     terms = {"hbm": t_hbm, "host_link": t_h2d, "tensor": t_tc}
     bound = max(terms, key=terms.get)
+    # the same bound against the nominal figures of the part (context; the headline uses measured peaks)
+    nominal = {"hbm": b_hbm / (NOMINAL["hbm_gbs"] * 1e9) * 1e3, "host_link": b_h2d / (NOMINAL["h2d_gbs"] * 1e9) * 1e3,
+               "tensor": flops / (NOMINAL["bf16_tflops"] * 1e12) * 1e3}
     return {"bound": bound, "t_roof_ms": terms[bound], "t_measured_ms": ms_per_step,
             "frac": terms[bound] / ms_per_step, "terms_ms": terms,
+            "frac_of_nominal": nominal[bound] / ms_per_step, "nominal_peaks": NOMINAL,
             "hbm_bytes_per_step": b_hbm, "h2d_bytes_per_step": b_h2d, "flops_per_step": flops}
 
 
