@@ -83,6 +83,63 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
   }
 }
 
+// Large steps with bf16 assignment outputs: eight elements per thread, so that every access is
+// a 16-byte vector (the four-element form above reads 8 bytes per lane and row).
+__global__ void __launch_bounds__(256)
+combine_bf16_wide_kernel(const uint16_t* __restrict__ y, const float* __restrict__ gate,
+                         const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
+                         const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next,
+                         uint32_t* __restrict__ zero_words, int n_zero_words) {
+  const int t = blockIdx.x;
+  griddep_launch_dependents();
+  griddep_wait();
+  if (t == 0 && zero_words != nullptr)
+    for (int i = threadIdx.x; i < n_zero_words; i += blockDim.x) zero_words[i] = 0u;
+  __shared__ float s_g[OLED_MAX_TOPK];
+  __shared__ int s_r[OLED_MAX_TOPK];
+  if (threadIdx.x < K) {
+    s_g[threadIdx.x] = gate[(size_t)t * K + threadIdx.x];
+    s_r[threadIdx.x] = pos[(size_t)t * K + threadIdx.x];
+  }
+  __syncthreads();
+  for (int h = threadIdx.x * 8; h < H; h += blockDim.x * 8) {
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int j = 0; j < K; ++j) {  // rank order
+      const uint4 p = *reinterpret_cast<const uint4*>(y + (size_t)s_r[j] * H + h);
+      const float g = s_g[j];
+      const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc[2 * i] = fmaf(g, __uint_as_float(w[i] << 16), acc[2 * i]);
+        acc[2 * i + 1] = fmaf(g, __uint_as_float(w[i] & 0xffff0000u), acc[2 * i + 1]);
+      }
+    }
+    uint32_t o[4];
+    __nv_bfloat162 ob[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      ob[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+      o[i] = *reinterpret_cast<uint32_t*>(&ob[i]);
+    }
+    *reinterpret_cast<uint4*>(out + (size_t)t * H + h) = make_uint4(o[0], o[1], o[2], o[3]);
+    if (x_next != nullptr) {  // residual on the rounded output: bf16(x + bf16(out))
+      const uint4 xv = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+      const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+      uint32_t r[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 of = __bfloat1622float2(ob[i]);
+        __nv_bfloat162 rb = __floats2bfloat162_rn(__uint_as_float(xw[i] << 16) + of.x,
+                                                  __uint_as_float(xw[i] & 0xffff0000u) + of.y);
+        r[i] = *reinterpret_cast<uint32_t*>(&rb);
+      }
+      *reinterpret_cast<uint4*>(x_next + (size_t)t * H + h) = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(256)
 residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ r,
                     uint16_t* __restrict__ y, size_t n) {
@@ -106,6 +163,9 @@ void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* ga
   if (y_bf16 && small)
     launch_pdl(combine_kernel<true, 8>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
+  else if (y_bf16 && H % 8 == 0)
+    launch_pdl(combine_bf16_wide_kernel, dim3(T), dim3(256), 0, st, reinterpret_cast<const uint16_t*>(y), gate, pos, H,
+               K, out, x, x_next, zero_words, n_zero_words);
   else if (y_bf16)
     launch_pdl(combine_kernel<true, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);

@@ -341,20 +341,29 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   }
 }
 
+// One warp per sorted row: the row's token number once, then the row's 16-byte vectors, four
+// loads in flight per lane.
 __global__ void __launch_bounds__(256)
 gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, int n_rows, int H,
               int K, uint16_t* __restrict__ xp) {
   const int vec_per_row = H / 8;
-  const size_t total = (size_t)n_rows * vec_per_row;
+  const int lane = threadIdx.x & 31;
+  const int warps = gridDim.x * (blockDim.x >> 5);
   griddep_launch_dependents();
   griddep_wait();
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-       i += (size_t)gridDim.x * blockDim.x) {
-    const int r = (int)(i / vec_per_row);
-    const int c = (int)(i % vec_per_row);
+  for (int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n_rows; r += warps) {
     const int t = perm[r] / K;
-    reinterpret_cast<uint4*>(xp)[(size_t)r * vec_per_row + c] =
-        reinterpret_cast<const uint4*>(x)[(size_t)t * vec_per_row + c];
+    const uint4* src = reinterpret_cast<const uint4*>(x) + (size_t)t * vec_per_row;
+    uint4* dst = reinterpret_cast<uint4*>(xp) + (size_t)r * vec_per_row;
+    for (int c0 = lane; c0 < vec_per_row; c0 += 128) {
+      uint4 v[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (c0 + 32 * j < vec_per_row) v[j] = src[c0 + 32 * j];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (c0 + 32 * j < vec_per_row) dst[c0 + 32 * j] = v[j];
+    }
   }
 }
 
