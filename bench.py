@@ -38,8 +38,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # (many-token regime) a launch processes, so the ratio scales a capture to any launch.
 NCU_TRAFFIC_RATIO = {
     # profiles/ffn_tc_kernel_cfg2_full_residency.md: 63 experts x 4 tokens, H 2048, I 1024
-    ("ffn_gate_up", "few_tokens"): (529.63 + 5.88) / 530.1,
-    ("ffn_down", "few_tokens"): (264.83 + 5.29) / 267.0,
+    ("ffn_gate_up", "few_tokens"): (529.62 + 5.63) / 530.1,
+    ("ffn_down", "few_tokens"): (264.86 + 5.34) / 267.0,
     # profiles/ffn_tc_kernel_fp8_cfg2_full_residency.md: the same launch with fp8 stores
     ("ffn_gate_up", "few_tokens", "fp8"): (265.88 + 4.06) / 266.6,
     ("ffn_down", "few_tokens", "fp8"): (133.23 + 4.07) / 135.2,
