@@ -124,6 +124,9 @@ int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob,
  *   out          device [n_tokens,H] bf16: sum_j g[t,j]*FFN_{e(t,j)}(hidden[t]); must not alias hidden.
  * Buffers are borrowed until the enqueued work completes on the context's stream.  The layer's
  * resident set and the counters are updated before the call returns.
+ * Non-finite activations do not break the step: a NaN gate logit ranks as -inf (the k expert
+ * ids of a token stay distinct), a NaN gate*confidence product adds nothing to the reuse score,
+ * the outputs of the affected tokens are NaN and those of the other tokens are unaffected.
  * Errors: INVALID_ARG, NOT_REGISTERED, TOO_MANY_TOKENS, NO_SLOT, CUDA, TIMEOUT (reported by
  * the next call that synchronises). */
 int oled_denoise_step(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
