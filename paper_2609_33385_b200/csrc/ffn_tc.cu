@@ -145,7 +145,7 @@ template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
-              void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int out_bf16,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int early_start, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -240,7 +240,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // that kernel, only the token tiles (hbuf) are its product - so a KIND 2 CTA, which gets its SM
   // when a KIND 1 CTA leaves it, sets up and streams its first weight tiles while the slower SMs
   // still finish KIND 1; its producer waits for the predecessor before the first token-tile load.
-  if (KIND == 1) griddep_wait();
+  // (early_start is set by the host only when a CTA of this kernel and a CTA of the KIND 1 kernel
+  // before it do not fit into one SM's shared memory together, which is what keeps a KIND 2 CTA
+  // from starting while a KIND 1 CTA on that SM still waits for the permutation)
+  const bool early = KIND == 2 && early_start != 0;
+  if (!early) griddep_wait();
   for (int g = threadIdx.x; g < grp.n; g += kThreads) {
     const int e = grp.expert[g];
     const int s = offsets[e];
@@ -321,7 +325,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
                       bar, (kb * k_atoms + atom) * kBlockK, it.row0);
       };
       int kb = 0;
-      if (KIND == 2 && seq == 0) {
+      if (early && seq == 0) {
         // the CTA's first stages (all free): weights now, token tiles once the predecessor is done
         const int pre = min(n_stages, k_blocks);
         for (int i = 0; i < pre; ++i) load_weights(i, i);
@@ -715,14 +719,18 @@ bool set_smem_attr() {
 template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
-                    const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter) {
+                    const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter,
+                    uint32_t smem_of_predecessor) {
   const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 1 ? H : I);
+  // KIND 2 may start ahead of its dependency wait only if one of its CTAs and one of the KIND 1
+  // kernel before it cannot share an SM (see the kernel's set-up)
+  const int early = (KIND == 2 && smem_of_predecessor + r.smem > 228u * 1024u) ? 1 : 0;
   if (fp8)
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, r.k_atoms, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
+               I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
   else
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
-               I, r.stages, r.k_atoms, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
+               I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter);
 }
 
 }  // namespace
@@ -815,20 +823,23 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     use_stacked = a ? atoi(a) : 1;
     force_dual = b ? atoi(b) : 0;
   }
-  if (kind == 1 && grp.n_box <= 32 && use_stacked == 1) {
+  // shared memory of a CTA of this group's KIND 1 launch
+  const bool stacked1 = grp.n_box <= 32 && use_stacked == 1;
+  const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
+  if (kind == 1 && stacked1) {
     launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
-                             0, maps.pool, maps.slot_bytes, status, work_counter);
+                             0, maps.pool, maps.slot_bytes, status, work_counter, smem1);
   } else if (kind == 1) {
     launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
-                            maps.pool, maps.slot_bytes, status, work_counter);
+                            maps.pool, maps.slot_bytes, status, work_counter, smem1);
   } else {
     const bool dual = grp.n_box == 256 || force_dual == 1;
     if (dual)
       launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
-                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter);
+                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1);
     else
       launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
-                               maps.pool, maps.slot_bytes, status, work_counter);
+                               maps.pool, maps.slot_bytes, status, work_counter, smem1);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
