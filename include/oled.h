@@ -50,7 +50,8 @@ typedef enum {
   OLED_ERR_CUDA = -6,           /* a CUDA call failed; see oled_last_cuda_error()               */
   OLED_ERR_TIMEOUT = -7,        /* a bounded device-side wait ran out; the step's out is invalid */
   OLED_ERR_NO_SLOT = -8,        /* staging_slots too small for this step's misses               */
-  OLED_ERR_STALE_DEBUG = -9     /* oled_debug_last(): the last step was on another layer        */
+  OLED_ERR_STALE_DEBUG = -9,    /* oled_debug_last(): the last step was on another layer        */
+  OLED_ERR_SELF_CHECK = -10     /* OLED_OPT_SELF_CHECK found a violation; oled_self_check_report() */
 } oled_status;
 
 typedef struct oled_ctx oled_ctx; /* opaque, owned by the library */
@@ -190,6 +191,22 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
 #define OLED_OPT_POLICY 4
 #define OLED_OPT_ADAPT_PERIOD 5
 #define OLED_OPT_TEST_WITHHOLD_LOADS 6
+/* OLED_OPT_SELF_CHECK: 1 = every step also runs two checking kernels (the paper has no counterpart;
+ * they stand in for a memory checker): after the permutation, the invariants all later addressing
+ * relies on (OLED_CHECK_* below); after the combine, the guard words behind the step's scratch
+ * buffers.  A violation is sticky like a time-out: the next synchronising call returns
+ * OLED_ERR_SELF_CHECK, oled_self_check_report() tells what was found, oled_clear_status() re-arms.
+ * OLED_OPT_TEST_CORRUPT_PERM: test aid for that path.  1 = the first two rows of the sorted order
+ * are exchanged after the permutation (both stay valid rows; the step's output is wrong). */
+#define OLED_OPT_SELF_CHECK 7
+#define OLED_OPT_TEST_CORRUPT_PERM 8
+#define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */
+#define OLED_CHECK_ID_DUPLICATE 0x02u  /* a token routed twice to one expert                        */
+#define OLED_CHECK_OFFSETS 0x04u       /* offsets are not the exclusive scan of the counts          */
+#define OLED_CHECK_PERM_RANGE 0x08u    /* a sorted row names no assignment                          */
+#define OLED_CHECK_INVERSE 0x10u       /* pos is not the inverse of perm                            */
+#define OLED_CHECK_ROW_EXPERT 0x20u    /* a sorted row lies outside the range of its expert         */
+#define OLED_CHECK_ORDER 0x40u         /* the rows of an expert are not in ascending (token, rank)  */
 #define OLED_POLICY_PRIORITY 0 /* confidence- and gate-guided priority, Sec. 4.3 (default) */
 #define OLED_POLICY_LRU 1      /* comparison point: least recently used (Sec. 5.1 Naive-LRU)  */
 #define OLED_POLICY_LFU 2      /* comparison point: least frequently used (Sec. 5.3)          */
@@ -228,6 +245,14 @@ int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_
 
 /* Clears a recorded device-side time-out (OLED_ERR_TIMEOUT is sticky until then).  Synchronises. */
 int oled_clear_status(oled_ctx* ctx);
+
+/* What OLED_OPT_SELF_CHECK has found since the status was last cleared.  Synchronises.
+ *   flags        OR of OLED_CHECK_* (0 = nothing).
+ *   first_index  the smallest offending index (assignment, expert or sorted row, by flag), -1 if none.
+ *   guard_mask   bit b set = the guard words behind scratch buffer b were overwritten (order:
+ *                logits, ids, gate, offsets, perm, pos, sorted token rows, intermediate, outputs).
+ * Any pointer may be NULL. */
+int oled_self_check_report(oled_ctx* ctx, uint32_t* flags, int32_t* first_index, uint32_t* guard_mask);
 
 /* Host time spent in the cache policy (hit/miss resolution, Top-C retention, slot plan) so far, in
  * nanoseconds, and the number of policy runs - the "policy overhead" of Sec. 5.4. */

@@ -24,6 +24,10 @@ ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -
 ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -9
 OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE, OPT_POLICY, OPT_ADAPT_PERIOD = 1, 2, 3, 4, 5
 OPT_TEST_WITHHOLD_LOADS = 6
+OPT_SELF_CHECK, OPT_TEST_CORRUPT_PERM = 7, 8
+ERR_SELF_CHECK = -10
+CHECK_FLAGS = {0x01: "id_range", 0x02: "id_duplicate", 0x04: "offsets", 0x08: "perm_range", 0x10: "inverse",
+               0x20: "row_expert", 0x40: "order"}
 POLICY_PRIORITY, POLICY_LRU, POLICY_LFU = 0, 1, 2
 POLICY_IDS = {"priority": 0, "lru": 1, "lfu": 2}
 KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
@@ -36,6 +40,7 @@ EXPORTS = [
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
     "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
     "oled_policy_adapt", "oled_clear_status", "oled_policy_time", "oled_expert_blob_bytes",
+    "oled_self_check_report",
 ]
 EXPERTS_BF16, EXPERTS_FP8 = 0, 1
 NOALLOC_MAX_TOKENS = 256
@@ -124,6 +129,7 @@ def load() -> C.CDLL:
     lib.oled_expert_blob_bytes.argtypes = [i32, i32, i32]
     lib.oled_expert_blob_bytes.restype = C.c_size_t
     lib.oled_clear_status.argtypes = [vp]
+    lib.oled_self_check_report.argtypes = [vp, vp, vp, vp]
     lib.oled_policy_time.argtypes = [vp, u64p, u64p]
     lib.oled_adapt_capacity.argtypes = [vp, vp]
     lib.oled_get_capacity.argtypes = [vp, vp]
@@ -261,6 +267,14 @@ class OledContext:
 
     def clear_status(self) -> None:
         self._check(self._lib.oled_clear_status(self._h), "oled_clear_status")
+
+    def self_check_report(self):
+        """(names of the violated invariants, smallest offending index or -1, guard mask)."""
+        flags, index, guard = C.c_uint32(0), C.c_int32(-1), C.c_uint32(0)
+        self._check(self._lib.oled_self_check_report(self._h, C.byref(flags), C.byref(index),
+                                                     C.byref(guard)), "oled_self_check_report")
+        names = [n for bit, n in CHECK_FLAGS.items() if flags.value & bit]
+        return names, index.value, guard.value
 
     def policy_time(self):
         """(nanoseconds spent in the host cache policy, number of policy runs)."""

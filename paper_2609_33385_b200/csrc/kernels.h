@@ -53,6 +53,18 @@ struct FfnGroup {
 
 // Device status word values (0 = ok).
 enum : uint32_t { kStatusOk = 0, kStatusWaitTimeout = 1 };
+// The context's status block (device words): a bounded wait that ran out; flags and smallest
+// offending index of the self-check; one bit per scratch buffer whose guard words were overwritten.
+enum : int { kStatusWait = 0, kStatusCheckFlags = 1, kStatusCheckIndex = 2, kStatusGuardMask = 3, kStatusWords = 4 };
+constexpr uint32_t kStatusNoIndex = 0x7fffffffu;  // initial value of the index word
+
+// Guard words behind the step's scratch buffers (checked when OLED_OPT_SELF_CHECK is on).
+constexpr int kGuardWords = 16;
+constexpr uint32_t kGuardPattern = 0xC0DEC0DEu;
+struct GuardList {
+  int n;
+  uint32_t* words[12];
+};
 
 // Where the gate kernel's last CTA publishes the step's counts and scores for the host: mapped
 // pinned host memory, one 8-byte word per value with the step's sequence number in the upper
@@ -116,5 +128,12 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, i
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
                   int I, int n_sms, uint32_t* status, uint32_t* work_counter);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
+
+// Self-check (check.cu): invariants of the routing and the permutation, guard words.
+void launch_self_check(cudaStream_t st, const int32_t* ids, const int32_t* counts, const int32_t* offsets,
+                       const int32_t* perm, const int32_t* pos, int T, int E, int K, uint32_t* status);
+void launch_guard_check(cudaStream_t st, const GuardList& guards, uint32_t* status);
+void launch_guard_fill(cudaStream_t st, const GuardList& guards);
+void launch_corrupt_perm(cudaStream_t st, int32_t* perm, int n);  // test aid
 
 }  // namespace oled

@@ -84,6 +84,9 @@ struct oled_ctx {
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
   int miss_chunk = 4;
   int withhold_loads = 0;      // test aid, see OLED_OPT_TEST_WITHHOLD_LOADS
+  int self_check = 0;          // OLED_OPT_SELF_CHECK
+  int corrupt_perm = 0;        // test aid, see OLED_OPT_TEST_CORRUPT_PERM
+  GuardList guards{};          // guard words behind the step's scratch buffers
   uint64_t policy_ns = 0, policy_runs = 0;
   long long total_capacity = 0;
   int adapt_period = 0;        // iterations between automatic capacity refreshes (0 = off)
@@ -119,14 +122,30 @@ int dev_alloc(oled_ctx* ctx, T** p, size_t n) {
   return OLED_OK;
 }
 
+// A scratch buffer of n elements followed by guard words (16-byte aligned), which the self-check
+// verifies after every step: a kernel that writes past its buffer shows up there.
+template <typename T>
+int dev_alloc_guarded(oled_ctx* ctx, T** p, size_t n) {
+  const size_t bytes = (std::max<size_t>(n, 1) * sizeof(T) + 15) / 16 * 16;
+  uint8_t* q = nullptr;
+  const int rc = dev_alloc(ctx, &q, bytes + kGuardWords * sizeof(uint32_t));
+  if (rc != OLED_OK) return rc;
+  *p = reinterpret_cast<T*>(q);
+  if (ctx->guards.n < (int)(sizeof(ctx->guards.words) / sizeof(ctx->guards.words[0])))
+    ctx->guards.words[ctx->guards.n++] = reinterpret_cast<uint32_t*>(q + bytes);
+  return OLED_OK;
+}
+
 int check_status(oled_ctx* ctx) {
-  if (ctx->h_status && *ctx->h_status != kStatusOk) return OLED_ERR_TIMEOUT;
+  if (!ctx->h_status) return OLED_OK;
+  if (ctx->h_status[kStatusWait] != kStatusOk) return OLED_ERR_TIMEOUT;
+  if (ctx->h_status[kStatusCheckFlags] != 0 || ctx->h_status[kStatusGuardMask] != 0) return OLED_ERR_SELF_CHECK;
   return OLED_OK;
 }
 
 int sync_all(oled_ctx* ctx) {
   OLED_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
-  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost,
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, kStatusWords * sizeof(uint32_t), cudaMemcpyDeviceToHost,
                                  ctx->stream));
   OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
   return check_status(ctx);
@@ -336,6 +355,7 @@ const char* oled_strerror(int code) {
     case OLED_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case OLED_ERR_NO_SLOT: return "not enough staging slots for this step's misses";
     case OLED_ERR_STALE_DEBUG: return "the most recent step was on another layer";
+    case OLED_ERR_SELF_CHECK: return "the self-check found a violation (see oled_self_check_report)";
     default: return "unknown error";
   }
 }
@@ -404,16 +424,16 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
   ctx->d_ticket = reinterpret_cast<unsigned int*>(ctrl + E * (sizeof(unsigned long long) + sizeof(int32_t)));
   ctx->d_work = reinterpret_cast<uint32_t*>(ctx->d_ticket) + 2;
-  if ((rc = dev_alloc(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_offsets, E + 1)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_perm, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_pos, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_xp, T * K * H)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_hbuf, T * K * I)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_y, T * K * H)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctx->d_status, 1)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_offsets, E + 1)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_perm, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_pos, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_xp, T * K * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_hbuf, T * K * I)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_y, T * K * H)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_status, kStatusWords)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_hidden_stage, T * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_conf_stage, T)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_out_stage, T * H)) != OLED_OK) return fail(rc);
@@ -424,14 +444,16 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
     if (s.has_router_bias && (rc = dev_alloc(ctx, &ctx->layers[l].bias, E)) != OLED_OK) return fail(rc);
   }
   if (cudaMallocHost(reinterpret_cast<void**>(&ctx->h_ctrl), 2 * E * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMallocHost(reinterpret_cast<void**>(&ctx->h_status), sizeof(uint32_t)) != cudaSuccess)
+      cudaMallocHost(reinterpret_cast<void**>(&ctx->h_status), kStatusWords * sizeof(uint32_t)) != cudaSuccess)
     return fail(OLED_ERR_OOM);
-  *ctx->h_status = kStatusOk;
+  memset(ctx->h_status, 0, kStatusWords * sizeof(uint32_t));
+  ctx->h_status[kStatusCheckIndex] = kStatusNoIndex;
   memset(ctx->h_ctrl, 0, 2 * E * sizeof(unsigned long long));
   ctx->h_report = reinterpret_cast<volatile unsigned long long*>(ctx->h_ctrl);
   ctx->host_scores.assign(E, 0);
   ctx->host_counts.assign(E, 0);
-  if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess ||
+  launch_guard_fill(ctx->stream, ctx->guards);
+  if (cudaMemcpy(ctx->d_status, ctx->h_status, kStatusWords * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemset(ctx->d_xp, 0, T * K * H * 2) != cudaSuccess ||
       cudaMemset(ctx->d_hbuf, 0, T * K * I * 2) != cudaSuccess ||
       cudaMemset(ctx->d_y, 0, T * K * H * 4) != cudaSuccess)
@@ -545,6 +567,14 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
   }
   ctx->launches += fuse_gather ? 2 : 3;
+  if (ctx->corrupt_perm) {
+    launch_corrupt_perm(st, ctx->d_perm, T * K);
+    ctx->launches += 1;
+  }
+  if (ctx->self_check) {
+    launch_self_check(st, ctx->d_ids, ctx->d_counts, ctx->d_offsets, ctx->d_perm, ctx->d_pos, T, E, K, ctx->d_status);
+    ctx->launches += 1;
+  }
   OLED_CUDA(ctx, cudaGetLastError());
 
   // 1b. cache hits need no decision: the FFN over the experts resident BEFORE the step is
@@ -635,6 +665,10 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
                    reinterpret_cast<uint32_t*>(ctx->d_scores), (int)(ctx->ctrl_bytes / 4));
   }
   ctx->launches += 1;
+  if (ctx->self_check) {
+    launch_guard_check(st, ctx->guards, ctx->d_status);
+    ctx->launches += 1;
+  }
   OLED_CUDA(ctx, cudaGetLastError());
   ctx->ctrl_dirty = false;  // combine's CTA 0 cleared the control block for the next step
 
@@ -831,6 +865,12 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
     case OLED_OPT_TEST_WITHHOLD_LOADS:
       ctx->withhold_loads = value != 0 ? 1 : 0;
       return OLED_OK;
+    case OLED_OPT_SELF_CHECK:
+      ctx->self_check = value != 0 ? 1 : 0;
+      return OLED_OK;
+    case OLED_OPT_TEST_CORRUPT_PERM:
+      ctx->corrupt_perm = value != 0 ? 1 : 0;
+      return OLED_OK;
     case OLED_OPT_MISS_CHUNK:
       if (value < 1) return OLED_ERR_INVALID_ARG;
       ctx->miss_chunk = (int)std::min<int64_t>(value, OLED_MAX_EXPERTS);
@@ -852,9 +892,22 @@ int oled_profile_read(oled_ctx* ctx, int32_t kernel, int32_t reset, oled_kernel_
 int oled_clear_status(oled_ctx* ctx) {
   if (!ctx) return OLED_ERR_INVALID_ARG;
   OLED_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
-  OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), ctx->stream));
+  memset(ctx->h_status, 0, kStatusWords * sizeof(uint32_t));
+  ctx->h_status[kStatusCheckIndex] = kStatusNoIndex;
+  OLED_CUDA(ctx, cudaMemcpyAsync(ctx->d_status, ctx->h_status, kStatusWords * sizeof(uint32_t), cudaMemcpyHostToDevice,
+                                 ctx->stream));
   OLED_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-  *ctx->h_status = kStatusOk;
+  return OLED_OK;
+}
+
+int oled_self_check_report(oled_ctx* ctx, uint32_t* flags, int32_t* first_index, uint32_t* guard_mask) {
+  if (!ctx) return OLED_ERR_INVALID_ARG;
+  const int rc = sync_all(ctx);
+  if (rc != OLED_OK && rc != OLED_ERR_SELF_CHECK && rc != OLED_ERR_TIMEOUT) return rc;
+  const uint32_t f = ctx->h_status[kStatusCheckFlags];
+  if (flags) *flags = f;
+  if (first_index) *first_index = f != 0 ? (int32_t)ctx->h_status[kStatusCheckIndex] : -1;
+  if (guard_mask) *guard_mask = ctx->h_status[kStatusGuardMask];
   return OLED_OK;
 }
 

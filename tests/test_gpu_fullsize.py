@@ -4,7 +4,8 @@ sequence of step + fused-residual launches that is replayed here layer by layer)
 
 Discrete results are compared for every token of every layer execution; the layer output is
 compared on sampled tokens (a token's output depends on no other token), within max-abs 2e-2
-and relative L2 1e-2.  To bound host memory and set-up time the stacks are shallower than the
+and relative L2 1e-2.  The library's own self-check (routing and permutation invariants, guard
+words behind the scratch buffers) runs in every step and must stay silent.  To bound host memory and set-up time the stacks are shallower than the
 named configurations and layers share a few distinct sets of expert weights; every layer
 execution has the configuration's full shape (H, E, k, I, tokens per step, capacity).
 """
@@ -25,6 +26,8 @@ def _setup(w, **kw):
     build.build()
     from paper_2609_33385_b200.runner import StackRunner
     run = StackRunner(w, **kw)
+    from paper_2609_33385_b200 import binding
+    run.ctx.set_option(binding.OPT_SELF_CHECK, 1)   # every step also checked on the device
     ora = OracleStack(w.n_layers, w.hidden, w.n_experts, w.top_k, w.intermediate, run.capacity)
     for l in range(w.n_layers):
         ora.register_router(l, run.router_bits[l], run.bias[l])
@@ -72,6 +75,9 @@ def _replay(run, ora, n_iters, sample_layers, n_sample_tokens, rng):
         a, b = run.ctx.stats(l), ora.stats(l)
         assert (a.steps, a.hits, a.misses, a.bytes_moved, a.evictions, a.active_experts) == \
                (b.steps, b.hits, b.misses, b.bytes_moved, b.evictions, b.active_experts)
+    # the device-side self-check ran in every step: invariants held, guard words intact
+    run.ctx.synchronize()
+    assert run.ctx.self_check_report() == ([], -1, 0)
     return worst
 
 

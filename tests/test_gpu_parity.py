@@ -374,6 +374,41 @@ def test_bounded_device_wait_reports_timeout_and_context_survives():
         run.close()
 
 
+def test_self_check_is_silent_on_valid_steps_and_flags_a_corrupted_permutation():
+    """OLED_OPT_SELF_CHECK: the checking kernels find nothing on valid steps (parity unchanged, guard
+    words intact); with the first two sorted rows exchanged by the test aid - both still valid
+    rows, so nothing faults - the next synchronising call returns OLED_ERR_SELF_CHECK and the
+    report names the broken invariant; after oled_clear_status() the context is in parity again."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(blocks=1, iters=3)
+    run = _runner(w, capacity=[3, 5], max_tokens=max(w.tokens, 9))
+    ora = _oracle_for(run, [3, 5])
+    try:
+        run.ctx.set_option(binding.OPT_SELF_CHECK, 1)
+        _run_stack(run, ora)                                     # every step checked, all in parity
+        run.ctx.synchronize()
+        assert run.ctx.self_check_report() == ([], -1, 0)
+        h_bits, conf = synth.flat_tokens(w, 9, 3)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((9, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.ctx.set_option(binding.OPT_TEST_CORRUPT_PERM, 1)
+        run.step(0, x, c, out)
+        ora.denoise_step(0, h_bits, conf)                        # keep the oracle's cache state in step
+        assert run.ctx.synchronize_rc() == binding.ERR_SELF_CHECK
+        names, index, guard = run.ctx.self_check_report()
+        assert "inverse" in names and index in (0, 1) and guard == 0
+        assert run.ctx.synchronize_rc() == binding.ERR_SELF_CHECK   # sticky until cleared
+        run.ctx.set_option(binding.OPT_TEST_CORRUPT_PERM, 0)
+        run.ctx.clear_status()
+        assert run.ctx.synchronize_rc() == binding.OLED_OK
+        run.step(0, x, c, out)
+        _check_step(run, 0, 9, out, ora.denoise_step(0, h_bits, conf))
+        assert run.ctx.self_check_report() == ([], -1, 0)
+    finally:
+        run.close()
+
+
 def test_maximum_expert_count_and_top_k():
     """512 experts (OLED_MAX_EXPERTS) with top-32 (OLED_MAX_TOPK): the widest gate the ABI allows."""
     from paper_2609_33385_b200.runner import bits_to_dev
