@@ -682,6 +682,13 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.stats.assignments += (uint64_t)T * K;
   L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
   L.stats.ideal_hits += (uint64_t)std::min<int64_t>(plan.n_active, plan.capacity_used);
+  static const bool log_steps = getenv("OLED_LOG") != nullptr;  // one line per layer execution on stderr
+  if (log_steps) {
+    int resident = 0;
+    for (uint8_t r : plan.after) resident += r;
+    fprintf(stderr, "oled: layer %d tokens %d active %d hits %zu misses %zu evicted %d resident %d/%d\n", (int)layer, T,
+            (int)plan.n_active, plan.hits.size(), n_miss, (int)plan.n_evictions, resident, (int)plan.capacity_used);
+  }
   return OLED_OK;
 }
 
