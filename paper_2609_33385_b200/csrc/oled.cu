@@ -257,14 +257,18 @@ void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
 
 // The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
 // known on the host yet (the group is the resident set and experts without tokens cost nothing).
-int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts) {
+// before_down: an event the down projection (and nothing before it) has to wait for, or null.
+int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts,
+                     cudaEvent_t before_down = nullptr) {
   if (grp.n <= 0) return OLED_OK;
   const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
   if (ctx->ffn_impl == 1) {
+    if (before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
                       ctx->d_y, H, I);
   } else {
     for (int kind = 1; kind <= 2; ++kind) {
+      if (kind == 2 && before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
       ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
       // a fresh (zero) work counter per launch; a layer execution has at most three launch pairs,
       // should there ever be more, a used word is cleared in stream order and taken again
@@ -283,7 +287,7 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
 
 // FFN over experts[begin, end) (ids) with known counts, weights through the layer's slot table.
 int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& experts, size_t begin, size_t end,
-                  const int32_t* counts) {
+                  const int32_t* counts, cudaEvent_t before_down = nullptr) {
   if (begin >= end) return OLED_OK;
   FfnGroup grp;
   grp.n = (int32_t)(end - begin);
@@ -300,7 +304,7 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
     rows += (uint64_t)counts[e];
   }
   prof_add_ffn(ctx, (uint64_t)grp.n, rows);
-  return run_ffn_launches(ctx, grp, max_count, counts);
+  return run_ffn_launches(ctx, grp, max_count, counts, before_down);
 }
 
 // Blocks until the gate kernel of step `seq` has published counts and scores, and decodes them.
@@ -623,8 +627,17 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   // 3. fills: one pinned-host -> HBM copy per miss on the side stream.  The misses form two
   // groups: everything but the last `miss_chunk` experts, then those last few.  The first group's
   // FFN is one large launch that runs under the copies of the second; only the small second
-  // group's FFN is exposed after the last byte has arrived.
+  // group's FFN is exposed after the last byte has arrived - and of that only the down
+  // projection: the step's LAST blob is copied in two parts, what the gate/up kernel reads (and
+  // the row scales of an fp8 blob) first, the down-projection weights after it, so the last
+  // group's gate/up kernel runs while the last down-projection weights are still on the link.
   const size_t n_miss = plan.misses.size();
+  // byte range of the down-projection weights inside a blob (bf16 elements or e4m3 codes)
+  const size_t esz = ctx->shape.expert_format == OLED_EXPERTS_FP8 ? 1 : 2;
+  const size_t hi_elems = (size_t)ctx->shape.hidden * (size_t)ctx->shape.intermediate;
+  const size_t down_off = 2 * hi_elems * esz, down_bytes = hi_elems * esz;
+  static const bool split_allowed = getenv("OLED_SPLIT_LAST") == nullptr || atoi(getenv("OLED_SPLIT_LAST")) != 0;
+  const bool split_last = split_allowed && n_miss > 0 && E >= 3;
   const size_t tail = std::min(n_miss, (size_t)ctx->miss_chunk);
   const size_t bounds[3] = {0, n_miss - tail, n_miss};
   size_t n_groups = 0;
@@ -633,11 +646,26 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     if (bounds[gi] == bounds[gi + 1]) continue;
     for (size_t i = bounds[gi]; i < bounds[gi + 1]; ++i) {
       const int32_t e = plan.misses[i];
-      OLED_CUDA(ctx, cudaMemcpyAsync(ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes,
-                                     L.host_blob + (size_t)e * L.host_stride, ctx->slot_bytes,
-                                     cudaMemcpyHostToDevice, ctx->copy_stream));
+      uint8_t* dst = ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes;
+      const uint8_t* src = L.host_blob + (size_t)e * L.host_stride;
+      if (i + 1 < n_miss || !split_last) {
+        OLED_CUDA(ctx, cudaMemcpyAsync(dst, src, ctx->slot_bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+      } else {  // the step's last blob: gate|up (and the scales behind the codes) now, down below
+        OLED_CUDA(ctx, cudaMemcpyAsync(dst, src, down_off, cudaMemcpyHostToDevice, ctx->copy_stream));
+        if (ctx->slot_bytes > down_off + down_bytes)
+          OLED_CUDA(ctx, cudaMemcpyAsync(dst + down_off + down_bytes, src + down_off + down_bytes,
+                                         ctx->slot_bytes - down_off - down_bytes, cudaMemcpyHostToDevice,
+                                         ctx->copy_stream));
+      }
     }
     OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[n_groups], ctx->copy_stream));
+    if (split_last && bounds[gi + 1] == n_miss) {
+      const int32_t e = plan.misses[n_miss - 1];
+      OLED_CUDA(ctx, cudaMemcpyAsync(ctx->pool + (size_t)L.cache.slot_of[e] * ctx->slot_bytes + down_off,
+                                     L.host_blob + (size_t)e * L.host_stride + down_off, down_bytes,
+                                     cudaMemcpyHostToDevice, ctx->copy_stream));
+      OLED_CUDA(ctx, cudaEventRecord(ctx->fill_events[2], ctx->copy_stream));
+    }
     group_begin[n_groups] = bounds[gi];
     group_end[n_groups] = bounds[gi + 1];
     ++n_groups;
@@ -652,7 +680,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   int rc = OLED_OK;
   for (size_t c = 0; c < n_groups; ++c) {
     OLED_CUDA(ctx, cudaStreamWaitEvent(st, ctx->fill_events[c], 0));
-    rc = run_ffn_group(ctx, L, plan.misses, group_begin[c], group_end[c], counts);
+    rc = run_ffn_group(ctx, L, plan.misses, group_begin[c], group_end[c], counts,
+                       split_last && group_end[c] == n_miss ? ctx->fill_events[2] : nullptr);
     if (rc != OLED_OK) return rc;
   }
 
