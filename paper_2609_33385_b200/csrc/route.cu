@@ -56,7 +56,8 @@ __device__ __forceinline__ void route_token_tail_n(const float* row, int t, int 
     for (int i = 0; i < kMaxEPerLane; ++i) {
       const int e = lane + 32 * i;
       const float x = e < E ? row[e] : 0.0f;
-      v[i] = (x == x) ? x : __int_as_float(0xff800000);  // a NaN logit is read as -inf: the order stays total
+      // a NaN logit is read as -inf: the order stays total; -0 becomes +0 (they compare equal)
+      v[i] = (x == x) ? __fadd_rn(x, 0.0f) : __int_as_float(0xff800000);
     }
     uint32_t used = 0;
     int my_id = 0;
@@ -74,17 +75,14 @@ __device__ __forceinline__ void route_token_tail_n(const float* row, int t, int 
           }
         }
       }
-#pragma unroll
-      for (int d = 16; d >= 1; d >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, d);
-        const bool take = (oe != 0x7fffffff) &&
-                          (be == 0x7fffffff || ov > bv || (ov == bv && oe < be));
-        if (take) {
-          bv = ov;
-          be = oe;
-        }
-      }
+      // the warp's best: largest logit, then lowest index - two integer warp reductions (the logit
+      // as an order-preserving unsigned key; a lane without a candidate holds key 0, below every
+      // logit's key) and one broadcast of the winning logit
+      const uint32_t bits = __float_as_uint(bv);
+      const uint32_t key = be == 0x7fffffff ? 0u : ((bits & 0x80000000u) ? ~bits : (bits | 0x80000000u));
+      const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+      be = (int)__reduce_min_sync(0xffffffffu, key == kmax ? (uint32_t)be : 0x7fffffffu);
+      bv = __shfl_sync(0xffffffffu, bv, be & 31);
       if ((be & 31) == lane) used |= 1u << (be >> 5);
       if (lane == r) {
         my_id = be;
