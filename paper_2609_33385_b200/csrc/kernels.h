@@ -46,7 +46,7 @@ struct FfnGroup {
   int32_t n;
   int32_t n_box;  // token rows per TMA box / MMA N tile of this launch
   int32_t withhold_loads;  // test aid: the producer issues nothing, the consumers' waits run out
-  int32_t pad;
+  int32_t pad;             // tuning aid: cap on the fp8 converter groups (0 = default)
   uint16_t expert[OLED_MAX_EXPERTS];
   uint16_t slot[OLED_MAX_EXPERTS];
 };
