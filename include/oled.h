@@ -1,10 +1,10 @@
 /*
  * oled.h — C ABI of the B200 MoE denoise-step library.
  *
- * One context holds, for an L-layer MoE stack, a bounded per-layer GPU expert cache
- * ("each MoE layer owns an independent cache pool", paper Sec. 4.1), the host expert store
- * (borrowed pinned host memory; "the rest reside in host CPU memory", Sec. 2.2) and the
- * scratch the step needs.  A call to oled_denoise_step() performs one layer execution of one
+ * One context holds, for an L-layer MoE stack, a bounded GPU expert cache per layer (every
+ * layer has a cache pool of its own, paper Sec. 4.1), the host expert store (borrowed pinned
+ * host memory, where the experts that are not cached live, Sec. 2.2) and the scratch the step
+ * needs.  A call to oled_denoise_step() performs one layer execution of one
  * denoising iteration over a block of tokens (Sec. 2.1, Sec. 4.1 per-layer flow):
  *
  *   gate -> top-k expert ids + gate scores -> token->expert permutation -> hits/misses
@@ -64,7 +64,10 @@ typedef struct {
   int32_t intermediate;    /* I (SwiGLU) */
   int32_t max_tokens;      /* upper bound on n_tokens of any step */
   int32_t has_router_bias; /* 1: oled_register_router() takes a per-expert fp32 bias */
-  int32_t staging_slots;   /* transient slots for misses beyond capacity; 0 = E - min capacity */
+  int32_t staging_slots;   /* transient slots for misses beyond capacity; 0 = E - 1, which can never
+                              run out; a smaller value s stops layer-adaptive sizing from shrinking
+                              a layer below E - s slots (a layer with C slots can need E - C
+                              transient ones while it executes) */
   int32_t expert_format;   /* OLED_EXPERTS_BF16 (0) or OLED_EXPERTS_FP8 */
 } oled_model_shape;
 
@@ -106,8 +109,8 @@ typedef struct {
 int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, void* cuda_stream,
                 oled_ctx** out_ctx);
 
-/* Give a layer its gate (Sec. 4.1: "the MoE gate first produces the routed expert IDs, gate
- * scores").  w_router: [E,H] bf16, host or device, copied by the call.  bias: fp32[E] host or
+/* Give a layer its gate, which yields the routed expert ids and the gate scores of every token
+ * (Sec. 4.1).  w_router: [E,H] bf16, host or device, copied by the call.  bias: fp32[E] host or
  * device, or NULL (must be non-NULL iff has_router_bias). */
 int oled_register_router(oled_ctx* ctx, int32_t layer, const void* w_router, const float* bias);
 
@@ -123,6 +126,8 @@ int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob,
  *   confidences  device fp32[n_tokens], token confidences c_t in [0,1] (Sec. 4.3).
  *   n_tokens     0 <= n_tokens <= max_tokens.
  *   out          device [n_tokens,H] bf16: sum_j g[t,j]*FFN_{e(t,j)}(hidden[t]); must not alias hidden.
+ * hidden and out must be 16-byte aligned (rows are moved with 16-byte vector accesses),
+ * confidences 4-byte aligned; a misaligned pointer is rejected with INVALID_ARG, nothing is launched.
  * Buffers are borrowed until the enqueued work completes on the context's stream.  The layer's
  * resident set and the counters are updated before the call returns.
  * Non-finite activations do not break the step: a NaN gate logit ranks as -inf (the k expert
@@ -162,6 +167,12 @@ int oled_stats(oled_ctx* ctx, int32_t layer, oled_stats_t* out);
 int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int32_t* perm,
                     int32_t* counts, uint64_t* scores, uint8_t* resident_before,
                     uint8_t* resident_after);
+
+/* Parity aid, the permutation's other two products of the most recent step (host buffers, NULL
+ * to skip): offsets int32[E+1], the exclusive scan of the counts (sorted rows of expert e are
+ * offsets[e] .. offsets[e+1]-1), and pos int32[T*k], the inverse of perm (pos[t*k+j] = sorted row
+ * of assignment (t,j)).  Synchronises. */
+int oled_debug_perm(oled_ctx* ctx, int32_t layer, int32_t* offsets, int32_t* pos);
 
 /* Gate logits fp32[T*E] of the most recent step (host buffer).  Synchronises. */
 int oled_debug_logits(oled_ctx* ctx, int32_t layer, float* logits);
@@ -283,6 +294,12 @@ int oled_last_cuda_error(oled_ctx* ctx);
  *   ids int32[n_tokens*top_k], gate fp32[n_tokens*top_k], counts int32[n_experts],
  *   offsets int32[n_experts+1], perm int32[n_tokens*top_k]: device, written; caller-owned.
  *   n_tokens <= OLED_NOALLOC_MAX_TOKENS, else OLED_ERR_TOO_MANY_TOKENS; other limits as above.
+ *   hidden, w_router and ids must be 16-byte aligned (they are accessed with 16-byte vectors), the
+ *   other arrays 4-byte aligned; a misaligned pointer is rejected with OLED_ERR_INVALID_ARG before
+ *   anything is launched.
+ * The launches use programmatic dependent launch when the calling thread's most recent
+ * oled_denoise_step() did (steps of at most 4096 token-expert assignments), and by default if the
+ * thread has run no step; either way the results are the same.
  * The work is enqueued on cuda_stream.  The first call on a device looks up the array's device
  * address (one-time set-up under a lock); make that first call before any stream capture.
  * All calls share the one array, which still holds the previous call's data: the accumulators
@@ -304,6 +321,12 @@ int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, 
 int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scores,
                      uint8_t* resident_before, uint8_t* resident_after, int32_t* slot_of,
                      int32_t* n_hits, int32_t* n_misses, int32_t* n_evictions);
+/* The layers of a simulated STACK: n_layers simulators that share one slot pool sized by the rule
+ * oled_create() uses (sum of the capacities + staging; staging_slots = 0 takes the default), with
+ * the same floor on the capacities oled_policy_adapt() may hand out.  out: oled_policy*[n_layers],
+ * each destroyed with oled_policy_destroy(); pool_slots (may be NULL) receives the pool size. */
+int oled_policy_create_stack(int32_t n_layers, int32_t n_experts, const int32_t* capacity,
+                             int32_t staging_slots, oled_policy** out, int32_t* pool_slots);
 void oled_policy_destroy(oled_policy* p);
 /* Retention value of the simulator's layer (OLED_POLICY_*). */
 int oled_policy_set_policy(oled_policy* p, int32_t policy);

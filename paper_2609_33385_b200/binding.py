@@ -40,7 +40,7 @@ EXPORTS = [
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
     "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
     "oled_policy_adapt", "oled_clear_status", "oled_policy_time", "oled_expert_blob_bytes",
-    "oled_self_check_report",
+    "oled_self_check_report", "oled_debug_perm", "oled_policy_create_stack",
 ]
 EXPERTS_BF16, EXPERTS_FP8 = 0, 1
 NOALLOC_MAX_TOKENS = 256
@@ -110,6 +110,8 @@ def load() -> C.CDLL:
     lib.oled_stats.argtypes = [vp, i32, C.POINTER(StatsStruct)]
     lib.oled_debug_last.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.oled_debug_logits.argtypes = [vp, i32, vp]
+    lib.oled_debug_perm.argtypes = [vp, i32, vp, vp]
+    lib.oled_policy_create_stack.argtypes = [i32, i32, C.POINTER(i32), i32, C.POINTER(vp), C.POINTER(i32)]
     lib.oled_reset_cache.argtypes = [vp]
     lib.oled_residual_add.argtypes = [vp, vp, vp, vp, C.c_size_t]
     lib.oled_set_option.argtypes = [vp, i32, C.c_int64]
@@ -219,6 +221,14 @@ class OledContext:
                     "oled_debug_last")
         return out
 
+    def debug_perm(self, layer: int, n_tokens: int) -> dict:
+        """offsets [E+1] and pos [T*k] (the inverse of perm) of the most recent step."""
+        out = dict(offsets=np.zeros(self.shape.n_experts + 1, np.int32),
+                   pos=np.zeros(n_tokens * self.shape.top_k, np.int32))
+        self._check(self._lib.oled_debug_perm(self._h, layer, _np_ptr(out["offsets"]), _np_ptr(out["pos"])),
+                    "oled_debug_perm")
+        return out
+
     def debug_logits(self, layer: int, n_tokens: int) -> np.ndarray:
         out = np.zeros((n_tokens, self.shape.n_experts), np.float32)
         self._check(self._lib.oled_debug_logits(self._h, layer, _np_ptr(out)), "oled_debug_logits")
@@ -307,17 +317,34 @@ def route_noalloc(hidden_ptr, w_router_ptr, bias_ptr, conf_ptr, n_tokens: int, h
 class PolicySim:
     """Host-only policy simulator (``oled_policy_*``): the library's C++ policy code, no GPU."""
 
-    def __init__(self, n_experts: int, capacity: int, pool_slots: int, policy: str = "priority"):
+    def __init__(self, n_experts: int, capacity: int, pool_slots: int, policy: str = "priority", _handle=None):
         self._lib = load()
         self.n_experts = n_experts
-        h = C.c_void_p()
-        rc = self._lib.oled_policy_create(n_experts, capacity, pool_slots, C.byref(h))
-        if rc != OLED_OK:
-            raise OledError(rc, "oled_policy_create")
-        self._h = h
+        if _handle is None:
+            h = C.c_void_p()
+            rc = self._lib.oled_policy_create(n_experts, capacity, pool_slots, C.byref(h))
+            if rc != OLED_OK:
+                raise OledError(rc, "oled_policy_create")
+            self._h = h
+        else:
+            self._h = _handle
         rc = self._lib.oled_policy_set_policy(self._h, POLICY_IDS[policy])
         if rc != OLED_OK:
             raise OledError(rc, "oled_policy_set_policy")
+
+    @staticmethod
+    def stack(n_experts: int, capacity: Sequence[int], staging_slots: int = 0, policy: str = "priority"):
+        """Simulators of the layers of one stack sharing one slot pool sized as ``oled_create``
+        sizes it (``oled_policy_create_stack``); returns (list of PolicySim, pool size)."""
+        n = len(capacity)
+        caps = (C.c_int32 * n)(*[int(c) for c in capacity])
+        arr = (C.c_void_p * n)()
+        slots = C.c_int32()
+        rc = load().oled_policy_create_stack(n, n_experts, caps, staging_slots, arr, C.byref(slots))
+        if rc != OLED_OK:
+            raise OledError(rc, "oled_policy_create_stack")
+        return [PolicySim(n_experts, int(c), 0, policy, _handle=C.c_void_p(arr[i]))
+                for i, c in enumerate(capacity)], int(slots.value)
 
     def fills_reused(self) -> int:
         v = C.c_uint64()

@@ -1,5 +1,5 @@
-// Grouped SwiGLU expert FFN on the 5th-generation tensor cores (paper Sec. 4.1: "cache-hit
-// experts execute directly on the GPU"; misses follow once their weights have landed).
+// Grouped SwiGLU expert FFN on the 5th-generation tensor cores (paper Sec. 4.1: experts that hit
+// the cache run on the GPU at once; misses follow once their weights have landed).
 //
 // Two persistent kernels per expert group, both "weights on M, tokens on N":
 //   KIND 1:  D_g[i,n] = sum_h Wg[i,h] x[n,h],  D_u likewise with Wu  (two TMEM accumulators),
@@ -619,6 +619,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   }
 
   // ---- teardown
+  // An early-start CTA reaches its dependency wait only on the path of its first item; every
+  // other way out (no item drawn, loads withheld, an abort) passes it here, so that NO kernel of
+  // a step completes before its predecessors have - the ordering of the kernels behind this one
+  // rests on that.
+  if (early) griddep_wait();
   tc_fence_before();
   __syncthreads();
   if (warp == kMmaWarp) {

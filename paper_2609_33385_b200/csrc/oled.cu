@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <memory>
 #include <new>
 #include <vector>
 
@@ -89,6 +90,7 @@ struct oled_ctx {
   GuardList guards{};          // guard words behind the step's scratch buffers
   uint64_t policy_ns = 0, policy_runs = 0;
   long long total_capacity = 0;
+  int adapt_lo = 1;            // smallest capacity layer-adaptive sizing may hand out (see pool_plan)
   int adapt_period = 0;        // iterations between automatic capacity refreshes (0 = off)
   uint64_t iterations = 0;     // oled_denoise_iteration() calls so far
   uint64_t launches = 0;
@@ -135,6 +137,8 @@ int dev_alloc_guarded(oled_ctx* ctx, T** p, size_t n) {
     ctx->guards.words[ctx->guards.n++] = reinterpret_cast<uint32_t*>(q + bytes);
   return OLED_OK;
 }
+
+inline bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
 
 int check_status(oled_ctx* ctx) {
   if (!ctx->h_status) return OLED_OK;
@@ -409,10 +413,12 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
     if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(OLED_ERR_CUDA);
   }
 
-  const int staging = s.staging_slots > 0 ? s.staging_slots : (s.n_experts - min_cap);
+  (void)min_cap;
+  const PoolPlan pp = pool_plan(s.n_experts, total_cap, s.staging_slots);
+  ctx->adapt_lo = pp.adapt_lo;
   ctx->slot_bytes = oled_expert_blob_bytes(s.hidden, s.intermediate, s.expert_format);
-  ctx->n_slots = (int)std::min<long long>(total_cap + staging, 65535);
-  if (total_cap + staging > 65535) return fail(OLED_ERR_INVALID_ARG);
+  if (pp.n_slots > 65535) return fail(OLED_ERR_INVALID_ARG);
+  ctx->n_slots = (int)pp.n_slots;
   ctx->slots.init(ctx->n_slots);
   ctx->total_capacity = total_cap;
   ctx->layers.resize(s.n_layers);
@@ -529,6 +535,9 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     const uint8_t* b = static_cast<const uint8_t*>(out);
     const size_t bytes = (size_t)T * H * 2;
     if (a < b + bytes && b < a + bytes) return OLED_ERR_INVALID_ARG;  // out aliases hidden
+    // the kernels read and write rows with 16-byte vector accesses
+    if (misaligned(hidden, 16) || misaligned(out, 16) || misaligned(x_next, 16) || misaligned(confidences, 4))
+      return OLED_ERR_INVALID_ARG;
   }
   cudaStream_t st = ctx->stream;
   ctx->last_layer = layer;
@@ -768,7 +777,7 @@ int oled_adapt_capacity(oled_ctx* ctx, int32_t* new_capacity) {
   if (!ctx) return OLED_ERR_INVALID_ARG;
   std::vector<LayerCacheState*> layers;
   for (auto& L : ctx->layers) layers.push_back(&L.cache);
-  const std::vector<int32_t> caps = adaptive_capacities(layers, ctx->total_capacity);
+  const std::vector<int32_t> caps = adaptive_capacities(layers, ctx->total_capacity, ctx->adapt_lo);
   // Slots of residents evicted here may still be read by kernels already enqueued; they are
   // reused only after the next step's gate report, which those kernels precede in stream order.
   for (size_t l = 0; l < layers.size(); ++l)
@@ -844,6 +853,21 @@ int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int
   }
   if (resident_before) memcpy(resident_before, ctx->last_before.data(), E);
   if (resident_after) memcpy(resident_after, ctx->last_after.data(), E);
+  return rc;
+}
+
+int oled_debug_perm(oled_ctx* ctx, int32_t layer, int32_t* offsets, int32_t* pos) {
+  if (!ctx || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  if (ctx->last_layer != layer) return OLED_ERR_STALE_DEBUG;
+  const int rc = sync_all(ctx);
+  if (rc != OLED_OK && rc != OLED_ERR_TIMEOUT) return rc;
+  const size_t n = (size_t)ctx->last_tokens * ctx->shape.top_k, E = (size_t)ctx->shape.n_experts;
+  if (n > 0) {
+    if (offsets) OLED_CUDA(ctx, cudaMemcpy(offsets, ctx->d_offsets, (E + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (pos) OLED_CUDA(ctx, cudaMemcpy(pos, ctx->d_pos, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  } else if (offsets) {
+    memset(offsets, 0, (E + 1) * sizeof(int32_t));
+  }
   return rc;
 }
 
@@ -972,9 +996,10 @@ int oled_last_cuda_error(oled_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0;
 // ---- host-only policy simulator -----------------------------------------------------------
 struct oled_policy {
   LayerCacheState cache;
-  SlotPool pool;
+  std::shared_ptr<SlotPool> pool;  // one per simulated layer, or shared by the layers of a simulated stack
   StepPlan plan;
   uint64_t fills_reused = 0;
+  int32_t adapt_lo = 1;
 };
 
 int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, oled_policy** out) {
@@ -984,8 +1009,36 @@ int oled_policy_create(int32_t n_experts, int32_t capacity, int32_t pool_slots, 
   oled_policy* p = new (std::nothrow) oled_policy();
   if (!p) return OLED_ERR_OOM;
   p->cache.init(n_experts, capacity);
-  p->pool.init(pool_slots);
+  p->pool = std::make_shared<SlotPool>();
+  p->pool->init(pool_slots);
   *out = p;
+  return OLED_OK;
+}
+
+int oled_policy_create_stack(int32_t n_layers, int32_t n_experts, const int32_t* capacity, int32_t staging_slots,
+                             oled_policy** out, int32_t* pool_slots) {
+  if (!out || !capacity || n_layers <= 0 || n_experts <= 0 || n_experts > OLED_MAX_EXPERTS || staging_slots < 0)
+    return OLED_ERR_INVALID_ARG;
+  long long total = 0;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    if (capacity[l] <= 0 || capacity[l] > n_experts) return OLED_ERR_INVALID_ARG;
+    total += capacity[l];
+  }
+  const PoolPlan pp = pool_plan(n_experts, total, staging_slots);  // the sizing rule of oled_create()
+  auto pool = std::make_shared<SlotPool>();
+  pool->init((int32_t)pp.n_slots);
+  for (int32_t l = 0; l < n_layers; ++l) {
+    oled_policy* p = new (std::nothrow) oled_policy();
+    if (!p) {
+      for (int32_t j = 0; j < l; ++j) delete out[j];
+      return OLED_ERR_OOM;
+    }
+    p->cache.init(n_experts, capacity[l]);
+    p->pool = pool;
+    p->adapt_lo = pp.adapt_lo;
+    out[l] = p;
+  }
+  if (pool_slots) *pool_slots = (int32_t)pp.n_slots;
   return OLED_OK;
 }
 
@@ -993,7 +1046,7 @@ int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scor
                      uint8_t* resident_after, int32_t* slot_of, int32_t* n_hits, int32_t* n_misses,
                      int32_t* n_evictions) {
   if (!p || !counts || !scores) return OLED_ERR_INVALID_ARG;
-  if (!plan_step(p->cache, p->pool, counts, scores, p->plan)) return OLED_ERR_NO_SLOT;
+  if (!plan_step(p->cache, *p->pool, counts, scores, p->plan)) return OLED_ERR_NO_SLOT;
   const size_t E = (size_t)p->cache.n_experts;
   if (resident_before) memcpy(resident_before, p->plan.before.data(), E);
   if (resident_after) memcpy(resident_after, p->plan.after.data(), E);
@@ -1003,7 +1056,7 @@ int oled_policy_step(oled_policy* p, const int32_t* counts, const uint64_t* scor
   if (n_misses) *n_misses = (int32_t)p->plan.misses.size();
   if (n_evictions) *n_evictions = p->plan.n_evictions;
   p->fills_reused += (uint64_t)p->plan.n_fills_reused;
-  finish_step(p->cache, p->pool, p->plan);
+  finish_step(p->cache, *p->pool, p->plan);
   return OLED_OK;
 }
 
@@ -1030,9 +1083,9 @@ int oled_policy_adapt(oled_policy** layers, int32_t n_layers, int32_t total_capa
   }
   if (total_capacity < n_layers || total_capacity > (int64_t)n_layers * ls[0]->n_experts)
     return OLED_ERR_INVALID_ARG;
-  const std::vector<int32_t> caps = adaptive_capacities(ls, total_capacity);
+  const std::vector<int32_t> caps = adaptive_capacities(ls, total_capacity, layers[0]->adapt_lo);
   for (int32_t l = 0; l < n_layers; ++l) {
-    shrink_to(*ls[l], layers[l]->pool, caps[l]);
+    shrink_to(*ls[l], *layers[l]->pool, caps[l]);
     new_capacity[l] = caps[l];
   }
   return OLED_OK;

@@ -239,7 +239,9 @@ inline std::vector<int32_t> apportion(std::vector<uint64_t> w, int64_t total, in
 
 // Layer-adaptive sizing (Sec. 4.3): w_l = a_l * u_l from the statistics of the period that just
 // ended, smoothed over periods by s <- (s + new) / 2 in Q16; returns the new capacities.
-inline std::vector<int32_t> adaptive_capacities(std::vector<LayerCacheState*>& layers, int64_t total) {
+// lo: smallest capacity a layer may be given (see pool_plan: a layer that shrinks further could
+// need more transient slots during one of its steps than the pool has).
+inline std::vector<int32_t> adaptive_capacities(std::vector<LayerCacheState*>& layers, int64_t total, int32_t lo = 1) {
   std::vector<uint64_t> w;
   for (LayerCacheState* L : layers) {
     if (L->period_steps > 0) {
@@ -251,7 +253,26 @@ inline std::vector<int32_t> adaptive_capacities(std::vector<LayerCacheState*>& l
     }
     w.push_back((uint64_t)std::max<int64_t>(0, L->a_q16) * (uint64_t)std::max<int64_t>(0, L->u_q16));
   }
-  return apportion(w, total, 1, layers.empty() ? 1 : layers[0]->n_experts);
+  return apportion(w, total, std::max<int32_t>(1, lo), layers.empty() ? 1 : layers[0]->n_experts);
+}
+
+// Size of the shared slot pool.  While layer l executes, the other layers hold at most
+// C_total - C_l slots (the resident sets never exceed the capacities, also right after a
+// resize) and layer l itself needs at most E (every expert activated), so the pool never runs
+// out iff C_total + staging - (C_total - C_l) >= E, i.e. staging >= E - C_l for every capacity a
+// layer can ever have.  Layer-adaptive sizing may shrink a layer down to `adapt_lo`; the default
+// staging (E - 1) allows 1, a smaller caller-chosen staging raises the floor accordingly.
+struct PoolPlan {
+  int32_t staging;   // transient slots beyond the capacities
+  int64_t n_slots;   // C_total + staging
+  int32_t adapt_lo;  // smallest capacity layer-adaptive sizing may hand out
+};
+inline PoolPlan pool_plan(int32_t n_experts, int64_t total_capacity, int32_t staging_requested) {
+  PoolPlan p;
+  p.staging = staging_requested > 0 ? staging_requested : std::max<int32_t>(1, n_experts - 1);
+  p.n_slots = total_capacity + p.staging;
+  p.adapt_lo = std::max<int32_t>(1, n_experts - p.staging);
+  return p;
 }
 
 }  // namespace oled

@@ -1,6 +1,6 @@
-// Gate of the MoE layer (paper Sec. 2.1 / Sec. 4.1: "the MoE gate first produces the routed
-// expert IDs, gate scores"), token->expert permutation, and the integer numerators of the
-// expert reuse priority (Sec. 4.3 priority equation).
+// Gate of the MoE layer (paper Sec. 2.1 / Sec. 4.1: the gate yields each token's routed expert
+// ids and gate scores), token->expert permutation, and the integer numerators of the expert
+// reuse priority (Sec. 4.3 priority equation).
 //
 // Everything a keep/evict or routing decision depends on is computed in a fixed operation
 // order so that it can be reproduced bit for bit elsewhere:
@@ -469,6 +469,12 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   if (n_tokens > OLED_NOALLOC_MAX_TOKENS) return OLED_ERR_TOO_MANY_TOKENS;
   if (n_tokens > 0 && (!hidden || !w_router || !confidences || !ids || !gate || !perm))
     return OLED_ERR_INVALID_ARG;
+  {  // rows and ids are accessed with 16-byte vectors, everything else as 32-bit words
+    auto off = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
+    if (off(hidden, 16) || off(w_router, 16) || off(ids, 16) || off(bias, 4) || off(confidences, 4) ||
+        off(gate, 4) || off(counts, 4) || off(offsets, 4) || off(perm, 4))
+      return OLED_ERR_INVALID_ARG;
+  }
   unsigned char* scratch = nullptr;
   const int rc = noalloc_scratch_ptr(&scratch);
   if (rc != OLED_OK) return rc;

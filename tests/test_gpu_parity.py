@@ -56,6 +56,9 @@ def _check_step(run, layer, n_tokens, out_t, ref, check_out=True):
     assert [int(v) for v in dbg["scores"]] == list(ref["scores"]), "reuse scores differ"
     assert set(np.flatnonzero(dbg["resident_before"])) == ref["resident_before"]
     assert set(np.flatnonzero(dbg["resident_after"])) == ref["resident_after"]
+    dbp = run.ctx.debug_perm(layer, n_tokens)
+    assert np.array_equal(dbp["offsets"], ref["offsets"]), "offsets differ"
+    assert np.array_equal(dbp["pos"], ref["pos"]), "inverse permutation differs"
     if n_tokens:
         logits = run.ctx.debug_logits(layer, n_tokens)
         assert np.array_equal(logits.view(np.uint32), ref["logits"].view(np.uint32)), "logits differ"
@@ -259,6 +262,10 @@ def test_errors_are_codes_not_crashes():
         assert ctx.denoise_step_rc(1, x.data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.ERR_INVALID_ARG
         assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, x.data_ptr()) == binding.ERR_INVALID_ARG
         assert ctx.denoise_step_rc(0, None, c.data_ptr(), 8, out.data_ptr()) == binding.ERR_INVALID_ARG
+        # rows are moved with 16-byte vector accesses: a view that starts inside one is refused
+        big = torch.zeros(8 * w.hidden + 8, dtype=torch.bfloat16, device="cuda:0")
+        assert ctx.denoise_step_rc(0, big[4:].data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.ERR_INVALID_ARG
+        assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, big[4:].data_ptr()) == binding.ERR_INVALID_ARG
         assert ctx.denoise_step_rc(0, x.data_ptr(), c.data_ptr(), 8, out.data_ptr()) == binding.OLED_OK
         ctx.synchronize()
         assert float(out.float().abs().max()) == 0.0          # zero weights -> zero output

@@ -124,3 +124,70 @@ def test_host_adaptive_sizing_matches_oracle(binding):
             assert binding.PolicySim.adapt(sims, sum(caps)) == want
             assert sum(want) == sum(caps)
     assert want[0] < want[-1]                        # slots moved to the layers with the larger working sets
+
+
+def test_shared_pool_never_runs_out_after_adaptive_shrinking(binding):
+    """The slot pool of a stack, sized by the rule oled_create() uses with default staging: a layer
+    that layer-adaptive sizing has shrunk to ONE slot, while the other layers fill their enlarged
+    capacities, must still be able to activate every expert in one step (Sec. 4.3 sizing on top of
+    the Sec. 4.2 cache update)."""
+    e, n_layers = 16, 4
+    caps = [4] * n_layers
+    sims, pool_slots = binding.PolicySim.stack(e, caps)
+    assert pool_slots == sum(caps) + e - 1
+    ones = np.ones(e, np.uint64)
+    # period 1: layer 0 activates one expert per step, the others all of them -> layer 0 starves
+    for it in range(5):
+        for l, sim in enumerate(sims):
+            counts = np.zeros(e, np.int32)
+            if l == 0:
+                counts[0] = 1
+            else:
+                counts[:] = 1
+            sim.step(counts, ones * (it + 1))
+    new = binding.PolicySim.adapt(sims, sum(caps))
+    assert sum(new) == sum(caps) and new[0] == 1 and max(new[1:]) > 4
+    # the grown layers fill their capacities, then the shrunk layer activates everything
+    for l in (1, 2, 3):
+        got = sims[l].step(np.ones(e, np.int32), np.arange(e, dtype=np.uint64) + 1)
+        assert int(got["resident_after"].sum()) == new[l]
+    got = sims[0].step(np.ones(e, np.int32), np.arange(e, dtype=np.uint64) + 1)
+    assert got["hits"] + got["misses"] == e and int(got["resident_after"].sum()) == 1
+    slots = got["slot_of"]
+    assert np.all(slots >= 0) and len(set(slots.tolist())) == e
+
+
+def test_small_caller_chosen_staging_raises_the_adaptive_floor(binding):
+    """With fewer staging slots than E - 1 a layer of capacity C could need E - C transient slots
+    that do not exist; the sizing then never hands out less than E - staging."""
+    e, caps, staging = 16, [6, 6, 6], 10
+    sims, pool_slots = binding.PolicySim.stack(e, caps, staging_slots=staging)
+    assert pool_slots == sum(caps) + staging
+    for it in range(5):
+        for l, sim in enumerate(sims):
+            counts = np.zeros(e, np.int32)
+            counts[: (1 if l == 0 else e)] = 1
+            sim.step(counts, np.ones(e, np.uint64))
+    new = binding.PolicySim.adapt(sims, sum(caps))
+    assert sum(new) == sum(caps) and min(new) == e - staging
+    for l in (1, 2, 0):                                   # worst case still fits
+        got = sims[l].step(np.ones(e, np.int32), np.arange(e, dtype=np.uint64) + 1)
+        assert got["hits"] + got["misses"] == e
+
+
+def test_misaligned_pointers_are_rejected_before_anything_is_launched(binding):
+    """oled_route_noalloc accesses rows and ids with 16-byte vectors: a pointer into the middle of
+    such a vector is an argument error (nothing touches the GPU, so this runs without one)."""
+    ok16, ok4 = 0x7000_0000_0100, 0x7000_0000_0204
+    args = dict(hidden=ok16, w_router=ok16 + 0x1000, bias=None, conf=ok4, ids=ok16 + 0x2000, gate=ok4 + 0x3000,
+                counts=ok4 + 0x4000, offsets=ok4 + 0x5000, perm=ok4 + 0x6000)
+
+    def call(**kw):
+        a = dict(args, **kw)
+        return binding.route_noalloc(a["hidden"], a["w_router"], a["bias"], a["conf"], 4, 256, 8, 2, 0, a["ids"],
+                                     a["gate"], a["counts"], a["offsets"], a["perm"])
+    for name in ("hidden", "w_router", "ids"):
+        assert call(**{name: args[name] + 8}) == binding.ERR_INVALID_ARG, name
+    for name in ("conf", "gate", "counts", "offsets", "perm"):
+        assert call(**{name: args[name] + 2}) == binding.ERR_INVALID_ARG, name
+    assert call(bias=ok4 + 1) == binding.ERR_INVALID_ARG

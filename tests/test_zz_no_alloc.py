@@ -5,7 +5,7 @@ synchronisation of cudaMalloc inside the decode loop; for them the library offer
 ``oled_route_noalloc``, whose scratch is a fixed array inside the library.  This test calls it
 through the C ABI twice in a row, with different inputs (so stale contents of the shared array
 would show), and checks every output bit for bit against what ``oled_denoise_step`` produced
-for the same inputs.  It is collected last on purpose: a run that stops at the first failure
+for the same inputs and against the CPU oracle's gate, top-k and permutation of the same bits.  It is collected last on purpose: a run that stops at the first failure
 has then already run every other test.
 """
 import numpy as np
@@ -13,6 +13,7 @@ import pytest
 
 torch = pytest.importorskip("torch")
 
+from oracle import moe_layer as oracle_moe  # noqa: E402
 from paper_2609_33385_b200 import synth  # noqa: E402
 
 pytestmark = pytest.mark.gpu
@@ -53,6 +54,16 @@ def test_route_noalloc_matches_denoise_step_twice_in_a_row():
             assert np.array_equal(perm.cpu().numpy(), ref["perm"])
             off = offsets.cpu().numpy()
             assert off[0] == 0 and np.array_equal(np.diff(off), ref["counts"])
+            # ... and against the oracle (independent of the CUDA path) on the same input bits
+            logits = oracle_moe.gate_logits(oracle_moe.bf16_to_f32(h_bits),
+                                            oracle_moe.bf16_to_f32(run.router_bits[0]), None)
+            o_ids, o_gate = oracle_moe.topk_route(logits, k)
+            o_counts, o_offsets, o_perm, _ = oracle_moe.permutation(o_ids, e)
+            assert np.array_equal(ids.cpu().numpy().reshape(n, k), o_ids)
+            assert np.array_equal(gate.cpu().numpy().view(np.uint32).reshape(n, k), o_gate.view(np.uint32))
+            assert np.array_equal(counts.cpu().numpy(), o_counts)
+            assert np.array_equal(off, o_offsets)
+            assert np.array_equal(perm.cpu().numpy(), o_perm)
         # beyond the stated maximum: a clear error, nothing launched
         big = binding.NOALLOC_MAX_TOKENS + 1
         rc = binding.route_noalloc(x.data_ptr(), wr_dev.data_ptr(), None, c.data_ptr(), big, h, e, k,
