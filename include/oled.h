@@ -211,6 +211,20 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * are exchanged after the permutation (both stay valid rows; the step's output is wrong). */
 #define OLED_OPT_SELF_CHECK 7
 #define OLED_OPT_TEST_CORRUPT_PERM 8
+/* Launch-structure switches, all on by default; the results do not depend on them (they exist
+ * to measure what each one buys):
+ * OLED_OPT_SPLIT_LAST_FILL: the step's last expert blob is copied in two parts, gate|up first,
+ *   so that the last group's gate/up kernel runs while its down-projection weights still arrive.
+ * OLED_OPT_FUSE_FFN: few-token steps on bf16 stores run gate/up and down projection of an expert
+ *   group as ONE launch.
+ * OLED_OPT_GATHER_IN_FFN: few-token steps on bf16 stores let the FFN kernel gather the token rows
+ *   it needs instead of reading a sorted copy of the input written by an earlier kernel.
+ * OLED_OPT_PDL: programmatic dependent launch between the kernels of a few-token step
+ *   (process-wide, not per context). */
+#define OLED_OPT_SPLIT_LAST_FILL 9
+#define OLED_OPT_FUSE_FFN 10
+#define OLED_OPT_GATHER_IN_FFN 11
+#define OLED_OPT_PDL 12
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */
 #define OLED_CHECK_ID_DUPLICATE 0x02u  /* a token routed twice to one expert                        */
 #define OLED_CHECK_OFFSETS 0x04u       /* offsets are not the exclusive scan of the counts          */
@@ -243,7 +257,8 @@ int oled_get_capacity(oled_ctx* ctx, int32_t* capacity);
 #define OLED_KERNEL_FFN_GATE_UP 3
 #define OLED_KERNEL_FFN_DOWN 4
 #define OLED_KERNEL_COMBINE 5
-#define OLED_N_KERNELS 6
+#define OLED_KERNEL_FFN_FUSED 6 /* gate/up + SwiGLU + down projection in one launch (few-token steps) */
+#define OLED_N_KERNELS 7
 typedef struct {
   uint64_t launches;
   double ms;       /* sum of CUDA-event durations */

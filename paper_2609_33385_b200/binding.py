@@ -17,7 +17,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("OLED_LIB_PATH") or os.path.join(_HERE, "liboled.so")
+LIB_PATH = os.path.join(_HERE, "liboled.so")
 
 OLED_OK = 0
 ERR_INVALID_ARG, ERR_NOT_PINNED, ERR_NOT_REGISTERED, ERR_TOO_MANY_TOKENS = -1, -2, -3, -4
@@ -25,12 +25,13 @@ ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -
 OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE, OPT_POLICY, OPT_ADAPT_PERIOD = 1, 2, 3, 4, 5
 OPT_TEST_WITHHOLD_LOADS = 6
 OPT_SELF_CHECK, OPT_TEST_CORRUPT_PERM = 7, 8
+OPT_SPLIT_LAST_FILL, OPT_FUSE_FFN, OPT_GATHER_IN_FFN, OPT_PDL = 9, 10, 11, 12
 ERR_SELF_CHECK = -10
 CHECK_FLAGS = {0x01: "id_range", 0x02: "id_duplicate", 0x04: "offsets", 0x08: "perm_range", 0x10: "inverse",
                0x20: "row_expert", 0x40: "order"}
 POLICY_PRIORITY, POLICY_LRU, POLICY_LFU = 0, 1, 2
 POLICY_IDS = {"priority": 0, "lru": 1, "lfu": 2}
-KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
+KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "ffn_fused"]
 
 EXPORTS = [
     "oled_create", "oled_register_router", "oled_register_experts", "oled_denoise_step",

@@ -10,8 +10,9 @@
 namespace oled {
 namespace {
 
-// BATCH: the number of assignment rows whose loads are issued together.  Small steps (a few CTAs,
-// latency-bound) take 8; large steps keep 1, where the extra registers cost occupancy.
+// BATCH: the number of assignment rows whose loads are issued together.  Small steps (latency-
+// bound) take 8 and split a token's row over gridDim.y CTAs, so that a 32-token step still puts
+// a CTA on most SMs; large steps keep 1, where the extra registers cost occupancy.
 template <bool Y_BF16, int BATCH>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
@@ -19,9 +20,10 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next,
                uint32_t* __restrict__ zero_words, int n_zero_words) {
   const int t = blockIdx.x;
+  const int slice = H / gridDim.y, h_begin = blockIdx.y * slice, h_end = h_begin + slice;
   griddep_launch_dependents();
   griddep_wait();
-  if (t == 0 && zero_words != nullptr)
+  if (t == 0 && blockIdx.y == 0 && zero_words != nullptr)
     for (int i = threadIdx.x; i < n_zero_words; i += blockDim.x) zero_words[i] = 0u;
   __shared__ float s_g[OLED_MAX_TOPK];
   __shared__ int s_r[OLED_MAX_TOPK];
@@ -30,7 +32,7 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
     s_r[threadIdx.x] = pos[(size_t)t * K + threadIdx.x];
   }
   __syncthreads();
-  for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
+  for (int h = h_begin + threadIdx.x * 4; h < h_end; h += blockDim.x * 4) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     // the rows of BATCH assignments are loaded together (independent requests in flight), then
     // accumulated in rank order
@@ -160,8 +162,13 @@ void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* ga
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
                     uint32_t* zero_words, int n_zero_words) {
   const bool small = (size_t)T * K <= 4096;
+  // small steps: slices of 512 columns (128 threads x 4) while that leaves at most ~4 CTAs per SM
+  int slices = 1;
+  if (small)
+    while (slices < 8 && H % (slices * 2 * 512) == 0 && (size_t)T * slices * 2 <= 592) slices *= 2;
+  const dim3 sgrid(T, slices), sblock(slices > 1 ? 128 : 256);
   if (y_bf16 && small)
-    launch_pdl(combine_kernel<true, 8>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+    launch_pdl(combine_kernel<true, 8>, sgrid, sblock, 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
   else if (y_bf16 && H % 8 == 0)
     launch_pdl(combine_bf16_wide_kernel, dim3(T), dim3(256), 0, st, reinterpret_cast<const uint16_t*>(y), gate, pos, H,
@@ -170,7 +177,7 @@ void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* ga
     launch_pdl(combine_kernel<true, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
   else if (small)
-    launch_pdl(combine_kernel<false, 8>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
+    launch_pdl(combine_kernel<false, 8>, sgrid, sblock, 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
                n_zero_words);
   else
     launch_pdl(combine_kernel<false, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,

@@ -21,8 +21,9 @@ __device__ __forceinline__ void griddep_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 #endif
-bool pdl_enabled();            // attribute on? (OLED_PDL=0 turns it off for good)
-void pdl_set_step(bool on);    // per step: used for small steps only (it costs ~2 % on many-token steps)
+bool pdl_enabled();            // attribute on?
+void pdl_set_step(bool on);    // per step and thread: used for small steps only (it costs ~2 % on many-token steps)
+void pdl_set_allowed(bool on); // process-wide switch (OLED_OPT_PDL)
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -79,9 +80,13 @@ struct RouteReport {
 // ---- route.cu -------------------------------------------------------------------------
 // Gate logits in the contract order, top-k (ties to the lower index), softmax over the selected
 // logits, per-expert counts and integer reuse-score numerators (atomics on zeroed arrays).
+// Small steps (route_fuses_permutation): with offsets/perm/pos non-null and a ticket in rep, the
+// kernel's last CTA also builds the permutation, and launch_permute is not needed.
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep);
+                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep,
+                  int32_t* offsets, int32_t* perm, int32_t* pos);
+bool route_fuses_permutation(int T, int E, int K);
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
 // kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
@@ -121,12 +126,30 @@ struct FfnTcMaps {
 // Builds the tensor maps; returns 0 or a negative oled_status.
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
-// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
-// work_counter: a device word that is ZERO when the kernel starts; its CTAs draw their work items
-// from it (every launch that can be in flight at the same time needs a word of its own).
+// Buffers of an FFN launch.
+struct FfnTcIo {
+  const int32_t* offsets = nullptr;   // [E+1]
+  uint16_t* hbuf = nullptr;           // [rows, I] bf16 intermediate
+  float* y = nullptr;                 // [rows, H] per-assignment outputs (fp32, or bf16 if y_bf16)
+  int y_bf16 = 0;
+  uint32_t* status = nullptr;
+  // a device word that is ZERO when the kernel starts; its CTAs draw their work items from it
+  // (every launch that can be in flight at the same time needs a word of its own)
+  uint32_t* work_counter = nullptr;
+  // bf16 stores, kinds 1 and 3: gather the token rows of the gate/up items from x [T, H] through
+  // perm instead of reading pre-sorted rows (x_gather == nullptr: read the sorted copy)
+  const uint16_t* x_gather = nullptr;
+  const int32_t* perm = nullptr;
+  int top_k = 0;
+  uint32_t* done = nullptr;           // kind 3: one ZERO word per expert of the group
+};
+// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y; kind 3: both in one launch
+// (bf16 stores and token tiles of at most 32 rows only: ask ffn_tc_can_fuse).  One launch each.
+// behind_event_wait: the launch follows a cudaStreamWaitEvent (with, for kind 2, at most its own
+// kind 1 launch in between), i.e. everything enqueued before that wait has completed.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
-                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
-                  int I, int n_sms, uint32_t* status, uint32_t* work_counter);
+                  const int32_t* host_counts, const FfnTcIo& io, int H, int I, int n_sms, bool behind_event_wait);
+bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 // Self-check (check.cu): invariants of the routing and the permutation, guard words.

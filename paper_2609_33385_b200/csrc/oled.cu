@@ -59,7 +59,8 @@ struct oled_ctx {
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
   unsigned int* d_ticket = nullptr;   // control block, after the counts
-  uint32_t* d_work = nullptr;         // control block, last: work-item counters of the step's FFN launches
+  uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
+  uint32_t* d_done = nullptr;         // control block, last: [kFfnWorkCounters][E] completion counters of fused FFN launches
   int work_next = 0;                  // next unused counter of the current layer execution
   bool ctrl_dirty = true;             // control block must be cleared before the next gate launch
   unsigned int seq = 0;               // step sequence number echoed by the gate kernel
@@ -82,8 +83,14 @@ struct oled_ctx {
   std::vector<cudaEvent_t> prof_free;
   oled_kernel_profile prof_acc[OLED_N_KERNELS] = {};
   int ffn_impl = 0;
+  bool fuse_ffn = true;        // small steps: gate/up and down projection in one launch where possible
+  bool gather_in_ffn = true;   // small steps, bf16 stores: the FFN kernel gathers the token rows itself
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
+  bool small_step = false;     // this step's gate kernel also made the permutation
+  const uint16_t* x_gather = nullptr;  // this step's FFN kernels gather token rows from here (else from d_xp)
+  bool hit_fused = false;      // this step's resident-group FFN ran as one fused launch
   int miss_chunk = 4;
+  bool split_last = true;      // the step's last blob is copied in two parts (gate|up first, down after)
   int withhold_loads = 0;      // test aid, see OLED_OPT_TEST_WITHHOLD_LOADS
   int self_check = 0;          // OLED_OPT_SELF_CHECK
   int corrupt_perm = 0;        // test aid, see OLED_OPT_TEST_CORRUPT_PERM
@@ -250,48 +257,76 @@ void prof_add(oled_ctx* ctx, int kernel, uint64_t bytes, uint64_t flops) {
 
 // Algorithmic bytes / flops of the two FFN kernels for n experts with `rows` token rows in total:
 // each expert's weights once, the token rows in, the result rows out.
-void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
+void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows, bool fused) {
   const uint64_t H = ctx->shape.hidden, I = ctx->shape.intermediate, hi = H * I;
   const bool fp8 = ctx->shape.expert_format == OLED_EXPERTS_FP8;
   // weight bytes of one expert per kernel: bf16 elements, or e4m3 codes plus the fp32 row scales
   const uint64_t w13 = fp8 ? 2 * hi + 2 * I * 4 : 2 * hi * 2, w2 = fp8 ? hi + H * 4 : hi * 2;
-  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * w13 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
-  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4), 2 * rows * hi);
+  const uint64_t b1 = n * w13 + rows * H * 2 + rows * I * 2, b2 = n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4);
+  if (fused) {
+    prof_add(ctx, OLED_KERNEL_FFN_FUSED, b1 + b2, 6 * rows * hi);
+  } else {
+    prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, b1, 4 * rows * hi);
+    prof_add(ctx, OLED_KERNEL_FFN_DOWN, b2, 2 * rows * hi);
+  }
 }
 
-// The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
-// known on the host yet (the group is the resident set and experts without tokens cost nothing).
+// The FFN launches over one group: one fused launch where the form exists (bf16 stores, token
+// tiles of at most 32 rows, nothing to wait for between the two projections), else gate/up and
+// down.  host_counts == nullptr: the per-expert counts are not known on the host yet (the group is
+// the resident set and experts without tokens cost nothing).
 // before_down: an event the down projection (and nothing before it) has to wait for, or null.
+// behind_event_wait: the caller has just enqueued a cudaStreamWaitEvent on the stream.
+// Returns the number of launches through *fused (1 = one fused launch).
 int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts,
-                     cudaEvent_t before_down = nullptr) {
+                     cudaEvent_t before_down, bool behind_event_wait, bool* fused_out) {
+  if (fused_out) *fused_out = false;
   if (grp.n <= 0) return OLED_OK;
   const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
   if (ctx->ffn_impl == 1) {
     if (before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
                       ctx->d_y, H, I);
+    ctx->launches += 2;
   } else {
-    for (int kind = 1; kind <= 2; ++kind) {
+    const bool fuse = ctx->small_step && ctx->fuse_ffn && before_down == nullptr && ffn_tc_can_fuse(ctx->maps, max_count);
+    for (int kind = fuse ? 3 : 1; kind <= (fuse ? 3 : 2); ++kind) {
       if (kind == 2 && before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
-      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
-      // a fresh (zero) work counter per launch; a layer execution has at most three launch pairs,
-      // should there ever be more, a used word is cleared in stream order and taken again
-      uint32_t* work = ctx->d_work + ctx->work_next % kFfnWorkCounters;
-      if (ctx->work_next >= kFfnWorkCounters) OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
+      ProfScope ps(ctx, kind == 3 ? OLED_KERNEL_FFN_FUSED : kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
+      // a fresh (zero) work counter and, for a fused launch, a fresh row of completion counters
+      // per launch; a layer execution has at most three launch pairs, should there ever be more,
+      // used words are cleared in stream order and taken again
+      const int li = ctx->work_next % kFfnWorkCounters;
+      FfnTcIo io;
+      io.work_counter = ctx->d_work + li;
+      io.done = ctx->d_done + (size_t)li * ctx->shape.n_experts;
+      if (ctx->work_next >= kFfnWorkCounters) {
+        OLED_CUDA(ctx, cudaMemsetAsync(io.work_counter, 0, sizeof(uint32_t), ctx->stream));
+        OLED_CUDA(ctx, cudaMemsetAsync(io.done, 0, (size_t)ctx->shape.n_experts * sizeof(uint32_t), ctx->stream));
+      }
       ctx->work_next += 1;
-      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
-                                   ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work);
+      io.offsets = ctx->d_offsets;
+      io.hbuf = ctx->d_hbuf;
+      io.y = ctx->d_y;
+      io.y_bf16 = ctx->y_bf16 ? 1 : 0;
+      io.status = ctx->d_status;
+      io.x_gather = ctx->x_gather;
+      io.perm = ctx->d_perm;
+      io.top_k = ctx->shape.top_k;
+      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, io, H, I, ctx->n_sms,
+                                   behind_event_wait || (kind == 2 && before_down != nullptr));
       if (rc != OLED_OK) return rc;
+      ctx->launches += 1;
     }
+    if (fused_out) *fused_out = fuse;
   }
-  ctx->launches += 2;
   OLED_CUDA(ctx, cudaGetLastError());
   return OLED_OK;
 }
 
 // FFN over experts[begin, end) (ids) with known counts, weights through the layer's slot table.
 int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& experts, size_t begin, size_t end,
-                  const int32_t* counts, cudaEvent_t before_down = nullptr) {
+                  const int32_t* counts, cudaEvent_t before_down, bool behind_event_wait) {
   if (begin >= end) return OLED_OK;
   FfnGroup grp;
   grp.n = (int32_t)(end - begin);
@@ -307,8 +342,10 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
     max_count = std::max(max_count, counts[e]);
     rows += (uint64_t)counts[e];
   }
-  prof_add_ffn(ctx, (uint64_t)grp.n, rows);
-  return run_ffn_launches(ctx, grp, max_count, counts, before_down);
+  bool fused = false;
+  const int rc = run_ffn_launches(ctx, grp, max_count, counts, before_down, behind_event_wait, &fused);
+  prof_add_ffn(ctx, (uint64_t)grp.n, rows, fused);
+  return rc;
 }
 
 // Blocks until the gate kernel of step `seq` has published counts and scores, and decodes them.
@@ -426,7 +463,8 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
-  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + (2 + kFfnWorkCounters) * sizeof(uint32_t);
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + (2 + kFfnWorkCounters) * sizeof(uint32_t) +
+                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t);
   uint8_t* ctrl = nullptr;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctrl, ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
@@ -434,6 +472,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
   ctx->d_ticket = reinterpret_cast<unsigned int*>(ctrl + E * (sizeof(unsigned long long) + sizeof(int32_t)));
   ctx->d_work = reinterpret_cast<uint32_t*>(ctx->d_ticket) + 2;
+  ctx->d_done = ctx->d_work + kFfnWorkCounters;
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
@@ -472,9 +511,6 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
                     s.expert_format == OLED_EXPERTS_FP8, ctx->d_xp,
                     ctx->d_hbuf, (int)(T * K));
   if (rc != OLED_OK) return fail(rc);
-  if (const char* env = getenv("OLED_FFN_IMPL"))
-    ctx->ffn_impl = (atoi(env) == 1 && s.expert_format == OLED_EXPERTS_BF16) ? 1 : 0;
-  if (const char* env = getenv("OLED_MISS_CHUNK")) ctx->miss_chunk = std::max(1, atoi(env));
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(OLED_ERR_CUDA);
   *out_ctx = ctx;
   return OLED_OK;
@@ -554,6 +590,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   // adds at most 2^-9 relative per term, far inside the output tolerance)
   ctx->y_bf16 = ctx->ffn_impl == 0 && (size_t)T * K > 4096;
   // 1. gate, counts and reuse-score numerators; the kernel's last CTA reports them to the host
+  // and, in a small step, also builds the permutation
   if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
   ctx->ctrl_dirty = true;
   ctx->work_next = 0;
@@ -563,23 +600,33 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   rep.host_scores = reinterpret_cast<unsigned long long*>(ctx->h_ctrl);
   rep.host_counts = reinterpret_cast<unsigned long long*>(ctx->h_ctrl) + E;
   rep.seq = ctx->seq;
+  ctx->small_step = T <= 1024 && route_fuses_permutation(T, E, K);
+  const bool small = ctx->small_step;
   {
-    ProfScope ps(ctx, OLED_KERNEL_ROUTE, ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * 8,
+    ProfScope ps(ctx, OLED_KERNEL_ROUTE, ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * (small ? 20 : 8),
                  2ull * T * H * E);
     launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
-                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, rep);
+                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, rep,
+                 small ? ctx->d_offsets : nullptr, small ? ctx->d_perm : nullptr, small ? ctx->d_pos : nullptr);
   }
-  const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
-  {
+  ctx->launches += 1;
+  // token rows in sorted order (xp): a small step on bf16 stores needs none - its FFN kernels
+  // gather the rows themselves; otherwise the permutation kernel copies them (few rows per
+  // expert: one CTA per expert) or a gather kernel does
+  ctx->x_gather = (small && ctx->gather_in_ffn && ctx->ffn_impl == 0 && ctx->shape.expert_format == OLED_EXPERTS_BF16)
+                      ? static_cast<const uint16_t*>(hidden) : nullptr;
+  const bool fuse_gather = !small && (size_t)T * K <= 4096;
+  if (!small) {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
     launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
                    static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H);
+    ctx->launches += 1;
   }
-  if (!fuse_gather) {
+  if (!fuse_gather && ctx->x_gather == nullptr) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
+    ctx->launches += 1;
   }
-  ctx->launches += fuse_gather ? 2 : 3;
   if (ctx->corrupt_perm) {
     launch_corrupt_perm(st, ctx->d_perm, T * K);
     ctx->launches += 1;
@@ -607,7 +654,9 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
       }
     // token tile of this launch: twice the mean load per expert (a fuller expert takes more tiles)
     const int mean_load = (int)(((size_t)T * K + E - 1) / E);
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr);
+    ctx->hit_fused = false;
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false,
+                                     &ctx->hit_fused);
     if (rc0 != OLED_OK) return rc0;
   }
 
@@ -645,8 +694,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   const size_t esz = ctx->shape.expert_format == OLED_EXPERTS_FP8 ? 1 : 2;
   const size_t hi_elems = (size_t)ctx->shape.hidden * (size_t)ctx->shape.intermediate;
   const size_t down_off = 2 * hi_elems * esz, down_bytes = hi_elems * esz;
-  static const bool split_allowed = getenv("OLED_SPLIT_LAST") == nullptr || atoi(getenv("OLED_SPLIT_LAST")) != 0;
-  const bool split_last = split_allowed && n_miss > 0 && E >= 3;
+  const bool split_last = ctx->split_last && n_miss > 0 && E >= 3;
   const size_t tail = std::min(n_miss, (size_t)ctx->miss_chunk);
   const size_t bounds[3] = {0, n_miss - tail, n_miss};
   size_t n_groups = 0;
@@ -684,13 +732,13 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   {
     uint64_t hit_rows = 0;
     for (int32_t e : plan.hits) hit_rows += (uint64_t)counts[e];
-    prof_add_ffn(ctx, plan.hits.size(), hit_rows);
+    prof_add_ffn(ctx, plan.hits.size(), hit_rows, ctx->hit_fused);
   }
   int rc = OLED_OK;
   for (size_t c = 0; c < n_groups; ++c) {
     OLED_CUDA(ctx, cudaStreamWaitEvent(st, ctx->fill_events[c], 0));
     rc = run_ffn_group(ctx, L, plan.misses, group_begin[c], group_end[c], counts,
-                       split_last && group_end[c] == n_miss ? ctx->fill_events[2] : nullptr);
+                       split_last && group_end[c] == n_miss ? ctx->fill_events[2] : nullptr, true);
     if (rc != OLED_OK) return rc;
   }
 
@@ -934,6 +982,18 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
     case OLED_OPT_MISS_CHUNK:
       if (value < 1) return OLED_ERR_INVALID_ARG;
       ctx->miss_chunk = (int)std::min<int64_t>(value, OLED_MAX_EXPERTS);
+      return OLED_OK;
+    case OLED_OPT_SPLIT_LAST_FILL:
+      ctx->split_last = value != 0;
+      return OLED_OK;
+    case OLED_OPT_FUSE_FFN:
+      ctx->fuse_ffn = value != 0;
+      return OLED_OK;
+    case OLED_OPT_GATHER_IN_FFN:
+      ctx->gather_in_ffn = value != 0;
+      return OLED_OK;
+    case OLED_OPT_PDL:
+      pdl_set_allowed(value != 0);
       return OLED_OK;
     default:
       return OLED_ERR_INVALID_ARG;

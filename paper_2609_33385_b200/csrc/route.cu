@@ -12,6 +12,7 @@
 //   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
 // The router stays off the tensor cores on purpose: their accumulation order is unspecified.
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <mutex>
 
@@ -243,6 +244,222 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   route_publish(rep, counts, scores, E, &s_last);
 }
 
+// ---- small steps: one kernel for gate, top-k, gate scores, counts, scores AND the permutation --
+// One CTA per token.  The logits are computed as in route_kernel (same chains, same butterfly).
+// The top-k is a rank computation spread over all warps: expert e is selected iff fewer than K
+// experts precede it in the order (logit descending, index ascending), and its rank is the number
+// that do - the same total order the round-by-round selection walks, so the ids and their order
+// are identical.  The last CTA to finish (a ticket) publishes counts and scores to the host and,
+// if asked to, builds offsets, the stable permutation and its inverse: with at most
+// kSmallMaxAssign assignments one CTA does that in a few microseconds, which removes a kernel
+// boundary from the latency chain of a few-token step.
+constexpr int kSmallMaxAssign = 2048;
+constexpr int kSmallMaxExperts = 128;
+
+__device__ __forceinline__ uint32_t order_key(float v) {  // v is not NaN and not -0
+  const uint32_t bits = __float_as_uint(v);
+  return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+
+template <int WARPS, int UNROLL, int kEPerWarp>
+__global__ void __launch_bounds__(WARPS * 32)
+route_small_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
+                   const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
+                   int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
+                   float* __restrict__ gate, int32_t* __restrict__ counts,
+                   unsigned long long* __restrict__ scores, int32_t* __restrict__ offsets,
+                   int32_t* __restrict__ perm, int32_t* __restrict__ pos, int do_perm, RouteReport rep) {
+  __shared__ float s_logits[OLED_MAX_EXPERTS];
+  __shared__ int s_sel_id[OLED_MAX_TOPK];
+  __shared__ float s_sel_logit[OLED_MAX_TOPK];
+  __shared__ int s_last;
+  __shared__ int s_off[kSmallMaxExperts + 1];
+  __shared__ int s_ids[kSmallMaxAssign];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x;
+  griddep_launch_dependents();
+  if (gridDim.x <= 128) {
+    // The router weights do not depend on the predecessor (the previous layer's combine), but the
+    // expert weights streamed since their last use have pushed them out of L2 - so they are
+    // called back in while this kernel still waits for its input.
+    for (int eb = warp * kEPerWarp; eb < E; eb += WARPS * kEPerWarp)
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        const int e = min(eb + b, E - 1);
+        for (int off = lane * 64; off < H; off += 32 * 64)  // 128-byte lines of the row
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(wr + (size_t)e * H + off));
+      }
+  }
+  griddep_wait();
+
+  for (int eb = warp * kEPerWarp; eb < E; eb += WARPS * kEPerWarp) {
+    float acc[kEPerWarp];
+#pragma unroll
+    for (int b = 0; b < kEPerWarp; ++b) acc[b] = 0.0f;
+#pragma unroll UNROLL
+    for (int hc = 0; hc < H; hc += 256) {
+      const int h = hc + lane * 8;
+      uint32_t xw[4], ww[kEPerWarp][4];
+      {
+        const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+        xw[0] = v.x; xw[1] = v.y; xw[2] = v.z; xw[3] = v.w;
+      }
+#pragma unroll
+      for (int b = 0; b < kEPerWarp; ++b) {
+        const int e = min(eb + b, E - 1);
+        const uint4 v = *reinterpret_cast<const uint4*>(wr + (size_t)e * H + h);
+        ww[b][0] = v.x; ww[b][1] = v.y; ww[b][2] = v.z; ww[b][3] = v.w;
+      }
+      // elements in ascending h: word 0 low half, word 0 high half, word 1 low half, ...
+#pragma unroll
+      for (int wi = 0; wi < 4; ++wi) {
+        const float xl = bf16_lo(xw[wi]), xh = bf16_hi(xw[wi]);
+#pragma unroll
+        for (int b = 0; b < kEPerWarp; ++b) acc[b] = __fmaf_rn(xl, bf16_lo(ww[b][wi]), acc[b]);
+#pragma unroll
+        for (int b = 0; b < kEPerWarp; ++b) acc[b] = __fmaf_rn(xh, bf16_hi(ww[b][wi]), acc[b]);
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < kEPerWarp; ++b) {
+      float v = acc[b];
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, d));
+      const int e = eb + b;
+      if (lane == 0 && e < E) {
+        if (bias != nullptr) v = __fadd_rn(v, bias[e]);
+        s_logits[e] = v;
+        if (logits_out != nullptr) logits_out[(size_t)t * E + e] = v;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- top-k by rank.  A NaN logit is read as -inf (the order stays total), -0 as +0 (they
+  // compare equal, the index decides); ties go to the lower index.
+  {
+    constexpr int kPerLane = OLED_MAX_EXPERTS / 32;
+    uint32_t key[kPerLane];
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+      const int e = lane + 32 * i;
+      if (e < E) {
+        const float xv = s_logits[e];
+        key[i] = order_key((xv == xv) ? __fadd_rn(xv, 0.0f) : __int_as_float(0xff800000));
+      } else {
+        key[i] = 0u;  // below every real key (the key of -inf is 0x007fffff)
+      }
+    }
+    for (int e = warp; e < E; e += WARPS) {
+      const float xv = s_logits[e];
+      const float ve = (xv == xv) ? __fadd_rn(xv, 0.0f) : __int_as_float(0xff800000);
+      const uint32_t ke = order_key(ve);
+      int before = 0;
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        const int a = lane + 32 * i;
+        if (32 * i < E) before += (a < E && (key[i] > ke || (key[i] == ke && a < e))) ? 1 : 0;
+      }
+      before = __reduce_add_sync(0xffffffffu, before);
+      if (lane == 0 && before < K) {
+        s_sel_id[before] = e;
+        s_sel_logit[before] = ve;
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int my_id = lane < K ? s_sel_id[lane] : 0;
+    const float my_logit = lane < K ? s_sel_logit[lane] : 0.0f;
+    const float top = __shfl_sync(0xffffffffu, my_logit, 0);
+    const float z = lane < K ? exp_spec(__fsub_rn(my_logit, top)) : 0.0f;
+    float sum = __shfl_sync(0xffffffffu, z, 0);
+    for (int j = 1; j < K; ++j) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, z, j));
+    if (lane < K) {
+      const float g = __fdiv_rn(z, sum);
+      ids[(size_t)t * K + lane] = my_id;
+      gate[(size_t)t * K + lane] = g;
+      float c = conf[t];
+      c = (c != c) ? 0.0f : fminf(fmaxf(c, 0.0f), 1.0f);  // psi(c) = c, clamped; NaN -> 0
+      const float pv = __fmul_rn(g, c);
+      // a NaN product (non-finite activations) adds nothing; the 64-bit conversion of a NaN
+      // would return 2^63
+      const unsigned long long q = (pv == pv) ? __float2ull_rz(__fmul_rn(pv, 4294967296.0f)) : 0ull;
+      atomicAdd(&counts[my_id], 1);
+      atomicAdd(&scores[my_id], q);
+    }
+    __syncwarp();
+    if (lane == 0) {
+      s_last = 0;
+      if (rep.ticket != nullptr) {
+        __threadfence();
+        s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+      }
+    }
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // ---- the last CTA: report to the host first (it plans the fills from it), then the permutation
+  if (rep.host_scores != nullptr) {
+    const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
+    const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+      // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
+      rep.host_scores[e] = tag16 | (__ldcg(&scores[e]) & 0xffffffffffffull);
+      rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
+    }
+  }
+  if (!do_perm) return;
+  const int n = T * K;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s_ids[i] = __ldcg(&ids[i]);
+  if (warp == 0) {  // exclusive scan of the counts
+    const int per = (E + 31) / 32;
+    int local = 0;
+    for (int i = 0; i < per; ++i) {
+      const int e = lane * per + i;
+      if (e < E) local += __ldcg(&counts[e]);
+    }
+    int incl = local;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
+    }
+    int run = incl - local;
+    for (int i = 0; i < per; ++i) {
+      const int e = lane * per + i;
+      if (e < E) {
+        s_off[e] = run;
+        offsets[e] = run;
+        run += __ldcg(&counts[e]);
+      }
+    }
+    if (lane == 31) {
+      s_off[E] = incl;
+      offsets[E] = incl;
+    }
+  }
+  __syncthreads();
+  // stable: the assignments of an expert keep their ascending (token, rank) order
+  for (int e = warp; e < E; e += WARPS) {
+    int base = s_off[e];
+    const int end = s_off[e + 1];
+    for (int a0 = 0; a0 < n && base < end; a0 += 32) {
+      const int a = a0 + lane;
+      const bool hit = a < n && s_ids[a] == e;
+      const uint32_t m = __ballot_sync(0xffffffffu, hit);
+      if (hit) {
+        const int r = base + __popc(m & ((1u << lane) - 1u));
+        perm[r] = a;
+        pos[a] = r;
+      }
+      base += __popc(m);
+    }
+  }
+}
+
 // One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
 // assignment list (ascending t*K+j) hands out consecutive sorted rows.
 // If xp != nullptr the CTA also copies the token rows of its expert into sorted order
@@ -367,29 +584,28 @@ gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm, 
 
 }  // namespace
 
+constexpr int kRouteSmallMax = 1024;  // largest step that takes the one-token-per-CTA gate kernel
+
 static thread_local bool g_pdl_step = true;
+static std::atomic<bool> g_pdl_allowed{true};
 void pdl_set_step(bool on) { g_pdl_step = on; }
-bool pdl_enabled() {
-  static int on = -1;
-  if (on < 0) {
-    const char* env = getenv("OLED_PDL");
-    on = (env && atoi(env) == 0) ? 0 : 1;
-  }
-  return on == 1 && g_pdl_step;
+void pdl_set_allowed(bool on) { g_pdl_allowed.store(on); }
+bool pdl_enabled() { return g_pdl_allowed.load() && g_pdl_step; }
+
+bool route_fuses_permutation(int T, int E, int K) {
+  return (size_t)T * K <= (size_t)kSmallMaxAssign && E <= kSmallMaxExperts;
 }
 
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep) {
-  static int small_max = -1;  // tuning aid: largest step that takes the one-token-per-CTA variant
-  if (small_max < 0) {
-    const char* a = getenv("OLED_ROUTE_SMALL_MAX");
-    small_max = a ? atoi(a) : 1024;
-  }
-  if (T <= small_max) {
-    constexpr int TT = 1, W = 16;
-    launch_pdl(route_kernel<TT, W, 4, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
-               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
+                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep,
+                  int32_t* offsets, int32_t* perm, int32_t* pos) {
+  if (T <= kRouteSmallMax) {  // one token per CTA
+    constexpr int W = 16;
+    const int do_perm = (offsets != nullptr && perm != nullptr && pos != nullptr && rep.ticket != nullptr &&
+                         route_fuses_permutation(T, E, K)) ? 1 : 0;
+    launch_pdl(route_small_kernel<W, 4, 4>, dim3(T), dim3(W * 32), 0, st, x, w_router, bias, conf, T, H, E, K, logits,
+               ids, gate, counts, scores, offsets, perm, pos, do_perm, rep);
   } else {
     constexpr int TT = 8, W = 8;
     launch_pdl(route_kernel<TT, W, 1, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
@@ -492,7 +708,7 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   if (n_tokens == 0) return OLED_OK;
   launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
                confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores,
-               RouteReport{});
+               RouteReport{}, nullptr, nullptr, nullptr);
   launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
                  hidden_dim);
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
