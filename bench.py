@@ -300,6 +300,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-residency", action="store_true")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    ap.add_argument("--opt", action="append", default=[], metavar="ID=VALUE",
+                    help="oled_set_option(ID, VALUE) on every context (launch-structure switches, see include/oled.h)")
     ap.add_argument("--expert-format", default="bf16", choices=["bf16", "fp8"],
                     help="fp8: e4m3 expert blobs with row scales (an extension; the headline is bf16)")
     args = ap.parse_args()
@@ -340,6 +342,9 @@ def main():
     t_setup = time.perf_counter()
     fp8 = args.expert_format == "fp8"
     run = StackRunner(w, device=device, gen_threads=threads, distinct_layers=args.distinct_layers, fp8=fp8)
+    opts = [tuple(int(v) for v in o.split("=")) for o in args.opt]
+    for oid, val in opts:
+        run.ctx.set_option(oid, val)
     xs, cs = [], []
     for _, _, h_bits, conf in synth.denoise_inputs(w):
         xs.append(bits_to_dev(h_bits, device))
@@ -426,6 +431,8 @@ def main():
     # 4. full residency on the same workload (C = E): the HBM-bound regime and the TPOT ratio
     if not args.no_full_residency and w.residency < 1.0:
         full = StackRunner(w.replace(residency=1.0), device=device, share_store_of=run, fp8=fp8)
+        for oid, val in opts:
+            full.ctx.set_option(oid, val)
         # dummy requests (i.i.d. tokens activate nearly every expert) so that no cold miss is left
         dummy = []
         for j, (_, _, h_bits, conf) in enumerate(synth.denoise_inputs(w.replace(shared_beta=0.0, seed=w.seed + 1))):

@@ -24,7 +24,7 @@
  *   - One context is used by one host thread at a time.  Work is ordered on the stream given
  *     to oled_create(); oled_denoise_step() blocks the host until the gate results of the step
  *     are known (a few hundred bytes are read back to plan the copies), not until the step ends.
- *   - Shape limits: hidden a multiple of 256; intermediate a multiple of 128;
+ *   - Shape limits: hidden a multiple of 256, at most 16384; intermediate a multiple of 128;
  *     1 <= top_k <= 32, top_k <= n_experts <= OLED_MAX_EXPERTS, max_tokens <= 65535.
  */
 #ifndef OLED_H_
@@ -174,6 +174,13 @@ int oled_debug_last(oled_ctx* ctx, int32_t layer, int32_t* ids, float* gate, int
  * of assignment (t,j)).  Synchronises. */
 int oled_debug_perm(oled_ctx* ctx, int32_t layer, int32_t* offsets, int32_t* pos);
 
+/* Tracing aid: the device-side timeline of the most recent step on `layer` that ran with
+ * OLED_OPT_TIMELINE on.  times: host uint64[3 * OLED_TIMELINE_SLOTS], nanoseconds of the GPU's
+ * global timer: [slot] earliest kernel entry, [SLOTS + slot] earliest pass of the dependency
+ * wait, [2*SLOTS + slot] latest CTA end; a slot that did not run holds UINT64_MAX / 0.
+ * Synchronises. */
+int oled_debug_timeline(oled_ctx* ctx, int32_t layer, uint64_t* times);
+
 /* Gate logits fp32[T*E] of the most recent step (host buffer).  Synchronises. */
 int oled_debug_logits(oled_ctx* ctx, int32_t layer, float* logits);
 
@@ -215,16 +222,20 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * to measure what each one buys):
  * OLED_OPT_SPLIT_LAST_FILL: the step's last expert blob is copied in two parts, gate|up first,
  *   so that the last group's gate/up kernel runs while its down-projection weights still arrive.
- * OLED_OPT_FUSE_FFN: few-token steps on bf16 stores run gate/up and down projection of an expert
- *   group as ONE launch.
- * OLED_OPT_GATHER_IN_FFN: few-token steps on bf16 stores let the FFN kernel gather the token rows
- *   it needs instead of reading a sorted copy of the input written by an earlier kernel.
+ * OLED_OPT_FUSE_COMBINE: inside oled_denoise_iteration(), steps of at most 1024 tokens leave a
+ *   layer's combine and residual to the next layer's gate kernel (one kernel boundary and one
+ *   reload of the hidden states less per layer).
  * OLED_OPT_PDL: programmatic dependent launch between the kernels of a few-token step
  *   (process-wide, not per context). */
 #define OLED_OPT_SPLIT_LAST_FILL 9
-#define OLED_OPT_FUSE_FFN 10
-#define OLED_OPT_GATHER_IN_FFN 11
+#define OLED_OPT_FUSE_COMBINE 10
 #define OLED_OPT_PDL 12
+/* OLED_OPT_TIMELINE: 1 = the kernels of every step record, per kernel, when its first CTA entered,
+ * when the first one got past its dependency wait and when the last one finished (GPU global
+ * timer); read with oled_debug_timeline().  Off by default (a few atomics per CTA). */
+#define OLED_OPT_TIMELINE 13
+#define OLED_TIMELINE_SLOTS 12 /* 0 gate, 1 permutation, 2 gather (not recorded),
+                                  3..10 the step's FFN launches in order, 11 combine */
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */
 #define OLED_CHECK_ID_DUPLICATE 0x02u  /* a token routed twice to one expert                        */
 #define OLED_CHECK_OFFSETS 0x04u       /* offsets are not the exclusive scan of the counts          */
@@ -257,8 +268,7 @@ int oled_get_capacity(oled_ctx* ctx, int32_t* capacity);
 #define OLED_KERNEL_FFN_GATE_UP 3
 #define OLED_KERNEL_FFN_DOWN 4
 #define OLED_KERNEL_COMBINE 5
-#define OLED_KERNEL_FFN_FUSED 6 /* gate/up + SwiGLU + down projection in one launch (few-token steps) */
-#define OLED_N_KERNELS 7
+#define OLED_N_KERNELS 6
 typedef struct {
   uint64_t launches;
   double ms;       /* sum of CUDA-event durations */

@@ -25,13 +25,14 @@ ERR_OOM, ERR_CUDA, ERR_TIMEOUT, ERR_NO_SLOT, ERR_STALE_DEBUG = -5, -6, -7, -8, -
 OPT_FFN_IMPL, OPT_MISS_CHUNK, OPT_PROFILE, OPT_POLICY, OPT_ADAPT_PERIOD = 1, 2, 3, 4, 5
 OPT_TEST_WITHHOLD_LOADS = 6
 OPT_SELF_CHECK, OPT_TEST_CORRUPT_PERM = 7, 8
-OPT_SPLIT_LAST_FILL, OPT_FUSE_FFN, OPT_GATHER_IN_FFN, OPT_PDL = 9, 10, 11, 12
+OPT_SPLIT_LAST_FILL, OPT_FUSE_COMBINE, OPT_PDL, OPT_TIMELINE = 9, 10, 12, 13
+TIMELINE_SLOTS = 12
 ERR_SELF_CHECK = -10
 CHECK_FLAGS = {0x01: "id_range", 0x02: "id_duplicate", 0x04: "offsets", 0x08: "perm_range", 0x10: "inverse",
                0x20: "row_expert", 0x40: "order"}
 POLICY_PRIORITY, POLICY_LRU, POLICY_LFU = 0, 1, 2
 POLICY_IDS = {"priority": 0, "lru": 1, "lfu": 2}
-KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine", "ffn_fused"]
+KERNEL_NAMES = ["route", "permute", "gather", "ffn_gate_up", "ffn_down", "combine"]
 
 EXPORTS = [
     "oled_create", "oled_register_router", "oled_register_experts", "oled_denoise_step",
@@ -41,7 +42,7 @@ EXPORTS = [
     "oled_policy_create", "oled_policy_step", "oled_policy_destroy", "oled_route_noalloc",
     "oled_adapt_capacity", "oled_get_capacity", "oled_policy_set_policy", "oled_policy_fills_reused",
     "oled_policy_adapt", "oled_clear_status", "oled_policy_time", "oled_expert_blob_bytes",
-    "oled_self_check_report", "oled_debug_perm", "oled_policy_create_stack",
+    "oled_self_check_report", "oled_debug_perm", "oled_policy_create_stack", "oled_debug_timeline",
 ]
 EXPERTS_BF16, EXPERTS_FP8 = 0, 1
 NOALLOC_MAX_TOKENS = 256
@@ -112,6 +113,7 @@ def load() -> C.CDLL:
     lib.oled_debug_last.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.oled_debug_logits.argtypes = [vp, i32, vp]
     lib.oled_debug_perm.argtypes = [vp, i32, vp, vp]
+    lib.oled_debug_timeline.argtypes = [vp, i32, vp]
     lib.oled_policy_create_stack.argtypes = [i32, i32, C.POINTER(i32), i32, C.POINTER(vp), C.POINTER(i32)]
     lib.oled_reset_cache.argtypes = [vp]
     lib.oled_residual_add.argtypes = [vp, vp, vp, vp, C.c_size_t]
@@ -228,6 +230,12 @@ class OledContext:
                    pos=np.zeros(n_tokens * self.shape.top_k, np.int32))
         self._check(self._lib.oled_debug_perm(self._h, layer, _np_ptr(out["offsets"]), _np_ptr(out["pos"])),
                     "oled_debug_perm")
+        return out
+
+    def debug_timeline(self, layer: int) -> np.ndarray:
+        """[3, TIMELINE_SLOTS] uint64: earliest entry, earliest start, latest end per kernel slot."""
+        out = np.zeros((3, TIMELINE_SLOTS), np.uint64)
+        self._check(self._lib.oled_debug_timeline(self._h, layer, _np_ptr(out)), "oled_debug_timeline")
         return out
 
     def debug_logits(self, layer: int, n_tokens: int) -> np.ndarray:

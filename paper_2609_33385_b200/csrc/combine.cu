@@ -18,11 +18,13 @@ __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
                const int32_t* __restrict__ pos, int H, int K, uint16_t* __restrict__ out,
                const uint16_t* __restrict__ x, uint16_t* __restrict__ x_next,
-               uint32_t* __restrict__ zero_words, int n_zero_words) {
+               uint32_t* __restrict__ zero_words, int n_zero_words, StepTimeline* timeline) {
   const int t = blockIdx.x;
   const int slice = H / gridDim.y, h_begin = blockIdx.y * slice, h_end = h_begin + slice;
   griddep_launch_dependents();
+  if (threadIdx.x == 0) timeline_entry(timeline, kTimelineSlots - 1);
   griddep_wait();
+  if (threadIdx.x == 0) timeline_start(timeline, kTimelineSlots - 1);
   if (t == 0 && blockIdx.y == 0 && zero_words != nullptr)
     for (int i = threadIdx.x; i < n_zero_words; i += blockDim.x) zero_words[i] = 0u;
   __shared__ float s_g[OLED_MAX_TOPK];
@@ -83,6 +85,7 @@ combine_kernel(const float* __restrict__ y, const float* __restrict__ gate,
       *reinterpret_cast<uint2*>(x_next + (size_t)t * H + h) = rk;
     }
   }
+  if (threadIdx.x == 0) timeline_end(timeline, kTimelineSlots - 1);
 }
 
 // Large steps with bf16 assignment outputs: eight elements per thread, so that every access is
@@ -160,7 +163,14 @@ residual_add_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__
 
 void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
-                    uint32_t* zero_words, int n_zero_words) {
+                    uint32_t* zero_words, int n_zero_words, StepTimeline* timeline) {
+  static bool carveout_done = false;
+  if (!carveout_done) {  // keep the FFN kernels' shared-memory carve-out: see gate_cluster.cu
+    cudaFuncSetAttribute(combine_kernel<true, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaFuncSetAttribute(combine_kernel<false, 8>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaGetLastError();
+    carveout_done = true;
+  }
   const bool small = (size_t)T * K <= 4096;
   // small steps: slices of 512 columns (128 threads x 4) while that leaves at most ~4 CTAs per SM
   int slices = 1;
@@ -169,19 +179,19 @@ void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* ga
   const dim3 sgrid(T, slices), sblock(slices > 1 ? 128 : 256);
   if (y_bf16 && small)
     launch_pdl(combine_kernel<true, 8>, sgrid, sblock, 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
-               n_zero_words);
+               n_zero_words, timeline);
   else if (y_bf16 && H % 8 == 0)
     launch_pdl(combine_bf16_wide_kernel, dim3(T), dim3(256), 0, st, reinterpret_cast<const uint16_t*>(y), gate, pos, H,
                K, out, x, x_next, zero_words, n_zero_words);
   else if (y_bf16)
     launch_pdl(combine_kernel<true, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
-               n_zero_words);
+               n_zero_words, timeline);
   else if (small)
     launch_pdl(combine_kernel<false, 8>, sgrid, sblock, 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
-               n_zero_words);
+               n_zero_words, timeline);
   else
     launch_pdl(combine_kernel<false, 1>, dim3(T), dim3(256), 0, st, y, gate, pos, H, K, out, x, x_next, zero_words,
-               n_zero_words);
+               n_zero_words, timeline);
 }
 
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {

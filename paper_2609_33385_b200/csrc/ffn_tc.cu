@@ -97,7 +97,6 @@ struct __align__(16) SharedCtl {
   int n_tiles_total;
   int pad;
   int item_ring[kItemRing];  // item numbers handed out by the producer; -1 = no more work
-  int gather_tok[256];       // token of every row of the current gate/up item (gathering warp only)
   int tile_prefix[OLED_MAX_EXPERTS + 1];
   int row_start[OLED_MAX_EXPERTS];
   int count[OLED_MAX_EXPERTS];
@@ -110,16 +109,6 @@ constexpr uint32_t kCtlBytes = (sizeof(SharedCtl) + 1023u) & ~1023u;
 
 struct Item {
   int slot, m0, row0, valid;
-  int kind;  // 1: gate/up (+SwiGLU), 2: down projection
-  int g;     // index of the expert in the launch's group
-};
-// Shape of the launch's work list.  Items [0, n1) are of the kernel's first kind; a FUSED launch
-// (KIND 3) appends the down-projection items [n1, n1 + n2) of the same experts and token tiles.
-struct WorkShape {
-  int n1, m_tiles1, m_rows1, k_blocks1;
-  int m_tiles2, m_rows2, k_blocks2;
-  int kind1;
-  int n_box;
 };
 // Items (expert, token tile, weight tile) are handed out DYNAMICALLY: the producer thread of a
 // CTA draws item numbers from a counter in global memory (one atomic per item, fetched one item
@@ -137,86 +126,39 @@ __device__ __forceinline__ int take_item(SharedCtl* ctl, int seq, volatile int* 
   mbar_arrive(smem_u32(&ctl->item_empty[slot]));
   return item;
 }
-// cursor: the role's position in the expert list (items arrive in ascending order within a
-// phase, so the search for an item's expert only moves forward; it restarts with the second phase).
-struct ItemCursor {
-  int g = 0;
-  int phase2 = 0;
-};
-__device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, const WorkShape& ws,
-                                            ItemCursor& cur, Item& it) {
-  int m_tiles = ws.m_tiles1, m_rows = ws.m_rows1;
-  it.kind = ws.kind1;
-  if (item >= ws.n1) {
-    item -= ws.n1;
-    m_tiles = ws.m_tiles2;
-    m_rows = ws.m_rows2;
-    it.kind = 2;
-    if (!cur.phase2) {
-      cur.phase2 = 1;
-      cur.g = 0;
-    }
-  }
+__device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int m_tiles,
+                                            int m_rows, int n_box, int& g, Item& it) {
   const int q = item / m_tiles;
   const int m = item - q * m_tiles;
-  int g = cur.g;
   while (ctl->tile_prefix[g + 1] <= q) ++g;
-  cur.g = g;
   const int nt = q - ctl->tile_prefix[g];
-  it.g = g;
   it.slot = grp.slot[g];
   it.m0 = m * m_rows;
-  it.row0 = ctl->row_start[g] + nt * ws.n_box;
-  it.valid = min(ws.n_box, ctl->count[g] - nt * ws.n_box);
+  it.row0 = ctl->row_start[g] + nt * n_box;
+  it.valid = min(n_box, ctl->count[g] - nt * n_box);
 }
-
-// What a launch needs beyond the tensor maps and the expert group.
-struct FfnArgs {
-  const int32_t* offsets;
-  void* out;         // KIND 1 and 3: hbuf (bf16 [rows, I]); KIND 2: y
-  void* out2;        // KIND 3: y
-  int H, I, n_stages, k_atoms, early_start, out_bf16;
-  const uint8_t* pool;
-  unsigned long long slot_bytes;
-  uint32_t* status;
-  uint32_t* work_counter;
-  // token rows of gate/up items gathered from the step's input by a warp of the CTA instead of a
-  // TMA load of pre-sorted rows (bf16 stores): x [T, H], perm [T*K], K; x_gather == nullptr: off
-  const uint16_t* x_gather;
-  const int32_t* perm;
-  int top_k;
-  uint32_t* done;    // KIND 3: per expert of the group, epilogue warps that have stored gate/up rows (zero at start)
-};
 
 // DUAL: two accumulators per item - gate and up (KIND 1, always), or two row blocks of Wd
 // (KIND 2 with the 256-token tile).
 // FP8: the slot pool holds fp8 expert blobs (tm_w is a byte map over the e4m3 codes).
-// KIND 3 (bf16 stores, token tiles of at most 32 rows): the gate/up items in their stacked form,
-// then the down-projection items of the same experts, in ONE launch.  A down item reads the
-// intermediate rows that the gate/up items of its expert wrote, so its producer waits (bounded)
-// until the expert's counter in `done` shows that all of them have been stored; items are handed
-// out in order, gate/up first, so that wait is over long before it is reached except in launches
-// with fewer items than SMs.  The weight stream never stops between the two projections.
 template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
-              const __grid_constant__ CUtensorMap tm_w2, const __grid_constant__ CUtensorMap tm_act2,
-              const __grid_constant__ FfnGroup grp, const __grid_constant__ FfnArgs args) {
+              const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
+              void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int early_start, int out_bf16,
+              const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
+              uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter, StepTimeline* timeline,
+              int timeline_slot) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_box = grp.n_box;
-  const int H = args.H, I = args.I, n_stages = args.n_stages, k_atoms = args.k_atoms, out_bf16 = args.out_bf16;
-  uint32_t* const status = args.status;
-  constexpr bool fused = KIND == 3;
-  static_assert(!(fused && (DUAL || FP8)), "the fused form exists for bf16 stores and single tiles only");
   constexpr bool dual = DUAL;
-  constexpr bool stacked = (KIND == 1 && !DUAL) || fused;  // gate/up items: 64 gate + 64 up rows in one 128-row tile
+  constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t b_bytes = (uint32_t)n_box * 128u;
-  const bool gather = !FP8 && KIND != 2 && args.x_gather != nullptr;
   // bf16 stores: a stage (shared memory) holds the weight tile(s) and the token tile of a k-block.
   // fp8 stores: a stage is a load slot in shared memory - the code tile (one byte per element)
   // followed by the token tile - plus a_cols columns of TENSOR memory, behind the accumulators,
@@ -229,22 +171,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const uint32_t stage_bytes = (uint32_t)k_atoms * atom_bytes;
   constexpr uint32_t atom_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
   const uint32_t a_cols = (uint32_t)k_atoms * atom_cols;
-  WorkShape ws;
-  ws.kind1 = fused ? 1 : KIND;
-  ws.n_box = n_box;
-  ws.k_blocks1 = ((KIND == 2) ? I : H) / (kBlockK * k_atoms);  // stages per item
-  ws.m_rows1 = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
-  ws.m_tiles1 = ((KIND == 2) ? H : I) / ws.m_rows1;
-  ws.k_blocks2 = I / (kBlockK * k_atoms);
-  ws.m_rows2 = kBlockM;
-  ws.m_tiles2 = H / kBlockM;
+  const int k_blocks = (KIND == 1 ? H : I) / (kBlockK * k_atoms);  // stages per item
+  constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
+  const int m_tiles = (KIND == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
   const int a_total = FP8 ? n_stages * (int)a_cols : 0;
   const int acc_stages = (2 * acc_cols + a_total <= 512) ? 2 : 1;
   const uint32_t a_col0 = (uint32_t)(acc_stages * acc_cols);  // first column of the weight stages
-  // warps that can own a 16-column chunk; the SwiGLU epilogue profits from all 16, the plain
-  // store epilogue of KIND 2 runs best with 8
-  const int epi_warps = min((KIND != 2 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+  // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
+  // plain store epilogue of KIND 2 runs best with 8
+  const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
   // fp8 stores: the four dedicated converter warps plus epilogue warps this token tile leaves
   // idle form conv_groups (at most two: more of them take issue slots from the MMA thread and
   // measured slower) groups of four warps, one warp per TMEM lane quarter.
@@ -265,19 +201,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // ---- set-up that depends on no earlier kernel: barriers, TMEM (overlaps the predecessor's tail)
   griddep_launch_dependents();
   if (threadIdx.x == 0) {
+    timeline_entry(timeline, timeline_slot);
     for (int s = 0; s < kMaxStages; ++s) {
-      // the stage's TMA transaction (plus the gathering warp where token rows are gathered), or
-      // every lane of the four converting warps
-      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 128u : gather ? 2u : 1u);
+      // the stage's TMA transaction, or every lane of the four converting warps
+      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 128u : 1u);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int s = 0; s < kMaxStages; ++s) mbar_init(smem_u32(&ctl->slot_full[s]), 1);
     for (int s = 0; s < kItemRing; ++s) {
       mbar_init(smem_u32(&ctl->item_full[s]), 1);
-      // consumers: the MMA thread, one lane of every epilogue warp, of every converter warp and
-      // of the gathering warp
-      mbar_init(smem_u32(&ctl->item_empty[s]),
-                1u + (uint32_t)epi_warps + (FP8 ? 4u * (uint32_t)conv_groups : 0u) + (gather ? 1u : 0u));
+      // consumers: the MMA thread, one lane of every epilogue warp and of every converter warp
+      mbar_init(smem_u32(&ctl->item_empty[s]), 1u + (uint32_t)epi_warps + (FP8 ? 4u * (uint32_t)conv_groups : 0u));
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
@@ -291,13 +225,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == kProducerWarp && lane == 0) {  // the tensor maps, ahead of the first copy
+  if (warp == kProducerWarp && lane == 0) {  // the two tensor maps, ahead of the first copy
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
-    if (fused) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w2)) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act2)) : "memory");
-    }
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -307,19 +237,20 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // ---- from here on the step's earlier kernels must have completed: work table from offsets.
-  // KIND 1 and 3 follow the permutation, whose products they read from the first instruction on.
-  // KIND 2 follows KIND 1 of the same expert group: the offsets and the expert weights are older
-  // than that kernel, only the token tiles (hbuf) are its product - so a KIND 2 CTA, which gets
-  // its SM when a KIND 1 CTA leaves it, sets up and streams its first weight tiles while the
-  // slower SMs still finish KIND 1; its producer waits for the predecessor before the first
-  // token-tile load.  (early_start is set by the host only where that is safe: see launch_ffn_tc.)
-  const bool early = KIND == 2 && args.early_start != 0;
+  // KIND 1 follows the permutation, whose products it reads from the first instruction on.  KIND 2
+  // follows KIND 1 of the same expert group: the offsets and the expert weights are older than
+  // that kernel, only the token tiles (hbuf) are its product - so a KIND 2 CTA, which gets its SM
+  // when a KIND 1 CTA leaves it, sets up and streams its first weight tiles while the slower SMs
+  // still finish KIND 1; its producer waits for the predecessor before the first token-tile load.
+  // (early_start is set by the host only where that is safe: see launch_ffn_tc and launch_variant)
+  const bool early = KIND == 2 && early_start != 0;
   if (!early) griddep_wait();
+  if (threadIdx.x == 0) timeline_start(timeline, timeline_slot);
   for (int g = threadIdx.x; g < grp.n; g += kThreads) {
     const int e = grp.expert[g];
-    const int s = args.offsets[e];
+    const int s = offsets[e];
     ctl->row_start[g] = s;
-    ctl->count[g] = args.offsets[e + 1] - s;
+    ctl->count[g] = offsets[e + 1] - s;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -339,27 +270,23 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr uint32_t nap_epi = FP8 ? OLED_NAP_EPI : 0u, nap_load = FP8 ? OLED_NAP_LOAD : 0u,
                      nap_conv = FP8 ? OLED_NAP_CONV : 0u;
   const uint32_t tmem_base = ctl->tmem_base;
-  ws.n1 = ctl->n_tiles_total * ws.m_tiles1;
-  const int total_items = ws.n1 + (fused ? ctl->n_tiles_total * ws.m_tiles2 : 0);
-  // KIND 3: epilogue warps that store intermediate rows, per gate/up item, times the items of an expert tile row
-  const uint32_t done_per_tile = (uint32_t)(ws.m_tiles1 * (epi_warps / 2));
+  const int total_items = ctl->n_tiles_total * m_tiles;
   volatile int* abort_flag = &ctl->abort;
 
   if (warp == kProducerWarp && lane == 0) {
     // ------------------------------------------------------------ TMA producer
     // bf16 stores: weight rows and token tile of a k-block go to one operand stage; fp8 stores:
     // code rows and token tile go to one load slot
-    int stage = 0, ready_g = -1;
-    ItemCursor cur;
+    int stage = 0, g = 0;
     uint32_t phase = 0;
     bool ok = true;
     const int ring = n_stages;
     // (with loads withheld - the test of the bounded waits - nothing is published either)
-    int item = grp.withhold_loads ? 0 : (int)atomicAdd(args.work_counter, 1u);
+    int item = grp.withhold_loads ? 0 : (int)atomicAdd(work_counter, 1u);
     for (int seq = 0; ok && !grp.withhold_loads; ++seq) {
       const bool none = item >= total_items;
       // the next item's number is fetched now: the atomic's latency lies under this item's loads
-      const int next = none ? item : (int)atomicAdd(args.work_counter, 1u);
+      const int next = none ? item : (int)atomicAdd(work_counter, 1u);
       const int ring_slot = seq % kItemRing;
       if (!mbar_wait(smem_u32(&ctl->item_empty[ring_slot]), ((uint32_t)(seq / kItemRing) & 1u) ^ 1u, abort_flag, status,
                      nap_load)) {
@@ -370,38 +297,31 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       mbar_arrive(smem_u32(&ctl->item_full[ring_slot]));
       if (none) break;
       Item it;
-      decode_item(ctl, grp, item, ws, cur, it);
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       item = next;
-      const bool second = fused && it.kind == 2;  // a down item of a fused launch
-      const CUtensorMap* map_w = second ? &tm_w2 : &tm_w;
-      const CUtensorMap* map_act = second ? &tm_act2 : &tm_act;
-      const bool tma_tokens = !(gather && it.kind == 1);
-      const int k_blocks = second ? ws.k_blocks2 : ws.k_blocks1;
       constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
       auto load_weights = [&](int st, int kb) {
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
-        mbar_expect_tx(bar, tma_tokens ? stage_bytes : stage_bytes - (uint32_t)k_atoms * b_bytes);
-        if (gather && tma_tokens) mbar_arrive(bar);  // stands in for the gathering warp, which skips this stage
+        mbar_expect_tx(bar, stage_bytes);
         for (int atom = 0; atom < k_atoms; ++atom) {
           const uint32_t w_addr = tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes;
           const int k0 = (kb * k_atoms + atom) * kBlockK;
-          if (stacked && it.kind == 1) {  // tm_w has 64-row boxes here
-            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
-            tma_load_3d(map_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
-          } else if (it.kind == 1) {
-            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);               // gate rows
-            tma_load_3d(map_w, w_addr + w_tile, bar, k0, I + it.m0, it.slot);  // up rows
+          if (stacked) {  // tm_w has 64-row boxes here
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
+            tma_load_3d(&tm_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
+          } else if (KIND == 1) {
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // gate rows
+            tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, I + it.m0, it.slot);  // up rows
           } else {
-            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
-            if (dual) tma_load_3d(map_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
+            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
+            if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
           }
         }
       };
       auto load_tokens = [&](int st, int kb) {
-        if (!tma_tokens) return;
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
         for (int atom = 0; atom < k_atoms; ++atom)
-          tma_load_2d(map_act,
+          tma_load_2d(&tm_act,
                       tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (FP8 ? raw_bytes : a_bytes),
                       bar, (kb * k_atoms + atom) * kBlockK, it.row0);
       };
@@ -415,57 +335,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         kb = pre;
         if (pre == n_stages) phase ^= 1u;
         else stage = pre;
-      }
-      if (second) {
-        // The intermediate rows of this expert's token tile must all be in memory.  If they are
-        // not yet (launches with fewer items than SMs), the weights of as many stages as the ring
-        // holds go first, then the wait, then those stages' token tiles.
-        const uint32_t* flag = args.done + it.g;
-        uint32_t seen = done_per_tile;  // (an expert seen complete stays complete: no second look)
-        if (it.g != ready_g) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
-        int pre = 0;
-        const int stage0 = stage;
-        if (seen < done_per_tile) {
-          pre = min(n_stages, k_blocks);
-          for (int i = 0; i < pre && ok; ++i) {
-            if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_load)) {
-              ok = false;
-              break;
-            }
-            load_weights(stage, i);
-            if (++stage == ring) {
-              stage = 0;
-              phase ^= 1u;
-            }
-          }
-          unsigned long long t0 = 0;
-          for (uint32_t spin = 0; ok; ++spin) {
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
-            if (seen >= done_per_tile) break;
-            if ((spin & 255u) == 255u) {
-              if (*abort_flag) ok = false;
-              const unsigned long long now = globaltimer();
-              if (t0 == 0) t0 = now;
-              if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(status, (uint32_t)kStatusWaitTimeout);
-                ok = false;
-              }
-            }
-          }
-          if (!ok) break;
-        }
-        ready_g = it.g;
-        // the rows were written through the generic proxy; the loads below read through the async proxy
-        asm volatile("fence.proxy.async;" ::: "memory");
-        if (pre > 0) {
-          int st = stage0;
-          for (int i = 0; i < pre; ++i) {
-            load_tokens(st, i);
-            if (++st == ring) st = 0;
-          }
-          kb = pre;
-        }
       }
       for (; kb < k_blocks; ++kb) {
         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_load)) {
@@ -487,8 +356,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
   } else if (warp == kMmaWarp && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
-    int stage = 0, local = 0;
-    ItemCursor cur;
+    int stage = 0, g = 0, local = 0;
     uint32_t phase = 0;
     bool ok = true;
     // Descriptor words of stage 0 (K-major, 128-byte swizzle, 8-row groups 1024 bytes apart); the
@@ -504,8 +372,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const int item = take_item(ctl, local, abort_flag, status, 0u);
       if (item < 0) break;
       Item it;
-      decode_item(ctl, grp, item, ws, cur, it);
-      const int k_blocks = (fused && it.kind == 2) ? ws.k_blocks2 : ws.k_blocks1;
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
       if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
@@ -549,88 +416,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       }
       if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));
     }
-  } else if (gather && warp == kConvWarp0) {
-    // ------------------------------------------------------------ token-row gatherer (bf16 stores)
-    // The token tile of a gate/up item is the rows x[perm[row0 + r] / K, :] of the step's input:
-    // this warp copies their k-blocks into the stages, in the 128-byte-swizzled layout a TMA box
-    // would have produced (16-byte chunk c of row r at r * 128 + ((c ^ (r & 7)) << 4)), so that no
-    // sorted copy of the input has to be written and read back.  Loads run one batch (one k-block
-    // of up to 32 rows: 8 x 16 bytes per lane) ahead of the stores, which wait for the stage.
-    int stage = 0;
-    uint32_t phase = 0;
-    ItemCursor cur;
-    bool live = true;
-    int* tok = ctl->gather_tok;
-    const int c = lane & 7, rs = lane >> 3;
-    const int groups = (n_box + 31) / 32;           // row groups of 32 per k-block
-    for (int seq = 0; live; ++seq) {
-      int item = 0;
-      if (lane == 0) item = take_item(ctl, seq, abort_flag, status, 0u);
-      item = __shfl_sync(0xffffffffu, item, 0);
-      if (item < 0) break;
-      Item it;
-      decode_item(ctl, grp, item, ws, cur, it);
-      if (it.kind != 1) {  // token tiles of down items arrive by TMA: only keep track of the ring
-        const int adv = ws.k_blocks2;
-        stage += adv;
-        phase ^= (uint32_t)(stage / n_stages) & 1u;
-        stage %= n_stages;
-        continue;
-      }
-      __syncwarp();
-      for (int r = lane; r < n_box; r += 32) tok[r] = r < it.valid ? args.perm[it.row0 + r] / args.top_k : -1;
-      __syncwarp();
-      const int k_blocks = ws.k_blocks1;
-      const int n_batches = k_blocks * k_atoms * groups;
-      uint4 cur_v[8], nxt_v[8];
-      auto load_batch = [&](int b, uint4 (&v)[8]) {
-        const int kblk = b / groups, grp_r = b - kblk * groups;  // kblk counts k-blocks of 64
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = grp_r * 32 + rs + 4 * i;
-          const int t = r < n_box ? tok[r] : -1;
-          v[i] = t >= 0 ? __ldg(reinterpret_cast<const uint4*>(args.x_gather + (size_t)t * H + kblk * kBlockK) + c)
-                        : make_uint4(0u, 0u, 0u, 0u);
-        }
-      };
-      load_batch(0, cur_v);
-      for (int b = 0; b < n_batches && live; ++b) {
-        if (b + 1 < n_batches) load_batch(b + 1, nxt_v);
-        const int kblk = b / groups, grp_r = b - kblk * groups;
-        const int atom = kblk % k_atoms;
-        if (atom == 0 && grp_r == 0) {  // first batch of a stage: the MMAs that read its last contents are done
-          int ok = 0;
-          if (lane == 0) ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status) ? 1 : 0;
-          ok = __shfl_sync(0xffffffffu, ok, 0);
-          if (!ok) {
-            live = false;
-            break;
-          }
-        }
-        const uint32_t dst = tiles_base + (uint32_t)stage * stage_bytes + (uint32_t)atom * atom_bytes + a_bytes;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = grp_r * 32 + rs + 4 * i;
-          if (r < n_box) {
-            const uint32_t addr = dst + (uint32_t)r * 128u + (uint32_t)((c ^ (r & 7)) << 4);
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(cur_v[i].x), "r"(cur_v[i].y),
-                         "r"(cur_v[i].z), "r"(cur_v[i].w)
-                         : "memory");
-          }
-        }
-        if (atom == k_atoms - 1 && grp_r == groups - 1) {  // last batch of the stage
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&ctl->full[stage]));
-          if (++stage == n_stages) {
-            stage = 0;
-            phase ^= 1u;
-          }
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) cur_v[i] = nxt_v[i];
-      }
-    }
   } else if (is_conv) {
     // ------------------------------------------------------------ fp8 -> bf16 converters
     // The four warps of a group widen the code tile of one load slot into the weight stage (tensor
@@ -649,7 +434,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     int stage = group, mine = group;
     uint32_t phase = 0;
     bool live = true;
-    const int k_blocks = ws.k_blocks1;
     for (int seq = 0; live; ++seq) {
       int item = 0;
       if (lane == 0) item = take_item(ctl, seq, abort_flag, status, nap_conv);
@@ -700,8 +484,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
-    int local = 0;
-    ItemCursor cur;
+    int g = 0, local = 0;
     uint32_t xn = 0;  // stacked mode: 16-column chunks this warp's chunk group has exchanged so far
     bool alive = true;
     for (; alive; ++local) {
@@ -710,8 +493,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       item = __shfl_sync(0xffffffffu, item, 0);
       if (item < 0) break;
       Item it;
-      decode_item(ctl, grp, item, ws, cur, it);
-      const bool first_kind = it.kind == 1;   // a gate/up item (always true for KIND 1, never for KIND 2)
+      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
       // one lane polls (keeps issue slots free for the producer and MMA threads); the outcome is
@@ -726,7 +508,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const int n_mma = max(16, (it.valid + 15) & ~15);
       const int col = it.m0 + quarter * 32 + lane;  // output feature owned by this thread
       // fp8 stores: one fp32 scale per weight row behind the codes: s_gate[I] | s_up[I] | s_down[H]
-      const float* sc = FP8 ? reinterpret_cast<const float*>(args.pool + (size_t)it.slot * args.slot_bytes + (size_t)3 * H * I)
+      const float* sc = FP8 ? reinterpret_cast<const float*>(pool + (size_t)it.slot * slot_bytes + (size_t)3 * H * I)
                             : nullptr;
       float s0 = 1.0f, s1 = 1.0f;
       if (FP8) {
@@ -744,7 +526,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
-        if (stacked && first_kind) {
+        if (stacked) {
           // lanes 0-63 hold silu's argument (gate rows), lanes 64-127 the up rows of the same
           // features: warps 2,3 hand their chunk to warps 0,1 through a double-buffered slot
           tmem_ld_wait();
@@ -781,7 +563,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
               u[j] = v.x; u[j + 1] = v.y; u[j + 2] = v.z; u[j + 3] = v.w;
             }
             mbar_arrive(smem_u32(&ctl->x_empty[buf][half]));
-            uint16_t* hb = reinterpret_cast<uint16_t*>(args.out);
+            uint16_t* hb = reinterpret_cast<uint16_t*>(out_ptr);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               if (c + j < it.valid) {
@@ -796,7 +578,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           uint32_t rb[16];
           tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
           tmem_ld_wait();
-          uint16_t* hb = reinterpret_cast<uint16_t*>(args.out);
+          uint16_t* hb = reinterpret_cast<uint16_t*>(out_ptr);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             if (c + j < it.valid) {
@@ -808,9 +590,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
           }
         } else {
-          void* const out_y = fused ? args.out2 : args.out;
-          float* y = reinterpret_cast<float*>(out_y);
-          uint16_t* yb = reinterpret_cast<uint16_t*>(out_y);  // many-token steps keep y in bf16
+          float* y = reinterpret_cast<float*>(out_ptr);
+          uint16_t* yb = reinterpret_cast<uint16_t*>(out_ptr);  // many-token steps keep y in bf16
           uint32_t rb[16];
           if (dual) tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
           tmem_ld_wait();
@@ -833,14 +614,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
       }
       if (!alive) break;
-      if (fused && first_kind && quarter < 2) {
-        // this warp's intermediate rows of the item are stored: make them visible device-wide,
-        // then count the warp in (the down items of this expert wait for the full count)
-        __threadfence();
-        asm volatile("fence.proxy.async;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) atomicAdd(args.done + it.g, 1u);
-      }
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
     }
@@ -860,6 +633,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
                  : "memory");
   }
+  if (threadIdx.x == 0) timeline_end(timeline, timeline_slot);
 }
 
 // ---------------------------------------------------------------- host side
@@ -901,7 +675,7 @@ struct Rings {
 };
 // Epilogue warps the kernel activates for a token tile (the others widen fp8 weights).
 int epi_warps_for(int kind, int out_bf16, int n_box) {
-  return std::min((kind != 2 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+  return std::min((kind == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
 }
 // Stage shape and count.  A stage holds two k-blocks where at least four such stages fit (small
 // token tiles, one weight tile) and the contraction has an even number of k-blocks.  bf16 stores:
@@ -909,8 +683,7 @@ int epi_warps_for(int kind, int out_bf16, int n_box) {
 // (eleven measured slower).  fp8 stores: a stage is a load slot in shared memory plus columns of
 // tensor memory behind the accumulators (two accumulator stages if at least two weight stages
 // still fit); the depth is a multiple of the number of converter groups (see the kernel).
-// k_dim2: the second contraction length of a fused launch (0 otherwise).
-Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim, int k_dim2 = 0) {
+Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim) {
   const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
   const uint32_t atom = fp8 ? a / 2 + b : a + b;  // one k-block in shared memory
@@ -921,7 +694,7 @@ Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_di
     kblocks = std::min(kblocks, free_cols / a_cols);
   }
   Rings r;
-  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0 && (k_dim2 / kBlockK) % 2 == 0) ? 2 : 1;
+  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0) ? 2 : 1;
   r.stages = std::min(kblocks / r.k_atoms, kMaxStages);
   if (fp8) {
     const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
@@ -939,24 +712,22 @@ bool set_smem_attr() {
 
 template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
-                    const CUtensorMap& tw2, const CUtensorMap& ta2, const FfnGroup& grp, FfnArgs args,
-                    bool early_allowed, uint32_t smem_of_predecessor) {
-  const Rings r = rings_for(KIND, DUAL, grp.n_box, args.out_bf16, fp8, KIND == 2 ? args.I : args.H,
-                            KIND == 3 ? args.I : 0);
+                    const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
+                    const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter,
+                    uint32_t smem_of_predecessor, bool early_allowed, StepTimeline* timeline, int timeline_slot) {
+  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 1 ? H : I);
   // KIND 2 may start ahead of its dependency wait only where the caller vouches for the ordering
   // (early_allowed, see launch_ffn_tc) AND one of its CTAs and one of the KIND 1 kernel before it
   // cannot share an SM, so that it gets an SM only when a KIND 1 CTA has left it
-  args.early_start = (KIND == 2 && early_allowed && smem_of_predecessor + r.smem > 228u * 1024u) ? 1 : 0;
-  args.n_stages = r.stages;
-  args.k_atoms = r.k_atoms;
-  if constexpr (KIND == 3) {
-    launch_pdl(ffn_tc_kernel<3, false, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, tw2, ta2, grp, args);
-  } else {
-    if (fp8)
-      launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, tw2, ta2, grp, args);
-    else
-      launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, tw2, ta2, grp, args);
-  }
+  const int early = (KIND == 2 && early_allowed && smem_of_predecessor + r.smem > 228u * 1024u) ? 1 : 0;
+  if (fp8)
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+               I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
+               timeline_slot);
+  else
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+               I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
+               timeline_slot);
 }
 
 }  // namespace
@@ -998,7 +769,7 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   if (!attr_done) {
     if (!set_smem_attr<1, true, false>() || !set_smem_attr<1, false, false>() || !set_smem_attr<2, true, false>() ||
         !set_smem_attr<2, false, false>() || !set_smem_attr<1, true, true>() || !set_smem_attr<1, false, true>() ||
-        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>() || !set_smem_attr<3, false, false>())
+        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>())
       return OLED_ERR_CUDA;
     attr_done = true;
   }
@@ -1011,10 +782,10 @@ static int box_index(int max_count, int cap) {
   return i;
 }
 
-int ffn_tc_token_tile(int max_count, bool fp8) { return 16 << box_index(max_count, fp8 ? 128 : 256); }
-
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
-                  const int32_t* host_counts, const FfnTcIo& io, int H, int I, int n_sms, bool behind_event_wait) {
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
+                  int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait, StepTimeline* timeline,
+                  int timeline_slot) {
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   const bool fp8 = maps.fp8;
@@ -1024,7 +795,6 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   // (fp8 stores stop at N = 128: the widened weights need tensor-memory columns of their own)
   const int ib = box_index(max_count, fp8 ? 128 : 256);
   grp.n_box = 16 << ib;
-  if (kind == 3 && (fp8 || grp.n_box > 32)) return OLED_ERR_INVALID_ARG;  // callers ask ffn_tc_can_fuse() first
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int m_tiles) {
     if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
@@ -1032,57 +802,30 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     for (int g = 0; g < grp.n; ++g) tiles += (host_counts[grp.expert[g]] + grp.n_box - 1) / grp.n_box;
     return (int)std::max<long long>(1, std::min<long long>(n_sms, tiles * m_tiles));
   };
-  FfnArgs args{};
-  args.offsets = io.offsets;
-  args.H = H;
-  args.I = I;
-  args.pool = maps.pool;
-  args.slot_bytes = maps.slot_bytes;
-  args.status = io.status;
-  args.work_counter = io.work_counter;
-  args.x_gather = fp8 ? nullptr : io.x_gather;
-  args.perm = io.perm;
-  args.top_k = io.top_k;
-  args.done = io.done;
   // shared memory of a CTA of this group's KIND 1 launch
   const bool stacked1 = grp.n_box <= 32;
-  const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
   // A KIND 2 launch may start early only if nothing it reads besides the token tiles can still be
   // in the making: either every SM holds a CTA of the KIND 1 launch before it (full grid: a KIND 2
   // CTA then gets an SM only after a KIND 1 CTA, which waited for the permutation, has left it),
   // or the launch pair sits behind an event wait, which completes everything enqueued before it.
-  const bool early_allowed = kind == 2 && (behind_event_wait || (host_counts == nullptr && 
-                                                                 grid_for(1) == n_sms));
-  if (kind == 3) {
-    args.out = io.hbuf;
-    args.out2 = io.y;
-    args.out_bf16 = 0;
-    launch_variant<3, false>(false, grid_for(I / (kBlockM / 2) + H / kBlockM), st, maps.w13_half, maps.xp[ib], maps.w2,
-                             maps.hbuf[ib], grp, args, false, 0u);
-  } else if (kind == 1 && stacked1) {
-    args.out = io.hbuf;
-    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], maps.w2, maps.hbuf[ib], grp,
-                             args, false, 0u);
+  const bool early_allowed = kind == 2 && (behind_event_wait || host_counts == nullptr);
+  const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
+  if (kind == 1 && stacked1) {
+    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
+                             0, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
   } else if (kind == 1) {
-    args.out = io.hbuf;
-    launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], maps.w2, maps.hbuf[ib], grp, args,
-                            false, 0u);
+    launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
+                            maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
   } else {
-    args.out = io.y;
-    args.out_bf16 = io.y_bf16;
-    args.x_gather = nullptr;
-    if (grp.n_box == 256)
-      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], maps.w2, maps.hbuf[ib], grp,
-                              args, early_allowed, smem1);
+    const bool dual = grp.n_box == 256;
+    if (dual)
+      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
+                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
     else
-      launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], maps.w2, maps.hbuf[ib], grp, args,
-                               early_allowed, smem1);
+      launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
+                               maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
-}
-
-bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count) {
-  return !maps.fp8 && ffn_tc_token_tile(max_count, false) <= 32;
 }
 
 }  // namespace oled

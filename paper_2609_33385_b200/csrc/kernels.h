@@ -41,6 +41,33 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// ---- device-side timeline (OLED_OPT_TIMELINE) ------------------------------------------------
+// Per kernel slot of a step: the earliest time a CTA entered the kernel, the earliest time one got
+// past its dependency wait, and the latest time one finished (GPU global timer, nanoseconds).
+constexpr int kTimelineSlots = 12;   // 0 gate, 1 permutation, 2 gather, 3..10 FFN launches, 11 combine
+struct StepTimeline {
+  unsigned long long entry_min[kTimelineSlots];
+  unsigned long long start_min[kTimelineSlots];
+  unsigned long long end_max[kTimelineSlots];
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ unsigned long long timeline_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// called by one thread per CTA; tl == nullptr: tracing off
+__device__ __forceinline__ void timeline_entry(StepTimeline* tl, int slot) {
+  if (tl) atomicMin(&tl->entry_min[slot], timeline_now());
+}
+__device__ __forceinline__ void timeline_start(StepTimeline* tl, int slot) {
+  if (tl) atomicMin(&tl->start_min[slot], timeline_now());
+}
+__device__ __forceinline__ void timeline_end(StepTimeline* tl, int slot) {
+  if (tl) atomicMax(&tl->end_max[slot], timeline_now());
+}
+#endif
+
 // The experts one FFN launch works on and the slot each one's weights sit in: the per-launch
 // image of the expert->slot indirection table, passed by value in kernel-parameter space.
 struct FfnGroup {
@@ -67,31 +94,44 @@ struct GuardList {
   uint32_t* words[12];
 };
 
-// Where the gate kernel's last CTA publishes the step's counts and scores for the host: mapped
+// Where the permutation kernel publishes the step's counts and scores for the host: mapped
 // pinned host memory, one 8-byte word per value with the step's sequence number in the upper
 // bits (scores: seq & 0xffff in bits 48..63; counts: seq in bits 32..63).  All-null = no report.
 struct RouteReport {
-  unsigned int* ticket = nullptr;               // device, zero before the launch
   unsigned long long* host_scores = nullptr;    // mapped host [E]
   unsigned long long* host_counts = nullptr;    // mapped host [E]
   unsigned int seq = 0;
+  StepTimeline* timeline = nullptr;             // device, or null
 };
 
 // ---- route.cu -------------------------------------------------------------------------
 // Gate logits in the contract order, top-k (ties to the lower index), softmax over the selected
 // logits, per-expert counts and integer reuse-score numerators (atomics on zeroed arrays).
-// Small steps (route_fuses_permutation): with offsets/perm/pos non-null and a ticket in rep, the
-// kernel's last CTA also builds the permutation, and launch_permute is not needed.
+// A layer's combine handed to the next layer's gate kernel (few-token steps inside a stack
+// iteration): out = bf16(sum_j gate[t,j] * y[pos[t*K+j],:]) in rank order, x_next = bf16(x + out),
+// and x_next is the gate kernel's input.  y == nullptr: nothing to carry out.
+struct CombinePrev {
+  const float* y = nullptr;        // [T*K,H] fp32 per-assignment outputs of the previous layer
+  const float* gate = nullptr;     // [T,K]   its gate scores
+  const int32_t* pos = nullptr;    // [T*K]   its inverse permutation
+  const uint16_t* x = nullptr;     // [T,H]   its input
+  uint16_t* out = nullptr;         // [T,H]   its MoE output
+  uint16_t* x_next = nullptr;      // [T,H]   its input plus its output
+  int K = 0;
+  uint32_t* zero_words = nullptr;  // the control block the previous step used, cleared by CTA 0
+  int n_zero_words = 0;
+};
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep,
-                  int32_t* offsets, int32_t* perm, int32_t* pos);
-bool route_fuses_permutation(int T, int E, int K);
+                  float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
+                  StepTimeline* timeline);
+bool route_can_take_combine(int T);  // does the gate kernel of a T-token step carry out a CombinePrev?
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
-// kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
-void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
-                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp,
-                    int H);
+// kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.  Also
+// publishes counts and scores to the host (rep; all-null: no report).
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, const unsigned long long* scores,
+                    int T, int E, int K, int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x,
+                    uint16_t* xp, int H, const RouteReport& rep);
 // xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);
@@ -104,7 +144,7 @@ void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int 
 // y_bf16 != 0: y holds bf16 rows (many-token steps) instead of fp32.
 void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* gate, const int32_t* pos, int T,
                     int H, int K, uint16_t* out, const uint16_t* x, uint16_t* x_next,
-                    uint32_t* zero_words, int n_zero_words);
+                    uint32_t* zero_words, int n_zero_words, StepTimeline* timeline = nullptr);
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n);
 
 // ---- ffn_simple.cu (bring-up path, plain FMA) ---------------------------------------------
@@ -126,30 +166,15 @@ struct FfnTcMaps {
 // Builds the tensor maps; returns 0 or a negative oled_status.
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
-// Buffers of an FFN launch.
-struct FfnTcIo {
-  const int32_t* offsets = nullptr;   // [E+1]
-  uint16_t* hbuf = nullptr;           // [rows, I] bf16 intermediate
-  float* y = nullptr;                 // [rows, H] per-assignment outputs (fp32, or bf16 if y_bf16)
-  int y_bf16 = 0;
-  uint32_t* status = nullptr;
-  // a device word that is ZERO when the kernel starts; its CTAs draw their work items from it
-  // (every launch that can be in flight at the same time needs a word of its own)
-  uint32_t* work_counter = nullptr;
-  // bf16 stores, kinds 1 and 3: gather the token rows of the gate/up items from x [T, H] through
-  // perm instead of reading pre-sorted rows (x_gather == nullptr: read the sorted copy)
-  const uint16_t* x_gather = nullptr;
-  const int32_t* perm = nullptr;
-  int top_k = 0;
-  uint32_t* done = nullptr;           // kind 3: one ZERO word per expert of the group
-};
-// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y; kind 3: both in one launch
-// (bf16 stores and token tiles of at most 32 rows only: ask ffn_tc_can_fuse).  One launch each.
+// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
+// work_counter: a device word that is ZERO when the kernel starts; its CTAs draw their work items
+// from it (every launch that can be in flight at the same time needs a word of its own).
 // behind_event_wait: the launch follows a cudaStreamWaitEvent (with, for kind 2, at most its own
 // kind 1 launch in between), i.e. everything enqueued before that wait has completed.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
-                  const int32_t* host_counts, const FfnTcIo& io, int H, int I, int n_sms, bool behind_event_wait);
-bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
+                  const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
+                  int I, int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait,
+                  StepTimeline* timeline, int timeline_slot);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 // Self-check (check.cu): invariants of the routing and the permutation, guard words.

@@ -45,12 +45,35 @@ struct oled_ctx {
   StepPlan plan;
 
   // scratch (device)
-  unsigned long long* d_scores = nullptr;  // [E]   } one block, zeroed per step
+  // The step's control block (scores, counts, work-item counters of its FFN launches), all zero
+  // when a step starts.  There are two, used by alternate steps: the kernel that clears a block -
+  // the step's combine or, when that has been left to it, the next step's gate kernel - runs
+  // after everything that used the block and never while the current step's atomics land in it.
+  uint8_t* d_ctrl[2] = {nullptr, nullptr};
+  int ctrl_sel = 0;
+  unsigned long long* d_scores = nullptr;  // [E]   } the current step's block
   int32_t* d_counts = nullptr;             // [E]   }
   size_t ctrl_bytes = 0;
   float* d_logits = nullptr;   // [T,E]
   int32_t* d_ids = nullptr;    // [T,k]
-  float* d_gate = nullptr;     // [T,k]
+  float* d_gate = nullptr;     // [T,k]  (the current step's of the two buffers below)
+  float* d_gate_buf[2] = {nullptr, nullptr};
+  int32_t* d_pos_buf[2] = {nullptr, nullptr};
+  int buf_sel = 0;
+  // a layer's combine that has been left to the next layer's gate kernel (few-token steps inside
+  // oled_denoise_iteration): what that kernel, or a stand-alone combine, needs to carry it out
+  struct PendingCombine {
+    bool valid = false;
+    int T = 0;
+    const float* gate = nullptr;
+    const int32_t* pos = nullptr;
+    const uint16_t* x = nullptr;
+    uint16_t* out = nullptr;
+    uint16_t* x_next = nullptr;
+    uint32_t* ctrl = nullptr;      // the control block that step used (to be cleared)
+  } pending;
+  bool fuse_combine = true;    // stack iterations of few-token steps: a layer's combine runs inside the
+                               // next layer's gate kernel (OLED_OPT_FUSE_COMBINE)
   int32_t* d_offsets = nullptr;// [E+1]
   int32_t* d_perm = nullptr;   // [T*k]
   int32_t* d_pos = nullptr;    // [T*k]
@@ -58,11 +81,9 @@ struct oled_ctx {
   uint16_t* d_hbuf = nullptr;  // [T*k,I]
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
-  unsigned int* d_ticket = nullptr;   // control block, after the counts
-  uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
-  uint32_t* d_done = nullptr;         // control block, last: [kFfnWorkCounters][E] completion counters of fused FFN launches
+  uint32_t* d_work = nullptr;         // control block, last: work-item counters of the step's FFN launches
   int work_next = 0;                  // next unused counter of the current layer execution
-  bool ctrl_dirty = true;             // control block must be cleared before the next gate launch
+  bool ctrl_dirty = true;             // both control blocks must be cleared before the next gate launch
   unsigned int seq = 0;               // step sequence number echoed by the gate kernel
   volatile unsigned long long* h_report = nullptr;  // pinned, mapped: tagged scores [E] | tagged counts [E]
   std::vector<unsigned long long> host_scores;       // decoded copy of the last report
@@ -83,12 +104,9 @@ struct oled_ctx {
   std::vector<cudaEvent_t> prof_free;
   oled_kernel_profile prof_acc[OLED_N_KERNELS] = {};
   int ffn_impl = 0;
-  bool fuse_ffn = true;        // small steps: gate/up and down projection in one launch where possible
-  bool gather_in_ffn = true;   // small steps, bf16 stores: the FFN kernel gathers the token rows itself
+  bool timeline_on = false;    // OLED_OPT_TIMELINE
+  StepTimeline* d_timeline = nullptr;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
-  bool small_step = false;     // this step's gate kernel also made the permutation
-  const uint16_t* x_gather = nullptr;  // this step's FFN kernels gather token rows from here (else from d_xp)
-  bool hit_fused = false;      // this step's resident-group FFN ran as one fused launch
   int miss_chunk = 4;
   bool split_last = true;      // the step's last blob is copied in two parts (gate|up first, down after)
   int withhold_loads = 0;      // test aid, see OLED_OPT_TEST_WITHHOLD_LOADS
@@ -117,6 +135,15 @@ namespace {
       return OLED_ERR_CUDA;                       \
     }                                             \
   } while (0)
+
+void select_ctrl(oled_ctx* ctx, int sel) {
+  const size_t E = (size_t)ctx->shape.n_experts;
+  uint8_t* b = ctx->d_ctrl[sel];
+  ctx->ctrl_sel = sel;
+  ctx->d_scores = reinterpret_cast<unsigned long long*>(b);
+  ctx->d_counts = reinterpret_cast<int32_t*>(b + E * sizeof(unsigned long long));
+  ctx->d_work = reinterpret_cast<uint32_t*>(b + E * (sizeof(unsigned long long) + sizeof(int32_t)));
+}
 
 template <typename T>
 int dev_alloc(oled_ctx* ctx, T** p, size_t n) {
@@ -154,7 +181,23 @@ int check_status(oled_ctx* ctx) {
   return OLED_OK;
 }
 
+// Carries out a combine that was left to the next layer's gate kernel and never got one.
+int flush_pending_combine(oled_ctx* ctx) {
+  if (!ctx->pending.valid) return OLED_OK;
+  const auto& p = ctx->pending;
+  launch_combine(ctx->stream, ctx->d_y, 0, p.gate, p.pos, p.T, ctx->shape.hidden, ctx->shape.top_k, p.out, p.x, p.x_next,
+                 p.ctrl, (int)(ctx->ctrl_bytes / 4));
+  ctx->pending.valid = false;
+  ctx->launches += 1;
+  OLED_CUDA(ctx, cudaGetLastError());
+  return OLED_OK;
+}
+
 int sync_all(oled_ctx* ctx) {
+  {
+    const int rcp = flush_pending_combine(ctx);
+    if (rcp != OLED_OK) return rcp;
+  }
   OLED_CUDA(ctx, cudaStreamSynchronize(ctx->copy_stream));
   OLED_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, kStatusWords * sizeof(uint32_t), cudaMemcpyDeviceToHost,
                                  ctx->stream));
@@ -170,17 +213,20 @@ void free_ctx(oled_ctx* ctx) {
     cudaFree(l.bias);
   }
   cudaFree(ctx->pool);
-  cudaFree(ctx->d_scores);
+  cudaFree(ctx->d_ctrl[0]);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_ids);
-  cudaFree(ctx->d_gate);
+  cudaFree(ctx->d_gate_buf[0]);
+  cudaFree(ctx->d_gate_buf[1]);
   cudaFree(ctx->d_offsets);
   cudaFree(ctx->d_perm);
-  cudaFree(ctx->d_pos);
+  cudaFree(ctx->d_pos_buf[0]);
+  cudaFree(ctx->d_pos_buf[1]);
   cudaFree(ctx->d_xp);
   cudaFree(ctx->d_hbuf);
   cudaFree(ctx->d_y);
   cudaFree(ctx->d_status);
+  cudaFree(ctx->d_timeline);
   cudaFree(ctx->d_hidden_stage);
   cudaFree(ctx->d_conf_stage);
   cudaFree(ctx->d_out_stage);
@@ -257,69 +303,45 @@ void prof_add(oled_ctx* ctx, int kernel, uint64_t bytes, uint64_t flops) {
 
 // Algorithmic bytes / flops of the two FFN kernels for n experts with `rows` token rows in total:
 // each expert's weights once, the token rows in, the result rows out.
-void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows, bool fused) {
+void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
   const uint64_t H = ctx->shape.hidden, I = ctx->shape.intermediate, hi = H * I;
   const bool fp8 = ctx->shape.expert_format == OLED_EXPERTS_FP8;
   // weight bytes of one expert per kernel: bf16 elements, or e4m3 codes plus the fp32 row scales
   const uint64_t w13 = fp8 ? 2 * hi + 2 * I * 4 : 2 * hi * 2, w2 = fp8 ? hi + H * 4 : hi * 2;
-  const uint64_t b1 = n * w13 + rows * H * 2 + rows * I * 2, b2 = n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4);
-  if (fused) {
-    prof_add(ctx, OLED_KERNEL_FFN_FUSED, b1 + b2, 6 * rows * hi);
-  } else {
-    prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, b1, 4 * rows * hi);
-    prof_add(ctx, OLED_KERNEL_FFN_DOWN, b2, 2 * rows * hi);
-  }
+  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * w13 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
+  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4), 2 * rows * hi);
 }
 
-// The FFN launches over one group: one fused launch where the form exists (bf16 stores, token
-// tiles of at most 32 rows, nothing to wait for between the two projections), else gate/up and
-// down.  host_counts == nullptr: the per-expert counts are not known on the host yet (the group is
-// the resident set and experts without tokens cost nothing).
+// The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
+// known on the host yet (the group is the resident set and experts without tokens cost nothing).
 // before_down: an event the down projection (and nothing before it) has to wait for, or null.
 // behind_event_wait: the caller has just enqueued a cudaStreamWaitEvent on the stream.
-// Returns the number of launches through *fused (1 = one fused launch).
 int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts,
-                     cudaEvent_t before_down, bool behind_event_wait, bool* fused_out) {
-  if (fused_out) *fused_out = false;
+                     cudaEvent_t before_down, bool behind_event_wait) {
   if (grp.n <= 0) return OLED_OK;
   const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
   if (ctx->ffn_impl == 1) {
     if (before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
                       ctx->d_y, H, I);
-    ctx->launches += 2;
   } else {
-    const bool fuse = ctx->small_step && ctx->fuse_ffn && before_down == nullptr && ffn_tc_can_fuse(ctx->maps, max_count);
-    for (int kind = fuse ? 3 : 1; kind <= (fuse ? 3 : 2); ++kind) {
+    for (int kind = 1; kind <= 2; ++kind) {
       if (kind == 2 && before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
-      ProfScope ps(ctx, kind == 3 ? OLED_KERNEL_FFN_FUSED : kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
-      // a fresh (zero) work counter and, for a fused launch, a fresh row of completion counters
-      // per launch; a layer execution has at most three launch pairs, should there ever be more,
-      // used words are cleared in stream order and taken again
+      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
+      // a fresh (zero) work counter per launch; a layer execution has at most three launch pairs,
+      // should there ever be more, a used word is cleared in stream order and taken again
       const int li = ctx->work_next % kFfnWorkCounters;
-      FfnTcIo io;
-      io.work_counter = ctx->d_work + li;
-      io.done = ctx->d_done + (size_t)li * ctx->shape.n_experts;
-      if (ctx->work_next >= kFfnWorkCounters) {
-        OLED_CUDA(ctx, cudaMemsetAsync(io.work_counter, 0, sizeof(uint32_t), ctx->stream));
-        OLED_CUDA(ctx, cudaMemsetAsync(io.done, 0, (size_t)ctx->shape.n_experts * sizeof(uint32_t), ctx->stream));
-      }
+      uint32_t* work = ctx->d_work + li;
+      if (ctx->work_next >= kFfnWorkCounters) OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
       ctx->work_next += 1;
-      io.offsets = ctx->d_offsets;
-      io.hbuf = ctx->d_hbuf;
-      io.y = ctx->d_y;
-      io.y_bf16 = ctx->y_bf16 ? 1 : 0;
-      io.status = ctx->d_status;
-      io.x_gather = ctx->x_gather;
-      io.perm = ctx->d_perm;
-      io.top_k = ctx->shape.top_k;
-      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, io, H, I, ctx->n_sms,
-                                   behind_event_wait || (kind == 2 && before_down != nullptr));
+      const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
+                                   ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work,
+                                   behind_event_wait || (kind == 2 && before_down != nullptr),
+                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li);
       if (rc != OLED_OK) return rc;
-      ctx->launches += 1;
     }
-    if (fused_out) *fused_out = fuse;
   }
+  ctx->launches += 2;
   OLED_CUDA(ctx, cudaGetLastError());
   return OLED_OK;
 }
@@ -342,10 +364,8 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
     max_count = std::max(max_count, counts[e]);
     rows += (uint64_t)counts[e];
   }
-  bool fused = false;
-  const int rc = run_ffn_launches(ctx, grp, max_count, counts, before_down, behind_event_wait, &fused);
-  prof_add_ffn(ctx, (uint64_t)grp.n, rows, fused);
-  return rc;
+  prof_add_ffn(ctx, (uint64_t)grp.n, rows);
+  return run_ffn_launches(ctx, grp, max_count, counts, before_down, behind_event_wait);
 }
 
 // Blocks until the gate kernel of step `seq` has published counts and scores, and decodes them.
@@ -410,7 +430,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   if (!shape || !cache_capacity || !out_ctx) return OLED_ERR_INVALID_ARG;
   *out_ctx = nullptr;
   const oled_model_shape& s = *shape;
-  if (s.n_layers <= 0 || s.hidden <= 0 || s.hidden % 256 != 0 || s.intermediate <= 0 ||
+  if (s.n_layers <= 0 || s.hidden <= 0 || s.hidden % 256 != 0 || s.hidden > 16384 || s.intermediate <= 0 ||
       s.intermediate % 128 != 0 || s.n_experts <= 0 || s.n_experts > OLED_MAX_EXPERTS || s.top_k <= 0 ||
       s.top_k > OLED_MAX_TOPK || s.top_k > s.n_experts || s.max_tokens <= 0 || s.max_tokens > 65535 ||
       s.staging_slots < 0 || (s.expert_format != OLED_EXPERTS_BF16 && s.expert_format != OLED_EXPERTS_FP8))
@@ -463,26 +483,27 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
-  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + (2 + kFfnWorkCounters) * sizeof(uint32_t) +
-                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t);
-  uint8_t* ctrl = nullptr;
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + kFfnWorkCounters * sizeof(uint32_t);
+  ctx->ctrl_bytes = (ctx->ctrl_bytes + 15) / 16 * 16;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc(ctx, &ctrl, ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
-  ctx->d_scores = reinterpret_cast<unsigned long long*>(ctrl);
-  ctx->d_counts = reinterpret_cast<int32_t*>(ctrl + E * sizeof(unsigned long long));
-  ctx->d_ticket = reinterpret_cast<unsigned int*>(ctrl + E * (sizeof(unsigned long long) + sizeof(int32_t)));
-  ctx->d_work = reinterpret_cast<uint32_t*>(ctx->d_ticket) + 2;
-  ctx->d_done = ctx->d_work + kFfnWorkCounters;
+  if ((rc = dev_alloc(ctx, &ctx->d_ctrl[0], 2 * ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
+  ctx->d_ctrl[1] = ctx->d_ctrl[0] + ctx->ctrl_bytes;
+  select_ctrl(ctx, 0);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_logits, T * E)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_ids, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc_guarded(ctx, &ctx->d_gate, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_gate_buf[0], T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_gate_buf[1], T * K)) != OLED_OK) return fail(rc);
+  ctx->d_gate = ctx->d_gate_buf[0];
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_offsets, E + 1)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_perm, T * K)) != OLED_OK) return fail(rc);
-  if ((rc = dev_alloc_guarded(ctx, &ctx->d_pos, T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_pos_buf[0], T * K)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc_guarded(ctx, &ctx->d_pos_buf[1], T * K)) != OLED_OK) return fail(rc);
+  ctx->d_pos = ctx->d_pos_buf[0];
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_xp, T * K * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_hbuf, T * K * I)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_y, T * K * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_status, kStatusWords)) != OLED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_timeline, (size_t)s.n_layers)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_hidden_stage, T * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_conf_stage, T)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_out_stage, T * H)) != OLED_OK) return fail(rc);
@@ -558,8 +579,10 @@ int oled_register_experts(oled_ctx* ctx, int32_t layer, const void* host_blob, s
 }
 
 // x_next != nullptr: also write x_next = bf16(hidden + out), the residual between layers.
+// defer_combine: the caller promises that the next step on this context takes x_next as its
+// input with the same n_tokens; the combine may then be left to that step's gate kernel.
 static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const float* confidences,
-                     int32_t n_tokens, void* out, void* x_next) {
+                     int32_t n_tokens, void* out, void* x_next, bool defer_combine = false) {
   if (!ctx || layer < 0 || layer >= ctx->shape.n_layers || n_tokens < 0) return OLED_ERR_INVALID_ARG;
   if (n_tokens > ctx->shape.max_tokens) return OLED_ERR_TOO_MANY_TOKENS;
   LayerData& L = ctx->layers[layer];
@@ -589,44 +612,66 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   // per-assignment outputs y: fp32 for small steps; bf16 once y's traffic matters (the rounding
   // adds at most 2^-9 relative per term, far inside the output tolerance)
   ctx->y_bf16 = ctx->ffn_impl == 0 && (size_t)T * K > 4096;
-  // 1. gate, counts and reuse-score numerators; the kernel's last CTA reports them to the host
-  // and, in a small step, also builds the permutation
-  if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_scores, 0, ctx->ctrl_bytes, st));
+  // 1. gate, counts and reuse-score numerators, permutation; the permutation kernel reports
+  // counts and scores to the host.  This step takes the control block the last step did not use.
+  if (ctx->ctrl_dirty) OLED_CUDA(ctx, cudaMemsetAsync(ctx->d_ctrl[0], 0, 2 * ctx->ctrl_bytes, st));
   ctx->ctrl_dirty = true;
+  select_ctrl(ctx, ctx->ctrl_sel ^ 1);
   ctx->work_next = 0;
   ctx->seq += 1;
   RouteReport rep;
-  rep.ticket = ctx->d_ticket;
   rep.host_scores = reinterpret_cast<unsigned long long*>(ctx->h_ctrl);
   rep.host_counts = reinterpret_cast<unsigned long long*>(ctx->h_ctrl) + E;
   rep.seq = ctx->seq;
-  ctx->small_step = T <= 1024 && route_fuses_permutation(T, E, K);
-  const bool small = ctx->small_step;
+  StepTimeline* const tl = ctx->timeline_on ? ctx->d_timeline + layer : nullptr;
+  rep.timeline = tl;
+  if (tl) {  // earliest times start at the maximum, latest at zero
+    OLED_CUDA(ctx, cudaMemsetAsync(tl, 0xff, 2 * kTimelineSlots * sizeof(unsigned long long), st));
+    OLED_CUDA(ctx, cudaMemsetAsync(tl->end_max, 0, kTimelineSlots * sizeof(unsigned long long), st));
+  }
+  // the current step's gate-score and inverse-permutation buffers (the previous step's stay
+  // intact for a combine that has been left to this step's gate kernel)
+  ctx->buf_sel ^= 1;
+  ctx->d_gate = ctx->d_gate_buf[ctx->buf_sel];
+  ctx->d_pos = ctx->d_pos_buf[ctx->buf_sel];
+  const bool fuse_prev = ctx->pending.valid && ctx->pending.T == T && route_can_take_combine(T) &&
+                         ctx->pending.x_next == static_cast<const uint16_t*>(hidden);
+  if (ctx->pending.valid && !fuse_prev) {
+    const int rcp = flush_pending_combine(ctx);
+    if (rcp != OLED_OK) return rcp;
+  }
   {
-    ProfScope ps(ctx, OLED_KERNEL_ROUTE, ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * (small ? 20 : 8),
-                 2ull * T * H * E);
+    ProfScope ps(ctx, OLED_KERNEL_ROUTE,
+                 ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * 8 +
+                     (fuse_prev ? (uint64_t)T * K * H * 4 + (uint64_t)T * H * 6 : 0),
+                 2ull * T * H * E + (fuse_prev ? 2ull * T * K * H : 0));
+    CombinePrev prev;
+    if (fuse_prev) {
+      prev.y = ctx->d_y;
+      prev.gate = ctx->pending.gate;
+      prev.pos = ctx->pending.pos;
+      prev.x = ctx->pending.x;
+      prev.out = ctx->pending.out;
+      prev.x_next = ctx->pending.x_next;
+      prev.K = K;
+      prev.zero_words = ctx->pending.ctrl;
+      prev.n_zero_words = (int)(ctx->ctrl_bytes / 4);
+      ctx->pending.valid = false;
+    }
     launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
-                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, rep,
-                 small ? ctx->d_offsets : nullptr, small ? ctx->d_perm : nullptr, small ? ctx->d_pos : nullptr);
+                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, prev, tl);
   }
-  ctx->launches += 1;
-  // token rows in sorted order (xp): a small step on bf16 stores needs none - its FFN kernels
-  // gather the rows themselves; otherwise the permutation kernel copies them (few rows per
-  // expert: one CTA per expert) or a gather kernel does
-  ctx->x_gather = (small && ctx->gather_in_ffn && ctx->ffn_impl == 0 && ctx->shape.expert_format == OLED_EXPERTS_BF16)
-                      ? static_cast<const uint16_t*>(hidden) : nullptr;
-  const bool fuse_gather = !small && (size_t)T * K <= 4096;
-  if (!small) {
+  const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
+  {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
-    launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
-                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H);
-    ctx->launches += 1;
+    launch_permute(st, ctx->d_ids, ctx->d_counts, ctx->d_scores, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
+                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, rep);
   }
-  if (!fuse_gather && ctx->x_gather == nullptr) {
+  if (!fuse_gather) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
-    ctx->launches += 1;
   }
+  ctx->launches += fuse_gather ? 2 : 3;
   if (ctx->corrupt_perm) {
     launch_corrupt_perm(st, ctx->d_perm, T * K);
     ctx->launches += 1;
@@ -654,9 +699,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
       }
     // token tile of this launch: twice the mean load per expert (a fuller expert takes more tiles)
     const int mean_load = (int)(((size_t)T * K + E - 1) / E);
-    ctx->hit_fused = false;
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false,
-                                     &ctx->hit_fused);
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false);
     if (rc0 != OLED_OK) return rc0;
   }
 
@@ -732,7 +775,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   {
     uint64_t hit_rows = 0;
     for (int32_t e : plan.hits) hit_rows += (uint64_t)counts[e];
-    prof_add_ffn(ctx, plan.hits.size(), hit_rows, ctx->hit_fused);
+    prof_add_ffn(ctx, plan.hits.size(), hit_rows);
   }
   int rc = OLED_OK;
   for (size_t c = 0; c < n_groups; ++c) {
@@ -742,21 +785,35 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     if (rc != OLED_OK) return rc;
   }
 
-  // 5. combine
-  {
-    ProfScope ps(ctx, OLED_KERNEL_COMBINE, (uint64_t)T * K * H * (ctx->y_bf16 ? 2 : 4) + (uint64_t)T * H * 2,
-                 2ull * T * K * H);
-    launch_combine(st, ctx->d_y, ctx->y_bf16 ? 1 : 0, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out),
-                   static_cast<const uint16_t*>(hidden), static_cast<uint16_t*>(x_next),
-                   reinterpret_cast<uint32_t*>(ctx->d_scores), (int)(ctx->ctrl_bytes / 4));
-  }
-  ctx->launches += 1;
-  if (ctx->self_check) {
-    launch_guard_check(st, ctx->guards, ctx->d_status);
+  // 5. combine - or, inside a stack iteration of few-token steps, left to the next layer's gate kernel
+  const bool defer = defer_combine && ctx->fuse_combine && route_can_take_combine(T) && x_next != nullptr &&
+                     !ctx->y_bf16 && !ctx->self_check && ctx->ffn_impl == 0;
+  if (defer) {
+    ctx->pending.valid = true;
+    ctx->pending.T = T;
+    ctx->pending.gate = ctx->d_gate;
+    ctx->pending.pos = ctx->d_pos;
+    ctx->pending.x = static_cast<const uint16_t*>(hidden);
+    ctx->pending.out = static_cast<uint16_t*>(out);
+    ctx->pending.x_next = static_cast<uint16_t*>(x_next);
+    ctx->pending.ctrl = reinterpret_cast<uint32_t*>(ctx->d_ctrl[ctx->ctrl_sel]);
+    ctx->ctrl_dirty = false;  // the gate kernel that carries the combine out clears this step's block
+  } else {
+    {
+      ProfScope ps(ctx, OLED_KERNEL_COMBINE, (uint64_t)T * K * H * (ctx->y_bf16 ? 2 : 4) + (uint64_t)T * H * 2,
+                   2ull * T * K * H);
+      launch_combine(st, ctx->d_y, ctx->y_bf16 ? 1 : 0, ctx->d_gate, ctx->d_pos, T, H, K, static_cast<uint16_t*>(out),
+                     static_cast<const uint16_t*>(hidden), static_cast<uint16_t*>(x_next),
+                     reinterpret_cast<uint32_t*>(ctx->d_scores), (int)(ctx->ctrl_bytes / 4), tl);
+    }
     ctx->launches += 1;
+    if (ctx->self_check) {
+      launch_guard_check(st, ctx->guards, ctx->d_status);
+      ctx->launches += 1;
+    }
+    OLED_CUDA(ctx, cudaGetLastError());
+    ctx->ctrl_dirty = false;  // combine's CTA 0 cleared this step's control block
   }
-  OLED_CUDA(ctx, cudaGetLastError());
-  ctx->ctrl_dirty = false;  // combine's CTA 0 cleared the control block for the next step
 
   finish_step(L.cache, ctx->slots, plan);
   L.stats.steps += 1;
@@ -811,7 +868,7 @@ int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confi
   const void* x = hidden;
   for (int l = 0; l < ctx->shape.n_layers; ++l) {
     void* nxt = (l + 1 == ctx->shape.n_layers) ? hidden_out : (void*)ctx->d_iter[l & 1];
-    const int rc = step_impl(ctx, l, x, confidences, n_tokens, ctx->d_out_stage, nxt);
+    const int rc = step_impl(ctx, l, x, confidences, n_tokens, ctx->d_out_stage, nxt, l + 1 < ctx->shape.n_layers);
     if (rc != OLED_OK) return rc;
     x = nxt;
   }
@@ -919,6 +976,14 @@ int oled_debug_perm(oled_ctx* ctx, int32_t layer, int32_t* offsets, int32_t* pos
   return rc;
 }
 
+int oled_debug_timeline(oled_ctx* ctx, int32_t layer, uint64_t* times) {
+  if (!ctx || !times || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
+  const int rc = sync_all(ctx);
+  if (rc != OLED_OK && rc != OLED_ERR_TIMEOUT) return rc;
+  OLED_CUDA(ctx, cudaMemcpy(times, ctx->d_timeline + layer, sizeof(StepTimeline), cudaMemcpyDeviceToHost));
+  return rc;
+}
+
 int oled_debug_logits(oled_ctx* ctx, int32_t layer, float* logits) {
   if (!ctx || !logits || layer < 0 || layer >= ctx->shape.n_layers) return OLED_ERR_INVALID_ARG;
   if (ctx->last_layer != layer) return OLED_ERR_STALE_DEBUG;
@@ -986,14 +1051,14 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
     case OLED_OPT_SPLIT_LAST_FILL:
       ctx->split_last = value != 0;
       return OLED_OK;
-    case OLED_OPT_FUSE_FFN:
-      ctx->fuse_ffn = value != 0;
-      return OLED_OK;
-    case OLED_OPT_GATHER_IN_FFN:
-      ctx->gather_in_ffn = value != 0;
+    case OLED_OPT_FUSE_COMBINE:
+      ctx->fuse_combine = value != 0;
       return OLED_OK;
     case OLED_OPT_PDL:
       pdl_set_allowed(value != 0);
+      return OLED_OK;
+    case OLED_OPT_TIMELINE:
+      ctx->timeline_on = value != 0;
       return OLED_OK;
     default:
       return OLED_ERR_INVALID_ARG;

@@ -11,39 +11,18 @@
 //   * gate scores: z_j = exp_spec(L_j - L_0); S = ((z_0+z_1)+z_2)...; g_j = z_j / S.
 //   * score numerators: v = g * psi(c) rounded once; floor(v * 2^32) summed as integers.
 // The router stays off the tensor cores on purpose: their accumulation order is unspecified.
+#include <cuda_bf16.h>
+
 #include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <mutex>
 
 #include "kernels.h"
+#include "route_math.h"
 
 namespace oled {
 namespace {
-
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-// exp(x) for x <= 0 from individually rounded fp32 operations (no contraction, no fast math).
-__device__ __forceinline__ float exp_spec(float x) {
-  if (x < -80.0f) return 0.0f;
-  const float kLog2e = __uint_as_float(0x3fb8aa3bu);  // fl32(1/ln 2)
-  const float kLn2Hi = __uint_as_float(0x3f317000u);  // fl32(ln 2), low 12 significand bits cleared
-  const float kLn2Lo = __uint_as_float(0x3805fdf4u);  // fl32(ln 2 - kLn2Hi)
-  const float n = rintf(__fmul_rn(x, kLog2e));
-  const float r = __fsub_rn(__fsub_rn(x, __fmul_rn(n, kLn2Hi)), __fmul_rn(n, kLn2Lo));
-  float p = __uint_as_float(0x39500d01u);                        // 1/5040
-  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3ab60b61u));  // 1/720
-  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3c088889u));  // 1/120
-  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3d2aaaabu));  // 1/24
-  p = __fadd_rn(__fmul_rn(p, r), __uint_as_float(0x3e2aaaabu));  // 1/6
-  p = __fadd_rn(__fmul_rn(p, r), 0.5f);
-  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
-  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
-  const float scale = __int_as_float(((int)n + 127) << 23);  // 2^n, n >= -116
-  return __fmul_rn(p, scale);
-}
-
 
 // Top-k (ties to the lower index), gate scores over the selected logits, counts and integer
 // reuse-score numerators of one token; executed by one warp.  row: the token's E logits.
@@ -119,48 +98,87 @@ __device__ __forceinline__ void route_token_tail(const float* row, int t, int la
   else route_token_tail_n<OLED_MAX_EXPERTS / 32>(row, t, lane, E, K, conf, ids, gate, counts, scores);
 }
 
-// The last CTA to finish publishes counts and scores to the host (mapped pinned memory).
-// Every 8-byte word carries the step's sequence tag in its upper bits, so the host can tell
-// word by word that the data is there: no ordering fence, no copy operation, no event.
-__device__ __forceinline__ void route_publish(const RouteReport& rep, const int32_t* counts,
-                                              const unsigned long long* scores, int E, int* s_last) {
-  if (rep.host_scores == nullptr) return;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    *s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+// The previous layer's gate-weighted combine and residual, done by the gate kernel of the next
+// layer for its own token (paper Sec. 2.1: the MoE output is the gate-score-weighted sum over the
+// top-k experts; the stack adds it to the layer's input).  Arithmetic and order are those of
+// combine_kernel: fp32 fused multiply-adds in rank order, out = bf16(sum), x = bf16(x_prev + out).
+__device__ __forceinline__ void combine_row(const CombinePrev& p, int t, int H, uint16_t* s_x, float* s_g, int* s_r) {
+  const int K = p.K;
+  if (threadIdx.x < K) {
+    s_g[threadIdx.x] = p.gate[(size_t)t * K + threadIdx.x];
+    s_r[threadIdx.x] = p.pos[(size_t)t * K + threadIdx.x];
   }
   __syncthreads();
-  if (!*s_last) return;
-  __threadfence();
-  const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
-  const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
-    rep.host_scores[e] = tag16 | (__ldcg(&scores[e]) & 0xffffffffffffull);
-    rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
+  for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint2 xv = *reinterpret_cast<const uint2*>(p.x + (size_t)t * H + h);
+    for (int j0 = 0; j0 < K; j0 += 8) {  // the rows of eight assignments are loaded together
+      float4 v[8];
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj)
+        if (j0 + jj < K) v[jj] = *reinterpret_cast<const float4*>(p.y + (size_t)s_r[j0 + jj] * H + h);
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj)
+        if (j0 + jj < K) {
+          const float g = s_g[j0 + jj];
+          acc.x = fmaf(g, v[jj].x, acc.x);
+          acc.y = fmaf(g, v[jj].y, acc.y);
+          acc.z = fmaf(g, v[jj].z, acc.z);
+          acc.w = fmaf(g, v[jj].w, acc.w);
+        }
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p.out + (size_t)t * H + h) = pk;
+    const float2 o0 = __bfloat1622float2(lo), o1 = __bfloat1622float2(hi);
+    __nv_bfloat162 r0 = __floats2bfloat162_rn(__uint_as_float(xv.x << 16) + o0.x,
+                                              __uint_as_float(xv.x & 0xffff0000u) + o0.y);
+    __nv_bfloat162 r1 = __floats2bfloat162_rn(__uint_as_float(xv.y << 16) + o1.x,
+                                              __uint_as_float(xv.y & 0xffff0000u) + o1.y);
+    uint2 rk;
+    rk.x = *reinterpret_cast<uint32_t*>(&r0);
+    rk.y = *reinterpret_cast<uint32_t*>(&r1);
+    *reinterpret_cast<uint2*>(p.x_next + (size_t)t * H + h) = rk;
+    *reinterpret_cast<uint2*>(s_x + h) = rk;
   }
 }
 
 // TT tokens per CTA, WARPS warps; each warp owns kEPerWarp experts per pass and all TT tokens.  Small
 // blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
 // chunks of loads in flight; the chain order of every logit is the same in all variants.
+// TT = 1 only: the token's row is staged in shared memory - copied from x, or produced by the
+// previous layer's combine (prev.y != nullptr), which this kernel then carries out for its token -
+// and the top-k is a rank computation spread over all warps: expert e is selected iff fewer than K
+// experts precede it in the order (logit descending, index ascending), and its rank is the number
+// that do - the same total order a round-by-round selection walks.
+// The kernel reports nothing to the host: the permutation kernel, which follows it in every step,
+// publishes the finished counts and scores without any ticket or fence.
 template <int TT, int WARPS, int UNROLL, int kEPerWarp>
 __global__ void __launch_bounds__(WARPS * 32)
 route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
              const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
              int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
              float* __restrict__ gate, int32_t* __restrict__ counts,
-             unsigned long long* __restrict__ scores, RouteReport rep) {
-  extern __shared__ float s_logits[];  // [TT][E]
-  __shared__ int s_last;
+             unsigned long long* __restrict__ scores, CombinePrev prev, StepTimeline* timeline) {
+  extern __shared__ __align__(16) uint8_t s_dyn[];
+  float* s_logits = reinterpret_cast<float*>(s_dyn);                       // [TT][E]
+  // [H] (TT == 1 only), on a 16-byte boundary: the row is moved with 16-byte vector accesses
+  uint16_t* s_x = reinterpret_cast<uint16_t*>(s_dyn + (((size_t)TT * E * 4 + 15) & ~(size_t)15));
+  __shared__ int s_sel_id[OLED_MAX_TOPK];
+  __shared__ float s_sel_logit[OLED_MAX_TOPK];
+  __shared__ float s_g[OLED_MAX_TOPK];
+  __shared__ int s_r[OLED_MAX_TOPK];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
   griddep_launch_dependents();
+  if (threadIdx.x == 0) timeline_entry(timeline, 0);
   constexpr int kRouteWarps = WARPS;
   if (TT == 1 && gridDim.x <= 128) {
     // Small steps: the router weights do not depend on the predecessor (the previous layer's
-    // combine), but the expert weights streamed since their last use have pushed them out of
+    // expert FFN), but the expert weights streamed since their last use have pushed them out of
     // L2 - so they are called back in while this kernel still waits for its input.
     for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp)
 #pragma unroll
@@ -171,6 +189,19 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
       }
   }
   griddep_wait();
+  if (threadIdx.x == 0) timeline_start(timeline, 0);
+  if (TT == 1) {
+    if (prev.y != nullptr) {
+      // CTA 0 also clears the control block the previous step used (its kernels have completed)
+      if (blockIdx.x == 0 && prev.zero_words != nullptr)
+        for (int i = threadIdx.x; i < prev.n_zero_words; i += blockDim.x) prev.zero_words[i] = 0u;
+      combine_row(prev, t0, H, s_x, s_g, s_r);
+    } else {
+      for (int c = threadIdx.x; c < H / 8; c += blockDim.x)
+        reinterpret_cast<uint4*>(s_x)[c] = reinterpret_cast<const uint4*>(x + (size_t)t0 * H)[c];
+    }
+    __syncthreads();
+  }
 
   for (int eb = warp * kEPerWarp; eb < E; eb += kRouteWarps * kEPerWarp) {
     float acc[TT][kEPerWarp];
@@ -186,7 +217,8 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 #pragma unroll
       for (int a = 0; a < TT; ++a) {
         const int t = min(t0 + a, T - 1);
-        const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+        const uint4 v = TT == 1 ? *reinterpret_cast<const uint4*>(s_x + h)
+                                : *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
         xw[a][0] = v.x; xw[a][1] = v.y; xw[a][2] = v.z; xw[a][3] = v.w;
       }
 #pragma unroll
@@ -234,131 +266,15 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   }
   __syncthreads();
 
-  // top-k, gate scores, counts and reuse-score numerators: one warp per token
-  for (int a = warp; a < TT; a += kRouteWarps) {
-    const int t = t0 + a;
-    if (t >= T) continue;
-    route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores);
-  }
-
-  route_publish(rep, counts, scores, E, &s_last);
-}
-
-// ---- small steps: one kernel for gate, top-k, gate scores, counts, scores AND the permutation --
-// One CTA per token.  The logits are computed as in route_kernel (same chains, same butterfly).
-// The top-k is a rank computation spread over all warps: expert e is selected iff fewer than K
-// experts precede it in the order (logit descending, index ascending), and its rank is the number
-// that do - the same total order the round-by-round selection walks, so the ids and their order
-// are identical.  The last CTA to finish (a ticket) publishes counts and scores to the host and,
-// if asked to, builds offsets, the stable permutation and its inverse: with at most
-// kSmallMaxAssign assignments one CTA does that in a few microseconds, which removes a kernel
-// boundary from the latency chain of a few-token step.
-constexpr int kSmallMaxAssign = 2048;
-constexpr int kSmallMaxExperts = 128;
-
-__device__ __forceinline__ uint32_t order_key(float v) {  // v is not NaN and not -0
-  const uint32_t bits = __float_as_uint(v);
-  return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-}
-
-template <int WARPS, int UNROLL, int kEPerWarp>
-__global__ void __launch_bounds__(WARPS * 32)
-route_small_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
-                   const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
-                   int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
-                   float* __restrict__ gate, int32_t* __restrict__ counts,
-                   unsigned long long* __restrict__ scores, int32_t* __restrict__ offsets,
-                   int32_t* __restrict__ perm, int32_t* __restrict__ pos, int do_perm, RouteReport rep) {
-  __shared__ float s_logits[OLED_MAX_EXPERTS];
-  __shared__ int s_sel_id[OLED_MAX_TOPK];
-  __shared__ float s_sel_logit[OLED_MAX_TOPK];
-  __shared__ int s_last;
-  __shared__ int s_off[kSmallMaxExperts + 1];
-  __shared__ int s_ids[kSmallMaxAssign];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x;
-  griddep_launch_dependents();
-  if (gridDim.x <= 128) {
-    // The router weights do not depend on the predecessor (the previous layer's combine), but the
-    // expert weights streamed since their last use have pushed them out of L2 - so they are
-    // called back in while this kernel still waits for its input.
-    for (int eb = warp * kEPerWarp; eb < E; eb += WARPS * kEPerWarp)
-#pragma unroll
-      for (int b = 0; b < kEPerWarp; ++b) {
-        const int e = min(eb + b, E - 1);
-        for (int off = lane * 64; off < H; off += 32 * 64)  // 128-byte lines of the row
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(wr + (size_t)e * H + off));
-      }
-  }
-  griddep_wait();
-
-  for (int eb = warp * kEPerWarp; eb < E; eb += WARPS * kEPerWarp) {
-    float acc[kEPerWarp];
-#pragma unroll
-    for (int b = 0; b < kEPerWarp; ++b) acc[b] = 0.0f;
-#pragma unroll UNROLL
-    for (int hc = 0; hc < H; hc += 256) {
-      const int h = hc + lane * 8;
-      uint32_t xw[4], ww[kEPerWarp][4];
-      {
-        const uint4 v = *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
-        xw[0] = v.x; xw[1] = v.y; xw[2] = v.z; xw[3] = v.w;
-      }
-#pragma unroll
-      for (int b = 0; b < kEPerWarp; ++b) {
-        const int e = min(eb + b, E - 1);
-        const uint4 v = *reinterpret_cast<const uint4*>(wr + (size_t)e * H + h);
-        ww[b][0] = v.x; ww[b][1] = v.y; ww[b][2] = v.z; ww[b][3] = v.w;
-      }
-      // elements in ascending h: word 0 low half, word 0 high half, word 1 low half, ...
-#pragma unroll
-      for (int wi = 0; wi < 4; ++wi) {
-        const float xl = bf16_lo(xw[wi]), xh = bf16_hi(xw[wi]);
-#pragma unroll
-        for (int b = 0; b < kEPerWarp; ++b) acc[b] = __fmaf_rn(xl, bf16_lo(ww[b][wi]), acc[b]);
-#pragma unroll
-        for (int b = 0; b < kEPerWarp; ++b) acc[b] = __fmaf_rn(xh, bf16_hi(ww[b][wi]), acc[b]);
-      }
-    }
-#pragma unroll
-    for (int b = 0; b < kEPerWarp; ++b) {
-      float v = acc[b];
-#pragma unroll
-      for (int d = 16; d >= 1; d >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, d));
-      const int e = eb + b;
-      if (lane == 0 && e < E) {
-        if (bias != nullptr) v = __fadd_rn(v, bias[e]);
-        s_logits[e] = v;
-        if (logits_out != nullptr) logits_out[(size_t)t * E + e] = v;
-      }
-    }
-  }
-  __syncthreads();
-
-  // ---- top-k by rank.  A NaN logit is read as -inf (the order stays total), -0 as +0 (they
-  // compare equal, the index decides); ties go to the lower index.
-  {
-    constexpr int kPerLane = OLED_MAX_EXPERTS / 32;
-    uint32_t key[kPerLane];
-#pragma unroll
-    for (int i = 0; i < kPerLane; ++i) {
-      const int e = lane + 32 * i;
-      if (e < E) {
-        const float xv = s_logits[e];
-        key[i] = order_key((xv == xv) ? __fadd_rn(xv, 0.0f) : __int_as_float(0xff800000));
-      } else {
-        key[i] = 0u;  // below every real key (the key of -inf is 0x007fffff)
-      }
-    }
-    for (int e = warp; e < E; e += WARPS) {
-      const float xv = s_logits[e];
-      const float ve = (xv == xv) ? __fadd_rn(xv, 0.0f) : __int_as_float(0xff800000);
+  if (TT == 1) {
+    // top-k by rank, all warps; then warp 0: gate scores, counts and reuse-score numerators
+    for (int e = warp; e < E; e += kRouteWarps) {
+      const float ve = topk_value(s_logits[e]);
       const uint32_t ke = order_key(ve);
       int before = 0;
-#pragma unroll
-      for (int i = 0; i < kPerLane; ++i) {
-        const int a = lane + 32 * i;
-        if (32 * i < E) before += (a < E && (key[i] > ke || (key[i] == ke && a < e))) ? 1 : 0;
+      for (int o = lane; o < E; o += 32) {
+        const uint32_t ko = order_key(topk_value(s_logits[o]));
+        before += (ko > ke || (ko == ke && o < e)) ? 1 : 0;
       }
       before = __reduce_add_sync(0xffffffffu, before);
       if (lane == 0 && before < K) {
@@ -366,114 +282,64 @@ route_small_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ 
         s_sel_logit[before] = ve;
       }
     }
-  }
-  __syncthreads();
-  if (warp == 0) {
-    const int my_id = lane < K ? s_sel_id[lane] : 0;
-    const float my_logit = lane < K ? s_sel_logit[lane] : 0.0f;
-    const float top = __shfl_sync(0xffffffffu, my_logit, 0);
-    const float z = lane < K ? exp_spec(__fsub_rn(my_logit, top)) : 0.0f;
-    float sum = __shfl_sync(0xffffffffu, z, 0);
-    for (int j = 1; j < K; ++j) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, z, j));
-    if (lane < K) {
-      const float g = __fdiv_rn(z, sum);
-      ids[(size_t)t * K + lane] = my_id;
-      gate[(size_t)t * K + lane] = g;
-      float c = conf[t];
-      c = (c != c) ? 0.0f : fminf(fmaxf(c, 0.0f), 1.0f);  // psi(c) = c, clamped; NaN -> 0
-      const float pv = __fmul_rn(g, c);
-      // a NaN product (non-finite activations) adds nothing; the 64-bit conversion of a NaN
-      // would return 2^63
-      const unsigned long long q = (pv == pv) ? __float2ull_rz(__fmul_rn(pv, 4294967296.0f)) : 0ull;
-      atomicAdd(&counts[my_id], 1);
-      atomicAdd(&scores[my_id], q);
-    }
-    __syncwarp();
-    if (lane == 0) {
-      s_last = 0;
-      if (rep.ticket != nullptr) {
-        __threadfence();
-        s_last = (atomicAdd(rep.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (warp == 0) {
+      const int t = t0;
+      const int my_id = lane < K ? s_sel_id[lane] : 0;
+      const float my_logit = lane < K ? s_sel_logit[lane] : 0.0f;
+      const float top = __shfl_sync(0xffffffffu, my_logit, 0);
+      const float z = lane < K ? exp_spec(__fsub_rn(my_logit, top)) : 0.0f;
+      float sum = __shfl_sync(0xffffffffu, z, 0);
+      for (int j = 1; j < K; ++j) sum = __fadd_rn(sum, __shfl_sync(0xffffffffu, z, j));
+      if (lane < K) {
+        const float g = __fdiv_rn(z, sum);
+        ids[(size_t)t * K + lane] = my_id;
+        gate[(size_t)t * K + lane] = g;
+        atomicAdd(&counts[my_id], 1);
+        atomicAdd(&scores[my_id], score_quantum(g, conf[t]));
       }
     }
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-
-  // ---- the last CTA: report to the host first (it plans the fills from it), then the permutation
-  if (rep.host_scores != nullptr) {
-    const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
-    const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
-    for (int e = threadIdx.x; e < E; e += blockDim.x) {
-      // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
-      rep.host_scores[e] = tag16 | (__ldcg(&scores[e]) & 0xffffffffffffull);
-      rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)__ldcg(&counts[e]);
+  } else {
+    // one warp per token
+    for (int a = warp; a < TT; a += kRouteWarps) {
+      const int t = t0 + a;
+      if (t >= T) continue;
+      route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores);
     }
   }
-  if (!do_perm) return;
-  const int n = T * K;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) s_ids[i] = __ldcg(&ids[i]);
-  if (warp == 0) {  // exclusive scan of the counts
-    const int per = (E + 31) / 32;
-    int local = 0;
-    for (int i = 0; i < per; ++i) {
-      const int e = lane * per + i;
-      if (e < E) local += __ldcg(&counts[e]);
-    }
-    int incl = local;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const int o = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += o;
-    }
-    int run = incl - local;
-    for (int i = 0; i < per; ++i) {
-      const int e = lane * per + i;
-      if (e < E) {
-        s_off[e] = run;
-        offsets[e] = run;
-        run += __ldcg(&counts[e]);
-      }
-    }
-    if (lane == 31) {
-      s_off[E] = incl;
-      offsets[E] = incl;
-    }
-  }
-  __syncthreads();
-  // stable: the assignments of an expert keep their ascending (token, rank) order
-  for (int e = warp; e < E; e += WARPS) {
-    int base = s_off[e];
-    const int end = s_off[e + 1];
-    for (int a0 = 0; a0 < n && base < end; a0 += 32) {
-      const int a = a0 + lane;
-      const bool hit = a < n && s_ids[a] == e;
-      const uint32_t m = __ballot_sync(0xffffffffu, hit);
-      if (hit) {
-        const int r = base + __popc(m & ((1u << lane) - 1u));
-        perm[r] = a;
-        pos[a] = r;
-      }
-      base += __popc(m);
-    }
-  }
+  if (threadIdx.x == 0) timeline_end(timeline, 0);
 }
 
 // One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
 // assignment list (ascending t*K+j) hands out consecutive sorted rows.
 // If xp != nullptr the CTA also copies the token rows of its expert into sorted order
 // (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
+// The gate kernel before it has completed, so counts and scores are final: the last CTA (the
+// highest expert, usually the first to finish its scan) publishes them to the host in mapped
+// pinned memory.  Every 8-byte word carries the step's sequence tag in its upper bits, so the
+// host can tell word by word that the data is there: no ticket, no fence, no copy, no event.
 __global__ void __launch_bounds__(256)
-permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
+permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts,
+               const unsigned long long* __restrict__ scores, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
-               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K) {
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, RouteReport rep) {
   __shared__ int s_red[8];
   __shared__ int s_base;
   const int e = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   griddep_launch_dependents();
+  if (threadIdx.x == 0) timeline_entry(rep.timeline, 1);
   griddep_wait();
+  if (threadIdx.x == 0) timeline_start(rep.timeline, 1);
+  if (e == E - 1 && rep.host_scores != nullptr) {
+    const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
+    const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
+    for (int i = threadIdx.x; i < E; i += blockDim.x) {
+      // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
+      rep.host_scores[i] = tag16 | (scores[i] & 0xffffffffffffull);
+      rep.host_counts[i] = tag32 | (unsigned long long)(uint32_t)counts[i];
+    }
+  }
   int part = 0;
   for (int i = threadIdx.x; i < e; i += blockDim.x) part += counts[i];
 #pragma unroll
@@ -488,7 +354,10 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     if (e == E - 1) offsets[E] = off + counts[e];
   }
   __syncthreads();
-  if (counts[e] == 0) return;
+  if (counts[e] == 0) {
+    if (threadIdx.x == 0) timeline_end(rep.timeline, 1);
+    return;
+  }
   int base = s_base;
   // stable scan, 8 consecutive assignments per thread and 2048 per round
   for (int a0 = 0; a0 < n; a0 += 8 * blockDim.x) {
@@ -533,7 +402,10 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
       }
     base += total;
   }
-  if (xp == nullptr) return;
+  if (xp == nullptr) {
+    if (threadIdx.x == 0) timeline_end(rep.timeline, 1);
+    return;
+  }
   __syncthreads();  // this CTA's perm entries are visible to all of its threads
   // eight rows at a time: their token numbers, then their loads, are independent memory
   // operations in flight together (a row-by-row loop is a chain of dependent round trips)
@@ -592,31 +464,34 @@ void pdl_set_step(bool on) { g_pdl_step = on; }
 void pdl_set_allowed(bool on) { g_pdl_allowed.store(on); }
 bool pdl_enabled() { return g_pdl_allowed.load() && g_pdl_step; }
 
-bool route_fuses_permutation(int T, int E, int K) {
-  return (size_t)T * K <= (size_t)kSmallMaxAssign && E <= kSmallMaxExperts;
-}
+bool route_can_take_combine(int T) { return T <= kRouteSmallMax; }
 
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
-                  float* gate, int32_t* counts, unsigned long long* scores, const RouteReport& rep,
-                  int32_t* offsets, int32_t* perm, int32_t* pos) {
-  if (T <= kRouteSmallMax) {  // one token per CTA
-    constexpr int W = 16;
-    const int do_perm = (offsets != nullptr && perm != nullptr && pos != nullptr && rep.ticket != nullptr &&
-                         route_fuses_permutation(T, E, K)) ? 1 : 0;
-    launch_pdl(route_small_kernel<W, 4, 4>, dim3(T), dim3(W * 32), 0, st, x, w_router, bias, conf, T, H, E, K, logits,
-               ids, gate, counts, scores, offsets, perm, pos, do_perm, rep);
+                  float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
+                  StepTimeline* timeline) {
+  if (T <= kRouteSmallMax) {
+    constexpr int TT = 1, W = 16;
+    static bool attr_done = false;
+    if (!attr_done) {  // the staged row: H up to 16 K elements
+      cudaFuncSetAttribute(route_kernel<TT, W, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+      cudaGetLastError();
+      attr_done = true;
+    }
+    launch_pdl(route_kernel<TT, W, 4, 4>, dim3(T), dim3(W * 32), (((size_t)E * sizeof(float) + 15) & ~(size_t)15) + (size_t)H * 2, st, x,
+               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, prev, timeline);
   } else {
     constexpr int TT = 8, W = 8;
     launch_pdl(route_kernel<TT, W, 1, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), TT * E * sizeof(float), st, x,
-               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, rep);
+               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, CombinePrev{}, timeline);
   }
 }
 
-void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
-                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp,
-                    int H) {
-  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K);
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, const unsigned long long* scores,
+                    int T, int E, int K, int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x,
+                    uint16_t* xp, int H, const RouteReport& rep) {
+  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, scores, T * K, E, offsets, perm, pos, x, xp, H, K,
+             rep);
 }
 
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
@@ -708,8 +583,8 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   if (n_tokens == 0) return OLED_OK;
   launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
                confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores,
-               RouteReport{}, nullptr, nullptr, nullptr);
-  launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
-                 hidden_dim);
+               CombinePrev{}, nullptr);
+  launch_permute(st, ids, counts, scores, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
+                 hidden_dim, RouteReport{});
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
