@@ -110,9 +110,9 @@ constexpr uint32_t kCtlBytes = (sizeof(SharedCtl) + 1023u) & ~1023u;
 struct Item {
   int slot, m0, row0, valid;
 };
-// Items (expert, token tile, weight tile) are handed out DYNAMICALLY: the producer thread of a
-// CTA draws item numbers from a counter in global memory (one atomic per item, fetched one item
-// ahead) and publishes them to the other roles of its CTA through a small ring in shared
+// Items (expert, token tile, weight tile) are handed out DYNAMICALLY: after its first item (its own
+// CTA number) the producer thread of a CTA draws item numbers from a counter in global memory
+// (one atomic per item, fetched one item ahead) and publishes them to the other roles of its CTA through a small ring in shared
 // memory.  SMs that stream faster take more items, so the launch ends when the work does, not
 // when the slowest SM has finished a fixed share.  Which CTA computes an item does not change
 // its arithmetic.
@@ -148,7 +148,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
               void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int early_start, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter, StepTimeline* timeline,
-              int timeline_slot) {
+              int timeline_slot, const __grid_constant__ RouteReport report) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
@@ -273,6 +273,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int total_items = ctl->n_tiles_total * m_tiles;
   volatile int* abort_flag = &ctl->abort;
 
+  if (KIND == 1 && blockIdx.x == 0 && warp == kProducerWarp && lane != 0) {
+    // the step's report to the host (see RouteReport): sent by lanes that have nothing else to do;
+    // its trip across the host link ends long before this kernel does
+    publish_report(report, lane - 1, 31);
+  }
   if (warp == kProducerWarp && lane == 0) {
     // ------------------------------------------------------------ TMA producer
     // bf16 stores: weight rows and token tile of a k-block go to one operand stage; fp8 stores:
@@ -282,11 +287,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     bool ok = true;
     const int ring = n_stages;
     // (with loads withheld - the test of the bounded waits - nothing is published either)
-    int item = grp.withhold_loads ? 0 : (int)atomicAdd(work_counter, 1u);
+    // the CTA's first item is its own number (no round trip to the counter before the first
+    // load); every later one is drawn from the counter, which hands out numbers from gridDim.x on
+    int item = (int)blockIdx.x;
     for (int seq = 0; ok && !grp.withhold_loads; ++seq) {
       const bool none = item >= total_items;
       // the next item's number is fetched now: the atomic's latency lies under this item's loads
-      const int next = none ? item : (int)atomicAdd(work_counter, 1u);
+      const int next = none ? item : (int)(atomicAdd(work_counter, 1u) + gridDim.x);
       const int ring_slot = seq % kItemRing;
       if (!mbar_wait(smem_u32(&ctl->item_empty[ring_slot]), ((uint32_t)(seq / kItemRing) & 1u) ^ 1u, abort_flag, status,
                      nap_load)) {
@@ -714,7 +721,8 @@ template <int KIND, bool DUAL>
 void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter,
-                    uint32_t smem_of_predecessor, bool early_allowed, StepTimeline* timeline, int timeline_slot) {
+                    uint32_t smem_of_predecessor, bool early_allowed, StepTimeline* timeline, int timeline_slot,
+                    const RouteReport& report) {
   const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 1 ? H : I);
   // KIND 2 may start ahead of its dependency wait only where the caller vouches for the ordering
   // (early_allowed, see launch_ffn_tc) AND one of its CTAs and one of the KIND 1 kernel before it
@@ -723,11 +731,11 @@ void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, 
   if (fp8)
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot);
+               timeline_slot, report);
   else
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot);
+               timeline_slot, report);
 }
 
 }  // namespace
@@ -785,7 +793,8 @@ static int box_index(int max_count, int cap) {
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
                   int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait, StepTimeline* timeline,
-                  int timeline_slot) {
+                  int timeline_slot, const RouteReport& report_in) {
+  const RouteReport report = kind == 1 ? report_in : RouteReport{};
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   const bool fp8 = maps.fp8;
@@ -812,18 +821,18 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
   if (kind == 1 && stacked1) {
     launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
-                             0, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
+                             0, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   } else if (kind == 1) {
     launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
-                            maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
+                            maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   } else {
     const bool dual = grp.n_box == 256;
     if (dual)
       launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
-                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
+                              y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
     else
       launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
-                               maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot);
+                               maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }

@@ -94,15 +94,39 @@ struct GuardList {
   uint32_t* words[12];
 };
 
-// Where the permutation kernel publishes the step's counts and scores for the host: mapped
-// pinned host memory, one 8-byte word per value with the step's sequence number in the upper
-// bits (scores: seq & 0xffff in bits 48..63; counts: seq in bits 32..63).  All-null = no report.
+// Where a step's counts and scores are published for the host: mapped pinned host memory, one
+// 8-byte word per value with the step's sequence number in the upper bits (scores: seq & 0xffff
+// in bits 48..63; counts: seq in bits 32..63), so the host can tell word by word that the data is
+// there: no ticket, no fence, no copy, no event.  The writer is a kernel that runs after the gate
+// kernel has completed (counts and scores are final then) and that does NOT stand between the
+// gate and the expert FFN: a kernel's completion waits for its writes to host memory to be
+// acknowledged across the link (~4 us), so the report leaves from the first CTA of the step's
+// first FFN launch - a kernel that runs for tens of microseconds anyway - or, in a step whose
+// layer has no resident expert yet, from a one-CTA kernel of its own.  host_scores == nullptr:
+// no report.
 struct RouteReport {
   unsigned long long* host_scores = nullptr;    // mapped host [E]
   unsigned long long* host_counts = nullptr;    // mapped host [E]
   unsigned int seq = 0;
+  const int32_t* counts = nullptr;              // device [E], final
+  const unsigned long long* scores = nullptr;   // device [E], final
+  int n_experts = 0;
   StepTimeline* timeline = nullptr;             // device, or null
 };
+#ifdef __CUDACC__
+// Executed by `n_threads` threads with ranks 0..n_threads-1.
+__device__ __forceinline__ void publish_report(const RouteReport& rep, int rank, int n_threads) {
+  if (rep.host_scores == nullptr) return;
+  const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
+  const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
+  for (int e = rank; e < rep.n_experts; e += n_threads) {
+    // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
+    rep.host_scores[e] = tag16 | (rep.scores[e] & 0xffffffffffffull);
+    rep.host_counts[e] = tag32 | (unsigned long long)(uint32_t)rep.counts[e];
+  }
+}
+#endif
+void launch_report(cudaStream_t st, const RouteReport& rep);  // the one-CTA kernel (route.cu)
 
 // ---- route.cu -------------------------------------------------------------------------
 // Gate logits in the contract order, top-k (ties to the lower index), softmax over the selected
@@ -127,11 +151,10 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
                   StepTimeline* timeline);
 bool route_can_take_combine(int T);  // does the gate kernel of a T-token step carry out a CombinePrev?
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
-// kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.  Also
-// publishes counts and scores to the host (rep; all-null: no report).
-void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, const unsigned long long* scores,
-                    int T, int E, int K, int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x,
-                    uint16_t* xp, int H, const RouteReport& rep);
+// kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
+                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
+                    StepTimeline* timeline);
 // xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);
@@ -169,12 +192,14 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
 // work_counter: a device word that is ZERO when the kernel starts; its CTAs draw their work items
 // from it (every launch that can be in flight at the same time needs a word of its own).
+// report (kind 1 only; host_scores == nullptr: none): the kernel's first CTA publishes the step's
+// counts and scores to the host.
 // behind_event_wait: the launch follows a cudaStreamWaitEvent (with, for kind 2, at most its own
 // kind 1 launch in between), i.e. everything enqueued before that wait has completed.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
                   int I, int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait,
-                  StepTimeline* timeline, int timeline_slot);
+                  StepTimeline* timeline, int timeline_slot, const RouteReport& report);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 // Self-check (check.cu): invariants of the routing and the permutation, guard words.

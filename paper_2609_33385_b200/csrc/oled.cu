@@ -316,8 +316,14 @@ void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
 // known on the host yet (the group is the resident set and experts without tokens cost nothing).
 // before_down: an event the down projection (and nothing before it) has to wait for, or null.
 // behind_event_wait: the caller has just enqueued a cudaStreamWaitEvent on the stream.
+// report: the step's report to the host, sent by the gate/up launch (the plain-FMA bring-up path
+// and an empty group send it from a kernel of its own).
 int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts,
-                     cudaEvent_t before_down, bool behind_event_wait) {
+                     cudaEvent_t before_down, bool behind_event_wait, const RouteReport& report = RouteReport{}) {
+  if ((grp.n <= 0 || max_count <= 0 || ctx->ffn_impl == 1) && report.host_scores != nullptr) {
+    launch_report(ctx->stream, report);
+    ctx->launches += 1;
+  }
   if (grp.n <= 0) return OLED_OK;
   const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
   if (ctx->ffn_impl == 1) {
@@ -337,7 +343,7 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
       const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
                                    ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work,
                                    behind_event_wait || (kind == 2 && before_down != nullptr),
-                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li);
+                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li, report);
       if (rc != OLED_OK) return rc;
     }
   }
@@ -623,6 +629,9 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   rep.host_scores = reinterpret_cast<unsigned long long*>(ctx->h_ctrl);
   rep.host_counts = reinterpret_cast<unsigned long long*>(ctx->h_ctrl) + E;
   rep.seq = ctx->seq;
+  rep.counts = ctx->d_counts;
+  rep.scores = ctx->d_scores;
+  rep.n_experts = E;
   StepTimeline* const tl = ctx->timeline_on ? ctx->d_timeline + layer : nullptr;
   rep.timeline = tl;
   if (tl) {  // earliest times start at the maximum, latest at zero
@@ -664,8 +673,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
-    launch_permute(st, ctx->d_ids, ctx->d_counts, ctx->d_scores, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
-                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, rep);
+    launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
+                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl);
   }
   if (!fuse_gather) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
@@ -699,7 +708,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
       }
     // token tile of this launch: twice the mean load per expert (a fuller expert takes more tiles)
     const int mean_load = (int)(((size_t)T * K + E - 1) / E);
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false);
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false, rep);
     if (rc0 != OLED_OK) return rc0;
   }
 

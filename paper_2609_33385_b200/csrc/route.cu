@@ -314,32 +314,18 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 // assignment list (ascending t*K+j) hands out consecutive sorted rows.
 // If xp != nullptr the CTA also copies the token rows of its expert into sorted order
 // (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
-// The gate kernel before it has completed, so counts and scores are final: the last CTA (the
-// highest expert, usually the first to finish its scan) publishes them to the host in mapped
-// pinned memory.  Every 8-byte word carries the step's sequence tag in its upper bits, so the
-// host can tell word by word that the data is there: no ticket, no fence, no copy, no event.
 __global__ void __launch_bounds__(256)
-permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts,
-               const unsigned long long* __restrict__ scores, int n, int E,
+permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
-               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, RouteReport rep) {
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, StepTimeline* timeline) {
   __shared__ int s_red[8];
   __shared__ int s_base;
   const int e = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   griddep_launch_dependents();
-  if (threadIdx.x == 0) timeline_entry(rep.timeline, 1);
+  if (threadIdx.x == 0) timeline_entry(timeline, 1);
   griddep_wait();
-  if (threadIdx.x == 0) timeline_start(rep.timeline, 1);
-  if (e == E - 1 && rep.host_scores != nullptr) {
-    const unsigned long long tag16 = (unsigned long long)(rep.seq & 0xffffu) << 48;
-    const unsigned long long tag32 = (unsigned long long)rep.seq << 32;
-    for (int i = threadIdx.x; i < E; i += blockDim.x) {
-      // score < 2^48 (at most 2^16 tokens of at most 2^32 each); masked so that no data can spoil the tag
-      rep.host_scores[i] = tag16 | (scores[i] & 0xffffffffffffull);
-      rep.host_counts[i] = tag32 | (unsigned long long)(uint32_t)counts[i];
-    }
-  }
+  if (threadIdx.x == 0) timeline_start(timeline, 1);
   int part = 0;
   for (int i = threadIdx.x; i < e; i += blockDim.x) part += counts[i];
 #pragma unroll
@@ -355,7 +341,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   }
   __syncthreads();
   if (counts[e] == 0) {
-    if (threadIdx.x == 0) timeline_end(rep.timeline, 1);
+    if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
   int base = s_base;
@@ -403,7 +389,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     base += total;
   }
   if (xp == nullptr) {
-    if (threadIdx.x == 0) timeline_end(rep.timeline, 1);
+    if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
   __syncthreads();  // this CTA's perm entries are visible to all of its threads
@@ -487,11 +473,22 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
   }
 }
 
-void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, const unsigned long long* scores,
-                    int T, int E, int K, int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x,
-                    uint16_t* xp, int H, const RouteReport& rep) {
-  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, scores, T * K, E, offsets, perm, pos, x, xp, H, K,
-             rep);
+void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
+                    int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
+                    StepTimeline* timeline) {
+  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
+             timeline);
+}
+
+namespace {
+__global__ void __launch_bounds__(128) report_kernel(RouteReport rep) {
+  griddep_launch_dependents();
+  griddep_wait();
+  publish_report(rep, (int)threadIdx.x, (int)blockDim.x);
+}
+}  // namespace
+void launch_report(cudaStream_t st, const RouteReport& rep) {
+  launch_pdl(report_kernel, dim3(1), dim3(128), 0, st, rep);
 }
 
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
@@ -584,7 +581,7 @@ extern "C" int oled_route_noalloc(const void* hidden, const void* w_router, cons
   launch_route(st, static_cast<const uint16_t*>(hidden), static_cast<const uint16_t*>(w_router), bias,
                confidences, n_tokens, hidden_dim, n_experts, top_k, logits, ids, gate, counts, scores,
                CombinePrev{}, nullptr);
-  launch_permute(st, ids, counts, scores, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr,
-                 hidden_dim, RouteReport{});
+  launch_permute(st, ids, counts, n_tokens, n_experts, top_k, offsets, perm, pos, nullptr, nullptr, hidden_dim,
+                 nullptr);
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
