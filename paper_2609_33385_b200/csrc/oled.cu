@@ -706,9 +706,12 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
         grp.slot[grp.n] = (uint16_t)L.cache.slot_of[e];
         ++grp.n;
       }
-    // token tile of this launch: twice the mean load per expert (a fuller expert takes more tiles)
+    // token tile of this launch (the counts are not known on the host yet): twice the mean load
+    // per expert, but at least 32 rows - an expert that received more rows than the tile holds
+    // has its weights streamed once per tile, and in a block of 32 tokens whose routing is
+    // concentrated on few experts (the regime the paper reports) counts of 17..32 are common
     const int mean_load = (int)(((size_t)T * K + E - 1) / E);
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(16, 2 * mean_load)), nullptr, nullptr, false, rep);
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(32, 2 * mean_load)), nullptr, nullptr, false, rep);
     if (rc0 != OLED_OK) return rc0;
   }
 

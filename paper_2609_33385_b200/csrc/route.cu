@@ -310,17 +310,25 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   if (threadIdx.x == 0) timeline_end(timeline, 0);
 }
 
-// One CTA per expert: offset = sum of the counts before it; then a stable scan of the flat
-// assignment list (ascending t*K+j) hands out consecutive sorted rows.
-// If xp != nullptr the CTA also copies the token rows of its expert into sorted order
-// (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
+// One CTA per expert (blockIdx.x): offset = sum of the counts before it; then a stable scan of the
+// flat assignment list (ascending t*K+j) hands out consecutive sorted rows.
+// If xp != nullptr the expert's CTAs (gridDim.y of them) also copy its token rows into sorted
+// order (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
+// Each of those CTAs repeats the scan for itself - a few hundred ids - keeps the token of every
+// sorted row in shared memory (reading the rows' numbers back from global memory would cost a
+// round trip before the first load), and takes every gridDim.y-th batch of eight rows, so that an
+// expert that received many tokens does not make the step wait for one CTA's chain of batches.
+// Only the CTAs with blockIdx.y == 0 write offsets, perm and pos.
+constexpr int kGatherTokMax = 4096;  // rows of one expert in a step that gathers here (T * K <= 4096)
 __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
                const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, StepTimeline* timeline) {
   __shared__ int s_red[8];
   __shared__ int s_base;
+  __shared__ int s_tok[kGatherTokMax];
   const int e = blockIdx.x;
+  const bool writer = blockIdx.y == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   griddep_launch_dependents();
   if (threadIdx.x == 0) timeline_entry(timeline, 1);
@@ -336,11 +344,14 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     int off = 0;
     for (int w = 0; w < 8; ++w) off += s_red[w];
     s_base = off;
-    offsets[e] = off;
-    if (e == E - 1) offsets[E] = off + counts[e];
+    if (writer) {
+      offsets[e] = off;
+      if (e == E - 1) offsets[E] = off + counts[e];
+    }
   }
   __syncthreads();
-  if (counts[e] == 0) {
+  // (a CTA beyond the first of an expert has work only if the expert has a batch of rows for it)
+  if (counts[e] == 0 || (int)blockIdx.y * 8 >= counts[e]) {
     if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
@@ -382,8 +393,11 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
 #pragma unroll
     for (int i = 0; i < 8; ++i)
       if ((m >> i) & 1u) {
-        perm[r] = first + i;
-        pos[first + i] = r;
+        if (writer) {
+          perm[r] = first + i;
+          pos[first + i] = r;
+        }
+        if (xp != nullptr) s_tok[r - s_base] = (first + i) / K;
         ++r;
       }
     base += total;
@@ -392,16 +406,16 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
-  __syncthreads();  // this CTA's perm entries are visible to all of its threads
+  __syncthreads();  // the tokens of this expert's rows are in shared memory
   // eight rows at a time: their token numbers, then their loads, are independent memory
   // operations in flight together (a row-by-row loop is a chain of dependent round trips)
   const int vec_per_row = H / 8, first = s_base, rows = counts[e];
   const uint4* src = reinterpret_cast<const uint4*>(x);
   uint4* dst = reinterpret_cast<uint4*>(xp);
-  for (int r0 = 0; r0 < rows; r0 += 8) {
+  for (int r0 = (int)blockIdx.y * 8; r0 < rows; r0 += 8 * (int)gridDim.y) {
     int tok[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) tok[j] = r0 + j < rows ? perm[first + r0 + j] / K : -1;
+    for (int j = 0; j < 8; ++j) tok[j] = r0 + j < rows ? s_tok[r0 + j] : -1;
     for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
       uint4 v[8];
 #pragma unroll
@@ -412,6 +426,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
         if (tok[j] >= 0) dst[(size_t)(first + r0 + j) * vec_per_row + c] = v[j];
     }
   }
+  if (threadIdx.x == 0) timeline_end(timeline, 1);
 }
 
 // One warp per sorted row: the row's token number once, then the row's 16-byte vectors, four
@@ -476,7 +491,9 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
                     StepTimeline* timeline) {
-  launch_pdl(permute_kernel, dim3(E), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
+  // gathering steps: up to four CTAs per expert share its rows (batches of eight)
+  const int split = xp != nullptr ? 4 : 1;
+  launch_pdl(permute_kernel, dim3(E, split), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
              timeline);
 }
 
