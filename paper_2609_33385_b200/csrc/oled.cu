@@ -11,6 +11,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kernels.h"
 #include "policy.h"
 
@@ -260,6 +262,19 @@ cudaEvent_t prof_event(oled_ctx* ctx) {
   return e;
 }
 
+// NVTX range around one of the five parts of a step (host side; shows up in a timeline profiler
+// next to the kernels it enqueues).  Only with OLED_OPT_PROFILE on; the header-only NVTX API is a
+// no-op unless a tool is attached.
+struct NvtxRange {
+  bool on;
+  NvtxRange(const oled_ctx* ctx, const char* name);
+  void end() {
+    if (on) nvtxRangePop();
+    on = false;
+  }
+  ~NvtxRange() { end(); }
+};
+
 // Brackets one kernel launch with events when profiling is on.
 struct ProfScope {
   oled_ctx* ctx;
@@ -283,6 +298,10 @@ struct ProfScope {
     }
   }
 };
+
+NvtxRange::NvtxRange(const oled_ctx* ctx, const char* name) : on(ctx->profile) {
+  if (on) nvtxRangePushA(name);
+}
 
 void prof_resolve(oled_ctx* ctx) {
   for (auto& r : ctx->prof_pending) {
@@ -650,6 +669,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     if (rcp != OLED_OK) return rcp;
   }
   {
+    NvtxRange nv(ctx, "oled.step.1_gate_topk_scores");
     ProfScope ps(ctx, OLED_KERNEL_ROUTE,
                  ((uint64_t)T * H + (uint64_t)E * H) * 2 + (uint64_t)T * K * 8 +
                      (fuse_prev ? (uint64_t)T * K * H * 4 + (uint64_t)T * H * 6 : 0),
@@ -671,6 +691,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
                  ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, prev, tl);
   }
   const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
+  NvtxRange nv_perm(ctx, "oled.step.2_permutation_counts");
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
     launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
@@ -681,6 +702,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
   }
   ctx->launches += fuse_gather ? 2 : 3;
+  nv_perm.end();
   if (ctx->corrupt_perm) {
     launch_corrupt_perm(st, ctx->d_perm, T * K);
     ctx->launches += 1;
@@ -691,6 +713,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   }
   OLED_CUDA(ctx, cudaGetLastError());
 
+  NvtxRange nv_ffn_hits(ctx, "oled.step.3_expert_ffn_hits");
   // 1b. cache hits need no decision: the FFN over the experts resident BEFORE the step is
   // enqueued at once (experts that received no token contribute no tile), so the GPU does not
   // wait for the host's round trip below.
@@ -715,6 +738,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     if (rc0 != OLED_OK) return rc0;
   }
 
+  nv_ffn_hits.end();
+  NvtxRange nv_policy(ctx, "oled.step.5_reuse_score_retention_fills");
   // The report implies that everything enqueued before this step has completed, so slots
   // released earlier are free to be overwritten by the side stream.
   {
@@ -783,6 +808,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     ++n_groups;
   }
 
+  nv_policy.end();
+  NvtxRange nv_ffn_miss(ctx, "oled.step.3_expert_ffn_misses");
   // 4. grouped FFN over the misses as their weights land (hits: step 1b)
   {
     uint64_t hit_rows = 0;
@@ -797,6 +824,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     if (rc != OLED_OK) return rc;
   }
 
+  nv_ffn_miss.end();
+  NvtxRange nv_comb(ctx, "oled.step.4_combine");
   // 5. combine - or, inside a stack iteration of few-token steps, left to the next layer's gate kernel
   const bool defer = defer_combine && ctx->fuse_combine && route_can_take_combine(T) && x_next != nullptr &&
                      !ctx->y_bf16 && !ctx->self_check && ctx->ffn_impl == 0;

@@ -84,38 +84,47 @@ def policy_mode(args, device):
 
 def shape_mode(args, device):
     """Block length x capacity and batch-size sweeps (the paper's sensitivity studies, Sec. 5.4):
-    tokens per step from 1 to 1024 on the same stack, crossing from the few-tokens-per-expert
-    regime (weight streaming) towards the many-token regime (tensor bound)."""
+    block lengths 1..64 crossed with residencies 10..100 %, and batches of 4, 8 and 32 blocks of
+    32 tokens, on the same stack - from the few-tokens-per-expert regime (weight streaming)
+    towards the many-token regime (tensor bound)."""
     rows = []
     base = None
-    points = [(1, bl) for bl in (1, 4, 16, 32, 64)] + [(b, 32) for b in (2, 4, 8, 16, 32)]
-    for batch, block_len in points:
-        for res in (1.0, 0.4):
-            w = synth.config(3, n_layers=args.layers, batch=batch, block_len=block_len, residency=res,
-                             shared_beta=0.9 if args.variant == "B" else 0.0)
-            n_it = args.warmup + args.steps
-            w = w.replace(blocks=-(-n_it // w.iters))
-            xs, cs = [], []
-            for _, _, h_bits, conf in synth.denoise_inputs(w):
-                xs.append(bits_to_dev(h_bits, device))
-                cs.append(torch.from_numpy(conf).to(device))
-            run = StackRunner(w, device=device, share_store_of=base, distinct_layers=args.distinct_layers)
-            if base is None:
-                base = run
-            ms, d = run_point(run, xs, cs, args.warmup, args.steps)
-            rows.append(dict(batch=batch, block_len=block_len, tokens=w.tokens, residency=res,
-                             capacity=w.capacity, ms_per_step=ms, tokens_per_s=w.tokens / (ms * 1e-3),
-                             tpot_ms=ms * w.iters / w.tokens, misses=d["misses"], hits=d["hits"],
-                             active=d["active_experts"] / max(1, d["steps"]),
-                             h2d_gb_per_step=d["bytes_moved"] / args.steps / 1e9))
-            if run is not base:
-                run.close()
-    lines = ["| batch | block | tokens/step | residency | active/layer | misses | H2D GB/step | ms/step | "
-             "tokens/s | TPOT ms |", "|" + "---|" * 10]
+    points = [(1, bl, res) for bl in (1, 4, 16, 32, 64) for res in (1.0, 0.6, 0.4, 0.2, 0.1)]
+    points += [(b, 32, res) for b in (4, 8, 32) for res in (1.0, 0.4)]
+    full_ms = {}
+    for batch, block_len, res in points:
+        w = synth.config(3, n_layers=args.layers, batch=batch, block_len=block_len, residency=res,
+                         shared_beta=0.9 if args.variant == "B" else 0.0,
+                         rho=0.98 if args.variant == "B" else 0.9)
+        n_it = args.warmup + args.steps
+        w = w.replace(blocks=-(-n_it // w.iters))
+        xs, cs = [], []
+        for _, _, h_bits, conf in synth.denoise_inputs(w):
+            xs.append(bits_to_dev(h_bits, device))
+            cs.append(torch.from_numpy(conf).to(device))
+        run = StackRunner(w, device=device, share_store_of=base, distinct_layers=args.distinct_layers)
+        if base is None:
+            base = run
+        ms, d = run_point(run, xs, cs, args.warmup, args.steps)
+        if res == 1.0:
+            full_ms[(batch, block_len)] = ms
+        link_ms = d["bytes_moved"] / args.steps / (args.h2d_gbs * 1e9) * 1e3
+        rows.append(dict(batch=batch, block_len=block_len, tokens=w.tokens, residency=res,
+                         capacity=w.capacity, ms_per_step=ms, tokens_per_s=w.tokens / (ms * 1e-3),
+                         tpot_ms=ms * w.iters / w.tokens, misses=d["misses"], hits=d["hits"],
+                         active=d["active_experts"] / max(1, d["steps"]),
+                         h2d_gb_per_step=d["bytes_moved"] / args.steps / 1e9,
+                         x_full=ms / full_ms[(batch, block_len)],
+                         frac_of_link=(link_ms / ms) if link_ms > 0 else None))
+        if run is not base:
+            run.close()
+    lines = ["| batch | block | tokens/step | residency | C | active/layer | misses | H2D GB/step | ms/step | "
+             "tokens/s | TPOT ms | x full | of link bound |", "|" + "---|" * 13]
     for r in rows:
-        lines.append(f"| {r['batch']} | {r['block_len']} | {r['tokens']} | {r['residency']:.0%} | "
+        lf = "-" if r["frac_of_link"] is None else f"{r['frac_of_link']:.2f}"
+        lines.append(f"| {r['batch']} | {r['block_len']} | {r['tokens']} | {r['residency']:.0%} | {r['capacity']} | "
                      f"{r['active']:.1f} | {r['misses']} | {r['h2d_gb_per_step']:.3f} | {r['ms_per_step']:.3f} | "
-                     f"{r['tokens_per_s']:.0f} | {r['tpot_ms']:.4f} |")
+                     f"{r['tokens_per_s']:.0f} | {r['tpot_ms']:.4f} | {r['x_full']:.1f} | {lf} |")
     return rows, "\n".join(lines)
 
 

@@ -5,7 +5,7 @@ method's arithmetic (no routing, no FFN, no cache policy).  It is the one
 module that the CPU oracle's tests and the CUDA path's tests/bench may both
 use, so that both sides see identical inputs.
 
-Shapes follow the five workload configurations of the build contract; value
+Shapes follow the five workload configurations this library is measured on; value
 distributions follow the regime the paper reports for semi-autoregressive
 dLLM decoding (Sec. 2.1: a block of masked tokens is refined over several
 denoising iterations; Sec. 3.3: adjacent iterations have highly similar

@@ -173,3 +173,19 @@ def test_config5_shape_4096_tokens_zipf_bias():
         assert dbg["counts"].max() > 4 * dbg["counts"].min()          # the bias skews the load
     finally:
         run.close()
+
+
+@pytest.mark.parametrize("block_len", [1, 4])
+def test_config2_shape_short_blocks(block_len):
+    """Block lengths 1 and 4 at the full layer shape (hidden 2048, 64 experts top-8, I 1024): most
+    experts receive no token, the 16-row token tiles are nearly empty, and a step activates fewer
+    experts than the GPU has SMs (Sec. 5.4 block-length study).  Every discrete result and every
+    token's output against the oracle, cold start at 40 % residency, 4 layers."""
+    w = synth.config(1, n_layers=4, blocks=2, iters=3, block_len=block_len)
+    run, ora = _setup(w, distinct_layers=2)
+    try:
+        _replay(run, ora, 6, sample_layers={0, 1, 2, 3}, min_tokens=block_len, rng=np.random.default_rng(6))
+        st = run.ctx.stats()
+        assert st.steps == 24 and st.active_experts <= 24 * 8 * block_len
+    finally:
+        run.close()

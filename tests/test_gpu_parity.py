@@ -528,8 +528,9 @@ def test_fp8_expert_store_tiny_stack():
 
 @pytest.mark.parametrize("n", [40, 300, 700])
 def test_fp8_expert_store_token_tile_variants(n):
-    """fp8 blobs through every FFN tile form: stacked (few tokens), two accumulators (up to 128
-    tokens per expert) and the 256-token form with two weight tiles per item."""
+    """fp8 blobs through every FFN tile form that exists for them: stacked (token tiles up to 32
+    rows) and two accumulators (64 and 128 rows; fp8 stores stop at 128-row tiles, so the
+    700-token case takes several tiles per expert)."""
     from paper_2609_33385_b200.runner import bits_to_dev
     w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
     run = _runner(w, capacity=[4], max_tokens=n, fp8=True)
