@@ -225,10 +225,16 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * OLED_OPT_FUSE_COMBINE: inside oled_denoise_iteration(), steps of at most 1024 tokens leave a
  *   layer's combine and residual to the next layer's gate kernel (one kernel boundary and one
  *   reload of the hidden states less per layer).
+ * OLED_OPT_FUSE_FFN: 0 = gate/up and down projection of an expert group always as two launches;
+ *   1 (default) = as ONE launch where few work items per SM are expected (bf16 stores, token tiles
+ *   of at most 32 rows): SMs that run out of gate/up items go on with the down projection of
+ *   experts that are complete instead of idling until the whole gate/up launch has ended;
+ *   2 = one launch wherever that form exists.
  * OLED_OPT_PDL: programmatic dependent launch between the kernels of a few-token step
  *   (process-wide, not per context). */
 #define OLED_OPT_SPLIT_LAST_FILL 9
 #define OLED_OPT_FUSE_COMBINE 10
+#define OLED_OPT_FUSE_FFN 11
 #define OLED_OPT_PDL 12
 /* OLED_OPT_TIMELINE: 1 = the kernels of every step record, per kernel, when its first CTA entered,
  * when the first one got past its dependency wait and when the last one finished (GPU global
@@ -268,7 +274,8 @@ int oled_get_capacity(oled_ctx* ctx, int32_t* capacity);
 #define OLED_KERNEL_FFN_GATE_UP 3
 #define OLED_KERNEL_FFN_DOWN 4
 #define OLED_KERNEL_COMBINE 5
-#define OLED_N_KERNELS 6
+#define OLED_KERNEL_FFN_FUSED 6 /* gate/up + SwiGLU + down projection in one launch */
+#define OLED_N_KERNELS 7
 typedef struct {
   uint64_t launches;
   double ms;       /* sum of CUDA-event durations */

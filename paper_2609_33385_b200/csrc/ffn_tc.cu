@@ -109,6 +109,20 @@ constexpr uint32_t kCtlBytes = (sizeof(SharedCtl) + 1023u) & ~1023u;
 
 struct Item {
   int slot, m0, row0, valid;
+  int kind;  // 1: gate/up (+SwiGLU), 2: down projection
+  int g;     // index of the expert in the launch's group
+};
+// The second half of a FUSED launch's work list (KIND 3): items [n1, n1 + n2) are the down-
+// projection items of the same experts and token tiles as the gate/up items [0, n1).
+struct SecondPhase {
+  int n1;            // number of first-phase items (INT_MAX: no second phase)
+  int m_tiles, m_rows;
+};
+// A role's position in the expert list: items arrive in ascending order within a phase, so the
+// search for an item's expert only moves forward; it restarts with the second phase.
+struct ItemCursor {
+  int g = 0;
+  int phase2 = 0;
 };
 // Items (expert, token tile, weight tile) are handed out DYNAMICALLY: after its first item (its own
 // CTA number) the producer thread of a CTA draws item numbers from a counter in global memory
@@ -126,21 +140,53 @@ __device__ __forceinline__ int take_item(SharedCtl* ctl, int seq, volatile int* 
   mbar_arrive(smem_u32(&ctl->item_empty[slot]));
   return item;
 }
-__device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int m_tiles,
-                                            int m_rows, int n_box, int& g, Item& it) {
+__device__ __forceinline__ void decode_item(const SharedCtl* ctl, const FfnGroup& grp, int item, int kind1, int m_tiles,
+                                            int m_rows, int n_box, const SecondPhase& second, ItemCursor& cur,
+                                            Item& it) {
+  it.kind = kind1;
+  if (item >= second.n1) {
+    item -= second.n1;
+    m_tiles = second.m_tiles;
+    m_rows = second.m_rows;
+    it.kind = 2;
+    if (!cur.phase2) {
+      cur.phase2 = 1;
+      cur.g = 0;
+    }
+  }
   const int q = item / m_tiles;
   const int m = item - q * m_tiles;
+  int g = cur.g;
   while (ctl->tile_prefix[g + 1] <= q) ++g;
+  cur.g = g;
   const int nt = q - ctl->tile_prefix[g];
+  it.g = g;
   it.slot = grp.slot[g];
   it.m0 = m * m_rows;
   it.row0 = ctl->row_start[g] + nt * n_box;
   it.valid = min(n_box, ctl->count[g] - nt * n_box);
 }
 
+// What a FUSED launch (KIND 3) needs on top: the down projection's tensor maps, its output and
+// the completion counters.
+struct FusedSecond {
+  CUtensorMap tm_w2;    // down-projection weights
+  CUtensorMap tm_act2;  // intermediate rows (hbuf)
+  void* out2;           // y
+  uint32_t* done;       // per expert of the group: epilogue warps that have stored gate/up rows; ZERO at start
+};
+
 // DUAL: two accumulators per item - gate and up (KIND 1, always), or two row blocks of Wd
 // (KIND 2 with the 256-token tile).
 // FP8: the slot pool holds fp8 expert blobs (tm_w is a byte map over the e4m3 codes).
+// KIND 3 (bf16 stores, token tiles of at most 32 rows): the gate/up items in their stacked form,
+// then the down-projection items of the same experts, in ONE launch.  A down item reads the
+// intermediate rows that the gate/up items of its expert wrote, so its producer waits (bounded)
+// until the expert's counter in `done` shows that all of them have been stored; items are handed
+// out in order, gate/up first, so that wait is over long before it is reached except in launches
+// with few items per SM - which is where this form pays: the two-kernel form leaves every SM that
+// runs out of gate/up items idle until the last gate/up item of the whole launch is done, this
+// one lets it go on with the down projection of experts that are already complete.
 template <int KIND, bool DUAL, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
@@ -148,15 +194,19 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
               void* __restrict__ out_ptr, int H, int I, int n_stages, int k_atoms, int early_start, int out_bf16,
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter, StepTimeline* timeline,
-              int timeline_slot, const __grid_constant__ RouteReport report) {
+              int timeline_slot, const __grid_constant__ RouteReport report,
+              const __grid_constant__ FusedSecond fs) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_box = grp.n_box;
+  constexpr bool fused = KIND == 3;
+  static_assert(!(fused && (DUAL || FP8)), "the fused form exists for bf16 stores and single tiles only");
+  constexpr int kind1 = fused ? 1 : KIND;  // kind of the launch's first-phase (or only) items
   constexpr bool dual = DUAL;
-  constexpr bool stacked = KIND == 1 && !DUAL;  // 64 gate + 64 up rows in one 128-row tile
+  constexpr bool stacked = (KIND == 1 && !DUAL) || fused;  // gate/up items: 64 gate + 64 up rows in one 128-row tile
   constexpr uint32_t a_bytes = (dual ? 2u : 1u) * kATile;
   const uint32_t b_bytes = (uint32_t)n_box * 128u;
   // bf16 stores: a stage (shared memory) holds the weight tile(s) and the token tile of a k-block.
@@ -171,16 +221,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const uint32_t stage_bytes = (uint32_t)k_atoms * atom_bytes;
   constexpr uint32_t atom_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
   const uint32_t a_cols = (uint32_t)k_atoms * atom_cols;
-  const int k_blocks = (KIND == 1 ? H : I) / (kBlockK * k_atoms);  // stages per item
+  const int k_blocks1 = (kind1 == 1 ? H : I) / (kBlockK * k_atoms);  // stages per (first-phase) item
+  const int k_blocks2 = I / (kBlockK * k_atoms);                    // stages per down item of a fused launch
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
-  const int m_tiles = (KIND == 1 ? I : H) / m_rows;
+  const int m_tiles = (kind1 == 1 ? I : H) / m_rows;
   const int acc_cols = (dual ? 2 : 1) * n_box;
   const int a_total = FP8 ? n_stages * (int)a_cols : 0;
   const int acc_stages = (2 * acc_cols + a_total <= 512) ? 2 : 1;
   const uint32_t a_col0 = (uint32_t)(acc_stages * acc_cols);  // first column of the weight stages
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
   // plain store epilogue of KIND 2 runs best with 8
-  const int epi_warps = min((KIND == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+  const int epi_warps = min((KIND != 2 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
   // fp8 stores: the four dedicated converter warps plus epilogue warps this token tile leaves
   // idle form conv_groups (at most two: more of them take issue slots from the MMA thread and
   // measured slower) groups of four warps, one warp per TMEM lane quarter.
@@ -228,6 +279,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   if (warp == kProducerWarp && lane == 0) {  // the two tensor maps, ahead of the first copy
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
+    if (fused) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&fs.tm_w2)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&fs.tm_act2)) : "memory");
+    }
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -270,10 +325,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   constexpr uint32_t nap_epi = FP8 ? OLED_NAP_EPI : 0u, nap_load = FP8 ? OLED_NAP_LOAD : 0u,
                      nap_conv = FP8 ? OLED_NAP_CONV : 0u;
   const uint32_t tmem_base = ctl->tmem_base;
-  const int total_items = ctl->n_tiles_total * m_tiles;
+  SecondPhase second;
+  second.n1 = fused ? ctl->n_tiles_total * m_tiles : 0x7fffffff;
+  second.m_rows = kBlockM;
+  second.m_tiles = H / kBlockM;
+  const int total_items = ctl->n_tiles_total * m_tiles + (fused ? ctl->n_tiles_total * second.m_tiles : 0);
+  // KIND 3: epilogue warps that store intermediate rows per gate/up item, times the items of one token tile
+  const uint32_t done_per_tile = (uint32_t)(m_tiles * (epi_warps / 2));
   volatile int* abort_flag = &ctl->abort;
 
-  if (KIND == 1 && blockIdx.x == 0 && warp == kProducerWarp && lane != 0) {
+  if (KIND != 2 && blockIdx.x == 0 && warp == kProducerWarp && lane != 0) {
     // the step's report to the host (see RouteReport): sent by lanes that have nothing else to do;
     // its trip across the host link ends long before this kernel does
     publish_report(report, lane - 1, 31);
@@ -282,7 +343,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     // ------------------------------------------------------------ TMA producer
     // bf16 stores: weight rows and token tile of a k-block go to one operand stage; fp8 stores:
     // code rows and token tile go to one load slot
-    int stage = 0, g = 0;
+    int stage = 0, ready_g = -1;
+    ItemCursor cur;
     uint32_t phase = 0;
     bool ok = true;
     const int ring = n_stages;
@@ -304,8 +366,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       mbar_arrive(smem_u32(&ctl->item_full[ring_slot]));
       if (none) break;
       Item it;
-      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
+      decode_item(ctl, grp, item, kind1, m_tiles, m_rows, n_box, second, cur, it);
       item = next;
+      const bool down_of_fused = fused && it.kind == 2;
+      const CUtensorMap* map_w = down_of_fused ? &fs.tm_w2 : &tm_w;
+      const CUtensorMap* map_act = down_of_fused ? &fs.tm_act2 : &tm_act;
+      const int k_blocks = down_of_fused ? k_blocks2 : k_blocks1;
       constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
       auto load_weights = [&](int st, int kb) {
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
@@ -313,22 +379,22 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         for (int atom = 0; atom < k_atoms; ++atom) {
           const uint32_t w_addr = tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes;
           const int k0 = (kb * k_atoms + atom) * kBlockK;
-          if (stacked) {  // tm_w has 64-row boxes here
-            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
-            tma_load_3d(&tm_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
-          } else if (KIND == 1) {
-            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // gate rows
-            tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, I + it.m0, it.slot);  // up rows
+          if (stacked && it.kind == 1) {  // the map has 64-row boxes here
+            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
+            tma_load_3d(map_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
+          } else if (it.kind == 1) {
+            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);               // gate rows
+            tma_load_3d(map_w, w_addr + w_tile, bar, k0, I + it.m0, it.slot);  // up rows
           } else {
-            tma_load_3d(&tm_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
-            if (dual) tma_load_3d(&tm_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
+            tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);               // down rows
+            if (dual) tma_load_3d(map_w, w_addr + w_tile, bar, k0, it.m0 + kBlockM, it.slot);
           }
         }
       };
       auto load_tokens = [&](int st, int kb) {
         const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
         for (int atom = 0; atom < k_atoms; ++atom)
-          tma_load_2d(&tm_act,
+          tma_load_2d(map_act,
                       tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (FP8 ? raw_bytes : a_bytes),
                       bar, (kb * k_atoms + atom) * kBlockK, it.row0);
       };
@@ -342,6 +408,58 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         kb = pre;
         if (pre == n_stages) phase ^= 1u;
         else stage = pre;
+      }
+      if (down_of_fused) {
+        // The intermediate rows of every token tile of this expert must be in memory.  If they are
+        // not yet (launches with few items per SM), the weights of as many stages as the ring
+        // holds go first, then the wait, then those stages' token tiles.
+        const uint32_t* flag = fs.done + it.g;
+        const uint32_t target = done_per_tile * (uint32_t)(ctl->tile_prefix[it.g + 1] - ctl->tile_prefix[it.g]);
+        uint32_t seen = target;  // (an expert seen complete stays complete: no second look)
+        if (it.g != ready_g) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+        int pre = 0;
+        const int stage0 = stage;
+        if (seen < target) {
+          pre = min(n_stages, k_blocks);
+          for (int i = 0; i < pre && ok; ++i) {
+            if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_load)) {
+              ok = false;
+              break;
+            }
+            load_weights(stage, i);
+            if (++stage == ring) {
+              stage = 0;
+              phase ^= 1u;
+            }
+          }
+          unsigned long long t0 = 0;
+          for (uint32_t spin = 0; ok; ++spin) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(flag) : "memory");
+            if (seen >= target) break;
+            if ((spin & 255u) == 255u) {
+              if (*abort_flag) ok = false;
+              const unsigned long long now = globaltimer();
+              if (t0 == 0) t0 = now;
+              if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, (uint32_t)kStatusWaitTimeout);
+                ok = false;
+              }
+            }
+          }
+          if (!ok) break;
+        }
+        ready_g = it.g;
+        // the rows were written through the generic proxy; the loads below read through the async proxy
+        asm volatile("fence.proxy.async;" ::: "memory");
+        if (pre > 0) {
+          int st = stage0;
+          for (int i = 0; i < pre; ++i) {
+            load_tokens(st, i);
+            if (++st == ring) st = 0;
+          }
+          kb = pre;
+        }
       }
       for (; kb < k_blocks; ++kb) {
         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status, nap_load)) {
@@ -363,7 +481,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     }
   } else if (warp == kMmaWarp && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
-    int stage = 0, g = 0, local = 0;
+    int stage = 0, local = 0;
+    ItemCursor cur;
     uint32_t phase = 0;
     bool ok = true;
     // Descriptor words of stage 0 (K-major, 128-byte swizzle, 8-row groups 1024 bytes apart); the
@@ -379,7 +498,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const int item = take_item(ctl, local, abort_flag, status, 0u);
       if (item < 0) break;
       Item it;
-      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
+      decode_item(ctl, grp, item, kind1, m_tiles, m_rows, n_box, second, cur, it);
+      const int k_blocks = (fused && it.kind == 2) ? k_blocks2 : k_blocks1;
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
       if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
@@ -441,6 +561,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     int stage = group, mine = group;
     uint32_t phase = 0;
     bool live = true;
+    const int k_blocks = k_blocks1;
     for (int seq = 0; live; ++seq) {
       int item = 0;
       if (lane == 0) item = take_item(ctl, seq, abort_flag, status, nap_conv);
@@ -491,7 +612,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   } else if (warp < epi_warps) {
     // ------------------------------------------------------------ epilogue
     // (only as many warps per quarter as the token tile has 16-column chunks)
-    int g = 0, local = 0;
+    int local = 0;
+    ItemCursor cur;
     uint32_t xn = 0;  // stacked mode: 16-column chunks this warp's chunk group has exchanged so far
     bool alive = true;
     for (; alive; ++local) {
@@ -500,7 +622,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       item = __shfl_sync(0xffffffffu, item, 0);
       if (item < 0) break;
       Item it;
-      decode_item(ctl, grp, item, m_tiles, m_rows, n_box, g, it);
+      decode_item(ctl, grp, item, kind1, m_tiles, m_rows, n_box, second, cur, it);
+      const bool gate_up_item = it.kind == 1;  // (always true for KIND 1, never for KIND 2)
       const int acc = local % acc_stages;
       const uint32_t acc_phase = (uint32_t)(local / acc_stages) & 1u;
       // one lane polls (keeps issue slots free for the producer and MMA threads); the outcome is
@@ -533,7 +656,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
-        if (stacked) {
+        if (stacked && gate_up_item) {
           // lanes 0-63 hold silu's argument (gate rows), lanes 64-127 the up rows of the same
           // features: warps 2,3 hand their chunk to warps 0,1 through a double-buffered slot
           tmem_ld_wait();
@@ -597,8 +720,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
           }
         } else {
-          float* y = reinterpret_cast<float*>(out_ptr);
-          uint16_t* yb = reinterpret_cast<uint16_t*>(out_ptr);  // many-token steps keep y in bf16
+          void* const out_y = fused ? fs.out2 : out_ptr;
+          float* y = reinterpret_cast<float*>(out_y);
+          uint16_t* yb = reinterpret_cast<uint16_t*>(out_y);  // many-token steps keep y in bf16
           uint32_t rb[16];
           if (dual) tmem_ld16(t_row + (uint32_t)(n_box + c), rb);
           tmem_ld_wait();
@@ -621,6 +745,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
       }
       if (!alive) break;
+      if (fused && gate_up_item && quarter < 2) {
+        // this warp's intermediate rows of the item are stored: make them visible device-wide,
+        // then count the warp in (the down items of this expert wait for the full count)
+        __threadfence();
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) atomicAdd(fs.done + it.g, 1u);
+      }
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
     }
@@ -682,7 +814,7 @@ struct Rings {
 };
 // Epilogue warps the kernel activates for a token tile (the others widen fp8 weights).
 int epi_warps_for(int kind, int out_bf16, int n_box) {
-  return std::min((kind == 1 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
+  return std::min((kind != 2 || out_bf16) ? kEpiWarps : 8, 4 * (n_box / 16));
 }
 // Stage shape and count.  A stage holds two k-blocks where at least four such stages fit (small
 // token tiles, one weight tile) and the contraction has an even number of k-blocks.  bf16 stores:
@@ -690,7 +822,8 @@ int epi_warps_for(int kind, int out_bf16, int n_box) {
 // (eleven measured slower).  fp8 stores: a stage is a load slot in shared memory plus columns of
 // tensor memory behind the accumulators (two accumulator stages if at least two weight stages
 // still fit); the depth is a multiple of the number of converter groups (see the kernel).
-Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim) {
+// k_dim2: the second contraction length of a fused launch (0 otherwise).
+Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim, int k_dim2 = 0) {
   const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
   const uint32_t atom = fp8 ? a / 2 + b : a + b;  // one k-block in shared memory
@@ -701,7 +834,7 @@ Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_di
     kblocks = std::min(kblocks, free_cols / a_cols);
   }
   Rings r;
-  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0) ? 2 : 1;
+  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0 && (k_dim2 / kBlockK) % 2 == 0) ? 2 : 1;
   r.stages = std::min(kblocks / r.k_atoms, kMaxStages);
   if (fp8) {
     const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
@@ -722,20 +855,25 @@ void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, 
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter,
                     uint32_t smem_of_predecessor, bool early_allowed, StepTimeline* timeline, int timeline_slot,
-                    const RouteReport& report) {
-  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 1 ? H : I);
+                    const RouteReport& report, const FusedSecond& fs = FusedSecond{}) {
+  const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 2 ? I : H, KIND == 3 ? I : 0);
   // KIND 2 may start ahead of its dependency wait only where the caller vouches for the ordering
   // (early_allowed, see launch_ffn_tc) AND one of its CTAs and one of the KIND 1 kernel before it
   // cannot share an SM, so that it gets an SM only when a KIND 1 CTA has left it
   const int early = (KIND == 2 && early_allowed && smem_of_predecessor + r.smem > 228u * 1024u) ? 1 : 0;
-  if (fp8)
+  if constexpr (KIND == 3) {
+    launch_pdl(ffn_tc_kernel<3, false, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H, I,
+               r.stages, r.k_atoms, 0, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
+               timeline_slot, report, fs);
+  } else if (fp8) {
     launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot, report);
-  else
+               timeline_slot, report, fs);
+  } else {
     launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot, report);
+               timeline_slot, report, fs);
+  }
 }
 
 }  // namespace
@@ -777,7 +915,7 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   if (!attr_done) {
     if (!set_smem_attr<1, true, false>() || !set_smem_attr<1, false, false>() || !set_smem_attr<2, true, false>() ||
         !set_smem_attr<2, false, false>() || !set_smem_attr<1, true, true>() || !set_smem_attr<1, false, true>() ||
-        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>())
+        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>() || !set_smem_attr<3, false, false>())
       return OLED_ERR_CUDA;
     attr_done = true;
   }
@@ -793,8 +931,8 @@ static int box_index(int max_count, int cap) {
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
                   int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait, StepTimeline* timeline,
-                  int timeline_slot, const RouteReport& report_in) {
-  const RouteReport report = kind == 1 ? report_in : RouteReport{};
+                  int timeline_slot, const RouteReport& report_in, uint32_t* done) {
+  const RouteReport report = kind != 2 ? report_in : RouteReport{};
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
   const bool fp8 = maps.fp8;
@@ -819,7 +957,17 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   // or the launch pair sits behind an event wait, which completes everything enqueued before it.
   const bool early_allowed = kind == 2 && (behind_event_wait || host_counts == nullptr);
   const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
-  if (kind == 1 && stacked1) {
+  if (kind == 3) {
+    if (fp8 || !stacked1 || done == nullptr) return OLED_ERR_INVALID_ARG;  // callers ask ffn_tc_can_fuse() first
+    FusedSecond fs;
+    fs.tm_w2 = maps.w2;
+    fs.tm_act2 = maps.hbuf[ib];
+    fs.out2 = y;
+    fs.done = done;
+    launch_variant<3, false>(false, grid_for(I / (kBlockM / 2) + H / kBlockM), st, maps.w13_half, maps.xp[ib], grp, offsets,
+                             hbuf, H, I, 0, maps.pool, maps.slot_bytes, status, work_counter, 0u, false, timeline,
+                             timeline_slot, report, fs);
+  } else if (kind == 1 && stacked1) {
     launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
                              0, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   } else if (kind == 1) {
@@ -835,6 +983,10 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
                                maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
+}
+
+bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count) {
+  return !maps.fp8 && (16 << box_index(max_count, 256)) <= 32;
 }
 
 }  // namespace oled

@@ -189,17 +189,20 @@ struct FfnTcMaps {
 // Builds the tensor maps; returns 0 or a negative oled_status.
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows);
-// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y.  One launch each.
+// kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y; kind 3: both in one launch
+// (bf16 stores and token tiles of at most 32 rows only: ask ffn_tc_can_fuse; `done` then points at
+// one ZERO word per expert of the group).  One launch each.
 // work_counter: a device word that is ZERO when the kernel starts; its CTAs draw their work items
 // from it (every launch that can be in flight at the same time needs a word of its own).
-// report (kind 1 only; host_scores == nullptr: none): the kernel's first CTA publishes the step's
+// report (kinds 1 and 3; host_scores == nullptr: none): the kernel's first CTA publishes the step's
 // counts and scores to the host.
 // behind_event_wait: the launch follows a cudaStreamWaitEvent (with, for kind 2, at most its own
 // kind 1 launch in between), i.e. everything enqueued before that wait has completed.
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
                   int I, int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait,
-                  StepTimeline* timeline, int timeline_slot, const RouteReport& report);
+                  StepTimeline* timeline, int timeline_slot, const RouteReport& report, uint32_t* done = nullptr);
+bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 // Self-check (check.cu): invariants of the routing and the permutation, guard words.

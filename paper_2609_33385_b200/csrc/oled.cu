@@ -22,6 +22,7 @@ namespace {
 
 struct LayerData {
   LayerCacheState cache;
+  int32_t last_active = -1;      // experts activated at the layer's previous execution (-1: none yet)
   const uint8_t* host_blob = nullptr;
   size_t host_stride = 0;
   uint16_t* w_router = nullptr;  // device [E,H]
@@ -74,6 +75,7 @@ struct oled_ctx {
     uint16_t* x_next = nullptr;
     uint32_t* ctrl = nullptr;      // the control block that step used (to be cleared)
   } pending;
+  int fuse_ffn = 1;            // OLED_OPT_FUSE_FFN: 0 never, 1 where few items per SM are expected, 2 wherever possible
   bool fuse_combine = true;    // stack iterations of few-token steps: a layer's combine runs inside the
                                // next layer's gate kernel (OLED_OPT_FUSE_COMBINE)
   int32_t* d_offsets = nullptr;// [E+1]
@@ -83,7 +85,8 @@ struct oled_ctx {
   uint16_t* d_hbuf = nullptr;  // [T*k,I]
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
-  uint32_t* d_work = nullptr;         // control block, last: work-item counters of the step's FFN launches
+  uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
+  uint32_t* d_done = nullptr;         // control block, last: [kFfnWorkCounters][E] completion counters of fused FFN launches
   int work_next = 0;                  // next unused counter of the current layer execution
   bool ctrl_dirty = true;             // both control blocks must be cleared before the next gate launch
   unsigned int seq = 0;               // step sequence number echoed by the gate kernel
@@ -109,6 +112,7 @@ struct oled_ctx {
   bool timeline_on = false;    // OLED_OPT_TIMELINE
   StepTimeline* d_timeline = nullptr;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
+  bool hit_fused = false;      // this step's resident-group FFN ran as one fused launch
   int miss_chunk = 4;
   bool split_last = true;      // the step's last blob is copied in two parts (gate|up first, down after)
   int withhold_loads = 0;      // test aid, see OLED_OPT_TEST_WITHHOLD_LOADS
@@ -145,6 +149,7 @@ void select_ctrl(oled_ctx* ctx, int sel) {
   ctx->d_scores = reinterpret_cast<unsigned long long*>(b);
   ctx->d_counts = reinterpret_cast<int32_t*>(b + E * sizeof(unsigned long long));
   ctx->d_work = reinterpret_cast<uint32_t*>(b + E * (sizeof(unsigned long long) + sizeof(int32_t)));
+  ctx->d_done = ctx->d_work + kFfnWorkCounters;
 }
 
 template <typename T>
@@ -322,23 +327,33 @@ void prof_add(oled_ctx* ctx, int kernel, uint64_t bytes, uint64_t flops) {
 
 // Algorithmic bytes / flops of the two FFN kernels for n experts with `rows` token rows in total:
 // each expert's weights once, the token rows in, the result rows out.
-void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows) {
+void prof_add_ffn(oled_ctx* ctx, uint64_t n, uint64_t rows, bool fused) {
   const uint64_t H = ctx->shape.hidden, I = ctx->shape.intermediate, hi = H * I;
   const bool fp8 = ctx->shape.expert_format == OLED_EXPERTS_FP8;
   // weight bytes of one expert per kernel: bf16 elements, or e4m3 codes plus the fp32 row scales
   const uint64_t w13 = fp8 ? 2 * hi + 2 * I * 4 : 2 * hi * 2, w2 = fp8 ? hi + H * 4 : hi * 2;
-  prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, n * w13 + rows * H * 2 + rows * I * 2, 4 * rows * hi);
-  prof_add(ctx, OLED_KERNEL_FFN_DOWN, n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4), 2 * rows * hi);
+  const uint64_t b1 = n * w13 + rows * H * 2 + rows * I * 2, b2 = n * w2 + rows * I * 2 + rows * H * (ctx->y_bf16 ? 2 : 4);
+  if (fused) {
+    prof_add(ctx, OLED_KERNEL_FFN_FUSED, b1 + b2, 6 * rows * hi);
+  } else {
+    prof_add(ctx, OLED_KERNEL_FFN_GATE_UP, b1, 4 * rows * hi);
+    prof_add(ctx, OLED_KERNEL_FFN_DOWN, b2, 2 * rows * hi);
+  }
 }
 
-// The two FFN launches over one group.  host_counts == nullptr: the per-expert counts are not
+// The FFN launches over one group: gate/up and down projection, or ONE fused launch where that
+// form exists (bf16 stores, token tiles of at most 32 rows, no event to wait for between the two
+// projections) and few items per SM are expected (expected_experts: how many of the group's
+// experts are expected to have tokens).  host_counts == nullptr: the per-expert counts are not
 // known on the host yet (the group is the resident set and experts without tokens cost nothing).
 // before_down: an event the down projection (and nothing before it) has to wait for, or null.
 // behind_event_wait: the caller has just enqueued a cudaStreamWaitEvent on the stream.
-// report: the step's report to the host, sent by the gate/up launch (the plain-FMA bring-up path
+// report: the step's report to the host, sent by the first launch (the plain-FMA bring-up path
 // and an empty group send it from a kernel of its own).
 int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const int32_t* host_counts,
-                     cudaEvent_t before_down, bool behind_event_wait, const RouteReport& report = RouteReport{}) {
+                     cudaEvent_t before_down, bool behind_event_wait, int expected_experts, bool* fused_out,
+                     const RouteReport& report = RouteReport{}) {
+  if (fused_out) *fused_out = false;
   if ((grp.n <= 0 || max_count <= 0 || ctx->ffn_impl == 1) && report.host_scores != nullptr) {
     launch_report(ctx->stream, report);
     ctx->launches += 1;
@@ -349,24 +364,37 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
     if (before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
                       ctx->d_y, H, I);
+    ctx->launches += 2;
   } else {
-    for (int kind = 1; kind <= 2; ++kind) {
+    // With many items per SM the two-kernel form is a little faster (the down projection's early
+    // start hides the boundary; measured 125 against 129 us for 63 experts); with few, the SMs
+    // that run out of gate/up items would idle until the whole gate/up launch has finished.
+    const bool few_items = (long long)expected_experts * (I / 64) < 4ll * ctx->n_sms;
+    const bool fuse = before_down == nullptr && !ctx->y_bf16 && ffn_tc_can_fuse(ctx->maps, max_count) &&
+                      (ctx->fuse_ffn == 2 || (ctx->fuse_ffn == 1 && few_items));
+    for (int kind = fuse ? 3 : 1; kind <= (fuse ? 3 : 2); ++kind) {
       if (kind == 2 && before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
-      ProfScope ps(ctx, kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
-      // a fresh (zero) work counter per launch; a layer execution has at most three launch pairs,
-      // should there ever be more, a used word is cleared in stream order and taken again
+      ProfScope ps(ctx, kind == 3 ? OLED_KERNEL_FFN_FUSED : kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);
+      // a fresh (zero) work counter and, for a fused launch, a fresh row of completion counters
+      // per launch; a layer execution has at most three launch pairs, should there ever be more,
+      // used words are cleared in stream order and taken again
       const int li = ctx->work_next % kFfnWorkCounters;
       uint32_t* work = ctx->d_work + li;
-      if (ctx->work_next >= kFfnWorkCounters) OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
+      uint32_t* done = ctx->d_done + (size_t)li * ctx->shape.n_experts;
+      if (ctx->work_next >= kFfnWorkCounters) {
+        OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
+        OLED_CUDA(ctx, cudaMemsetAsync(done, 0, (size_t)ctx->shape.n_experts * sizeof(uint32_t), ctx->stream));
+      }
       ctx->work_next += 1;
       const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
                                    ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work,
                                    behind_event_wait || (kind == 2 && before_down != nullptr),
-                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li, report);
+                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li, report, done);
       if (rc != OLED_OK) return rc;
+      ctx->launches += 1;
     }
+    if (fused_out) *fused_out = fuse;
   }
-  ctx->launches += 2;
   OLED_CUDA(ctx, cudaGetLastError());
   return OLED_OK;
 }
@@ -389,8 +417,10 @@ int run_ffn_group(oled_ctx* ctx, LayerData& L, const std::vector<int32_t>& exper
     max_count = std::max(max_count, counts[e]);
     rows += (uint64_t)counts[e];
   }
-  prof_add_ffn(ctx, (uint64_t)grp.n, rows);
-  return run_ffn_launches(ctx, grp, max_count, counts, before_down, behind_event_wait);
+  bool fused = false;
+  const int rc = run_ffn_launches(ctx, grp, max_count, counts, before_down, behind_event_wait, grp.n, &fused);
+  prof_add_ffn(ctx, (uint64_t)grp.n, rows, fused);
+  return rc;
 }
 
 // Blocks until the gate kernel of step `seq` has published counts and scores, and decodes them.
@@ -508,7 +538,8 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
-  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + kFfnWorkCounters * sizeof(uint32_t);
+  ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + kFfnWorkCounters * sizeof(uint32_t) +
+                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t);
   ctx->ctrl_bytes = (ctx->ctrl_bytes + 15) / 16 * 16;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_ctrl[0], 2 * ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
@@ -734,7 +765,11 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     // has its weights streamed once per tile, and in a block of 32 tokens whose routing is
     // concentrated on few experts (the regime the paper reports) counts of 17..32 are common
     const int mean_load = (int)(((size_t)T * K + E - 1) / E);
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(32, 2 * mean_load)), nullptr, nullptr, false, rep);
+    // (how many of the residents will have tokens is not known yet: the layer's previous
+    // execution is the estimate - adjacent iterations activate mostly the same experts, Sec. 3.3)
+    const int expected = std::min<int>(grp.n, L.last_active >= 0 ? L.last_active : E);
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(32, 2 * mean_load)), nullptr, nullptr, false,
+                                     expected, &ctx->hit_fused, rep);
     if (rc0 != OLED_OK) return rc0;
   }
 
@@ -814,7 +849,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   {
     uint64_t hit_rows = 0;
     for (int32_t e : plan.hits) hit_rows += (uint64_t)counts[e];
-    prof_add_ffn(ctx, plan.hits.size(), hit_rows);
+    prof_add_ffn(ctx, plan.hits.size(), hit_rows, ctx->hit_fused);
   }
   int rc = OLED_OK;
   for (size_t c = 0; c < n_groups; ++c) {
@@ -863,6 +898,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.stats.bytes_moved += (uint64_t)n_miss * ctx->slot_bytes;
   L.stats.evictions += (uint64_t)plan.n_evictions;
   L.stats.active_experts += (uint64_t)plan.n_active;
+  L.last_active = plan.n_active;
   L.stats.assignments += (uint64_t)T * K;
   L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
   L.stats.ideal_hits += (uint64_t)std::min<int64_t>(plan.n_active, plan.capacity_used);
@@ -1091,6 +1127,10 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       return OLED_OK;
     case OLED_OPT_SPLIT_LAST_FILL:
       ctx->split_last = value != 0;
+      return OLED_OK;
+    case OLED_OPT_FUSE_FFN:
+      if (value < 0 || value > 2) return OLED_ERR_INVALID_ARG;
+      ctx->fuse_ffn = (int)value;
       return OLED_OK;
     case OLED_OPT_FUSE_COMBINE:
       ctx->fuse_combine = value != 0;

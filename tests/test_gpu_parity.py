@@ -571,3 +571,34 @@ def test_fp8_subnormal_codes_decode_exactly():
         _check_step(run, 0, 24, out, ref)
     finally:
         run.close()
+
+
+def test_one_launch_and_two_launch_ffn_forms_agree_bit_for_bit():
+    """OLED_OPT_FUSE_FFN: gate/up + down projection as one launch (down items wait on per-expert
+    completion counters) or as two launches.  Which kernel computes an item does not change its
+    arithmetic, so the layer outputs must be bit-identical, and both in parity with the oracle;
+    block sizes with one and with two token tiles per expert, cold start so that launches of
+    fetched experts (behind event waits) are covered too."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1, n_experts=6, top_k=3, hidden=512, intermediate=256)
+    outs = {}
+    for mode in (0, 2):
+        run = _runner(w, capacity=[3], max_tokens=160)
+        run.ctx.set_option(binding.OPT_FUSE_FFN, mode)
+        ora = _oracle_for(run, [3])
+        try:
+            res = []
+            for rep, n in enumerate((7, 33, 60, 150)):      # 150 tokens: 64-row tiles, always two launches
+                h_bits, conf = synth.flat_tokens(w, n, 80 + rep)
+                x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+                out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+                run.step(0, x, c, out)
+                _check_step(run, 0, n, out, ora.denoise_step(0, h_bits, conf))
+                res.append(dev_to_bits(out).copy())
+            outs[mode] = res
+            _check_stats(run, ora)
+        finally:
+            run.close()
+    for a, b in zip(outs[0], outs[2]):
+        assert np.array_equal(a, b)
