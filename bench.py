@@ -37,9 +37,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captured launch).  Traffic grows in proportion to the experts (few-token regime) or token rows
 # (many-token regime) a launch processes, so the ratio scales a capture to any launch.
 NCU_TRAFFIC_RATIO = {
-    # profiles/ffn_tc_kernel_cfg2_full_residency.md: 63 experts x 4 tokens, H 2048, I 1024
-    ("ffn_gate_up", "few_tokens"): (529.62 + 5.63) / 530.1,
-    ("ffn_down", "few_tokens"): (264.86 + 5.34) / 267.0,
+    # profiles/ffn_tc_kernel_cfg2_full_residency.md: 60 experts x 4 tokens, H 2048, I 1024
+    ("ffn_gate_up", "few_tokens"): (504.42 + 4.48) / 504.9,
+    ("ffn_down", "few_tokens"): (252.23 + 7.01) / 254.4,
+    # the one-launch form runs the same items as those two kernels together
+    ("ffn_fused", "few_tokens"): (504.42 + 4.48 + 252.23 + 7.01) / (504.9 + 254.4),
     # profiles/ffn_tc_kernel_fp8_cfg2_full_residency.md: the same launch with fp8 stores
     ("ffn_gate_up", "few_tokens", "fp8"): (265.88 + 4.06) / 266.6,
     ("ffn_down", "few_tokens", "fp8"): (133.23 + 4.07) / 135.2,
