@@ -102,13 +102,21 @@ __device__ __forceinline__ void route_token_tail(const float* row, int t, int la
 // layer for its own token (paper Sec. 2.1: the MoE output is the gate-score-weighted sum over the
 // top-k experts; the stack adds it to the layer's input).  Arithmetic and order are those of
 // combine_kernel: fp32 fused multiply-adds in rank order, out = bf16(sum), x = bf16(x_prev + out).
-__device__ __forceinline__ void combine_row(const CombinePrev& p, int t, int H, uint16_t* s_x, float* s_g, int* s_r) {
+// n_rows tokens t0 .. t0 + n_rows - 1; their rows end up in s_x[row][H] as well.
+__device__ __forceinline__ void combine_rows(const CombinePrev& p, int t0, int n_rows, int H, uint16_t* s_x_all,
+                                             float* s_g_all, int* s_r_all) {
   const int K = p.K;
-  if (threadIdx.x < K) {
-    s_g[threadIdx.x] = p.gate[(size_t)t * K + threadIdx.x];
-    s_r[threadIdx.x] = p.pos[(size_t)t * K + threadIdx.x];
+  // the small operands of all rows first (one round trip), then row after row
+  for (int i = threadIdx.x; i < n_rows * K; i += blockDim.x) {
+    s_g_all[i] = p.gate[(size_t)t0 * K + i];
+    s_r_all[i] = p.pos[(size_t)t0 * K + i];
   }
   __syncthreads();
+  for (int row = 0; row < n_rows; ++row) {
+  const int t = t0 + row;
+  const float* s_g = s_g_all + row * K;
+  const int* s_r = s_r_all + row * K;
+  uint16_t* s_x = s_x_all + (size_t)row * H;
   for (int h = threadIdx.x * 4; h < H; h += blockDim.x * 4) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint2 xv = *reinterpret_cast<const uint2*>(p.x + (size_t)t * H + h);
@@ -144,16 +152,19 @@ __device__ __forceinline__ void combine_row(const CombinePrev& p, int t, int H, 
     *reinterpret_cast<uint2*>(p.x_next + (size_t)t * H + h) = rk;
     *reinterpret_cast<uint2*>(s_x + h) = rk;
   }
+  }
 }
 
 // TT tokens per CTA, WARPS warps; each warp owns kEPerWarp experts per pass and all TT tokens.  Small
 // blocks use TT = 1 with 16 warps (one pass covers 64 experts) and keep several 256-wide
 // chunks of loads in flight; the chain order of every logit is the same in all variants.
-// TT = 1 only: the token's row is staged in shared memory - copied from x, or produced by the
-// previous layer's combine (prev.y != nullptr), which this kernel then carries out for its token -
-// and the top-k is a rank computation spread over all warps: expert e is selected iff fewer than K
-// experts precede it in the order (logit descending, index ascending), and its rank is the number
-// that do - the same total order a round-by-round selection walks.
+// TT <= 4 (few-token steps): the tokens' rows are staged in shared memory - copied from x, or
+// produced by the previous layer's combine (prev.y != nullptr), which this kernel then carries
+// out for its tokens - and the top-k is a rank computation spread over all warps: expert e is
+// selected iff fewer than K experts precede it in the order (logit descending, index ascending),
+// and its rank is the number that do - the same total order a round-by-round selection walks.
+// One token per CTA while that gives at most one wave of CTAs; two or four beyond (every CTA
+// streams the whole router matrix, so a second wave costs as much as the first).
 // The kernel reports nothing to the host: the permutation kernel, which follows it in every step,
 // publishes the finished counts and scores without any ticket or fence.
 template <int TT, int WARPS, int UNROLL, int kEPerWarp>
@@ -165,18 +176,21 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
              unsigned long long* __restrict__ scores, CombinePrev prev, StepTimeline* timeline) {
   extern __shared__ __align__(16) uint8_t s_dyn[];
   float* s_logits = reinterpret_cast<float*>(s_dyn);                       // [TT][E]
-  // [H] (TT == 1 only), on a 16-byte boundary: the row is moved with 16-byte vector accesses
+  constexpr bool staged = TT <= 4;
+  constexpr int kST = staged ? TT : 1;
+  // [TT][H] (staged forms only), on a 16-byte boundary: rows are moved with 16-byte vector accesses
   uint16_t* s_x = reinterpret_cast<uint16_t*>(s_dyn + (((size_t)TT * E * 4 + 15) & ~(size_t)15));
-  __shared__ int s_sel_id[OLED_MAX_TOPK];
-  __shared__ float s_sel_logit[OLED_MAX_TOPK];
-  __shared__ float s_g[OLED_MAX_TOPK];
-  __shared__ int s_r[OLED_MAX_TOPK];
+  __shared__ int s_sel_id[kST][OLED_MAX_TOPK];
+  __shared__ float s_sel_logit[kST][OLED_MAX_TOPK];
+  __shared__ float s_g[kST * OLED_MAX_TOPK];
+  __shared__ int s_r[kST * OLED_MAX_TOPK];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t0 = blockIdx.x * TT;
   griddep_launch_dependents();
   if (threadIdx.x == 0) timeline_entry(timeline, 0);
   constexpr int kRouteWarps = WARPS;
-  if (TT == 1 && gridDim.x <= 128) {
+  const int my_tokens = min(TT, T - t0);
+  if (staged && gridDim.x <= 148) {
     // Small steps: the router weights do not depend on the predecessor (the previous layer's
     // expert FFN), but the expert weights streamed since their last use have pushed them out of
     // L2 - so they are called back in while this kernel still waits for its input.
@@ -190,14 +204,14 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   }
   griddep_wait();
   if (threadIdx.x == 0) timeline_start(timeline, 0);
-  if (TT == 1) {
+  if (staged) {
     if (prev.y != nullptr) {
       // CTA 0 also clears the control block the previous step used (its kernels have completed)
       if (blockIdx.x == 0 && prev.zero_words != nullptr)
         for (int i = threadIdx.x; i < prev.n_zero_words; i += blockDim.x) prev.zero_words[i] = 0u;
-      combine_row(prev, t0, H, s_x, s_g, s_r);
+      combine_rows(prev, t0, my_tokens, H, s_x, s_g, s_r);
     } else {
-      for (int c = threadIdx.x; c < H / 8; c += blockDim.x)
+      for (int c = threadIdx.x; c < my_tokens * (H / 8); c += blockDim.x)
         reinterpret_cast<uint4*>(s_x)[c] = reinterpret_cast<const uint4*>(x + (size_t)t0 * H)[c];
     }
     __syncthreads();
@@ -217,8 +231,9 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 #pragma unroll
       for (int a = 0; a < TT; ++a) {
         const int t = min(t0 + a, T - 1);
-        const uint4 v = TT == 1 ? *reinterpret_cast<const uint4*>(s_x + h)
-                                : *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
+        // (staged rows beyond the step's last token hold stale shared memory: their logits are never used)
+        const uint4 v = staged ? *reinterpret_cast<const uint4*>(s_x + (size_t)a * H + h)
+                               : *reinterpret_cast<const uint4*>(x + (size_t)t * H + h);
         xw[a][0] = v.x; xw[a][1] = v.y; xw[a][2] = v.z; xw[a][3] = v.w;
       }
 #pragma unroll
@@ -266,27 +281,30 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   }
   __syncthreads();
 
-  if (TT == 1) {
-    // top-k by rank, all warps; then warp 0: gate scores, counts and reuse-score numerators
-    for (int e = warp; e < E; e += kRouteWarps) {
-      const float ve = topk_value(s_logits[e]);
+  if (staged) {
+    // top-k by rank, work items (token, expert) over all warps; then one warp per token: gate
+    // scores, counts and reuse-score numerators
+    for (int w = warp; w < my_tokens * E; w += kRouteWarps) {
+      const int a = w / E, e = w - a * E;
+      const float* row = s_logits + a * E;
+      const float ve = topk_value(row[e]);
       const uint32_t ke = order_key(ve);
       int before = 0;
       for (int o = lane; o < E; o += 32) {
-        const uint32_t ko = order_key(topk_value(s_logits[o]));
+        const uint32_t ko = order_key(topk_value(row[o]));
         before += (ko > ke || (ko == ke && o < e)) ? 1 : 0;
       }
       before = __reduce_add_sync(0xffffffffu, before);
       if (lane == 0 && before < K) {
-        s_sel_id[before] = e;
-        s_sel_logit[before] = ve;
+        s_sel_id[a][before] = e;
+        s_sel_logit[a][before] = ve;
       }
     }
     __syncthreads();
-    if (warp == 0) {
-      const int t = t0;
-      const int my_id = lane < K ? s_sel_id[lane] : 0;
-      const float my_logit = lane < K ? s_sel_logit[lane] : 0.0f;
+    for (int a = warp; a < my_tokens; a += kRouteWarps) {
+      const int t = t0 + a;
+      const int my_id = lane < K ? s_sel_id[a][lane] : 0;
+      const float my_logit = lane < K ? s_sel_logit[a][lane] : 0.0f;
       const float top = __shfl_sync(0xffffffffu, my_logit, 0);
       const float z = lane < K ? exp_spec(__fsub_rn(my_logit, top)) : 0.0f;
       float sum = __shfl_sync(0xffffffffu, z, 0);
@@ -472,15 +490,25 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
                   float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
                   StepTimeline* timeline) {
   if (T <= kRouteSmallMax) {
-    constexpr int TT = 1, W = 16;
+    constexpr int W = 16;
     static bool attr_done = false;
-    if (!attr_done) {  // the staged row: H up to 16 K elements
-      cudaFuncSetAttribute(route_kernel<TT, W, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    if (!attr_done) {  // the staged rows: up to 4 x 16 K elements
+      cudaFuncSetAttribute(route_kernel<1, W, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+      cudaFuncSetAttribute(route_kernel<2, W, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+      cudaFuncSetAttribute(route_kernel<4, W, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
       cudaGetLastError();
       attr_done = true;
     }
-    launch_pdl(route_kernel<TT, W, 4, 4>, dim3(T), dim3(W * 32), (((size_t)E * sizeof(float) + 15) & ~(size_t)15) + (size_t)H * 2, st, x,
-               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, prev, timeline);
+    auto smem = [&](int tt) { return ((((size_t)tt * E * sizeof(float)) + 15) & ~(size_t)15) + (size_t)tt * H * 2; };
+    if (T <= 148)
+      launch_pdl(route_kernel<1, W, 4, 4>, dim3(T), dim3(W * 32), smem(1), st, x, w_router, bias, conf, T, H, E, K,
+                 logits, ids, gate, counts, scores, prev, timeline);
+    else if (T <= 296)  // (four tokens per CTA measured slower at 256 tokens x 128 experts: 33 against 20 us)
+      launch_pdl(route_kernel<2, W, 4, 4>, dim3((T + 1) / 2), dim3(W * 32), smem(2), st, x, w_router, bias, conf, T, H,
+                 E, K, logits, ids, gate, counts, scores, prev, timeline);
+    else
+      launch_pdl(route_kernel<4, W, 2, 4>, dim3((T + 3) / 4), dim3(W * 32), smem(4), st, x, w_router, bias, conf, T, H,
+                 E, K, logits, ids, gate, counts, scores, prev, timeline);
   } else {
     // (tilings with more tokens or experts per warp, more warps per CTA or deeper unrolling were
     // measured at 4096 tokens x 64 experts x 4096: all slower - they cost occupancy)
