@@ -328,6 +328,156 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
   if (threadIdx.x == 0) timeline_end(timeline, 0);
 }
 
+// Many-token steps: TT tokens per CTA, eight warps, every warp a register tile of TT tokens x 8
+// experts.  The plain kernel above re-reads the router matrix once per eight tokens through the L1
+// path and spends an ALU instruction on every bf16 -> fp32 conversion; it reaches a third of the
+// FP32 pipe.  Here
+//  - the operands are staged in shared memory by cp.async, a ring of k-chunks of 256 elements (the
+//    TT token rows and 64 router rows of a chunk), so that the warps read only shared memory
+//    (conflict-free 16-byte reads) and the global loads of later chunks are always in flight;
+//  - the multiply-adds take their bf16 operands directly (fma.rn.f32.bf16: exact product, one
+//    rounding - bit for bit the fp32 fused multiply-add of the converted operands), which removes
+//    the conversions;
+//  - TT is chosen by the launcher so that the CTAs fill whole waves of SMs (4096 tokens: 14 per
+//    CTA, 293 CTAs, two waves on 148 SMs), and a larger TT re-reads the router matrix less often.
+// Same chains, same order: lane q still owns the elements h with (h/8) mod 32 == q and walks them
+// in ascending order.  Experts beyond 64 take further passes over the rows.
+constexpr int kManyWarps = 8, kManyExperts = 64, kManyStages = 4;
+__host__ __device__ constexpr int many_stage_bytes(int tt) { return (tt + kManyExperts) * 512; }  // one k-chunk of 256 bf16 per row
+
+// acc += x.lo * w.lo, then acc += x.hi * w.hi (ascending h), each an fp32 fused multiply-add
+__device__ __forceinline__ void fma_bf16_pair(float& acc, uint32_t x, uint32_t w) {
+  asm("{\n .reg .b16 xl, xh, wl, wh;\n mov.b32 {xl, xh}, %1;\n mov.b32 {wl, wh}, %2;\n"
+      " fma.rn.f32.bf16 %0, xl, wl, %0;\n fma.rn.f32.bf16 %0, xh, wh, %0;\n}"
+      : "+f"(acc)
+      : "r"(x), "r"(w));
+}
+
+template <int TT>
+__global__ void __launch_bounds__(kManyWarps * 32, 1)
+route_many_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
+                  const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
+                  int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
+                  float* __restrict__ gate, int32_t* __restrict__ counts,
+                  unsigned long long* __restrict__ scores, StepTimeline* timeline) {
+  constexpr int kStageBytes = many_stage_bytes(TT);
+  constexpr int kRows = TT + kManyExperts;
+  extern __shared__ __align__(16) uint8_t s_dyn[];
+  uint8_t* s_ring = s_dyn;                                                        // [stages][TT + 64 rows][512 B]
+  float* s_logits = reinterpret_cast<float*>(s_dyn + kManyStages * kStageBytes);  // [TT][E]
+  __shared__ const uint16_t* s_rowptr[kRows];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = blockIdx.x * TT;
+  griddep_launch_dependents();
+  if (threadIdx.x == 0) timeline_entry(timeline, 0);
+  griddep_wait();
+  if (threadIdx.x == 0) timeline_start(timeline, 0);
+  const int n_chunks = H / 256;
+  const uint32_t ring_base = (uint32_t)__cvta_generic_to_shared(s_ring);
+
+  for (int e0 = 0; e0 < E; e0 += kManyExperts) {
+    // one stage: rows 0..TT-1 = tokens t0.., rows TT.. = experts e0..; each row 32 pieces of 16 bytes.
+    // The rows' addresses are looked up in a table (one 8-byte read instead of a clamp and a 64-bit
+    // multiply per copy: the copies' own instructions are a tenth of the loop otherwise).
+    __syncthreads();  // the previous pass has finished with the ring and the table
+    for (int row = threadIdx.x; row < kRows; row += kManyWarps * 32)
+      s_rowptr[row] = row < TT ? x + (size_t)min(t0 + row, T - 1) * H
+                               : wr + (size_t)min(e0 + row - TT, E - 1) * H;
+    auto issue = [&](int chunk) {
+      const uint32_t dst0 = ring_base + (uint32_t)(chunk % kManyStages) * kStageBytes + (uint32_t)lane * 16u;
+#pragma unroll
+      for (int j = 0; j < (kRows + kManyWarps - 1) / kManyWarps; ++j) {
+        const int row = warp + j * kManyWarps;
+        if (row < kRows)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (uint32_t)row * 512u),
+                       "l"(s_rowptr[row] + (size_t)chunk * 256 + lane * 8)
+                       : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float acc[TT][8];
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < 8; ++b) acc[a][b] = 0.0f;
+    __syncthreads();  // the table is complete
+    for (int c = 0; c < kManyStages - 1; ++c) {
+      if (c < n_chunks) issue(c);
+      else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+      asm volatile("cp.async.wait_group %0;" ::"n"(kManyStages - 2) : "memory");  // chunk c has landed (this thread's part)
+      __syncthreads();                                                            // ... everyone's; and chunk c-1 is consumed
+      if (c + kManyStages - 1 < n_chunks) issue(c + kManyStages - 1);
+      else asm volatile("cp.async.commit_group;" ::: "memory");
+      const uint8_t* st = s_ring + (size_t)(c % kManyStages) * kStageBytes;
+      uint4 xw[TT], ww[8];
+#pragma unroll
+      for (int a = 0; a < TT; ++a) xw[a] = *reinterpret_cast<const uint4*>(st + a * 512 + lane * 16);
+#pragma unroll
+      for (int b = 0; b < 8; ++b) ww[b] = *reinterpret_cast<const uint4*>(st + (TT + warp * 8 + b) * 512 + lane * 16);
+      // elements in ascending h: word 0 low half, word 0 high half, word 1 low half, ...
+#pragma unroll
+      for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) fma_bf16_pair(acc[a][b], xw[a].x, ww[b].x);
+#pragma unroll
+      for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) fma_bf16_pair(acc[a][b], xw[a].y, ww[b].y);
+#pragma unroll
+      for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) fma_bf16_pair(acc[a][b], xw[a].z, ww[b].z);
+#pragma unroll
+      for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) fma_bf16_pair(acc[a][b], xw[a].w, ww[b].w);
+    }
+    // The 32 partial sums of every (token, expert) pair are added in the order of the xor butterfly
+    // (offsets 16, 8, 4, 2, 1; at every step a lane adds its partner's value to its own).  Addition
+    // is commutative bit for bit, so every lane of the butterfly ends with the same value, and the
+    // 32 pairs of a group can share the steps: at offset d a lane keeps the half of its pairs
+    // whose index has bit d equal to its own lane's bit and hands the other half to its partner -
+    // 31 shuffles per 32 pairs instead of 160, and lane l ends with the sum of pair l.
+#pragma unroll
+    for (int g = 0; g < (TT * 8 + 31) / 32; ++g) {
+      float v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int p = g * 32 + i;  // pair p: token p / 8, expert column p % 8
+        v[i] = p < TT * 8 ? acc[p / 8][p % 8] : 0.0f;
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        const bool upper = (lane & d) != 0;
+#pragma unroll
+        for (int i = 0; i < d; ++i) {
+          const float keep = upper ? v[i + d] : v[i];
+          const float send = upper ? v[i] : v[i + d];
+          v[i] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, d));
+        }
+      }
+      const int p = g * 32 + lane, a = p / 8, e = e0 + warp * 8 + p % 8;
+      if (p < TT * 8 && e < E && t0 + a < T) {
+        float r = v[0];
+        if (bias != nullptr) r = __fadd_rn(r, bias[e]);
+        s_logits[a * E + e] = r;
+        if (logits_out != nullptr) logits_out[(size_t)(t0 + a) * E + e] = r;
+      }
+    }
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  // one warp per token
+  for (int a = warp; a < TT; a += kManyWarps) {
+    const int t = t0 + a;
+    if (t >= T) continue;
+    route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores);
+  }
+  if (threadIdx.x == 0) timeline_end(timeline, 0);
+}
+
 // One CTA per expert (blockIdx.x): offset = sum of the counts before it; then a stable scan of the
 // flat assignment list (ascending t*K+j) hands out consecutive sorted rows.
 // If xp != nullptr the expert's CTAs (gridDim.y of them) also copy its token rows into sorted
@@ -510,11 +660,39 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
       launch_pdl(route_kernel<4, W, 2, 4>, dim3((T + 3) / 4), dim3(W * 32), smem(4), st, x, w_router, bias, conf, T, H,
                  E, K, logits, ids, gate, counts, scores, prev, timeline);
   } else {
-    // (tilings with more tokens or experts per warp, more warps per CTA or deeper unrolling were
-    // measured at 4096 tokens x 64 experts x 4096: all slower - they cost occupancy)
-    constexpr int TT = 8, W = 8;
-    launch_pdl(route_kernel<TT, W, 1, 4>, dim3((T + TT - 1) / TT), dim3(W * 32), (size_t)TT * E * sizeof(float), st, x,
-               w_router, bias, conf, T, H, E, K, logits, ids, gate, counts, scores, CombinePrev{}, timeline);
+    // (re-tilings of the plain kernel - more tokens or experts per warp, more warps per CTA, deeper
+    // unrolling - were all slower at 4096 tokens x 64 experts x 4096)
+    // tokens per CTA: the time is (waves of CTAs) x (tokens per CTA); ties go to the larger tile,
+    // which reads the router matrix less often
+    static int n_sms = 0;
+    if (n_sms == 0) {
+      int dev = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+      if (n_sms <= 0) n_sms = 148;
+    }
+    int best_tt = 8;
+    long best_cost = -1;
+    for (int tt : {8, 10, 12, 14}) {
+      const int ctas = (T + tt - 1) / tt;
+      const long cost = (long)((ctas + n_sms - 1) / n_sms) * tt;
+      if (best_cost < 0 || cost <= best_cost) {
+        best_cost = cost;
+        best_tt = tt;
+      }
+    }
+    auto go = [&](auto kernel, int tt) {
+      const size_t smem = (size_t)kManyStages * many_stage_bytes(tt) + (size_t)tt * E * sizeof(float);
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+      launch_pdl(kernel, dim3((T + tt - 1) / tt), dim3(kManyWarps * 32), smem, st, x, w_router, bias, conf, T, H, E,
+                 K, logits, ids, gate, counts, scores, timeline);
+    };
+    switch (best_tt) {
+      case 8: go(route_many_kernel<8>, 8); break;
+      case 10: go(route_many_kernel<10>, 10); break;
+      case 12: go(route_many_kernel<12>, 12); break;
+      default: go(route_many_kernel<14>, 14); break;
+    }
   }
 }
 
