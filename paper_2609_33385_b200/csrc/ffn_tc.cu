@@ -47,11 +47,13 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 
 #include <algorithm>
 #include <cstddef>
 #include <cstdlib>
 
+#include "fp8_split.h"
 #include "kernels.h"
 #include "sm100_ptx.h"
 
@@ -187,7 +189,7 @@ struct FusedSecond {
 // with few items per SM - which is where this form pays: the two-kernel form leaves every SM that
 // runs out of gate/up items idle until the last gate/up item of the whole launch is done, this
 // one lets it go on with the down projection of experts that are already complete.
-template <int KIND, bool DUAL, bool FP8>
+template <int KIND, bool DUAL, int FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
               const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
@@ -195,7 +197,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
               const uint8_t* __restrict__ pool, unsigned long long slot_bytes,
               uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter, StepTimeline* timeline,
               int timeline_slot, const __grid_constant__ RouteReport report,
-              const __grid_constant__ FusedSecond fs) {
+              const __grid_constant__ FusedSecond fs, const uint32_t* __restrict__ amax_in,
+              uint32_t* __restrict__ amax_out) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;
@@ -204,6 +207,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   const int n_box = grp.n_box;
   constexpr bool fused = KIND == 3;
   static_assert(!(fused && (DUAL || FP8)), "the fused form exists for bf16 stores and single tiles only");
+  constexpr bool WIDEN = FP8 == 1;   // fp8 stores, codes widened to bf16 by converter warps
+  constexpr bool DIRECT = FP8 == 2;  // fp8 stores, codes read by the MMA as they are (see the header comment)
+  static_assert(!(DIRECT && DUAL), "the direct fp8 form exists for single 128-row tiles only");
+  constexpr int kK = DIRECT ? 128 : kBlockK;  // k-values of a k-block (one 128-byte swizzle atom of weights)
   constexpr int kind1 = fused ? 1 : KIND;  // kind of the launch's first-phase (or only) items
   constexpr bool dual = DUAL;
   constexpr bool stacked = (KIND == 1 && !DUAL) || fused;  // gate/up items: 64 gate + 64 up rows in one 128-row tile
@@ -216,17 +223,20 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // A stage spans k_atoms (1 or 2) k-blocks of 64, laid out one after the other, each as
   // described above: small token tiles take two, which halves the waits and commits per byte on
   // the serial path of the MMA thread.
-  constexpr uint32_t raw_bytes = FP8 ? a_bytes / 2 : 0u;
-  const uint32_t atom_bytes = FP8 ? raw_bytes + b_bytes : a_bytes + b_bytes;  // one k-block in shared memory
+  // direct fp8 form: a stage is the code tile of a k-block of 128 (16 KB) and the two e4m3 term
+  // tiles of the tokens (2 n_box rows of 128 bytes, term 2 behind term 1) - the MMA's B operand.
+  constexpr uint32_t raw_bytes = WIDEN ? a_bytes / 2 : 0u;
+  const uint32_t atom_bytes = DIRECT ? kATile + 2u * b_bytes
+                              : WIDEN ? raw_bytes + b_bytes : a_bytes + b_bytes;  // one k-block in shared memory
   const uint32_t stage_bytes = (uint32_t)k_atoms * atom_bytes;
   constexpr uint32_t atom_cols = dual ? 64u : 32u;  // 64 k-values of one (two) 128-row tile(s), two per column
   const uint32_t a_cols = (uint32_t)k_atoms * atom_cols;
-  const int k_blocks1 = (kind1 == 1 ? H : I) / (kBlockK * k_atoms);  // stages per (first-phase) item
-  const int k_blocks2 = I / (kBlockK * k_atoms);                    // stages per down item of a fused launch
+  const int k_blocks1 = (kind1 == 1 ? H : I) / (kK * k_atoms);  // stages per (first-phase) item
+  const int k_blocks2 = I / (kK * k_atoms);                    // stages per down item of a fused launch
   constexpr int m_rows = (KIND == 2 && dual) ? 2 * kBlockM : stacked ? kBlockM / 2 : kBlockM;  // output features per item
   const int m_tiles = (kind1 == 1 ? I : H) / m_rows;
-  const int acc_cols = (dual ? 2 : 1) * n_box;
-  const int a_total = FP8 ? n_stages * (int)a_cols : 0;
+  const int acc_cols = (dual || DIRECT ? 2 : 1) * n_box;  // (direct fp8 form: one accumulator per token term)
+  const int a_total = WIDEN ? n_stages * (int)a_cols : 0;
   const int acc_stages = (2 * acc_cols + a_total <= 512) ? 2 : 1;
   const uint32_t a_col0 = (uint32_t)(acc_stages * acc_cols);  // first column of the weight stages
   // warps that can own a 16-column chunk; the SwiGLU epilogue (KIND 1) profits from all 16, the
@@ -239,13 +249,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   // depths, so every load slot and every weight stage belongs to ONE group, which visits the
   // rounds of its barriers in order - a parity wait can then never take an older phase for the
   // one it wants.
-  int conv_groups = FP8 ? 1 + (kEpiWarps - epi_warps) / 4 : 0;
+  int conv_groups = WIDEN ? 1 + (kEpiWarps - epi_warps) / 4 : 0;
   if (conv_groups > 2) conv_groups = 2;
   if (conv_groups > 1 && n_stages % conv_groups != 0) conv_groups = 1;
-  const int conv_group = !FP8 ? -1
+  const int conv_group = !WIDEN ? -1
                          : (warp >= kConvWarp0 && warp < kConvWarp0 + 4) ? 0
                          : (warp >= epi_warps && warp < kEpiWarps) ? 1 + (warp - epi_warps) / 4 : -1;
-  const bool is_conv = FP8 && conv_group >= 0 && conv_group < conv_groups;
+  const bool is_conv = WIDEN && conv_group >= 0 && conv_group < conv_groups;
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < acc_stages * acc_cols + a_total) tmem_cols <<= 1;
 
@@ -255,14 +265,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     timeline_entry(timeline, timeline_slot);
     for (int s = 0; s < kMaxStages; ++s) {
       // the stage's TMA transaction, or every lane of the four converting warps
-      mbar_init(smem_u32(&ctl->full[s]), FP8 ? 128u : 1u);
+      mbar_init(smem_u32(&ctl->full[s]), WIDEN ? 128u : 1u);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int s = 0; s < kMaxStages; ++s) mbar_init(smem_u32(&ctl->slot_full[s]), 1);
     for (int s = 0; s < kItemRing; ++s) {
       mbar_init(smem_u32(&ctl->item_full[s]), 1);
       // consumers: the MMA thread, one lane of every epilogue warp and of every converter warp
-      mbar_init(smem_u32(&ctl->item_empty[s]), 1u + (uint32_t)epi_warps + (FP8 ? 4u * (uint32_t)conv_groups : 0u));
+      mbar_init(smem_u32(&ctl->item_empty[s]), 1u + (uint32_t)epi_warps + (WIDEN ? 4u * (uint32_t)conv_groups : 0u));
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
@@ -322,8 +332,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   tc_fence_after();
 
   // polling back-off of the fp8 form, by role (the MMA thread never sleeps)
-  constexpr uint32_t nap_epi = FP8 ? OLED_NAP_EPI : 0u, nap_load = FP8 ? OLED_NAP_LOAD : 0u,
-                     nap_conv = FP8 ? OLED_NAP_CONV : 0u;
+  constexpr uint32_t nap_epi = WIDEN ? OLED_NAP_EPI : 0u, nap_load = WIDEN ? OLED_NAP_LOAD : 0u,
+                     nap_conv = WIDEN ? OLED_NAP_CONV : 0u;
   const uint32_t tmem_base = ctl->tmem_base;
   SecondPhase second;
   second.n1 = fused ? ctl->n_tiles_total * m_tiles : 0x7fffffff;
@@ -372,13 +382,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       const CUtensorMap* map_w = down_of_fused ? &fs.tm_w2 : &tm_w;
       const CUtensorMap* map_act = down_of_fused ? &fs.tm_act2 : &tm_act;
       const int k_blocks = down_of_fused ? k_blocks2 : k_blocks1;
-      constexpr uint32_t w_tile = FP8 ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
+      constexpr uint32_t w_tile = WIDEN ? kATile / 2 : kATile;  // bytes of 128 weight rows of a k-block
       auto load_weights = [&](int st, int kb) {
-        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
+        const uint32_t bar = smem_u32(WIDEN ? &ctl->slot_full[st] : &ctl->full[st]);
         mbar_expect_tx(bar, stage_bytes);
         for (int atom = 0; atom < k_atoms; ++atom) {
           const uint32_t w_addr = tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes;
-          const int k0 = (kb * k_atoms + atom) * kBlockK;
+          const int k0 = (kb * k_atoms + atom) * kK;
           if (stacked && it.kind == 1) {  // the map has 64-row boxes here
             tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
             tma_load_3d(map_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
@@ -392,11 +402,18 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         }
       };
       auto load_tokens = [&](int st, int kb) {
-        const uint32_t bar = smem_u32(FP8 ? &ctl->slot_full[st] : &ctl->full[st]);
-        for (int atom = 0; atom < k_atoms; ++atom)
-          tma_load_2d(map_act,
-                      tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (FP8 ? raw_bytes : a_bytes),
-                      bar, (kb * k_atoms + atom) * kBlockK, it.row0);
+        const uint32_t bar = smem_u32(WIDEN ? &ctl->slot_full[st] : &ctl->full[st]);
+        for (int atom = 0; atom < k_atoms; ++atom) {
+          const uint32_t t_addr =
+              tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (WIDEN ? raw_bytes : a_bytes);
+          const int k0 = (kb * k_atoms + atom) * kK;
+          if (DIRECT) {  // (the map is over [term][row][k])
+            tma_load_3d(map_act, t_addr, bar, k0, it.row0, 0);
+            tma_load_3d(map_act, t_addr + b_bytes, bar, k0, it.row0, 1);
+          } else {
+            tma_load_2d(map_act, t_addr, bar, k0, it.row0);
+          }
+        }
       };
       int kb = 0;
       if (early && seq == 0) {
@@ -490,7 +507,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
     const uint32_t ring_step = atom_bytes >> 4;  // one k-block further in shared memory
     const uint32_t a_lo0 = (uint32_t)make_smem_desc(tiles_base);
-    const uint32_t b_lo0 = (uint32_t)make_smem_desc(tiles_base + (FP8 ? raw_bytes : a_bytes));
+    const uint32_t b_lo0 = (uint32_t)make_smem_desc(tiles_base + (WIDEN ? raw_bytes : a_bytes));
     const uint32_t a_tmem0 = tmem_base + a_col0;  // fp8 stores: weights come from tensor memory
     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
     uint32_t a_lo = a_lo0, b_lo = b_lo0, a_tmem = a_tmem0;
@@ -505,7 +522,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status)) break;
       tc_fence_after();
       const int n_mma = max(16, (it.valid + 15) & ~15);
-      const uint32_t idesc = make_idesc(n_mma);
+      const uint32_t idesc = DIRECT ? make_idesc_e4m3(2 * n_box) : make_idesc(n_mma);
       const uint32_t d0 = tmem_base + (uint32_t)(acc * acc_cols);
       for (int kb = 0; kb < k_blocks; ++kb) {
         // (fp8 stores: the converters arrive on full[] only after the stage's slot has landed)
@@ -519,7 +536,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < kBlockK / 16; ++k) {  // 32 bytes along K = 2 address units
             const uint32_t accum = k != 0 ? 1u : first;
-            if (FP8) {
+            if (DIRECT) {
+              tc_mma_e4m3_lo(d0, a_lo + k * 2, b_lo + k * 2, desc_hi, idesc, accum);
+            } else if (WIDEN) {
               tc_mma_ts_lo(d0, a_tmem + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
               if (dual) tc_mma_ts_lo(d0 + (uint32_t)n_box, a_tmem + 32 + k * 8, b_lo + k * 2, desc_hi, idesc, accum);
             } else {
@@ -656,6 +675,17 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
       for (int c = half * 16; c < n_mma; c += 16 * (epi_warps / 4 > 0 ? epi_warps / 4 : 1)) {
         uint32_t ra[16];
         tmem_ld16(t_row + (uint32_t)c, ra);
+        if (DIRECT) {
+          // the two terms' accumulators: D = (D1 + D2 / 16) / row scale of the token
+          uint32_t rt[16];
+          tmem_ld16(t_row + (uint32_t)(n_box + c), rt);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float inv = c + j < it.valid ? token_scale_inverse(amax_in[it.row0 + c + j]) : 0.0f;
+            ra[j] = __float_as_uint(__fmaf_rn(__uint_as_float(rt[j]), 0.0625f, __uint_as_float(ra[j])) * inv);
+          }
+        }
         if (stacked && gate_up_item) {
           // lanes 0-63 hold silu's argument (gate rows), lanes 64-127 the up rows of the same
           // features: warps 2,3 hand their chunk to warps 0,1 through a double-buffered slot
@@ -694,14 +724,28 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
             }
             mbar_arrive(smem_u32(&ctl->x_empty[buf][half]));
             uint16_t* hb = reinterpret_cast<uint16_t*>(out_ptr);
+            uint32_t mag[16];  // direct fp8 form: magnitudes of the stored values (bf16 bit patterns)
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
+              mag[j] = 0u;
               if (c + j < it.valid) {
                 const float a = __uint_as_float(ra[j]) * s0;
                 const float hm = __fdividef(a, 1.0f + __expf(-a)) * u[j];
                 const __nv_bfloat16 b = __float2bfloat16_rn(hm);
                 hb[(size_t)(it.row0 + c + j) * I + it.m0 + xrow] = *reinterpret_cast<const uint16_t*>(&b);
+                mag[j] = (uint32_t)(*reinterpret_cast<const uint16_t*>(&b) & 0x7fffu);
               }
+            }
+            if (DIRECT) {
+              // the rows' largest magnitudes, for the down projection's token scaling: the warp's
+              // 32 features of token c + j are reduced, lane j raises the row's word
+              uint32_t top = 0u;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const uint32_t m = __reduce_max_sync(0xffffffffu, mag[j]);
+                if (lane == j) top = m;
+              }
+              if (lane < 16 && c + lane < it.valid && top != 0u) atomicMax(amax_out + it.row0 + c + lane, top << 16);
             }
           }
         } else if (KIND == 1) {
@@ -775,6 +819,34 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
   if (threadIdx.x == 0) timeline_end(timeline, timeline_slot);
 }
 
+// fp8 direct form, between the two projections: the intermediate rows of the group's experts
+// (bf16, written by the gate/up epilogue together with every row's largest magnitude) as two e4m3
+// terms per element.  One CTA per expert of the group; a warp takes a row at a time.
+__global__ void __launch_bounds__(256)
+split_rows_kernel(const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
+                  const uint16_t* __restrict__ hbuf, const uint32_t* __restrict__ amax_mid,
+                  uint8_t* __restrict__ terms_mid, int I, int rows_total) {
+  griddep_launch_dependents();
+  griddep_wait();
+  const int e = grp.expert[blockIdx.x];
+  const int first = offsets[e], last = offsets[e + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = first + warp; r < last; r += 8) {
+    const float scale = token_scale(amax_mid[r]);
+    const uint4* src = reinterpret_cast<const uint4*>(hbuf + (size_t)r * I);
+    uint2* out1 = reinterpret_cast<uint2*>(terms_mid + (size_t)r * I);
+    uint2* out2 = reinterpret_cast<uint2*>(terms_mid + ((size_t)rows_total + r) * I);
+    for (int c = lane; c < I / 8; c += 32) {
+      const uint4 v = src[c];
+      uint2 t1, t2;
+      split_bf16x4(v.x, v.y, scale, t1.x, t2.x);
+      split_bf16x4(v.z, v.w, scale, t1.y, t2.y);
+      out1[c] = t1;
+      out2[c] = t2;
+    }
+  }
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -794,16 +866,18 @@ EncodeTiledFn get_encode_fn() {
 }
 
 bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, const cuuint64_t* strides,
-            const cuuint32_t* box, bool bytes = false) {
+            const cuuint32_t* box, bool bytes = false, bool bytes_swizzle_128 = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint32_t estr[3] = {1, 1, 1};
   const CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-  // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; e4m3 rows (64 bytes per
-  // k-block) land with the 64-byte swizzle, which lets 32 lanes read 32 rows free of bank conflicts
+  // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; e4m3 rows for the
+  // widening form (64 bytes per k-block) land with the 64-byte swizzle, which lets 32 lanes read
+  // 32 rows free of bank conflicts; e4m3 rows the MMA reads itself (128 bytes per k-block) land
+  // in the 128-byte-swizzled layout again
   return fn(m, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
             const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            bytes ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, promo,
+            bytes && !bytes_swizzle_128 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, promo,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -823,20 +897,21 @@ int epi_warps_for(int kind, int out_bf16, int n_box) {
 // tensor memory behind the accumulators (two accumulator stages if at least two weight stages
 // still fit); the depth is a multiple of the number of converter groups (see the kernel).
 // k_dim2: the second contraction length of a fused launch (0 otherwise).
-Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_dim, int k_dim2 = 0) {
+// fp8: 0 = bf16 stores, 1 = fp8 stores widened by converter warps, 2 = fp8 stores read directly.
+Rings rings_for(int kind, bool dual, int n_box, int out_bf16, int fp8, int k_dim, int k_dim2 = 0) {
   const uint32_t a = (dual ? 2u : 1u) * kATile, b = (uint32_t)n_box * 128u;
   const uint32_t avail = kSmemMax - kCtlBytes - 1024u;
-  const uint32_t atom = fp8 ? a / 2 + b : a + b;  // one k-block in shared memory
-  int kblocks = (int)std::min<uint32_t>((uint32_t)(fp8 ? 2 * kMaxStages : 10), avail / atom);
-  if (fp8) {
+  const uint32_t atom = fp8 == 2 ? kATile + 2u * b : fp8 ? a / 2 + b : a + b;  // one k-block in shared memory
+  int kblocks = (int)std::min<uint32_t>((uint32_t)(fp8 == 2 ? kMaxStages : fp8 ? 2 * kMaxStages : 10), avail / atom);
+  if (fp8 == 1) {
     const int acc_cols = (dual ? 2 : 1) * n_box, a_cols = dual ? 64 : 32;
     const int free_cols = 512 - 2 * acc_cols >= 2 * a_cols ? 512 - 2 * acc_cols : 512 - acc_cols;
     kblocks = std::min(kblocks, free_cols / a_cols);
   }
   Rings r;
-  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0 && (k_dim2 / kBlockK) % 2 == 0) ? 2 : 1;
+  r.k_atoms = (fp8 != 2 && !dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0 && (k_dim2 / kBlockK) % 2 == 0) ? 2 : 1;
   r.stages = std::min(kblocks / r.k_atoms, kMaxStages);
-  if (fp8) {
+  if (fp8 == 1) {
     const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
     if (r.stages >= groups) r.stages -= r.stages % groups;
   }
@@ -844,42 +919,48 @@ Rings rings_for(int kind, bool dual, int n_box, int out_bf16, bool fp8, int k_di
   return r;
 }
 
-template <int KIND, bool DUAL, bool FP8>
+template <int KIND, bool DUAL, int FP8>
 bool set_smem_attr() {
   return cudaFuncSetAttribute(ffn_tc_kernel<KIND, DUAL, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)kSmemMax) == cudaSuccess;
 }
 
 template <int KIND, bool DUAL>
-void launch_variant(bool fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
+void launch_variant(int fp8, int grid, cudaStream_t st, const CUtensorMap& tw, const CUtensorMap& ta,
                     const FfnGroup& grp, const int32_t* offsets, void* out, int H, int I, int out_bf16,
                     const uint8_t* pool, size_t slot_bytes, uint32_t* status, uint32_t* work_counter,
                     uint32_t smem_of_predecessor, bool early_allowed, StepTimeline* timeline, int timeline_slot,
-                    const RouteReport& report, const FusedSecond& fs = FusedSecond{}) {
+                    const RouteReport& report, const FusedSecond& fs = FusedSecond{}, const uint32_t* amax_in = nullptr,
+                    uint32_t* amax_out = nullptr) {
   const Rings r = rings_for(KIND, DUAL, grp.n_box, out_bf16, fp8, KIND == 2 ? I : H, KIND == 3 ? I : 0);
   // KIND 2 may start ahead of its dependency wait only where the caller vouches for the ordering
   // (early_allowed, see launch_ffn_tc) AND one of its CTAs and one of the KIND 1 kernel before it
   // cannot share an SM, so that it gets an SM only when a KIND 1 CTA has left it
   const int early = (KIND == 2 && early_allowed && smem_of_predecessor + r.smem > 228u * 1024u) ? 1 : 0;
   if constexpr (KIND == 3) {
-    launch_pdl(ffn_tc_kernel<3, false, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H, I,
+    launch_pdl(ffn_tc_kernel<3, false, 0>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H, I,
                r.stages, r.k_atoms, 0, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot, report, fs);
+               timeline_slot, report, fs, amax_in, amax_out);
+  } else if (fp8 == 2) {
+    if constexpr (!DUAL)
+      launch_pdl(ffn_tc_kernel<KIND, false, 2>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+                 I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter,
+                 timeline, timeline_slot, report, fs, amax_in, amax_out);
   } else if (fp8) {
-    launch_pdl(ffn_tc_kernel<KIND, DUAL, true>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, 1>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot, report, fs);
+               timeline_slot, report, fs, amax_in, amax_out);
   } else {
-    launch_pdl(ffn_tc_kernel<KIND, DUAL, false>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
+    launch_pdl(ffn_tc_kernel<KIND, DUAL, 0>, dim3(grid), dim3(kThreads), r.smem, st, tw, ta, grp, offsets, out, H,
                I, r.stages, r.k_atoms, early, out_bf16, pool, (unsigned long long)slot_bytes, status, work_counter, timeline,
-               timeline_slot, report, fs);
+               timeline_slot, report, fs, amax_in, amax_out);
   }
 }
 
 }  // namespace
 
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
-                 const uint16_t* xp, const uint16_t* hbuf, int rows) {
+                 const uint16_t* xp, const uint16_t* hbuf, int rows, const TokenSplit* split) {
   maps->fp8 = fp8;
   maps->pool = pool;
   maps->slot_bytes = slot_bytes;
@@ -898,6 +979,24 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
     const cuuint32_t box[3] = {kBlockK, kBlockM, 1};
     if (!encode(&maps->w2, 3, pool + (size_t)2 * I * H * esz, dims, strides, box, fp8)) return OLED_ERR_CUDA;
   }
+  // fp8 stores: maps for the form whose MMAs read the codes themselves - k-blocks of 128 bytes
+  maps->e4m3_direct = fp8 && H % 128 == 0 && I % 128 == 0 && split != nullptr && split->complete() && split->rows == rows;
+  if (maps->e4m3_direct) {
+    for (int i = 0; i < 2; ++i) {
+      const cuuint32_t tbox[3] = {128, (cuuint32_t)(16 << i), 1};
+      const cuuint64_t dims_in[3] = {(cuuint64_t)H, (cuuint64_t)rows, 2}, dims_mid[3] = {(cuuint64_t)I, (cuuint64_t)rows, 2};
+      const cuuint64_t str_in[2] = {(cuuint64_t)H, (cuuint64_t)rows * H}, str_mid[2] = {(cuuint64_t)I, (cuuint64_t)rows * I};
+      if (!encode(&maps->xp_terms[i], 3, split->terms_in, dims_in, str_in, tbox, true, true)) return OLED_ERR_CUDA;
+      if (!encode(&maps->hbuf_terms[i], 3, split->terms_mid, dims_mid, str_mid, tbox, true, true)) return OLED_ERR_CUDA;
+    }
+    const cuuint32_t box_half[3] = {128, kBlockM / 2, 1}, box[3] = {128, kBlockM, 1};
+    const cuuint64_t dims13[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
+    const cuuint64_t strides13[2] = {(cuuint64_t)H, (cuuint64_t)slot_bytes};
+    const cuuint64_t dims2[3] = {(cuuint64_t)I, (cuuint64_t)H, (cuuint64_t)n_slots};
+    const cuuint64_t strides2[2] = {(cuuint64_t)I, (cuuint64_t)slot_bytes};
+    if (!encode(&maps->w13_half_e4m3, 3, pool, dims13, strides13, box_half, true, true)) return OLED_ERR_CUDA;
+    if (!encode(&maps->w2_e4m3, 3, pool + (size_t)2 * I * H, dims2, strides2, box, true, true)) return OLED_ERR_CUDA;
+  }
   for (int i = 0; i < 5; ++i) {
     const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(16 << i)};
     {
@@ -913,9 +1012,10 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   }
   static bool attr_done = false;
   if (!attr_done) {
-    if (!set_smem_attr<1, true, false>() || !set_smem_attr<1, false, false>() || !set_smem_attr<2, true, false>() ||
-        !set_smem_attr<2, false, false>() || !set_smem_attr<1, true, true>() || !set_smem_attr<1, false, true>() ||
-        !set_smem_attr<2, true, true>() || !set_smem_attr<2, false, true>() || !set_smem_attr<3, false, false>())
+    if (!set_smem_attr<1, true, 0>() || !set_smem_attr<1, false, 0>() || !set_smem_attr<2, true, 0>() ||
+        !set_smem_attr<2, false, 0>() || !set_smem_attr<1, true, 1>() || !set_smem_attr<1, false, 1>() ||
+        !set_smem_attr<2, true, 1>() || !set_smem_attr<2, false, 1>() || !set_smem_attr<3, false, 0>() ||
+        !set_smem_attr<1, false, 2>() || !set_smem_attr<2, false, 2>())
       return OLED_ERR_CUDA;
     attr_done = true;
   }
@@ -931,7 +1031,7 @@ static int box_index(int max_count, int cap) {
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H, int I,
                   int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait, StepTimeline* timeline,
-                  int timeline_slot, const RouteReport& report_in, uint32_t* done) {
+                  int timeline_slot, const RouteReport& report_in, uint32_t* done, const TokenSplit* split) {
   const RouteReport report = kind != 2 ? report_in : RouteReport{};
   if (grp_in.n <= 0 || max_count <= 0) return OLED_OK;
   FfnGroup grp = grp_in;
@@ -942,6 +1042,10 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   // (fp8 stores stop at N = 128: the widened weights need tensor-memory columns of their own)
   const int ib = box_index(max_count, fp8 ? 128 : 256);
   grp.n_box = 16 << ib;
+  // fp8 stores, token tiles of at most 32 rows, row magnitudes at hand: the MMAs read the codes
+  // themselves (mode 2); otherwise converter warps widen them to bf16 (mode 1)
+  const bool direct = fp8 && maps.e4m3_direct && grp.n_box <= 32 && split != nullptr && split->complete();
+  const int mode = direct ? 2 : fp8 ? 1 : 0;
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int m_tiles) {
     if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
@@ -956,7 +1060,7 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   // CTA then gets an SM only after a KIND 1 CTA, which waited for the permutation, has left it),
   // or the launch pair sits behind an event wait, which completes everything enqueued before it.
   const bool early_allowed = kind == 2 && (behind_event_wait || host_counts == nullptr);
-  const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, fp8, H).smem : 0u;
+  const uint32_t smem1 = kind == 2 ? rings_for(1, !stacked1, grp.n_box, 0, mode, H).smem : 0u;
   if (kind == 3) {
     if (fp8 || !stacked1 || done == nullptr) return OLED_ERR_INVALID_ARG;  // callers ask ffn_tc_can_fuse() first
     FusedSecond fs;
@@ -964,25 +1068,39 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
     fs.tm_act2 = maps.hbuf[ib];
     fs.out2 = y;
     fs.done = done;
-    launch_variant<3, false>(false, grid_for(I / (kBlockM / 2) + H / kBlockM), st, maps.w13_half, maps.xp[ib], grp, offsets,
+    launch_variant<3, false>(0, grid_for(I / (kBlockM / 2) + H / kBlockM), st, maps.w13_half, maps.xp[ib], grp, offsets,
                              hbuf, H, I, 0, maps.pool, maps.slot_bytes, status, work_counter, 0u, false, timeline,
                              timeline_slot, report, fs);
   } else if (kind == 1 && stacked1) {
-    launch_variant<1, false>(fp8, grid_for(I / (kBlockM / 2)), st, maps.w13_half, maps.xp[ib], grp, offsets, hbuf, H, I,
-                             0, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
+    launch_variant<1, false>(mode, grid_for(I / (kBlockM / 2)), st, direct ? maps.w13_half_e4m3 : maps.w13_half,
+                             direct ? maps.xp_terms[ib] : maps.xp[ib], grp, offsets, hbuf, H, I, 0, maps.pool,
+                             maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report,
+                             FusedSecond{}, direct ? split->amax_in : nullptr, direct ? split->amax_mid : nullptr);
   } else if (kind == 1) {
-    launch_variant<1, true>(fp8, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
+    launch_variant<1, true>(mode, grid_for(I / kBlockM), st, maps.w13, maps.xp[ib], grp, offsets, hbuf, H, I, 0,
                             maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
   } else {
     const bool dual = grp.n_box == 256;
     if (dual)
-      launch_variant<2, true>(fp8, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
+      launch_variant<2, true>(mode, grid_for(H / (2 * kBlockM)), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I,
                               y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
-    else
-      launch_variant<2, false>(fp8, grid_for(H / kBlockM), st, maps.w2, maps.hbuf[ib], grp, offsets, y, H, I, y_bf16,
-                               maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
+    else {
+      if (direct)  // the intermediate rows as e4m3 terms, now that their magnitudes are complete
+        launch_pdl(split_rows_kernel, dim3(grp.n), dim3(256), 0, st, grp, offsets, (const uint16_t*)hbuf,
+                   (const uint32_t*)split->amax_mid, split->terms_mid, I, split->rows);
+      launch_variant<2, false>(mode, grid_for(H / kBlockM), st, direct ? maps.w2_e4m3 : maps.w2,
+                               direct ? maps.hbuf_terms[ib] : maps.hbuf[ib], grp, offsets, y, H, I, y_bf16, maps.pool,
+                               maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot,
+                               report, FusedSecond{}, direct ? split->amax_mid : nullptr, nullptr);
+    }
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
+}
+
+int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenSplit* split) {
+  const bool direct = maps.fp8 && maps.e4m3_direct && (16 << box_index(max_count, 128)) <= 32 && split != nullptr &&
+                      split->complete();
+  return kind == 2 && direct ? 2 : 1;
 }
 
 bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count) {

@@ -150,11 +150,29 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
                   float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
                   StepTimeline* timeline);
 bool route_can_take_combine(int T);  // does the gate kernel of a T-token step carry out a CombinePrev?
+// fp8 expert stores, direct form: the two token operands of a step's expert FFN - the gathered
+// input rows and the intermediate rows - as sums of two e4m3 terms each, after scaling every row
+// by a power of two taken from its largest magnitude (fp8_split.h).  The magnitudes are kept as the
+// bit pattern of a non-negative fp32, so that an unsigned integer maximum orders them.
+//   amax_in, terms_in:   written by the gathering permutation kernel, which also zeroes amax_mid
+//   amax_mid:            raised with atomicMax by the gate/up epilogue
+//   terms_mid:           written by the split kernel between the two projections
+struct TokenSplit {
+  uint32_t* amax_in = nullptr;   // [rows]
+  uint32_t* amax_mid = nullptr;  // [rows]
+  uint8_t* terms_in = nullptr;   // [2][rows][H] e4m3 codes: term 1 of every row, then term 2
+  uint8_t* terms_mid = nullptr;  // [2][rows][I]
+  int rows = 0;                  // rows of the buffers above (tokens x top-k of the context)
+  bool complete() const { return amax_in && amax_mid && terms_in && terms_mid && rows > 0; }
+};
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
 // kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
+// split (gathering launches only; nullptr: none): the kernel also writes, per sorted row, the
+// largest magnitude of the row it copied and the row's two e4m3 terms, and zeroes amax_mid (see
+// TokenSplit).
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
-                    StepTimeline* timeline);
+                    StepTimeline* timeline, const TokenSplit* split = nullptr);
 // xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);
@@ -177,6 +195,11 @@ void launch_ffn_simple(cudaStream_t st, const FfnGroup& grp, const uint8_t* pool
 
 // ---- ffn_tc.cu (tcgen05 / TMEM / TMA) ------------------------------------------------------
 struct FfnTcMaps {
+  CUtensorMap w13_half_e4m3;  // fp8 stores: [slots][2I][H] bytes, box {128,64,1}, 128-byte swizzle
+  CUtensorMap w2_e4m3;        // fp8 stores: [slots][H][I] bytes, box {128,128,1}, 128-byte swizzle
+  CUtensorMap xp_terms[2];    // [2][rows][H] bytes (TokenSplit::terms_in), box {128, 16<<i, 1}
+  CUtensorMap hbuf_terms[2];  // [2][rows][I] bytes (TokenSplit::terms_mid), box {128, 16<<i, 1}
+  bool e4m3_direct = false;   // the maps above exist (fp8 stores, H and I multiples of 128, term buffers given)
   CUtensorMap w13;       // [slots][2I][H] bf16, box {64,128,1}
   CUtensorMap w13_half;  // the same, box {64,64,1}
   CUtensorMap w2;        // [slots][H][I]  bf16, box {64,128,1}
@@ -188,7 +211,7 @@ struct FfnTcMaps {
 };
 // Builds the tensor maps; returns 0 or a negative oled_status.
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
-                 const uint16_t* xp, const uint16_t* hbuf, int rows);
+                 const uint16_t* xp, const uint16_t* hbuf, int rows, const TokenSplit* split = nullptr);
 // kind 1: gate/up + SwiGLU into hbuf; kind 2: down projection into y; kind 3: both in one launch
 // (bf16 stores and token tiles of at most 32 rows only: ask ffn_tc_can_fuse; `done` then points at
 // one ZERO word per expert of the group).  One launch each.
@@ -198,10 +221,15 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
 // counts and scores to the host.
 // behind_event_wait: the launch follows a cudaStreamWaitEvent (with, for kind 2, at most its own
 // kind 1 launch in between), i.e. everything enqueued before that wait has completed.
+// split (fp8 stores; nullptr: none): the token operands as e4m3 terms.  With them, token tiles of
+// at most 32 rows take the form whose MMAs read the experts' e4m3 codes as they are; a kind 2
+// launch is then preceded by the split kernel (ffn_tc_launches tells how many launches a call makes).
 int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int max_count, int kind,
                   const int32_t* host_counts, const int32_t* offsets, uint16_t* hbuf, float* y, int y_bf16, int H,
                   int I, int n_sms, uint32_t* status, uint32_t* work_counter, bool behind_event_wait,
-                  StepTimeline* timeline, int timeline_slot, const RouteReport& report, uint32_t* done = nullptr);
+                  StepTimeline* timeline, int timeline_slot, const RouteReport& report, uint32_t* done = nullptr,
+                  const TokenSplit* split = nullptr);
+int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenSplit* split);
 bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 

@@ -83,6 +83,8 @@ struct oled_ctx {
   int32_t* d_pos = nullptr;    // [T*k]
   uint16_t* d_xp = nullptr;    // [T*k,H]
   uint16_t* d_hbuf = nullptr;  // [T*k,I]
+  TokenSplit split;            // fp8 stores: the FFN's token operands as e4m3 terms (see TokenSplit)
+  const TokenSplit* step_split = nullptr;  // &split in steps whose permutation kernel fills it
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
   uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
@@ -231,6 +233,10 @@ void free_ctx(oled_ctx* ctx) {
   cudaFree(ctx->d_pos_buf[1]);
   cudaFree(ctx->d_xp);
   cudaFree(ctx->d_hbuf);
+  cudaFree(ctx->split.amax_in);
+  cudaFree(ctx->split.amax_mid);
+  cudaFree(ctx->split.terms_in);
+  cudaFree(ctx->split.terms_mid);
   cudaFree(ctx->d_y);
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_timeline);
@@ -389,9 +395,10 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
       const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
                                    ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work,
                                    behind_event_wait || (kind == 2 && before_down != nullptr),
-                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li, report, done);
+                                   ctx->timeline_on ? ctx->d_timeline + ctx->last_layer : nullptr, 3 + li, report, done,
+                                   ctx->step_split);
       if (rc != OLED_OK) return rc;
-      ctx->launches += 1;
+      ctx->launches += ffn_tc_launches(ctx->maps, max_count, kind, ctx->step_split);
     }
     if (fused_out) *fused_out = fuse;
   }
@@ -557,6 +564,13 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   ctx->d_pos = ctx->d_pos_buf[0];
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_xp, T * K * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_hbuf, T * K * I)) != OLED_OK) return fail(rc);
+  if (s.expert_format == OLED_EXPERTS_FP8 && H % 128 == 0 && I % 128 == 0) {
+    if ((rc = dev_alloc(ctx, &ctx->split.amax_in, T * K)) != OLED_OK) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->split.amax_mid, T * K)) != OLED_OK) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->split.terms_in, 2 * T * K * H)) != OLED_OK) return fail(rc);
+    if ((rc = dev_alloc(ctx, &ctx->split.terms_mid, 2 * T * K * I)) != OLED_OK) return fail(rc);
+    ctx->split.rows = (int)(T * K);
+  }
   if ((rc = dev_alloc_guarded(ctx, &ctx->d_y, T * K * H)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_status, kStatusWords)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_timeline, (size_t)s.n_layers)) != OLED_OK) return fail(rc);
@@ -586,7 +600,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
     return fail(OLED_ERR_CUDA);
   rc = ffn_tc_setup(&ctx->maps, ctx->pool, ctx->slot_bytes, ctx->n_slots, s.hidden, s.intermediate,
                     s.expert_format == OLED_EXPERTS_FP8, ctx->d_xp,
-                    ctx->d_hbuf, (int)(T * K));
+                    ctx->d_hbuf, (int)(T * K), ctx->split.complete() ? &ctx->split : nullptr);
   if (rc != OLED_OK) return fail(rc);
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(OLED_ERR_CUDA);
   *out_ctx = ctx;
@@ -725,8 +739,10 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   NvtxRange nv_perm(ctx, "oled.step.2_permutation_counts");
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
+    // (fp8 stores: a gathering permutation kernel also leaves the rows' magnitudes for the FFN)
+    ctx->step_split = fuse_gather && ctx->split.complete() ? &ctx->split : nullptr;
     launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
-                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl);
+                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl, ctx->step_split);
   }
   if (!fuse_gather) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);

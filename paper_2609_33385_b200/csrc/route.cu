@@ -19,6 +19,7 @@
 #include <mutex>
 
 #include "kernels.h"
+#include "fp8_split.h"
 #include "route_math.h"
 
 namespace oled {
@@ -491,10 +492,14 @@ constexpr int kGatherTokMax = 4096;  // rows of one expert in a step that gather
 __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
-               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, StepTimeline* timeline) {
+               const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, StepTimeline* timeline,
+               TokenSplit split) {
+  uint32_t* const amax_in = split.amax_in;
+  uint32_t* const amax_mid = split.amax_mid;
   __shared__ int s_red[8];
   __shared__ int s_base;
   __shared__ int s_tok[kGatherTokMax];
+  __shared__ uint32_t s_amax[8];
   const int e = blockIdx.x;
   const bool writer = blockIdx.y == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -584,6 +589,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     int tok[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) tok[j] = r0 + j < rows ? s_tok[r0 + j] : -1;
+    uint32_t big[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // per row: max of |bf16| bit patterns, two per word
     for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
       uint4 v[8];
 #pragma unroll
@@ -591,7 +597,46 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
         if (tok[j] >= 0) v[j] = src[(size_t)tok[j] * vec_per_row + c];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (tok[j] >= 0) dst[(size_t)(first + r0 + j) * vec_per_row + c] = v[j];
+        if (tok[j] >= 0) {
+          dst[(size_t)(first + r0 + j) * vec_per_row + c] = v[j];
+          if (amax_in != nullptr)
+            big[j] = __vmaxu2(__vmaxu2(big[j], __vmaxu2(v[j].x & 0x7fff7fffu, v[j].y & 0x7fff7fffu)),
+                              __vmaxu2(v[j].z & 0x7fff7fffu, v[j].w & 0x7fff7fffu));
+        }
+    }
+    if (amax_in != nullptr) {
+      // the rows' largest magnitudes (a bf16 magnitude's bits order like the value) and a cleared
+      // word per row for the intermediate rows' maxima
+      __syncthreads();  // the previous batch's s_amax has been read
+      if (threadIdx.x < 8) s_amax[threadIdx.x] = 0u;
+      __syncthreads();
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t m = __reduce_max_sync(0xffffffffu, max(big[j] & 0xffffu, big[j] >> 16));
+        if (lane == 0) atomicMax(&s_amax[j], m);
+      }
+      __syncthreads();
+      if (threadIdx.x < 8 && r0 + (int)threadIdx.x < rows) {
+        amax_in[first + r0 + threadIdx.x] = s_amax[threadIdx.x] << 16;
+        amax_mid[first + r0 + threadIdx.x] = 0u;
+      }
+      // the rows' two e4m3 terms (each thread re-reads the vectors it has just stored)
+      for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (tok[j] >= 0) {
+            const size_t r = (size_t)(first + r0 + j);
+            const uint4 v = dst[r * vec_per_row + c];
+            const float scale = token_scale(s_amax[j] << 16);
+            uint2 t1, t2;
+            split_bf16x4(v.x, v.y, scale, t1.x, t2.x);
+            split_bf16x4(v.z, v.w, scale, t1.y, t2.y);
+            uint2* out1 = reinterpret_cast<uint2*>(split.terms_in + r * H);
+            uint2* out2 = reinterpret_cast<uint2*>(split.terms_in + ((size_t)split.rows + r) * H);
+            out1[c] = t1;
+            out2[c] = t2;
+          }
+      }
     }
   }
   if (threadIdx.x == 0) timeline_end(timeline, 1);
@@ -698,11 +743,12 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
-                    StepTimeline* timeline) {
+                    StepTimeline* timeline, const TokenSplit* split) {
   // gathering steps: up to four CTAs per expert share its rows (batches of eight)
-  const int split = xp != nullptr ? 4 : 1;
-  launch_pdl(permute_kernel, dim3(E, split), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
-             timeline);
+  const int split_ctas = xp != nullptr ? 4 : 1;
+  const TokenSplit sp = xp != nullptr && split != nullptr && split->complete() ? *split : TokenSplit{};
+  launch_pdl(permute_kernel, dim3(E, split_ctas), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
+             timeline, sp);
 }
 
 namespace {
