@@ -389,7 +389,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
         for (int atom = 0; atom < k_atoms; ++atom) {
           const uint32_t w_addr = tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes;
           const int k0 = (kb * k_atoms + atom) * kK;
-          if (stacked && it.kind == 1) {  // the map has 64-row boxes here
+          if (DIRECT && stacked && it.kind == 1) {
+            // one copy: the map is over [slot][gate | up][row][k], the box takes 64 rows of either
+            // half (the copy instructions are the serial cost of this thread, see rings_for)
+            tma_load_4d(map_w, w_addr, bar, k0, it.m0, 0, it.slot);
+          } else if (stacked && it.kind == 1) {  // the map has 64-row boxes here
             tma_load_3d(map_w, w_addr, bar, k0, it.m0, it.slot);                  // 64 gate rows
             tma_load_3d(map_w, w_addr + w_tile / 2, bar, k0, I + it.m0, it.slot);  // 64 up rows
           } else if (it.kind == 1) {
@@ -407,9 +411,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
           const uint32_t t_addr =
               tiles_base + (uint32_t)st * stage_bytes + (uint32_t)atom * atom_bytes + (WIDEN ? raw_bytes : a_bytes);
           const int k0 = (kb * k_atoms + atom) * kK;
-          if (DIRECT) {  // (the map is over [term][row][k])
+          if (DIRECT) {  // (the map is over [term][row][k], the box takes both terms)
             tma_load_3d(map_act, t_addr, bar, k0, it.row0, 0);
-            tma_load_3d(map_act, t_addr + b_bytes, bar, k0, it.row0, 1);
           } else {
             tma_load_2d(map_act, t_addr, bar, k0, it.row0);
           }
@@ -869,7 +872,7 @@ bool encode(CUtensorMap* m, int rank, const void* base, const cuuint64_t* dims, 
             const cuuint32_t* box, bool bytes = false, bool bytes_swizzle_128 = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
-  cuuint32_t estr[3] = {1, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   const CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
   // bf16 operand tiles land in the 128-byte-swizzled layout the MMA reads; e4m3 rows for the
   // widening form (64 bytes per k-block) land with the 64-byte swizzle, which lets 32 lanes read
@@ -983,18 +986,18 @@ int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_
   maps->e4m3_direct = fp8 && H % 128 == 0 && I % 128 == 0 && split != nullptr && split->complete() && split->rows == rows;
   if (maps->e4m3_direct) {
     for (int i = 0; i < 2; ++i) {
-      const cuuint32_t tbox[3] = {128, (cuuint32_t)(16 << i), 1};
+      const cuuint32_t tbox[3] = {128, (cuuint32_t)(16 << i), 2};
       const cuuint64_t dims_in[3] = {(cuuint64_t)H, (cuuint64_t)rows, 2}, dims_mid[3] = {(cuuint64_t)I, (cuuint64_t)rows, 2};
       const cuuint64_t str_in[2] = {(cuuint64_t)H, (cuuint64_t)rows * H}, str_mid[2] = {(cuuint64_t)I, (cuuint64_t)rows * I};
       if (!encode(&maps->xp_terms[i], 3, split->terms_in, dims_in, str_in, tbox, true, true)) return OLED_ERR_CUDA;
       if (!encode(&maps->hbuf_terms[i], 3, split->terms_mid, dims_mid, str_mid, tbox, true, true)) return OLED_ERR_CUDA;
     }
-    const cuuint32_t box_half[3] = {128, kBlockM / 2, 1}, box[3] = {128, kBlockM, 1};
-    const cuuint64_t dims13[3] = {(cuuint64_t)H, (cuuint64_t)(2 * I), (cuuint64_t)n_slots};
-    const cuuint64_t strides13[2] = {(cuuint64_t)H, (cuuint64_t)slot_bytes};
+    const cuuint32_t box_half[4] = {128, kBlockM / 2, 2, 1}, box[3] = {128, kBlockM, 1};
+    const cuuint64_t dims13[4] = {(cuuint64_t)H, (cuuint64_t)I, 2, (cuuint64_t)n_slots};
+    const cuuint64_t strides13[3] = {(cuuint64_t)H, (cuuint64_t)I * H, (cuuint64_t)slot_bytes};
     const cuuint64_t dims2[3] = {(cuuint64_t)I, (cuuint64_t)H, (cuuint64_t)n_slots};
     const cuuint64_t strides2[2] = {(cuuint64_t)I, (cuuint64_t)slot_bytes};
-    if (!encode(&maps->w13_half_e4m3, 3, pool, dims13, strides13, box_half, true, true)) return OLED_ERR_CUDA;
+    if (!encode(&maps->w13_half_e4m3, 4, pool, dims13, strides13, box_half, true, true)) return OLED_ERR_CUDA;
     if (!encode(&maps->w2_e4m3, 3, pool + (size_t)2 * I * H, dims2, strides2, box, true, true)) return OLED_ERR_CUDA;
   }
   for (int i = 0; i < 5; ++i) {

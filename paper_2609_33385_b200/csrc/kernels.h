@@ -195,10 +195,10 @@ void launch_ffn_simple(cudaStream_t st, const FfnGroup& grp, const uint8_t* pool
 
 // ---- ffn_tc.cu (tcgen05 / TMEM / TMA) ------------------------------------------------------
 struct FfnTcMaps {
-  CUtensorMap w13_half_e4m3;  // fp8 stores: [slots][2I][H] bytes, box {128,64,1}, 128-byte swizzle
+  CUtensorMap w13_half_e4m3;  // fp8 stores: [slots][2][I][H] bytes, box {128,64,2,1}, 128-byte swizzle
   CUtensorMap w2_e4m3;        // fp8 stores: [slots][H][I] bytes, box {128,128,1}, 128-byte swizzle
-  CUtensorMap xp_terms[2];    // [2][rows][H] bytes (TokenSplit::terms_in), box {128, 16<<i, 1}
-  CUtensorMap hbuf_terms[2];  // [2][rows][I] bytes (TokenSplit::terms_mid), box {128, 16<<i, 1}
+  CUtensorMap xp_terms[2];    // [2][rows][H] bytes (TokenSplit::terms_in), box {128, 16<<i, 2}
+  CUtensorMap hbuf_terms[2];  // [2][rows][I] bytes (TokenSplit::terms_mid), box {128, 16<<i, 2}
   bool e4m3_direct = false;   // the maps above exist (fp8 stores, H and I multiples of 128, term buffers given)
   CUtensorMap w13;       // [slots][2I][H] bf16, box {64,128,1}
   CUtensorMap w13_half;  // the same, box {64,64,1}
