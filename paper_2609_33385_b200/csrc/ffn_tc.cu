@@ -824,7 +824,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
 
 // fp8 direct form, between the two projections: the intermediate rows of the group's experts
 // (bf16, written by the gate/up epilogue together with every row's largest magnitude) as two e4m3
-// terms per element.  One CTA per expert of the group; a warp takes a row at a time.
+// terms per element.  Four CTAs per expert of the group (a quarter of the columns each); a warp
+// takes a row at a time.
 __global__ void __launch_bounds__(256)
 split_rows_kernel(const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets,
                   const uint16_t* __restrict__ hbuf, const uint32_t* __restrict__ amax_mid,
@@ -839,7 +840,7 @@ split_rows_kernel(const __grid_constant__ FfnGroup grp, const int32_t* __restric
     const uint4* src = reinterpret_cast<const uint4*>(hbuf + (size_t)r * I);
     uint2* out1 = reinterpret_cast<uint2*>(terms_mid + (size_t)r * I);
     uint2* out2 = reinterpret_cast<uint2*>(terms_mid + ((size_t)rows_total + r) * I);
-    for (int c = lane; c < I / 8; c += 32) {
+    for (int c = lane + 32 * (int)blockIdx.y; c < I / 8; c += 32 * (int)gridDim.y) {
       const uint4 v = src[c];
       uint2 t1, t2;
       split_bf16x4(v.x, v.y, scale, t1.x, t2.x);
@@ -912,7 +913,8 @@ Rings rings_for(int kind, bool dual, int n_box, int out_bf16, int fp8, int k_dim
     kblocks = std::min(kblocks, free_cols / a_cols);
   }
   Rings r;
-  r.k_atoms = (fp8 != 2 && !dual && kblocks >= 8 && (k_dim / kBlockK) % 2 == 0 && (k_dim2 / kBlockK) % 2 == 0) ? 2 : 1;
+  const int kk = fp8 == 2 ? 128 : kBlockK;  // k-values of a k-block
+  r.k_atoms = (!dual && kblocks >= 8 && (k_dim / kk) % 2 == 0 && (k_dim2 / kk) % 2 == 0) ? 2 : 1;
   r.stages = std::min(kblocks / r.k_atoms, kMaxStages);
   if (fp8 == 1) {
     const int groups = std::min(2, 1 + (kEpiWarps - epi_warps_for(kind, out_bf16, n_box)) / 4);
@@ -1089,7 +1091,7 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
                               y_bf16, maps.pool, maps.slot_bytes, status, work_counter, smem1, early_allowed, timeline, timeline_slot, report);
     else {
       if (direct)  // the intermediate rows as e4m3 terms, now that their magnitudes are complete
-        launch_pdl(split_rows_kernel, dim3(grp.n), dim3(256), 0, st, grp, offsets, (const uint16_t*)hbuf,
+        launch_pdl(split_rows_kernel, dim3(grp.n, 4), dim3(256), 0, st, grp, offsets, (const uint16_t*)hbuf,
                    (const uint32_t*)split->amax_mid, split->terms_mid, I, split->rows);
       launch_variant<2, false>(mode, grid_for(H / kBlockM), st, direct ? maps.w2_e4m3 : maps.w2,
                                direct ? maps.hbuf_terms[ib] : maps.hbuf[ib], grp, offsets, y, H, I, y_bf16, maps.pool,

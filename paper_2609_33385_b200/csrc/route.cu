@@ -489,6 +489,10 @@ route_many_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w
 // expert that received many tokens does not make the step wait for one CTA's chain of batches.
 // Only the CTAs with blockIdx.y == 0 write offsets, perm and pos.
 constexpr int kGatherTokMax = 4096;  // rows of one expert in a step that gathers here (T * K <= 4096)
+// RB: rows a CTA copies at a time.  Eight for a plain copy; two (and eight CTAs per expert) where
+// the rows' e4m3 terms are produced too: the conversions are the long pole there, and an
+// expert's handful of rows is then spread over several SMs.
+template <int RB>
 __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
@@ -499,7 +503,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   __shared__ int s_red[8];
   __shared__ int s_base;
   __shared__ int s_tok[kGatherTokMax];
-  __shared__ uint32_t s_amax[8];
+  __shared__ uint32_t s_amax[3][RB];  // per batch of eight rows, three batches in rotation (see the gather loop)
   const int e = blockIdx.x;
   const bool writer = blockIdx.y == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -524,7 +528,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   }
   __syncthreads();
   // (a CTA beyond the first of an expert has work only if the expert has a batch of rows for it)
-  if (counts[e] == 0 || (int)blockIdx.y * 8 >= counts[e]) {
+  if (counts[e] == 0 || (int)blockIdx.y * RB >= counts[e]) {
     if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
@@ -579,24 +583,30 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
+  if (threadIdx.x < 3 * RB) s_amax[threadIdx.x / RB][threadIdx.x % RB] = 0u;
   __syncthreads();  // the tokens of this expert's rows are in shared memory
   // eight rows at a time: their token numbers, then their loads, are independent memory
   // operations in flight together (a row-by-row loop is a chain of dependent round trips)
   const int vec_per_row = H / 8, first = s_base, rows = counts[e];
   const uint4* src = reinterpret_cast<const uint4*>(x);
   uint4* dst = reinterpret_cast<uint4*>(xp);
-  for (int r0 = (int)blockIdx.y * 8; r0 < rows; r0 += 8 * (int)gridDim.y) {
-    int tok[8];
+  int batch = 0;
+  for (int r0 = (int)blockIdx.y * RB; r0 < rows; r0 += RB * (int)gridDim.y, ++batch) {
+    int tok[RB];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) tok[j] = r0 + j < rows ? s_tok[r0 + j] : -1;
-    uint32_t big[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // per row: max of |bf16| bit patterns, two per word
+    for (int j = 0; j < RB; ++j) tok[j] = r0 + j < rows ? s_tok[r0 + j] : -1;
+    uint32_t big[RB];  // per row: max of |bf16| bit patterns, two per word
+#pragma unroll
+    for (int j = 0; j < RB; ++j) big[j] = 0u;
+    uint4 v[RB];  // (the last vectors stay in registers for the e4m3 terms below)
+    int c_last = -1;
     for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
-      uint4 v[8];
+      c_last = c;
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+      for (int j = 0; j < RB; ++j)
         if (tok[j] >= 0) v[j] = src[(size_t)tok[j] * vec_per_row + c];
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+      for (int j = 0; j < RB; ++j)
         if (tok[j] >= 0) {
           dst[(size_t)(first + r0 + j) * vec_per_row + c] = v[j];
           if (amax_in != nullptr)
@@ -606,31 +616,33 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     }
     if (amax_in != nullptr) {
       // the rows' largest magnitudes (a bf16 magnitude's bits order like the value) and a cleared
-      // word per row for the intermediate rows' maxima
-      __syncthreads();  // the previous batch's s_amax has been read
-      if (threadIdx.x < 8) s_amax[threadIdx.x] = 0u;
-      __syncthreads();
+      // word per row for the intermediate rows' maxima.  One barrier per batch: a batch's words
+      // were cleared two batches (two barriers) ago, and it clears the words of the batch after next.
+      uint32_t* amax_now = s_amax[batch % 3];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < RB; ++j) {
         const uint32_t m = __reduce_max_sync(0xffffffffu, max(big[j] & 0xffffu, big[j] >> 16));
-        if (lane == 0) atomicMax(&s_amax[j], m);
+        if (lane == 0 && m != 0u) atomicMax(&amax_now[j], m);
       }
       __syncthreads();
-      if (threadIdx.x < 8 && r0 + (int)threadIdx.x < rows) {
-        amax_in[first + r0 + threadIdx.x] = s_amax[threadIdx.x] << 16;
-        amax_mid[first + r0 + threadIdx.x] = 0u;
+      if (threadIdx.x < RB) {
+        s_amax[(batch + 2) % 3][threadIdx.x] = 0u;
+        if (r0 + (int)threadIdx.x < rows) {
+          amax_in[first + r0 + threadIdx.x] = amax_now[threadIdx.x] << 16;
+          amax_mid[first + r0 + threadIdx.x] = 0u;
+        }
       }
-      // the rows' two e4m3 terms (each thread re-reads the vectors it has just stored)
+      // the rows' two e4m3 terms (vectors of earlier rounds of the loop above are read back)
       for (int c = threadIdx.x; c < vec_per_row; c += blockDim.x) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
+        for (int j = 0; j < RB; ++j)
           if (tok[j] >= 0) {
             const size_t r = (size_t)(first + r0 + j);
-            const uint4 v = dst[r * vec_per_row + c];
-            const float scale = token_scale(s_amax[j] << 16);
+            const uint4 vv = c == c_last ? v[j] : dst[r * vec_per_row + c];
+            const float scale = token_scale(amax_now[j] << 16);
             uint2 t1, t2;
-            split_bf16x4(v.x, v.y, scale, t1.x, t2.x);
-            split_bf16x4(v.z, v.w, scale, t1.y, t2.y);
+            split_bf16x4(vv.x, vv.y, scale, t1.x, t2.x);
+            split_bf16x4(vv.z, vv.w, scale, t1.y, t2.y);
             uint2* out1 = reinterpret_cast<uint2*>(split.terms_in + r * H);
             uint2* out2 = reinterpret_cast<uint2*>(split.terms_in + ((size_t)split.rows + r) * H);
             out1[c] = t1;
@@ -745,10 +757,13 @@ void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, 
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
                     StepTimeline* timeline, const TokenSplit* split) {
   // gathering steps: up to four CTAs per expert share its rows (batches of eight)
-  const int split_ctas = xp != nullptr ? 4 : 1;
   const TokenSplit sp = xp != nullptr && split != nullptr && split->complete() ? *split : TokenSplit{};
-  launch_pdl(permute_kernel, dim3(E, split_ctas), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
-             timeline, sp);
+  if (sp.complete())
+    launch_pdl(permute_kernel<2>, dim3(E, 8), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
+               timeline, sp);
+  else
+    launch_pdl(permute_kernel<8>, dim3(E, xp != nullptr ? 4 : 1), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm,
+               pos, x, xp, H, K, timeline, sp);
 }
 
 namespace {
