@@ -76,8 +76,13 @@ typedef struct {
  *   OLED_EXPERTS_FP8:  the same three matrices as fp8 e4m3 codes (1 byte each), followed by one
  *     fp32 scale per weight row, s_gate[I] | s_up[I] | s_down[H]; a weight is code * scale of its
  *     row.  3*H*I + 4*(2*I+H) bytes, padded to a multiple of 256.  Half the host-link and HBM
- *     traffic per expert (the paper names quantisation as the complementary lever for H2D volume);
- *     the codes are widened to bf16 on chip (exactly), the arithmetic is the bf16 path's. */
+ *     traffic per expert (the paper names quantisation as the complementary lever for H2D volume).
+ *     Token tiles of at most 32 rows (hidden and intermediate multiples of 128, steps of at most
+ *     4096 token-expert assignments): the tensor cores read the codes as they are; a bf16 token
+ *     row, scaled by a power of two, enters as the sum of two e4m3 terms, which represents every
+ *     element within 2^-14 of the row's largest magnitude exactly (OLED_OPT_FP8_DIRECT).
+ *     Otherwise the codes are widened to bf16 on chip (exactly) and the arithmetic is the bf16
+ *     path's. */
 #define OLED_EXPERTS_BF16 0
 #define OLED_EXPERTS_FP8 1
 /* Bytes of one expert blob in the given format. */
@@ -240,6 +245,9 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * when the first one got past its dependency wait and when the last one finished (GPU global
  * timer); read with oled_debug_timeline().  Off by default (a few atomics per CTA). */
 #define OLED_OPT_TIMELINE 13
+/* OLED_OPT_FP8_DIRECT (fp8 expert stores): 1 (default) = token tiles of at most 32 rows take the
+ * form whose MMAs read the e4m3 codes directly; 0 = every tile widens the codes to bf16. */
+#define OLED_OPT_FP8_DIRECT 14
 #define OLED_TIMELINE_SLOTS 12 /* 0 gate, 1 permutation, 2 gather (not recorded),
                                   3..10 the step's FFN launches in order, 11 combine */
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */

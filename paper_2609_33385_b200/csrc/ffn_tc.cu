@@ -31,7 +31,8 @@
 // warp 16 lane 0 TMA producer, warp 17 lane 0 MMA issuer (warp 17 also owns the TMEM allocation),
 // warps 18-21 widen fp8 weight tiles (fp8 expert stores only, idle otherwise).
 //
-// fp8 expert stores (e4m3 codes + one fp32 scale per weight row): a pipeline stage is a load
+// fp8 expert stores (e4m3 codes + one fp32 scale per weight row), token tiles of 64 and 128 rows
+// (FP8 = 1, "widening"): a pipeline stage is a load
 // slot in shared memory - the code tile of a k-block (64 bytes per weight row, half the bytes in
 // flight of the bf16 form) next to its token tile - plus 32 (64) columns of TENSOR memory.
 // Groups of four converter warps, one per TMEM lane quarter, read the codes, widen them to bf16
@@ -41,6 +42,25 @@
 // never touch shared memory.  The accumulators keep their place in front of the weight stages,
 // which is why the fp8 form stops at token tiles of 128.  The epilogue multiplies each output
 // row by its scale - the rows of a weight tile are the accumulator's lanes.
+//
+// fp8 expert stores, token tiles of at most 32 rows (FP8 = 2, "direct"): the widening form above
+// is bound by the thread that issues the MMAs - an M = 128 instruction consumes 128 weight rows x
+// 16 k whatever the element size, so half the bytes are not half the instructions.  Here the
+// MMAs are kind::f8f6f4 (K = 32 per instruction) and read the e4m3 code tile as the TMA laid it
+// down: a k-block is 128 rows x 128 k, the same 16 KB and the same four instructions as a bf16
+// k-block of 64.  An MMA takes both operands in the same 8-bit kind, so the token rows enter as
+// e4m3 too: every row, scaled by a power of two that brings its largest magnitude into
+// [128, 256), is the sum of two e4m3 terms (fp8_split.h; exact for every element within 2^-14 of
+// the row's maximum, which is as exact as bf16 tokens get next to an fp32 accumulator).  The
+// terms are made once per step and operand - by the gathering permutation kernel for the input
+// rows, by split_rows_kernel between the two projections for the intermediate rows, whose
+// largest magnitudes the gate/up epilogue collects with atomicMax - and loaded as the B tile
+// [term 1 rows | term 2 rows], N = 2 n_box; the epilogue adds the two accumulators (D1 + D2/16)
+// and undoes the row's scale.  No converter warps and no proxy fences in the streaming loop:
+// a form that split the tokens inside the kernel was bound by the fence between the converters'
+// shared-memory writes and the MMA's reads (one per stage, each waiting for the copies in flight).
+// The TMA thread issues one copy for the code tile (a 4-D map whose box takes the 64 gate and
+// the 64 up rows at once) and one for both term tiles per k-block.
 //
 // Every mbarrier wait is bounded: on a timeout the CTA raises a flag in the status word, gives
 // in-flight copies time to land, frees its TMEM and returns.

@@ -112,6 +112,7 @@ struct oled_ctx {
   oled_kernel_profile prof_acc[OLED_N_KERNELS] = {};
   int ffn_impl = 0;
   bool timeline_on = false;    // OLED_OPT_TIMELINE
+  bool fp8_direct = true;      // OLED_OPT_FP8_DIRECT
   StepTimeline* d_timeline = nullptr;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
   bool hit_fused = false;      // this step's resident-group FFN ran as one fused launch
@@ -740,7 +741,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
     // (fp8 stores: a gathering permutation kernel also leaves the rows' magnitudes for the FFN)
-    ctx->step_split = fuse_gather && ctx->split.complete() ? &ctx->split : nullptr;
+    ctx->step_split = fuse_gather && ctx->fp8_direct && ctx->split.complete() ? &ctx->split : nullptr;
     launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
                    static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl, ctx->step_split);
   }
@@ -1156,6 +1157,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       return OLED_OK;
     case OLED_OPT_TIMELINE:
       ctx->timeline_on = value != 0;
+      return OLED_OK;
+    case OLED_OPT_FP8_DIRECT:
+      ctx->fp8_direct = value != 0;
       return OLED_OK;
     default:
       return OLED_ERR_INVALID_ARG;

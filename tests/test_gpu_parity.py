@@ -545,6 +545,49 @@ def test_fp8_expert_store_token_tile_variants(n):
         run.close()
 
 
+def test_fp8_direct_form_agrees_with_widening_form_on_wide_range_rows():
+    """Token tiles of at most 32 rows take the form whose MMAs read the e4m3 codes directly, the
+    token rows entering as two e4m3 terms after a per-row power-of-two scale.  Rows with a wide
+    dynamic range (elements 2^-12 below the row's maximum), an all-zero row and a row 2^10 larger
+    than the rest: same discrete results, outputs within tolerance of the oracle, and the two
+    forms (OLED_OPT_FP8_DIRECT 1 / 0) agree far more closely than either has to with the oracle."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    n = 24
+    run = _runner(w, capacity=[4], max_tokens=n, fp8=True)
+    ora = _oracle_for(run, [4])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 51)
+        f = (h_bits.astype(np.uint32) << 16).view(np.float32).copy()
+        f[:, ::3] *= 2.0 ** -12          # a third of every row far below the row's maximum
+        f[3, :] = 0.0                    # an all-zero row
+        f[5, :] *= 2.0 ** 10             # one row far above the others
+        h_bits = (f.view(np.uint32) >> 16).astype(np.uint16)   # (scaling by powers of two is exact in bf16)
+        c = torch.from_numpy(conf).to(run.device)
+        with np.errstate(over="ignore"):   # exp(-a) of the large row's gate values overflows to inf: silu -> -0
+            ref = ora.denoise_step(0, h_bits, conf)
+        outs = []
+        for direct in (1, 0):
+            run.ctx.set_option(binding.OPT_FP8_DIRECT, direct)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, bits_to_dev(h_bits, run.device), c, out)
+            if direct:
+                _check_step(run, 0, n, out, ref, check_out=False)
+            outs.append(out.float().cpu().numpy().astype(np.float64))
+            run.ctx.reset_cache()
+        a, b = outs
+        assert np.all(a[3] == 0.0) and np.all(b[3] == 0.0) and np.all(ref["out"][3] == 0.0)
+        for t in range(n):   # row by row and relative: the rows differ in scale by orders of magnitude
+            den = np.linalg.norm(ref["out"][t])
+            if den > 0:
+                assert np.linalg.norm(a[t] - ref["out"][t]) / den <= REL_L2, ("direct form against the oracle", t)
+                assert np.linalg.norm(b[t] - ref["out"][t]) / den <= REL_L2, ("widening form against the oracle", t)
+                assert np.linalg.norm(a[t] - b[t]) / den < 3e-3, ("the two forms", t)
+    finally:
+        run.close()
+
+
 def test_fp8_subnormal_codes_decode_exactly():
     """Blobs whose row scales are so large that every code is an e4m3 subnormal (exponent field
     0): the on-chip widening must reproduce them exactly, not flush them."""
