@@ -248,6 +248,10 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
 /* OLED_OPT_FP8_DIRECT (fp8 expert stores): 1 (default) = token tiles of at most 32 rows take the
  * form whose MMAs read the e4m3 codes directly; 0 = every tile widens the codes to bf16. */
 #define OLED_OPT_FP8_DIRECT 14
+/* OLED_OPT_FFN_PAIRS: 1 (default) = many-token steps (token tiles of 256 rows, bf16 stores,
+ * intermediate a multiple of 256, hidden a multiple of 512) run the expert FFN on pairs of CTAs
+ * that share a token tile (tcgen05 cta_group::2); 0 = always one CTA per tile. */
+#define OLED_OPT_FFN_PAIRS 15
 #define OLED_TIMELINE_SLOTS 12 /* 0 gate, 1 permutation, 2 gather (not recorded),
                                   3..10 the step's FFN launches in order, 11 combine */
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "liboled.so")
-SOURCES = ["oled.cu", "route.cu", "combine.cu", "ffn_simple.cu", "ffn_tc.cu", "check.cu"]
+SOURCES = ["oled.cu", "route.cu", "combine.cu", "ffn_simple.cu", "ffn_tc.cu", "ffn_pair.cu", "check.cu"]
 HEADERS = [os.path.join(CSRC, "kernels.h"), os.path.join(CSRC, "policy.h"), os.path.join(CSRC, "sm100_ptx.h"), os.path.join(CSRC, "route_math.h"), os.path.join(CSRC, "fp8_split.h"),
            os.path.join(INCLUDE, "oled.h")]
 

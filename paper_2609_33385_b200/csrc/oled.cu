@@ -1161,6 +1161,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
     case OLED_OPT_FP8_DIRECT:
       ctx->fp8_direct = value != 0;
       return OLED_OK;
+    case OLED_OPT_FFN_PAIRS:
+      ctx->maps.use_pairs = value != 0;
+      return OLED_OK;
     default:
       return OLED_ERR_INVALID_ARG;
   }

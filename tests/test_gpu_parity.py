@@ -165,6 +165,35 @@ def test_many_tokens_per_expert_multi_tile(n):
         run.close()
 
 
+@pytest.mark.parametrize("n", [700, 2100])
+def test_cta_pair_ffn_form_many_tokens(n):
+    """Token tiles of 256 rows with hidden a multiple of 512 and intermediate a multiple of 256: the
+    expert FFN runs on CTA pairs (cta_group::2), each CTA holding half of a token tile.  Ragged
+    last tiles, several tiles per expert; against the oracle, and against the one-CTA form
+    (OLED_OPT_FFN_PAIRS 0), which accumulates every output in the same order."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    run = _runner(w, capacity=[4], max_tokens=n)
+    ora = _oracle_for(run, [4])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 9)
+        c = torch.from_numpy(conf).to(run.device)
+        ref = ora.denoise_step(0, h_bits, conf)
+        assert ref["counts"].max() > 256
+        outs = []
+        for pairs in (1, 0):
+            run.ctx.set_option(binding.OPT_FFN_PAIRS, pairs)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, bits_to_dev(h_bits, run.device), c, out)
+            _check_step(run, 0, n, out, ref)
+            outs.append(out.float().cpu().numpy().astype(np.float64))
+            run.ctx.reset_cache()
+        assert np.linalg.norm(outs[0] - outs[1]) <= 1e-3 * np.linalg.norm(outs[1])
+    finally:
+        run.close()
+
+
 def test_output_bit_identical_at_every_capacity():
     """Offloading is lossless (Sec. 5.1): routing and output do not depend on the capacity."""
     from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
