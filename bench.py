@@ -43,11 +43,11 @@ NCU_TRAFFIC_RATIO = {
     # the one-launch form runs the same items as those two kernels together
     ("ffn_fused", "few_tokens"): (504.42 + 4.48 + 252.23 + 7.01) / (504.9 + 254.4),
     # profiles/ffn_tc_kernel_fp8_cfg2_full_residency.md: the same launch with fp8 stores
-    ("ffn_gate_up", "few_tokens", "fp8"): (265.88 + 4.06) / 266.6,
-    ("ffn_down", "few_tokens", "fp8"): (133.23 + 4.07) / 135.2,
-    # profiles/ffn_tc_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
-    ("ffn_gate_up", "many_tokens"): (1916.5 + 102.1) / 1979.7,
-    ("ffn_down", "many_tokens"): (911.8 + 264.5) / 1174.4,
+    ("ffn_gate_up", "few_tokens", "fp8"): (261.71 + 4.15) / 270.6,
+    ("ffn_down", "few_tokens", "fp8"): (131.12 + 4.37) / 136.9,
+    # profiles/ffn_pair_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
+    ("ffn_gate_up", "many_tokens"): (1944.0 + 100.7) / 1979.7,
+    ("ffn_down", "many_tokens"): (909.4 + 264.2) / 1174.4,
 }
 
 
