@@ -191,3 +191,33 @@ def test_misaligned_pointers_are_rejected_before_anything_is_launched(binding):
     for name in ("conf", "gate", "counts", "offsets", "perm"):
         assert call(**{name: args[name] + 2}) == binding.ERR_INVALID_ARG, name
     assert call(bias=ok4 + 1) == binding.ERR_INVALID_ARG
+
+
+def test_two_e4m3_terms_hold_a_scaled_bf16_row():
+    """The arithmetic the direct fp8 tensor-core form rests on (csrc/fp8_split.h), restated in numpy
+    with the oracle's decoder: a bf16 row scaled by the power of two that brings its largest
+    magnitude into [128, 256) equals t1 + t2/16 with t1 = e4m3(v), t2 = e4m3(16 (v - t1)) -
+    exactly for every element within 2^-14 of the row's maximum, and to 2^-22 of the maximum
+    below that."""
+    from oracle.moe_layer import fp8_e4m3_to_f32
+    from paper_2609_33385_b200 import synth
+    rng = np.random.default_rng(5)
+    rows = []
+    for spread in (0, 6, 14, 20, 30):                      # binades between a row's largest and smallest elements
+        mant = rng.integers(128, 256, size=(64, 512)).astype(np.float64)          # 8 significant bits
+        expo = rng.integers(-spread, 1, size=(64, 512)) + rng.integers(-40, 40, size=(64, 1))
+        rows.append(np.ldexp(mant, expo - 7) * rng.choice([-1.0, 1.0], size=(64, 512)))
+    x = np.concatenate(rows)
+    x[3] = 0.0                                              # an all-zero row
+    assert np.array_equal(synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(x.astype(np.float32))).astype(np.float64), x)
+    amax = np.abs(x).max(axis=1, keepdims=True)
+    _, ex = np.frexp(np.where(amax > 0, amax, 1.0))        # amax = m * 2^ex, m in [0.5, 1)
+    scale = np.ldexp(1.0, 8 - ex)                          # amax * scale in [128, 256)
+    v = x * scale
+    assert np.all((np.abs(v).max(axis=1) >= 128) | (amax[:, 0] == 0)) and np.abs(v).max() < 256
+    t1 = fp8_e4m3_to_f32(synth.f32_to_e4m3_codes(v)).astype(np.float64)
+    t2 = fp8_e4m3_to_f32(synth.f32_to_e4m3_codes((v - t1) * 16.0)).astype(np.float64)
+    err = np.abs(t1 + t2 / 16.0 - v)
+    exact_zone = np.abs(v) >= 2.0 ** -6                    # within 2^-14 of a maximum of at least 128
+    assert exact_zone.mean() > 0.5 and np.all(err[exact_zone] == 0.0)
+    assert err.max() <= 2.0 ** -14 and (~exact_zone).any()  # 2^-22 of the smallest scaled maximum (128)
