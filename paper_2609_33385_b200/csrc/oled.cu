@@ -23,6 +23,7 @@ namespace {
 struct LayerData {
   LayerCacheState cache;
   int32_t last_active = -1;      // experts activated at the layer's previous execution (-1: none yet)
+  int32_t last_max_count = -1;   // most token rows any expert received then
   const uint8_t* host_blob = nullptr;
   size_t host_stride = 0;
   uint16_t* w_router = nullptr;  // device [E,H]
@@ -785,7 +786,10 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     // (how many of the residents will have tokens is not known yet: the layer's previous
     // execution is the estimate - adjacent iterations activate mostly the same experts, Sec. 3.3)
     const int expected = std::min<int>(grp.n, L.last_active >= 0 ? L.last_active : E);
-    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(32, 2 * mean_load)), nullptr, nullptr, false,
+    // (direct fp8 form: its token operand is two rows per token and a third of a stage at 32, so
+    // where the layer's previous execution gave no expert more than 16 rows the tile is 16)
+    const int floor_rows = ctx->step_split != nullptr && L.last_max_count >= 0 && L.last_max_count <= 16 ? 16 : 32;
+    const int rc0 = run_ffn_launches(ctx, grp, std::min(T, std::max(floor_rows, 2 * mean_load)), nullptr, nullptr, false,
                                      expected, &ctx->hit_fused, rep);
     if (rc0 != OLED_OK) return rc0;
   }
@@ -916,6 +920,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.stats.evictions += (uint64_t)plan.n_evictions;
   L.stats.active_experts += (uint64_t)plan.n_active;
   L.last_active = plan.n_active;
+  L.last_max_count = 0;
+  for (int32_t e = 0; e < E; ++e) L.last_max_count = std::max(L.last_max_count, counts[e]);
   L.stats.assignments += (uint64_t)T * K;
   L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
   L.stats.ideal_hits += (uint64_t)std::min<int64_t>(plan.n_active, plan.capacity_used);
