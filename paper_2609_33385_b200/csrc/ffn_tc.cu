@@ -1071,9 +1071,16 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   // themselves (mode 2); otherwise converter warps widen them to bf16 (mode 1)
   const bool direct = fp8 && maps.e4m3_direct && grp.n_box <= 32 && split != nullptr && split->complete();
   const int mode = direct ? 2 : fp8 ? 1 : 0;
-  if (kind != 3 && maps.use_pairs && ffn_pair_usable(maps, grp.n_box, H, I))
-    return launch_ffn_pair(st, maps, grp, kind, offsets, hbuf, y, y_bf16, H, I, n_sms, status, work_counter, timeline,
-                           timeline_slot, report);
+  // many-token tiles: the CTA-pair kernel, unless its cluster launch has failed before on this
+  // device (the one-CTA form below computes the same) or the test aid that withholds loads is on
+  static bool pairs_refused = false;
+  if (kind != 3 && maps.use_pairs && !pairs_refused && !grp.withhold_loads && ffn_pair_usable(maps, grp.n_box, H, I)) {
+    if (launch_ffn_pair(st, maps, grp, kind, offsets, hbuf, y, y_bf16, H, I, n_sms, status, work_counter, timeline,
+                        timeline_slot, report) == OLED_OK)
+      return OLED_OK;
+    cudaGetLastError();  // (a refused launch enqueues nothing)
+    pairs_refused = true;
+  }
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int m_tiles) {
     if (host_counts == nullptr) return n_sms;  // counts not known on the host yet
