@@ -245,25 +245,11 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
       }
       // elements in ascending h: word 0 low half, word 0 high half, word 1 low half, ...
 #pragma unroll
-      for (int wi = 0; wi < 4; ++wi) {
-        float xf[TT], wf[kEPerWarp];
-#pragma unroll
-        for (int a = 0; a < TT; ++a) xf[a] = bf16_lo(xw[a][wi]);
-#pragma unroll
-        for (int b = 0; b < kEPerWarp; ++b) wf[b] = bf16_lo(ww[b][wi]);
+      for (int wi = 0; wi < 4; ++wi)
 #pragma unroll
         for (int a = 0; a < TT; ++a)
 #pragma unroll
-          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf[a], wf[b], acc[a][b]);
-#pragma unroll
-        for (int a = 0; a < TT; ++a) xf[a] = bf16_hi(xw[a][wi]);
-#pragma unroll
-        for (int b = 0; b < kEPerWarp; ++b) wf[b] = bf16_hi(ww[b][wi]);
-#pragma unroll
-        for (int a = 0; a < TT; ++a)
-#pragma unroll
-          for (int b = 0; b < kEPerWarp; ++b) acc[a][b] = __fmaf_rn(xf[a], wf[b], acc[a][b]);
-      }
+          for (int b = 0; b < kEPerWarp; ++b) fma_bf16_pair(acc[a][b], xw[a][wi], ww[b][wi]);
     }
 #pragma unroll
     for (int a = 0; a < TT; ++a)
@@ -345,14 +331,6 @@ route_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wr,
 // in ascending order.  Experts beyond 64 take further passes over the rows.
 constexpr int kManyWarps = 8, kManyExperts = 64, kManyStages = 4;
 __host__ __device__ constexpr int many_stage_bytes(int tt) { return (tt + kManyExperts) * 512; }  // one k-chunk of 256 bf16 per row
-
-// acc += x.lo * w.lo, then acc += x.hi * w.hi (ascending h), each an fp32 fused multiply-add
-__device__ __forceinline__ void fma_bf16_pair(float& acc, uint32_t x, uint32_t w) {
-  asm("{\n .reg .b16 xl, xh, wl, wh;\n mov.b32 {xl, xh}, %1;\n mov.b32 {wl, wh}, %2;\n"
-      " fma.rn.f32.bf16 %0, xl, wl, %0;\n fma.rn.f32.bf16 %0, xh, wh, %0;\n}"
-      : "+f"(acc)
-      : "r"(x), "r"(w));
-}
 
 template <int TT>
 __global__ void __launch_bounds__(kManyWarps * 32, 1)

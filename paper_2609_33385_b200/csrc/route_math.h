@@ -9,6 +9,17 @@ namespace oled {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// acc += x.lo * w.lo, then acc += x.hi * w.hi (ascending h) for two packed bf16 pairs, each step
+// an fp32 fused multiply-add: fma.rn.f32.bf16 forms the exact product of its bf16 operands and
+// rounds once - bit for bit __fmaf_rn of the widened operands - and saves the widening
+// instructions, which outnumber the multiply-adds in the gate kernels' small register tiles.
+__device__ __forceinline__ void fma_bf16_pair(float& acc, uint32_t x, uint32_t w) {
+  asm("{\n .reg .b16 xl, xh, wl, wh;\n mov.b32 {xl, xh}, %1;\n mov.b32 {wl, wh}, %2;\n"
+      " fma.rn.f32.bf16 %0, xl, wl, %0;\n fma.rn.f32.bf16 %0, xh, wh, %0;\n}"
+      : "+f"(acc)
+      : "r"(x), "r"(w));
+}
+
 // exp(x) for x <= 0 from individually rounded fp32 operations (no contraction, no fast math).
 __device__ __forceinline__ float exp_spec(float x) {
   if (x < -80.0f) return 0.0f;
