@@ -73,16 +73,42 @@ constexpr uint32_t kPairSmem = kPairCtlBytes + 1024u + kPairStages * kPairStage;
 
 struct PairItem {
   int slot, m0, row0, valid;
+  int kind;  // 1: gate/up (+SwiGLU), 2: down projection
+  int g;     // index of the expert in the launch's group
 };
-// item -> (expert, token tile, feature block of the pair); cur_g only moves forward
-__device__ __forceinline__ void pair_decode(const PairCtl* ctl, const FfnGroup& grp, int item, int m_blocks, int m_rows,
-                                            int& cur_g, PairItem& it) {
+// A role's position in the expert list: items arrive in ascending order within a phase, so the
+// search for an item's expert only moves forward; it restarts with the second phase of a fused launch.
+struct PairCursor {
+  int g = 0;
+  int phase2 = 0;
+};
+// How a launch's item numbers divide: [0, n1) items of kind1 with m_blocks1 feature blocks per
+// token tile, then (a fused launch) the down items of the same token tiles with m_blocks2 blocks.
+struct PairPlan {
+  int kind1, n1, m_blocks1, m_blocks2;
+};
+// item -> (kind, expert, token tile, feature block of the pair)
+__device__ __forceinline__ void pair_decode(const PairCtl* ctl, const FfnGroup& grp, int item, const PairPlan& plan,
+                                            PairCursor& cur, PairItem& it) {
+  int m_blocks = plan.m_blocks1;
+  it.kind = plan.kind1;
+  if (item >= plan.n1) {
+    item -= plan.n1;
+    m_blocks = plan.m_blocks2;
+    it.kind = 2;
+    if (!cur.phase2) {
+      cur.phase2 = 1;
+      cur.g = 0;
+    }
+  }
+  const int m_rows = it.kind == 1 ? 256 : 512;  // features / output rows per pair item
   const int q = item / m_blocks;
   const int m = item - q * m_blocks;
-  int g = cur_g;
+  int g = cur.g;
   while (ctl->tile_prefix[g + 1] <= q) ++g;
-  cur_g = g;
+  cur.g = g;
   const int nt = q - ctl->tile_prefix[g];
+  it.g = g;
   it.slot = grp.slot[g];
   it.m0 = m * m_rows;
   it.row0 = ctl->row_start[g] + nt * kPairN;
@@ -126,12 +152,30 @@ __device__ __forceinline__ int take_pair_item(PairCtl* ctl, int seq, volatile in
   return *reinterpret_cast<volatile int*>(&ctl->item_ring[slot]);
 }
 
+// What a FUSED launch (KIND 3) needs on top: the down projection's tensor maps, its output and the
+// completion counters (one ZERO word per expert of the group).
+struct PairSecond {
+  CUtensorMap tm_w2;    // down-projection weights
+  CUtensorMap tm_act2;  // intermediate rows (hbuf)
+  void* out2;           // y
+  uint32_t* done;       // per expert: epilogue warps (of either CTA) that have stored gate/up rows
+};
+
+// KIND 3: the gate/up items, then the down items of the same experts, in ONE launch (a launch
+// boundary between cluster kernels is a full stop: a dependent cluster launch was never seen to
+// start before its predecessor had finished, so the last gate/up items' uneven end and the next
+// launch's set-up would leave SMs idle).  A down item reads the intermediate rows the gate/up
+// items of its expert wrote; its TMA threads wait (bounded) until the expert's counter shows
+// that all of them are stored - items are handed out in order, gate/up first, so that wait is
+// over long before it is reached except at the switch of phases.
 template <int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_act,
                 const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets, void* __restrict__ out_ptr,
                 int H, int I, int out_bf16, uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter,
-                StepTimeline* timeline, int timeline_slot, const __grid_constant__ RouteReport report) {
+                StepTimeline* timeline, int timeline_slot, const __grid_constant__ RouteReport report,
+                const __grid_constant__ PairSecond sec) {
+  constexpr bool fused = KIND == 3;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   PairCtl* ctl = reinterpret_cast<PairCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kPairCtlBytes + 1023u) & ~1023u;
@@ -156,6 +200,10 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   if (warp == kPairProducerWarp && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_act)) : "memory");
+    if (fused) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&sec.tm_w2)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&sec.tm_act2)) : "memory");
+    }
   }
   if (warp == kPairMmaWarp) {  // all 512 columns, allocated by the same warp of both CTAs
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
@@ -187,21 +235,26 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   tc_fence_after();
 
   const uint32_t tmem_base = ctl->tmem_base;
-  // features (KIND 1) / output rows (KIND 2) per CTA and per pair item
-  constexpr int kCtaRows = KIND == 1 ? 128 : 256;
-  const int m_rows = 2 * kCtaRows;
-  const int m_blocks = (KIND == 1 ? I : H) / m_rows;
-  const int k_blocks = (KIND == 1 ? H : I) / kPairK;
-  const int total_items = ctl->n_tiles_total * m_blocks;
+  // per pair item: 256 features (kind 1: 128 per CTA, their gate and up rows) or 512 output rows
+  // (kind 2: 256 per CTA, two row blocks of Wd)
+  PairPlan plan;
+  plan.kind1 = KIND == 2 ? 2 : 1;
+  plan.m_blocks1 = KIND == 2 ? H / 512 : I / 256;
+  plan.m_blocks2 = H / 512;
+  plan.n1 = fused ? ctl->n_tiles_total * plan.m_blocks1 : 0x7fffffff;
+  const int total_items = ctl->n_tiles_total * (plan.m_blocks1 + (fused ? plan.m_blocks2 : 0));
+  // (fused) gate/up epilogue warps of both CTAs that store rows per item, times the gate/up items of a token tile
+  const uint32_t done_per_tile = (uint32_t)(2 * kPairEpiWarps * (I / 256));
   volatile int* abort_flag = &ctl->abort;
   const uint32_t full_on_first = map_to_cta(smem_u32(&ctl->full[0]), 0);         // cluster-wide addresses
   const uint32_t tmem_empty_on_first = map_to_cta(smem_u32(&ctl->tmem_empty), 0);
 
-  if (KIND == 1 && blockIdx.x == 0 && warp == kPairProducerWarp && lane != 0) publish_report(report, lane - 1, 31);
+  if (KIND != 2 && blockIdx.x == 0 && warp == kPairProducerWarp && lane != 0) publish_report(report, lane - 1, 31);
 
   if (warp == kPairProducerWarp && lane == 0) {
     // ------------------------------------------------------------ TMA producer (one per CTA)
-    int stage = 0, cur_g = 0;
+    int stage = 0, ready_g = -1;
+    PairCursor cur;
     uint32_t phase = 0;
     bool ok = true;
     int next_item = pair;  // (first CTA) the pair's first item is its own number
@@ -222,10 +275,38 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       }
       if (item < 0) break;
       PairItem it;
-      pair_decode(ctl, grp, item, m_blocks, m_rows, cur_g, it);
+      pair_decode(ctl, grp, item, plan, cur, it);
+      const bool down_of_fused = fused && it.kind == 2;
+      const CUtensorMap* map_w = down_of_fused ? &sec.tm_w2 : &tm_w;
+      const CUtensorMap* map_act = down_of_fused ? &sec.tm_act2 : &tm_act;
+      const int k_blocks = (it.kind == 1 ? H : I) / kPairK;
+      if (down_of_fused && it.g != ready_g) {
+        // all intermediate rows of this expert stored?  (an expert seen complete stays complete)
+        const uint32_t target = (uint32_t)(ctl->tile_prefix[it.g + 1] - ctl->tile_prefix[it.g]) * done_per_tile;
+        unsigned long long t0 = 0;
+        for (uint32_t spin = 0; ok; ++spin) {
+          uint32_t seen;
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(sec.done + it.g) : "memory");
+          if (seen >= target) break;
+          if ((spin & 255u) == 255u) {
+            if (*abort_flag) ok = false;
+            const unsigned long long now = globaltimer();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
+              *abort_flag = 1;
+              atomicExch(status, (uint32_t)kStatusWaitTimeout);
+              ok = false;
+            }
+          }
+        }
+        if (!ok) break;
+        ready_g = it.g;
+        // the rows were written through the generic proxy; the copies below read through the async proxy
+        asm volatile("fence.proxy.async;" ::: "memory");
+      }
       const int n_mma = max(32, (it.valid + 31) & ~31);
       const int my_row0 = it.row0 + (int)rank * (n_mma >> 1);  // this CTA's half of the tile's token rows
-      const int my_m0 = it.m0 + (int)rank * kCtaRows;
+      const int my_m0 = it.m0 + (int)rank * (it.kind == 1 ? 128 : 256);
       for (int kb = 0; kb < k_blocks; ++kb) {
         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, status)) {
           ok = false;
@@ -235,14 +316,14 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[stage]), 2u * kPairStage);
         const uint32_t base = tiles_base + (uint32_t)stage * kPairStage;
         const int k0 = kb * kPairK;
-        if (KIND == 1) {
-          tma_load_3d_pair(&tm_w, base, bar, k0, my_m0, it.slot);                   // gate rows
-          tma_load_3d_pair(&tm_w, base + kPairATile, bar, k0, I + my_m0, it.slot);  // up rows
+        if (it.kind == 1) {
+          tma_load_3d_pair(map_w, base, bar, k0, my_m0, it.slot);                   // gate rows
+          tma_load_3d_pair(map_w, base + kPairATile, bar, k0, I + my_m0, it.slot);  // up rows
         } else {
-          tma_load_3d_pair(&tm_w, base, bar, k0, my_m0, it.slot);
-          tma_load_3d_pair(&tm_w, base + kPairATile, bar, k0, my_m0 + 128, it.slot);
+          tma_load_3d_pair(map_w, base, bar, k0, my_m0, it.slot);
+          tma_load_3d_pair(map_w, base + kPairATile, bar, k0, my_m0 + 128, it.slot);
         }
-        tma_load_2d_pair(&tm_act, base + 2 * kPairATile, bar, k0, my_row0);
+        tma_load_2d_pair(map_act, base + 2 * kPairATile, bar, k0, my_row0);
         if (++stage == kPairStages) {
           stage = 0;
           phase ^= 1u;
@@ -256,7 +337,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     }
   } else if (warp == kPairMmaWarp && lane == 0 && rank == 0) {
     // ------------------------------------------------------------ MMA issuer (first CTA only)
-    int stage = 0, cur_g = 0, local = 0;
+    int stage = 0, local = 0;
+    PairCursor cur;
     uint32_t phase = 0;
     bool ok = true;
     const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
@@ -268,7 +350,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       const int item = take_pair_item(ctl, local, abort_flag, status);
       if (item < 0) break;
       PairItem it;
-      pair_decode(ctl, grp, item, m_blocks, m_rows, cur_g, it);
+      pair_decode(ctl, grp, item, plan, cur, it);
+      const int k_blocks = (it.kind == 1 ? H : I) / kPairK;
       // one accumulator stage: both CTAs' epilogues must have drained the previous item
       if (!mbar_wait(smem_u32(&ctl->tmem_empty), ((uint32_t)local & 1u) ^ 1u, abort_flag, status)) break;
       tc_fence_after();
@@ -302,7 +385,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   } else if (warp < kPairEpiWarps) {
     // ------------------------------------------------------------ epilogue (both CTAs)
     // warp w: TMEM lane quarter w mod 4 (32 of the CTA's 128 rows), every fourth 16-column chunk
-    int cur_g = 0, local = 0;
+    int local = 0;
+    PairCursor cur;
     const int quarter = warp & 3, part = warp >> 2;
     for (;; ++local) {
       int item = 0;
@@ -310,7 +394,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       item = __shfl_sync(0xffffffffu, item, 0);
       if (item < 0) break;
       PairItem it;
-      pair_decode(ctl, grp, item, m_blocks, m_rows, cur_g, it);
+      pair_decode(ctl, grp, item, plan, cur, it);
       int ready = 0;
       if (lane == 0) ready = mbar_wait(smem_u32(&ctl->tmem_full), (uint32_t)local & 1u, abort_flag, status) ? 1 : 0;
       ready = __shfl_sync(0xffffffffu, ready, 0);
@@ -318,7 +402,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
       const int n_mma = max(32, (it.valid + 31) & ~31);
-      const int col = it.m0 + (int)rank * kCtaRows + quarter * 32 + lane;  // feature / output row of this thread
+      const int col = it.m0 + (int)rank * (it.kind == 1 ? 128 : 256) + quarter * 32 + lane;  // feature / output row of this thread
+      void* const out_y = fused ? sec.out2 : out_ptr;
       // The warp's chunks, one in registers while the next one's TMEM loads are in flight; the
       // accumulators are handed back as soon as the LAST chunk has been read - its arithmetic and
       // stores run while the MMAs of the next item already write the columns.
@@ -348,7 +433,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           released = true;
         }
         const bool whole = c + 16 <= it.valid;  // no ragged end inside this chunk
-        if (KIND == 1) {
+        if (it.kind == 1) {
           uint16_t* p = reinterpret_cast<uint16_t*>(out_ptr) + (size_t)(it.row0 + c) * I + col;
 #pragma unroll
           for (int j = 0; j < 16; ++j, p += I)
@@ -359,7 +444,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
               *p = *reinterpret_cast<const uint16_t*>(&b);
             }
         } else if (out_bf16) {  // many-token steps keep y in bf16
-          uint16_t* p = reinterpret_cast<uint16_t*>(out_ptr) + (size_t)(it.row0 + c) * H + col;
+          uint16_t* p = reinterpret_cast<uint16_t*>(out_y) + (size_t)(it.row0 + c) * H + col;
 #pragma unroll
           for (int j = 0; j < 16; ++j, p += H)
             if (whole || c + j < it.valid) {
@@ -369,7 +454,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
               p[128] = *reinterpret_cast<const uint16_t*>(&b1);
             }
         } else {
-          float* p = reinterpret_cast<float*>(out_ptr) + (size_t)(it.row0 + c) * H + col;
+          float* p = reinterpret_cast<float*>(out_y) + (size_t)(it.row0 + c) * H + col;
 #pragma unroll
           for (int j = 0; j < 16; ++j, p += H)
             if (whole || c + j < it.valid) {
@@ -382,6 +467,14 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(tmem_empty_on_first);
+      }
+      if (fused && it.kind == 1) {
+        // this warp's intermediate rows of the item are stored: visible device-wide (and to the
+        // async proxy of the down items' copies), then counted
+        __threadfence();
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) atomicAdd(sec.done + it.g, 1u);
       }
     }
   }
@@ -406,22 +499,33 @@ bool ffn_pair_usable(const FfnTcMaps& maps, int n_box, int H, int I) {
 
 int launch_ffn_pair(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int kind, const int32_t* offsets,
                     uint16_t* hbuf, float* y, int y_bf16, int H, int I, int n_sms, uint32_t* status,
-                    uint32_t* work_counter, StepTimeline* timeline, int timeline_slot, const RouteReport& report) {
+                    uint32_t* work_counter, StepTimeline* timeline, int timeline_slot, const RouteReport& report,
+                    uint32_t* done) {
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(ffn_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem) != cudaSuccess)
+        cudaFuncSetAttribute(ffn_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_pair_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmem) != cudaSuccess)
       return OLED_ERR_CUDA;
     attr_done = true;
   }
   const int grid = 2 * (n_sms / 2);  // one CTA per SM, in pairs
   cudaError_t err;
-  if (kind == 1)
+  PairSecond sec;
+  sec.tm_w2 = maps.w2;
+  sec.tm_act2 = maps.hbuf[3];
+  sec.out2 = y;
+  sec.done = done;
+  if (kind == 3) {
+    if (done == nullptr) return OLED_ERR_INVALID_ARG;
+    err = launch_pdl(ffn_pair_kernel<3>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w13, maps.xp[3], grp, offsets,
+                     (void*)hbuf, H, I, y_bf16, status, work_counter, timeline, timeline_slot, report, sec);
+  } else if (kind == 1)
     err = launch_pdl(ffn_pair_kernel<1>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w13, maps.xp[3], grp, offsets,
-                     (void*)hbuf, H, I, 0, status, work_counter, timeline, timeline_slot, report);
+                     (void*)hbuf, H, I, 0, status, work_counter, timeline, timeline_slot, report, sec);
   else
     err = launch_pdl(ffn_pair_kernel<2>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w2, maps.hbuf[3], grp,
-                     offsets, (void*)y, H, I, y_bf16, status, work_counter, timeline, timeline_slot, RouteReport{});
+                     offsets, (void*)y, H, I, y_bf16, status, work_counter, timeline, timeline_slot, RouteReport{}, sec);
   return err == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
 

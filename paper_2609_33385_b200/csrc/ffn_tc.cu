@@ -984,6 +984,8 @@ void launch_variant(int fp8, int grid, cudaStream_t st, const CUtensorMap& tw, c
 
 }  // namespace
 
+static bool g_pairs_refused = false;  // a cluster launch of the pair kernel failed on this device once
+
 int ffn_tc_setup(FfnTcMaps* maps, const uint8_t* pool, size_t slot_bytes, int n_slots, int H, int I, bool fp8,
                  const uint16_t* xp, const uint16_t* hbuf, int rows, const TokenSplit* split) {
   maps->fp8 = fp8;
@@ -1073,13 +1075,22 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   const int mode = direct ? 2 : fp8 ? 1 : 0;
   // many-token tiles: the CTA-pair kernel, unless its cluster launch has failed before on this
   // device (the one-CTA form below computes the same) or the test aid that withholds loads is on
-  static bool pairs_refused = false;
-  if (kind != 3 && maps.use_pairs && !pairs_refused && !grp.withhold_loads && ffn_pair_usable(maps, grp.n_box, H, I)) {
+  if (maps.use_pairs && !g_pairs_refused && !grp.withhold_loads && ffn_pair_usable(maps, grp.n_box, H, I)) {
     if (launch_ffn_pair(st, maps, grp, kind, offsets, hbuf, y, y_bf16, H, I, n_sms, status, work_counter, timeline,
-                        timeline_slot, report) == OLED_OK)
+                        timeline_slot, report, done) == OLED_OK)
       return OLED_OK;
     cudaGetLastError();  // (a refused launch enqueues nothing)
-    pairs_refused = true;
+    g_pairs_refused = true;
+  }
+  if (kind == 3 && grp.n_box > 32) {
+    // (only reached when the pair launch was refused: the two launches of the one-CTA form, the
+    // work counter cleared in stream order between them)
+    int rc = launch_ffn_tc(st, maps, grp_in, max_count, 1, host_counts, offsets, hbuf, y, y_bf16, H, I, n_sms, status,
+                           work_counter, behind_event_wait, timeline, timeline_slot, report_in, done, split);
+    if (rc != OLED_OK) return rc;
+    if (cudaMemsetAsync(work_counter, 0, sizeof(uint32_t), st) != cudaSuccess) return OLED_ERR_CUDA;
+    return launch_ffn_tc(st, maps, grp_in, max_count, 2, host_counts, offsets, hbuf, y, y_bf16, H, I, n_sms, status,
+                         work_counter, false, timeline, timeline_slot, report_in, done, split);
   }
   // one CTA per SM, fewer if the group has fewer (weight tile, token tile) items than SMs
   auto grid_for = [&](int m_tiles) {
@@ -1140,6 +1151,9 @@ int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenS
 
 bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count) {
   return !maps.fp8 && (16 << box_index(max_count, 256)) <= 32;
+}
+bool ffn_pair_can_fuse(const FfnTcMaps& maps, int max_count, int H, int I) {
+  return maps.use_pairs && !g_pairs_refused && ffn_pair_usable(maps, 16 << box_index(max_count, maps.fp8 ? 128 : 256), H, I);
 }
 
 }  // namespace oled

@@ -232,12 +232,15 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, i
                   const TokenSplit* split = nullptr);
 int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenSplit* split);
 bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
+bool ffn_pair_can_fuse(const FfnTcMaps& maps, int max_count, int H, int I);  // kind 3 on CTA pairs
 // ---- ffn_pair.cu: the many-token form on CTA pairs (bf16 stores, token tiles of 256 rows,
-// intermediate a multiple of 256 and hidden a multiple of 512); kinds 1 and 2 as above.
+// intermediate a multiple of 256 and hidden a multiple of 512); kinds 1 and 2 as above, kind 3 both
+// in one launch (`done`: one ZERO word per expert of the group).
 bool ffn_pair_usable(const FfnTcMaps& maps, int n_box, int H, int I);
 int launch_ffn_pair(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, int kind, const int32_t* offsets,
                     uint16_t* hbuf, float* y, int y_bf16, int H, int I, int n_sms, uint32_t* status,
-                    uint32_t* work_counter, StepTimeline* timeline, int timeline_slot, const RouteReport& report);
+                    uint32_t* work_counter, StepTimeline* timeline, int timeline_slot, const RouteReport& report,
+                    uint32_t* done = nullptr);
 constexpr int kFfnWorkCounters = 8;  // FFN launches of one layer execution: 3 groups x 2 kinds, rounded up
 
 // Self-check (check.cu): invariants of the routing and the permutation, guard words.

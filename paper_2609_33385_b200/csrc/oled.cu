@@ -378,8 +378,11 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
     // start hides the boundary; measured 125 against 129 us for 63 experts); with few, the SMs
     // that run out of gate/up items would idle until the whole gate/up launch has finished.
     const bool few_items = (long long)expected_experts * (I / 64) < 4ll * ctx->n_sms;
-    const bool fuse = before_down == nullptr && !ctx->y_bf16 && ffn_tc_can_fuse(ctx->maps, max_count) &&
-                      (ctx->fuse_ffn == 2 || (ctx->fuse_ffn == 1 && few_items));
+    // Many-token tiles on CTA pairs: always one launch (a boundary between cluster kernels is a full stop).
+    const bool fuse_pairs = before_down == nullptr && ctx->fuse_ffn != 0 && ffn_pair_can_fuse(ctx->maps, max_count, H, I);
+    const bool fuse = fuse_pairs ||
+                      (before_down == nullptr && !ctx->y_bf16 && ffn_tc_can_fuse(ctx->maps, max_count) &&
+                       (ctx->fuse_ffn == 2 || (ctx->fuse_ffn == 1 && few_items)));
     for (int kind = fuse ? 3 : 1; kind <= (fuse ? 3 : 2); ++kind) {
       if (kind == 2 && before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
       ProfScope ps(ctx, kind == 3 ? OLED_KERNEL_FFN_FUSED : kind == 1 ? OLED_KERNEL_FFN_GATE_UP : OLED_KERNEL_FFN_DOWN, 0, 0);

@@ -169,8 +169,10 @@ def test_many_tokens_per_expert_multi_tile(n):
 def test_cta_pair_ffn_form_many_tokens(n):
     """Token tiles of 256 rows with hidden a multiple of 512 and intermediate a multiple of 256: the
     expert FFN runs on CTA pairs (cta_group::2), each CTA holding half of a token tile.  Ragged
-    last tiles, several tiles per expert; against the oracle, and against the one-CTA form
-    (OLED_OPT_FFN_PAIRS 0), which accumulates every output in the same order."""
+    last tiles, several tiles per expert; against the oracle, against the one-CTA form
+    (OLED_OPT_FFN_PAIRS 0), which accumulates every output in the same order, and the one-launch
+    pair form (gate/up items, then down items behind per-expert counters) against the two-launch
+    one (OLED_OPT_FUSE_FFN 0)."""
     from paper_2609_33385_b200 import binding
     from paper_2609_33385_b200.runner import bits_to_dev
     w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
@@ -182,14 +184,16 @@ def test_cta_pair_ffn_form_many_tokens(n):
         ref = ora.denoise_step(0, h_bits, conf)
         assert ref["counts"].max() > 256
         outs = []
-        for pairs in (1, 0):
+        for pairs, fuse in ((1, 1), (0, 1), (1, 0)):   # one launch on pairs; one CTA per tile; two launches on pairs
             run.ctx.set_option(binding.OPT_FFN_PAIRS, pairs)
+            run.ctx.set_option(binding.OPT_FUSE_FFN, fuse)
             out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
             run.step(0, bits_to_dev(h_bits, run.device), c, out)
             _check_step(run, 0, n, out, ref)
             outs.append(out.float().cpu().numpy().astype(np.float64))
             run.ctx.reset_cache()
         assert np.linalg.norm(outs[0] - outs[1]) <= 1e-3 * np.linalg.norm(outs[1])
+        assert np.array_equal(outs[0], outs[2])   # the same items in the same arithmetic, one launch or two
     finally:
         run.close()
 
