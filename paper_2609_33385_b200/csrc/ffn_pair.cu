@@ -258,10 +258,12 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     uint32_t phase = 0;
     bool ok = true;
     int next_item = pair;  // (first CTA) the pair's first item is its own number
-    for (int seq = 0; ok; ++seq) {
+    // (with loads withheld - the test of the bounded waits - nothing is published either: every
+    // other role of both CTAs runs into the limit of its wait for the first item)
+    for (int seq = 0; ok && !(grp.withhold_loads && rank == 0); ++seq) {
       int item;
       if (rank == 0) {
-        item = next_item < total_items && !grp.withhold_loads ? next_item : -1;
+        item = next_item < total_items ? next_item : -1;
         // the following item's number is fetched now: the atomic's latency lies under this item's copies
         if (item >= 0) next_item = (int)atomicAdd(work_counter, 1u) + n_pairs;
         const int slot = seq % kPairRing;

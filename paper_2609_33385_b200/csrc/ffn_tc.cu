@@ -1074,8 +1074,8 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   const bool direct = fp8 && maps.e4m3_direct && grp.n_box <= 32 && split != nullptr && split->complete();
   const int mode = direct ? 2 : fp8 ? 1 : 0;
   // many-token tiles: the CTA-pair kernel, unless its cluster launch has failed before on this
-  // device (the one-CTA form below computes the same) or the test aid that withholds loads is on
-  if (maps.use_pairs && !g_pairs_refused && !grp.withhold_loads && ffn_pair_usable(maps, grp.n_box, H, I)) {
+  // device (the one-CTA form below computes the same)
+  if (maps.use_pairs && !g_pairs_refused && ffn_pair_usable(maps, grp.n_box, H, I)) {
     if (launch_ffn_pair(st, maps, grp, kind, offsets, hbuf, y, y_bf16, H, I, n_sms, status, work_counter, timeline,
                         timeline_slot, report, done) == OLED_OK)
       return OLED_OK;

@@ -414,6 +414,37 @@ def test_bounded_device_wait_reports_timeout_and_context_survives():
         run.close()
 
 
+def test_bounded_device_wait_in_the_cta_pair_kernel():
+    """The same failure path in the many-token FFN on CTA pairs: no item is ever published, the
+    bounded waits of every role of both CTAs run out, the cluster's kernels return, the host
+    reads OLED_ERR_TIMEOUT, and afterwards the same context is in parity again."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    n = 700
+    run = _runner(w, capacity=[4], max_tokens=n)
+    ora = _oracle_for(run, [4])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 11)
+        x, c = bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device)
+        out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+        run.step(0, x, c, out)                                   # warm: everything resident
+        ref = ora.denoise_step(0, h_bits, conf)
+        assert ref["counts"].max() > 256                         # token tiles of 256 rows: the pair kernel
+        _check_out(dev_to_bits(out), ref["out"])
+        run.ctx.set_option(binding.OPT_TEST_WITHHOLD_LOADS, 1)
+        run.step(0, x, c, out)
+        assert run.ctx.synchronize_rc() == binding.ERR_TIMEOUT
+        run.ctx.set_option(binding.OPT_TEST_WITHHOLD_LOADS, 0)
+        run.ctx.clear_status()
+        assert run.ctx.synchronize_rc() == binding.OLED_OK
+        ora.denoise_step(0, h_bits, conf)                        # keep the oracle's counters in step
+        run.step(0, x, c, out)
+        _check_out(dev_to_bits(out), ora.denoise_step(0, h_bits, conf)["out"])
+    finally:
+        run.close()
+
+
 def test_self_check_is_silent_on_valid_steps_and_flags_a_corrupted_permutation():
     """OLED_OPT_SELF_CHECK: the checking kernels find nothing on valid steps (parity unchanged, guard
     words intact); with the first two sorted rows exchanged by the test aid - both still valid
