@@ -652,6 +652,32 @@ def test_fp8_direct_form_agrees_with_widening_form_on_wide_range_rows():
         run.close()
 
 
+def test_fp8_direct_form_takes_several_token_tiles_per_expert():
+    """After a step in which no expert received more than 16 rows, the direct fp8 form's hit launch
+    uses 16-row token tiles; a following step that sends all 24 tokens to the same two experts
+    then needs two tiles per expert (the second one ragged)."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    w = synth.tiny(n_layers=1, n_experts=8, top_k=2, hidden=256, intermediate=128)
+    n = 24
+    run = _runner(w, capacity=[8], max_tokens=n, fp8=True)
+    ora = _oracle_for(run, [8])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n, 52)
+        same = np.repeat(h_bits[:1], n, axis=0)                  # every token the same row: one routing decision
+        c = torch.from_numpy(conf).to(run.device)
+        out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+        for rep, bits in enumerate((h_bits, h_bits, same, h_bits)):
+            run.step(0, bits_to_dev(bits, run.device), c, out)
+            ref = ora.denoise_step(0, bits, conf)
+            if rep < 2:
+                assert ref["counts"].max() <= 16
+            if rep == 2:
+                assert sorted(ref["counts"])[-2:] == [n, n]
+            _check_step(run, 0, n, out, ref)
+    finally:
+        run.close()
+
+
 def test_fp8_subnormal_codes_decode_exactly():
     """Blobs whose row scales are so large that every code is an e4m3 subnormal (exponent field
     0): the on-chip widening must reproduce them exactly, not flush them."""
