@@ -463,13 +463,14 @@ route_many_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w
 // order (xp[r,:] = x[perm[r]/K,:]); used for small steps, larger ones run gather_kernel instead.
 // Each of those CTAs repeats the scan for itself - a few hundred ids - keeps the token of every
 // sorted row in shared memory (reading the rows' numbers back from global memory would cost a
-// round trip before the first load), and takes every gridDim.y-th batch of eight rows, so that an
+// round trip before the first load), and takes every gridDim.y-th batch of RB rows, so that an
 // expert that received many tokens does not make the step wait for one CTA's chain of batches.
 // Only the CTAs with blockIdx.y == 0 write offsets, perm and pos.
 constexpr int kGatherTokMax = 4096;  // rows of one expert in a step that gathers here (T * K <= 4096)
-// RB: rows a CTA copies at a time.  Eight for a plain copy; two (and eight CTAs per expert) where
-// the rows' e4m3 terms are produced too: the conversions are the long pole there, and an
-// expert's handful of rows is then spread over several SMs.
+// RB: rows a CTA copies at a time.  Two, with eight CTAs per expert, in gathering launches: an
+// expert's handful of rows is then spread over several SMs (with one CTA taking eight rows the
+// step waited 3 us longer whenever an expert had more than eight, and the e4m3 terms of fp8
+// steps, whose conversions are the long pole, came to 7 us).  (Eight: launches that do not gather.)
 template <int RB>
 __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
@@ -481,7 +482,7 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   __shared__ int s_red[8];
   __shared__ int s_base;
   __shared__ int s_tok[kGatherTokMax];
-  __shared__ uint32_t s_amax[3][RB];  // per batch of eight rows, three batches in rotation (see the gather loop)
+  __shared__ uint32_t s_amax[3][RB];  // per batch of RB rows, three batches in rotation (see the gather loop)
   const int e = blockIdx.x;
   const bool writer = blockIdx.y == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -734,14 +735,13 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
                     StepTimeline* timeline, const TokenSplit* split) {
-  // gathering steps: up to four CTAs per expert share its rows (batches of eight)
   const TokenSplit sp = xp != nullptr && split != nullptr && split->complete() ? *split : TokenSplit{};
-  if (sp.complete())
+  if (xp != nullptr)  // gathering steps: two rows per CTA, eight CTAs per expert (see the kernel)
     launch_pdl(permute_kernel<2>, dim3(E, 8), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
                timeline, sp);
   else
-    launch_pdl(permute_kernel<8>, dim3(E, xp != nullptr ? 4 : 1), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm,
-               pos, x, xp, H, K, timeline, sp);
+    launch_pdl(permute_kernel<8>, dim3(E, 1), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
+               timeline, sp);
 }
 
 namespace {
