@@ -18,8 +18,9 @@
 // the launch.  The up values cross to the gate rows' warps through shared memory.
 //
 // In the many-token regime (N tile 256) both kernels work on two 128-row weight tiles that share
-// one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs,
-// which is what keeps the L2->shared-memory traffic under the tensor pipe's appetite.
+// one token tile (gate+up, or two row blocks of Wd): 64 KB of operands per 128x2x256x64 MACs.
+// (By default those steps run on CTA pairs instead, ffn_pair.cu; this form is what remains where
+// the pair form does not apply - shapes, fp8 stores - or is switched off.)
 //
 // Work items (expert, token tile, weight tile) are drawn from a global counter by each CTA's
 // producer and handed to its other roles through a ring in shared memory (see take_item); a
