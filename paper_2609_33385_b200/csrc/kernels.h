@@ -145,10 +145,14 @@ struct CombinePrev {
   uint32_t* zero_words = nullptr;  // the control block the previous step used, cleared by CTA 0
   int n_zero_words = 0;
 };
+// seg_counts (many-token steps; nullptr: none): ZERO words [kPermuteSegments][E]; the kernel also
+// counts every expert's assignments per segment of seg_tokens consecutive tokens, so that the
+// permutation kernel can work on the segments in parallel.
+constexpr int kPermuteSegments = 16;
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
-                  StepTimeline* timeline);
+                  StepTimeline* timeline, int32_t* seg_counts = nullptr, int seg_tokens = 0);
 bool route_can_take_combine(int T);  // does the gate kernel of a T-token step carry out a CombinePrev?
 // fp8 expert stores, direct form: the two token operands of a step's expert FFN - the gathered
 // input rows and the intermediate rows - as sums of two e4m3 terms each, after scaling every row
@@ -167,12 +171,15 @@ struct TokenSplit {
 };
 // Offsets (exclusive scan), stable permutation by expert and its inverse.  With xp != nullptr the
 // kernel also gathers the token rows (xp[r,:] = x[perm[r]/K,:]); meant for small steps.
+// seg_counts (launches that do not gather; nullptr: none): the gate kernel's per-segment counts (see
+// launch_route): kPermuteSegments CTAs per expert then scan one segment of the assignment list each.
 // split (gathering launches only; nullptr: none): the kernel also writes, per sorted row, the
 // largest magnitude of the row it copied and the row's two e4m3 terms, and zeroes amax_mid (see
 // TokenSplit).
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
-                    StepTimeline* timeline, const TokenSplit* split = nullptr);
+                    StepTimeline* timeline, const TokenSplit* split = nullptr, const int32_t* seg_counts = nullptr,
+                    int seg_tokens = 0);
 // xp[r,:] = x[perm[r] / K, :] for the T*K sorted rows.
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);

@@ -89,7 +89,8 @@ struct oled_ctx {
   float* d_y = nullptr;        // [T*k,H]
   uint32_t* d_status = nullptr;
   uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
-  uint32_t* d_done = nullptr;         // control block, last: [kFfnWorkCounters][E] completion counters of fused FFN launches
+  uint32_t* d_done = nullptr;         // control block: [kFfnWorkCounters][E] completion counters of fused FFN launches
+  int32_t* d_seg = nullptr;           // control block, last: [kPermuteSegments][E] per-segment counts of many-token steps
   int work_next = 0;                  // next unused counter of the current layer execution
   bool ctrl_dirty = true;             // both control blocks must be cleared before the next gate launch
   unsigned int seq = 0;               // step sequence number echoed by the gate kernel
@@ -154,6 +155,7 @@ void select_ctrl(oled_ctx* ctx, int sel) {
   ctx->d_counts = reinterpret_cast<int32_t*>(b + E * sizeof(unsigned long long));
   ctx->d_work = reinterpret_cast<uint32_t*>(b + E * (sizeof(unsigned long long) + sizeof(int32_t)));
   ctx->d_done = ctx->d_work + kFfnWorkCounters;
+  ctx->d_seg = reinterpret_cast<int32_t*>(ctx->d_done + (size_t)kFfnWorkCounters * E);
 }
 
 template <typename T>
@@ -551,7 +553,7 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
   ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + kFfnWorkCounters * sizeof(uint32_t) +
-                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t);
+                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t) + (size_t)kPermuteSegments * E * sizeof(int32_t);
   ctx->ctrl_bytes = (ctx->ctrl_bytes + 15) / 16 * 16;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_ctrl[0], 2 * ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
@@ -707,6 +709,10 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     OLED_CUDA(ctx, cudaMemsetAsync(tl, 0xff, 2 * kTimelineSlots * sizeof(unsigned long long), st));
     OLED_CUDA(ctx, cudaMemsetAsync(tl->end_max, 0, kTimelineSlots * sizeof(unsigned long long), st));
   }
+  // many-token steps: the gate kernel counts every expert's assignments per segment of the token
+  // range, and the permutation kernel then scans the segments in parallel
+  int32_t* const seg_counts = (size_t)T * K > 4096 && !route_can_take_combine(T) ? ctx->d_seg : nullptr;
+  const int seg_tokens = ((T + kPermuteSegments - 1) / kPermuteSegments + 3) / 4 * 4;
   // the current step's gate-score and inverse-permutation buffers (the previous step's stay
   // intact for a combine that has been left to this step's gate kernel)
   ctx->buf_sel ^= 1;
@@ -738,7 +744,7 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
       ctx->pending.valid = false;
     }
     launch_route(st, static_cast<const uint16_t*>(hidden), L.w_router, L.bias, confidences, T, H, E, K,
-                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, prev, tl);
+                 ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, prev, tl, seg_counts, seg_tokens);
   }
   const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
   NvtxRange nv_perm(ctx, "oled.step.2_permutation_counts");
@@ -747,7 +753,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
     // (fp8 stores: a gathering permutation kernel also leaves the rows' magnitudes for the FFN)
     ctx->step_split = fuse_gather && ctx->fp8_direct && ctx->split.complete() ? &ctx->split : nullptr;
     launch_permute(st, ctx->d_ids, ctx->d_counts, T, E, K, ctx->d_offsets, ctx->d_perm, ctx->d_pos,
-                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl, ctx->step_split);
+                   static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl, ctx->step_split,
+                   seg_counts, seg_tokens);
   }
   if (!fuse_gather) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);

@@ -31,7 +31,8 @@ template <int kMaxEPerLane>  // E <= 32 * kMaxEPerLane: bounds the per-lane cand
 __device__ __forceinline__ void route_token_tail_n(const float* row, int t, int lane, int E, int K,
                                                  const float* __restrict__ conf, int32_t* __restrict__ ids,
                                                  float* __restrict__ gate, int32_t* __restrict__ counts,
-                                                 unsigned long long* __restrict__ scores) {
+                                                 unsigned long long* __restrict__ scores,
+                                                 int32_t* __restrict__ seg_counts, int seg_tokens) {
     float v[kMaxEPerLane];
 #pragma unroll
     for (int i = 0; i < kMaxEPerLane; ++i) {
@@ -86,6 +87,7 @@ __device__ __forceinline__ void route_token_tail_n(const float* row, int t, int 
       const unsigned long long q = (pv == pv) ? __float2ull_rz(__fmul_rn(pv, 4294967296.0f)) : 0ull;
       atomicAdd(&counts[my_id], 1);
       atomicAdd(&scores[my_id], q);
+      if (seg_counts != nullptr) atomicAdd(&seg_counts[(t / seg_tokens) * E + my_id], 1);
     }
   }
 
@@ -93,10 +95,11 @@ __device__ __forceinline__ void route_token_tail_n(const float* row, int t, int 
 __device__ __forceinline__ void route_token_tail(const float* row, int t, int lane, int E, int K,
                                                  const float* __restrict__ conf, int32_t* __restrict__ ids,
                                                  float* __restrict__ gate, int32_t* __restrict__ counts,
-                                                 unsigned long long* __restrict__ scores) {
-  if (E <= 64) route_token_tail_n<2>(row, t, lane, E, K, conf, ids, gate, counts, scores);
-  else if (E <= 128) route_token_tail_n<4>(row, t, lane, E, K, conf, ids, gate, counts, scores);
-  else route_token_tail_n<OLED_MAX_EXPERTS / 32>(row, t, lane, E, K, conf, ids, gate, counts, scores);
+                                                 unsigned long long* __restrict__ scores,
+                                                 int32_t* __restrict__ seg_counts = nullptr, int seg_tokens = 1) {
+  if (E <= 64) route_token_tail_n<2>(row, t, lane, E, K, conf, ids, gate, counts, scores, seg_counts, seg_tokens);
+  else if (E <= 128) route_token_tail_n<4>(row, t, lane, E, K, conf, ids, gate, counts, scores, seg_counts, seg_tokens);
+  else route_token_tail_n<OLED_MAX_EXPERTS / 32>(row, t, lane, E, K, conf, ids, gate, counts, scores, seg_counts, seg_tokens);
 }
 
 // The previous layer's gate-weighted combine and residual, done by the gate kernel of the next
@@ -338,7 +341,8 @@ route_many_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w
                   const float* __restrict__ bias, const float* __restrict__ conf, int T, int H, int E,
                   int K, float* __restrict__ logits_out, int32_t* __restrict__ ids,
                   float* __restrict__ gate, int32_t* __restrict__ counts,
-                  unsigned long long* __restrict__ scores, StepTimeline* timeline) {
+                  unsigned long long* __restrict__ scores, StepTimeline* timeline,
+                  int32_t* __restrict__ seg_counts, int seg_tokens) {
   constexpr int kStageBytes = many_stage_bytes(TT);
   constexpr int kRows = TT + kManyExperts;
   extern __shared__ __align__(16) uint8_t s_dyn[];
@@ -452,7 +456,7 @@ route_many_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w
   for (int a = warp; a < TT; a += kManyWarps) {
     const int t = t0 + a;
     if (t >= T) continue;
-    route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores);
+    route_token_tail(s_logits + a * E, t, lane, E, K, conf, ids, gate, counts, scores, seg_counts, seg_tokens);
   }
   if (threadIdx.x == 0) timeline_end(timeline, 0);
 }
@@ -476,7 +480,7 @@ __global__ void __launch_bounds__(256)
 permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ counts, int n, int E,
                int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ pos,
                const uint16_t* __restrict__ x, uint16_t* __restrict__ xp, int H, int K, StepTimeline* timeline,
-               TokenSplit split) {
+               TokenSplit split, const int32_t* __restrict__ seg_counts, int seg_tokens) {
   uint32_t* const amax_in = split.amax_in;
   uint32_t* const amax_mid = split.amax_mid;
   __shared__ int s_red[8];
@@ -484,7 +488,10 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
   __shared__ int s_tok[kGatherTokMax];
   __shared__ uint32_t s_amax[3][RB];  // per batch of RB rows, three batches in rotation (see the gather loop)
   const int e = blockIdx.x;
-  const bool writer = blockIdx.y == 0;
+  // segmented launches (no gathering): CTA (e, s) scans segment s of the assignment list only and
+  // starts behind the expert's rows of the earlier segments, whose number the gate kernel counted
+  const bool segmented = seg_counts != nullptr;
+  const bool writer = blockIdx.y == 0 || segmented;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   griddep_launch_dependents();
   if (threadIdx.x == 0) timeline_entry(timeline, 1);
@@ -500,30 +507,36 @@ permute_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ coun
     int off = 0;
     for (int w = 0; w < 8; ++w) off += s_red[w];
     s_base = off;
-    if (writer) {
+    if (blockIdx.y == 0) {
       offsets[e] = off;
       if (e == E - 1) offsets[E] = off + counts[e];
+    }
+    if (segmented) {
+      for (int s = 0; s < (int)blockIdx.y; ++s) off += seg_counts[s * E + e];
+      s_base = off;
     }
   }
   __syncthreads();
   // (a CTA beyond the first of an expert has work only if the expert has a batch of rows for it)
-  if (counts[e] == 0 || (int)blockIdx.y * RB >= counts[e]) {
+  if (segmented ? seg_counts[blockIdx.y * E + e] == 0 : (counts[e] == 0 || (int)blockIdx.y * RB >= counts[e])) {
     if (threadIdx.x == 0) timeline_end(timeline, 1);
     return;
   }
   int base = s_base;
+  const int a_first = segmented ? (int)blockIdx.y * seg_tokens * K : 0;
+  const int a_end = segmented ? min(n, a_first + seg_tokens * K) : n;
   // stable scan, 8 consecutive assignments per thread and 2048 per round
-  for (int a0 = 0; a0 < n; a0 += 8 * blockDim.x) {
+  for (int a0 = a_first; a0 < a_end; a0 += 8 * blockDim.x) {
     const int first = a0 + threadIdx.x * 8;
     int v[8];
-    if (first + 8 <= n) {
+    if (first + 8 <= a_end) {
       const int4 lo = *reinterpret_cast<const int4*>(ids + first);
       const int4 hi = *reinterpret_cast<const int4*>(ids + first + 4);
       v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w;
       v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
     } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = first + i < n ? ids[first + i] : -1;
+      for (int i = 0; i < 8; ++i) v[i] = first + i < a_end ? ids[first + i] : -1;
     }
     uint32_t m = 0;
 #pragma unroll
@@ -674,7 +687,7 @@ bool route_can_take_combine(int T) { return T <= kRouteSmallMax; }
 void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, const float* bias,
                   const float* conf, int T, int H, int E, int K, float* logits, int32_t* ids,
                   float* gate, int32_t* counts, unsigned long long* scores, const CombinePrev& prev,
-                  StepTimeline* timeline) {
+                  StepTimeline* timeline, int32_t* seg_counts, int seg_tokens) {
   if (T <= kRouteSmallMax) {
     constexpr int W = 16;
     static bool attr_done = false;
@@ -721,7 +734,7 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
       const size_t smem = (size_t)kManyStages * many_stage_bytes(tt) + (size_t)tt * E * sizeof(float);
       cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
       launch_pdl(kernel, dim3((T + tt - 1) / tt), dim3(kManyWarps * 32), smem, st, x, w_router, bias, conf, T, H, E,
-                 K, logits, ids, gate, counts, scores, timeline);
+                 K, logits, ids, gate, counts, scores, timeline, seg_counts, seg_tokens);
     };
     switch (best_tt) {
       case 8: go(route_many_kernel<8>, 8); break;
@@ -734,14 +747,14 @@ void launch_route(cudaStream_t st, const uint16_t* x, const uint16_t* w_router, 
 
 void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, int T, int E, int K,
                     int32_t* offsets, int32_t* perm, int32_t* pos, const uint16_t* x, uint16_t* xp, int H,
-                    StepTimeline* timeline, const TokenSplit* split) {
+                    StepTimeline* timeline, const TokenSplit* split, const int32_t* seg_counts, int seg_tokens) {
   const TokenSplit sp = xp != nullptr && split != nullptr && split->complete() ? *split : TokenSplit{};
   if (xp != nullptr)  // gathering steps: two rows per CTA, eight CTAs per expert (see the kernel)
     launch_pdl(permute_kernel<2>, dim3(E, 8), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
-               timeline, sp);
+               timeline, sp, (const int32_t*)nullptr, 0);
   else
-    launch_pdl(permute_kernel<8>, dim3(E, 1), dim3(256), 0, st, ids, counts, T * K, E, offsets, perm, pos, x, xp, H, K,
-               timeline, sp);
+    launch_pdl(permute_kernel<8>, dim3(E, seg_counts != nullptr ? kPermuteSegments : 1), dim3(256), 0, st, ids, counts,
+               T * K, E, offsets, perm, pos, x, xp, H, K, timeline, sp, seg_counts, seg_tokens);
 }
 
 namespace {
