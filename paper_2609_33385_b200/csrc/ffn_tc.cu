@@ -339,14 +339,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ 
     ctl->count[g] = offsets[e + 1] - s;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int acc = 0;
-    for (int g = 0; g < grp.n; ++g) {
-      ctl->tile_prefix[g] = acc;
-      acc += (ctl->count[g] + n_box - 1) / n_box;
+  if (warp == 0) {  // exclusive scan of the experts' token-tile counts, 32 experts at a time
+    int carry = 0;
+    for (int g0 = 0; g0 < grp.n; g0 += 32) {
+      const int g = g0 + lane;
+      const int tiles = g < grp.n ? (ctl->count[g] + n_box - 1) / n_box : 0;
+      int incl = tiles;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += o;
+      }
+      if (g < grp.n) ctl->tile_prefix[g] = carry + incl - tiles;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    ctl->tile_prefix[grp.n] = acc;
-    ctl->n_tiles_total = acc;
+    if (lane == 0) {
+      ctl->tile_prefix[grp.n] = carry;
+      ctl->n_tiles_total = carry;
+    }
   }
   tc_fence_before();
   __syncthreads();
