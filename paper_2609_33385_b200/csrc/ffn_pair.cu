@@ -1,14 +1,15 @@
 // Grouped SwiGLU expert FFN for many-token steps on CTA PAIRS (tcgen05 cta_group::2).
 //
-// In the many-token regime (token tiles of 256 rows) the single-CTA kernel of ffn_tc.cu is bound
-// by the traffic from L2 to shared memory: its tile - two 128-row weight tiles against 256 token
-// rows, all 512 TMEM columns - needs 64 KB of operands per k-block of 64, and at the tensor
-// pipe's pace that is more than L2 delivers to 148 SMs (8.9 TB/s measured at 51 % of the pipe).
-// TMEM fixes the tile an SM can accumulate, so fewer operand bytes per multiply-add need two SMs
-// to share a token tile: here a cluster of two CTAs computes 512 output features x 256 tokens
-// with M = 256 MMAs.  Each CTA holds its own two 128-row weight tiles, its own accumulators (its
-// 128 lanes x 512 columns of TMEM) and HALF of the token tile; the MMA, issued by one thread of
-// the pair's first CTA, reads both halves.  48 KB of operands per CTA and k-block instead of 64.
+// In the many-token regime (token tiles of 256 rows) the expert FFN is a tensor-core GEMM, and
+// TMEM fixes the tile one SM can accumulate: two 128-row weight tiles against 256 token rows use
+// all 512 columns and take 64 KB of operands per k-block of 64.  Fewer operand bytes per
+// multiply-add need two SMs to share a token tile: here a cluster of two CTAs computes 512
+// output features x 256 tokens with M = 256 MMAs.  Each CTA holds its own two 128-row weight
+// tiles, its own accumulators (its 128 lanes x 512 columns of TMEM) and HALF of the token tile;
+// the MMA, issued by one thread of the pair's first CTA, reads both halves.  48 KB of operands per
+// CTA and k-block instead of 64 (the tensor pipe's share of the active cycles went from 67 to
+// 71 % on 4096 tokens x 4096 x 1536; the traffic alone was worth little - L2 runs at 39 % of its
+// peak - the dynamic items across the pair, the pipelined epilogue and the single launch the rest).
 //   KIND 1: features f0 + 128 r .. + 127 for CTA r: gate rows and up rows of those features,
 //           epilogue hbuf[n, f] = bf16(silu(D_gate) * D_up)
 //   KIND 2: output rows c0 + 256 r .. + 255 for CTA r (two row blocks of Wd), epilogue y[n, c] = D
