@@ -252,6 +252,12 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * intermediate a multiple of 256, hidden a multiple of 512) run the expert FFN on pairs of CTAs
  * that share a token tile (tcgen05 cta_group::2); 0 = always one CTA per tile. */
 #define OLED_OPT_FFN_PAIRS 15
+/* OLED_OPT_L2_PREFETCH: 1 (default) = inside oled_denoise_iteration(), while a layer whose previous
+ * execution had no miss runs its gate and permutation kernels (the HBM is idle then), the weights
+ * of the first experts its FFN will stream - the residents activated at that previous execution,
+ * adjacent iterations activating mostly the same experts (Sec. 3.3) - are called into L2 from
+ * the side stream; 0 = off. */
+#define OLED_OPT_L2_PREFETCH 16
 #define OLED_TIMELINE_SLOTS 12 /* 0 gate, 1 permutation, 2 gather (not recorded),
                                   3..10 the step's FFN launches in order, 11 combine */
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */

@@ -194,6 +194,33 @@ void launch_combine(cudaStream_t st, const float* y, int y_bf16, const float* ga
                n_zero_words, timeline);
 }
 
+namespace {
+constexpr uint32_t kPrefetchChunk = 16384;
+// one thread per 16 KB chunk of a listed slot. (Pacing the requests - 1024 threads, a pause between a
+// thread's chunks - was measured and made every workload slower.)
+__global__ void __launch_bounds__(128)
+l2_prefetch_kernel(const uint8_t* __restrict__ pool, unsigned long long slot_bytes, const __grid_constant__ SlotList slots,
+                   unsigned long long bytes_per_slot) {
+  const unsigned long long chunks_per_slot = (bytes_per_slot + kPrefetchChunk - 1) / kPrefetchChunk;
+  const unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= chunks_per_slot * (unsigned long long)slots.n) return;
+  const unsigned long long s = i / chunks_per_slot, c = i - s * chunks_per_slot;
+  const unsigned long long off = c * kPrefetchChunk;
+  const uint32_t bytes = (uint32_t)min((unsigned long long)kPrefetchChunk, bytes_per_slot - off) & ~15u;
+  if (bytes == 0) return;
+  const uint8_t* src = pool + (unsigned long long)slots.slot[s] * slot_bytes + off;
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+}  // namespace
+
+void launch_l2_prefetch(cudaStream_t st, const uint8_t* pool, size_t slot_bytes, const SlotList& slots,
+                        size_t bytes_per_slot) {
+  if (slots.n <= 0 || bytes_per_slot == 0) return;
+  const unsigned long long chunks = ((bytes_per_slot + kPrefetchChunk - 1) / kPrefetchChunk) * (unsigned long long)slots.n;
+  l2_prefetch_kernel<<<(unsigned)((chunks + 127) / 128), 128, 0, st>>>(pool, (unsigned long long)slot_bytes, slots,
+                                                                       (unsigned long long)bytes_per_slot);
+}
+
 void launch_residual_add(cudaStream_t st, const uint16_t* x, const uint16_t* r, uint16_t* y, size_t n) {
   const int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
   launch_pdl(residual_add_kernel, dim3(blocks), dim3(256), 0, st, x, r, y, n);

@@ -184,6 +184,15 @@ void launch_permute(cudaStream_t st, const int32_t* ids, const int32_t* counts, 
 void launch_gather(cudaStream_t st, const uint16_t* x, const int32_t* perm, int T, int H, int K,
                    uint16_t* xp);
 
+// Calls the first `bytes_per_slot` bytes of the listed slots of the pool into L2 (prefetch only:
+// nothing is read into registers, nothing waits).  combine.cu.
+struct SlotList {
+  int32_t n;
+  uint16_t slot[OLED_MAX_EXPERTS];
+};
+void launch_l2_prefetch(cudaStream_t st, const uint8_t* pool, size_t slot_bytes, const SlotList& slots,
+                        size_t bytes_per_slot);
+
 // ---- combine.cu -----------------------------------------------------------------------
 // out[t,:] = bf16( sum_j gate[t,j] * y[pos[t*K+j],:] ), j ascending, fp32 accumulation.  With
 // x_next != nullptr also x_next[t,:] = bf16(x[t,:] + out[t,:]) (the residual between layers).

@@ -24,6 +24,8 @@ struct LayerData {
   LayerCacheState cache;
   int32_t last_active = -1;      // experts activated at the layer's previous execution (-1: none yet)
   int32_t last_max_count = -1;   // most token rows any expert received then
+  int32_t last_misses = -1;      // its misses
+  std::vector<int32_t> last_counts;  // its per-expert row counts
   const uint8_t* host_blob = nullptr;
   size_t host_stride = 0;
   uint16_t* w_router = nullptr;  // device [E,H]
@@ -115,6 +117,8 @@ struct oled_ctx {
   int ffn_impl = 0;
   bool timeline_on = false;    // OLED_OPT_TIMELINE
   bool fp8_direct = true;      // OLED_OPT_FP8_DIRECT
+  bool l2_prefetch = true;     // OLED_OPT_L2_PREFETCH
+  cudaEvent_t ev_layer_done = nullptr;  // recorded behind a layer's last kernel (L2 prefetch of the next layer)
   StepTimeline* d_timeline = nullptr;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
   bool hit_fused = false;      // this step's resident-group FFN ran as one fused launch
@@ -258,6 +262,7 @@ void free_ctx(oled_ctx* ctx) {
   }
   for (auto ev : ctx->prof_free) cudaEventDestroy(ev);
   if (ctx->gate_event) cudaEventDestroy(ctx->gate_event);
+  if (ctx->ev_layer_done) cudaEventDestroy(ctx->ev_layer_done);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   cudaGetLastError();
   delete ctx;
@@ -932,6 +937,8 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
   L.last_active = plan.n_active;
   L.last_max_count = 0;
   for (int32_t e = 0; e < E; ++e) L.last_max_count = std::max(L.last_max_count, counts[e]);
+  L.last_misses = n_miss;
+  L.last_counts.assign(counts, counts + E);
   L.stats.assignments += (uint64_t)T * K;
   L.stats.fills_reused += (uint64_t)plan.n_fills_reused;
   L.stats.ideal_hits += (uint64_t)std::min<int64_t>(plan.n_active, plan.capacity_used);
@@ -970,6 +977,41 @@ int oled_denoise_step_host(oled_ctx* ctx, int32_t layer, const void* host_hidden
   return OLED_OK;
 }
 
+// While the next layer's gate and permutation kernels run the HBM is idle: if that layer's
+// previous execution hit the cache with every activated expert, the weights its FFN will stream
+// first - the residents activated then, in the order of the FFN's expert list - are called into
+// L2 from the side stream (idle as well when nothing misses), behind the current layer's last
+// kernel.  A prefetch only: what the gate then decides changes nothing but the hit rate in L2.
+static int prefetch_next_layer(oled_ctx* ctx, int32_t next) {
+  if (!ctx->l2_prefetch || ctx->ffn_impl != 0) return OLED_OK;
+  const LayerData& N = ctx->layers[next];
+  if (N.last_misses != 0 || (int32_t)N.last_counts.size() != ctx->shape.n_experts) return OLED_OK;
+  constexpr size_t kPrefetchBytes = 64u << 20;  // about what the HBM delivers during gate + permutation (32-96 MB measured alike, more costs)
+  // the gate/up matrices only (they lead a blob): the down matrices are read a whole gate/up launch later
+  const size_t esz = ctx->shape.expert_format == OLED_EXPERTS_FP8 ? 1 : 2;
+  const size_t lead_bytes = (size_t)2 * ctx->shape.hidden * ctx->shape.intermediate * esz;
+  // Worth it only in front of a long expert stream: measured, streams of 0.4 and 0.8 GB per layer gained
+  // 2-3 % and one of 0.27 GB lost 2 % (the prefetch delays the gate kernel's own loads by 2 us now and then).
+  size_t stream_bytes = 0;
+  for (int32_t e = 0; e < ctx->shape.n_experts; ++e)
+    if (N.last_counts[e] > 0) stream_bytes += (size_t)3 * ctx->shape.hidden * ctx->shape.intermediate * esz;
+  if (stream_bytes < 5 * kPrefetchBytes) return OLED_OK;
+  SlotList list;
+  list.n = 0;
+  const int cap = (int)std::max<size_t>(1, kPrefetchBytes / lead_bytes);
+  for (int32_t e = 0; e < ctx->shape.n_experts && list.n < cap; ++e)
+    if (N.cache.resident[e] && N.cache.slot_of[e] >= 0 && N.last_counts[e] > 0) list.slot[list.n++] = (uint16_t)N.cache.slot_of[e];
+  if (list.n == 0) return OLED_OK;
+  if (ctx->ev_layer_done == nullptr)
+    OLED_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_layer_done, cudaEventDisableTiming));
+  OLED_CUDA(ctx, cudaEventRecord(ctx->ev_layer_done, ctx->stream));
+  OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_layer_done, 0));
+  launch_l2_prefetch(ctx->copy_stream, ctx->pool, ctx->slot_bytes, list, lead_bytes);
+  ctx->launches += 1;
+  OLED_CUDA(ctx, cudaGetLastError());
+  return OLED_OK;
+}
+
 int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confidences, int32_t n_tokens,
                            void* hidden_out) {
   if (!ctx || n_tokens < 0) return OLED_ERR_INVALID_ARG;
@@ -981,6 +1023,10 @@ int oled_denoise_iteration(oled_ctx* ctx, const void* hidden, const float* confi
     const int rc = step_impl(ctx, l, x, confidences, n_tokens, ctx->d_out_stage, nxt, l + 1 < ctx->shape.n_layers);
     if (rc != OLED_OK) return rc;
     x = nxt;
+    {  // (behind the last layer: the first layer of the iteration that is likely to follow)
+      const int rcp = prefetch_next_layer(ctx, l + 1 < ctx->shape.n_layers ? l + 1 : 0);
+      if (rcp != OLED_OK) return rcp;
+    }
   }
   ctx->iterations += 1;
   if (ctx->adapt_period > 0 && ctx->iterations % (uint64_t)ctx->adapt_period == 0)
@@ -1176,6 +1222,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       return OLED_OK;
     case OLED_OPT_FP8_DIRECT:
       ctx->fp8_direct = value != 0;
+      return OLED_OK;
+    case OLED_OPT_L2_PREFETCH:
+      ctx->l2_prefetch = value != 0;
       return OLED_OK;
     case OLED_OPT_FFN_PAIRS:
       ctx->maps.use_pairs = value != 0;
