@@ -258,6 +258,11 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * adjacent iterations activating mostly the same experts (Sec. 3.3) - are called into L2 from
  * the side stream; 0 = off. */
 #define OLED_OPT_L2_PREFETCH 16
+/* OLED_OPT_GATHER_IN_FFN: 1 (default) = a many-token step whose FFN launches all run on CTA pairs
+ * has no gather kernel: each gate/up launch copies its own experts' token rows into sorted order
+ * while its first items run (one thread per CTA, bulk copies through shared memory, a counter
+ * per expert that the items wait for); 0 = a gather kernel in front, as for every other step. */
+#define OLED_OPT_GATHER_IN_FFN 17
 #define OLED_TIMELINE_SLOTS 12 /* 0 gate, 1 permutation, 2 gather (not recorded),
                                   3..10 the step's FFN launches in order, 11 combine */
 #define OLED_CHECK_ID_RANGE 0x01u      /* an expert id outside [0, E)                               */

@@ -28,6 +28,7 @@ OPT_SELF_CHECK, OPT_TEST_CORRUPT_PERM = 7, 8
 OPT_SPLIT_LAST_FILL, OPT_FUSE_COMBINE, OPT_FUSE_FFN, OPT_PDL, OPT_TIMELINE, OPT_FP8_DIRECT = 9, 10, 11, 12, 13, 14
 OPT_FFN_PAIRS = 15
 OPT_L2_PREFETCH = 16
+OPT_GATHER_IN_FFN = 17
 TIMELINE_SLOTS = 12
 ERR_SELF_CHECK = -10
 CHECK_FLAGS = {0x01: "id_range", 0x02: "id_duplicate", 0x04: "offsets", 0x08: "perm_range", 0x10: "inverse",

@@ -45,7 +45,8 @@ namespace {
 constexpr int kPairEpiWarps = 16;
 constexpr int kPairProducerWarp = kPairEpiWarps;
 constexpr int kPairMmaWarp = kPairEpiWarps + 1;
-constexpr int kPairThreads = (kPairEpiWarps + 2) * 32;
+constexpr int kPairGatherWarp = kPairEpiWarps + 2;
+constexpr int kPairThreads = (kPairEpiWarps + 3) * 32;
 constexpr int kPairK = 64;                              // k-values of a k-block (one 128-byte swizzle atom of bf16)
 constexpr uint32_t kPairATile = 128 * kPairK * 2;       // 128 weight rows of a k-block
 constexpr uint32_t kPairBHalf = 128 * kPairK * 2;       // this CTA's half of the token tile
@@ -60,6 +61,10 @@ struct __align__(16) PairCtl {
   unsigned long long tmem_full;
   unsigned long long tmem_empty;
   unsigned long long item_full[kPairRing];
+  unsigned long long row_full[4];  // (gathering thread) a row chunk has landed in its slot
+  unsigned long long row_dst[4];   // where the slot's chunk goes
+  uint32_t row_bytes[4];
+  int row_tile[8];                 // the token tile (number within the launch) of the last chunks issued
   int item_ring[kPairRing];
   uint32_t tmem_base;
   int abort;
@@ -70,7 +75,7 @@ struct __align__(16) PairCtl {
   int count[OLED_MAX_EXPERTS];
 };
 constexpr uint32_t kPairCtlBytes = (sizeof(PairCtl) + 1023u) & ~1023u;
-constexpr uint32_t kPairSmem = kPairCtlBytes + 1024u + kPairStages * kPairStage;
+constexpr uint32_t kPairSmem = kPairCtlBytes + 1024u + kPairStages * kPairStage + 3u * 8192u;  // + the row ring
 
 struct PairItem {
   int slot, m0, row0, valid;
@@ -162,6 +167,23 @@ struct PairSecond {
   uint32_t* done;       // per expert: epilogue warps (of either CTA) that have stored gate/up rows
 };
 
+// The launch gathers its experts' token rows itself (kinds 1 and 3; perm == nullptr: the rows are in
+// place already): sorted row r of the group's experts is row perm[r] / K of the step's input.  One
+// thread per CTA moves the rows (CTA c takes every gridDim-th row of the group, in the order the items
+// need them) through a small ring in shared memory with bulk copies, and counts each finished chunk
+// on its token tile's word of `ready` (ZERO at the start); the TMA threads hold a gate/up item back
+// until its tile's rows are complete.  The tensor pipe is the bound of these launches, so the
+// copies ride along; a gather kernel in front would cost its full length.
+struct PairTokens {
+  const uint16_t* x;     // [T][H] the step's input
+  uint16_t* xp;          // [rows][H] the sorted copy (read back through tm_act)
+  const int32_t* perm;
+  uint32_t* ready;       // per token tile of the launch (numbered expert by expert): chunks copied
+  int K;
+};
+constexpr uint32_t kRowChunk = 8192;  // bytes per bulk copy of a row piece
+constexpr int kRowSlots = 3;
+
 // KIND 3: the gate/up items, then the down items of the same experts, in ONE launch (a launch
 // boundary between cluster kernels is a full stop: a dependent cluster launch was never seen to
 // start before its predecessor had finished, so the last gate/up items' uneven end and the next
@@ -175,8 +197,9 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
                 const __grid_constant__ FfnGroup grp, const int32_t* __restrict__ offsets, void* __restrict__ out_ptr,
                 int H, int I, int out_bf16, uint32_t* __restrict__ status, uint32_t* __restrict__ work_counter,
                 StepTimeline* timeline, int timeline_slot, const __grid_constant__ RouteReport report,
-                const __grid_constant__ PairSecond sec) {
+                const __grid_constant__ PairSecond sec, const __grid_constant__ PairTokens tok) {
   constexpr bool fused = KIND == 3;
+  const bool gathers = KIND != 2 && tok.perm != nullptr;  // the launch gathers its token rows itself
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   PairCtl* ctl = reinterpret_cast<PairCtl*>(smem_raw);
   const uint32_t tiles_base = (smem_u32(smem_raw) + kPairCtlBytes + 1023u) & ~1023u;
@@ -192,6 +215,7 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int s = 0; s < kPairRing; ++s) mbar_init(smem_u32(&ctl->item_full[s]), 1);
+    for (int s = 0; s < kRowSlots; ++s) mbar_init(smem_u32(&ctl->row_full[s]), 1);
     mbar_init(smem_u32(&ctl->tmem_full), 1);
     mbar_init(smem_u32(&ctl->tmem_empty), 2u * kPairEpiWarps);
     ctl->abort = 0;
@@ -254,6 +278,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   plan.m_blocks2 = H / 512;
   plan.n1 = fused ? ctl->n_tiles_total * plan.m_blocks1 : 0x7fffffff;
   const int total_items = ctl->n_tiles_total * (plan.m_blocks1 + (fused ? plan.m_blocks2 : 0));
+  // (a launch that gathers) the token tiles the pairs' first items read: copied by the epilogue warps
+  const int first_tiles = min(ctl->n_tiles_total, (n_pairs + plan.m_blocks1 - 1) / plan.m_blocks1);
   // (fused) gate/up epilogue warps of both CTAs that store rows per item, times the gate/up items of a token tile
   const uint32_t done_per_tile = (uint32_t)(2 * kPairEpiWarps * (I / 256));
   volatile int* abort_flag = &ctl->abort;
@@ -293,13 +319,20 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
       const CUtensorMap* map_w = down_of_fused ? &sec.tm_w2 : &tm_w;
       const CUtensorMap* map_act = down_of_fused ? &sec.tm_act2 : &tm_act;
       const int k_blocks = (it.kind == 1 ? H : I) / kPairK;
-      if (down_of_fused && it.g != ready_g) {
-        // all intermediate rows of this expert stored?  (an expert seen complete stays complete)
-        const uint32_t target = (uint32_t)(ctl->tile_prefix[it.g + 1] - ctl->tile_prefix[it.g]) * done_per_tile;
+      // what the item's token operand waits for: (down items of a fused launch) all intermediate rows of
+      // the expert stored by its gate/up items; (gate/up items of a launch that gathers) the tile's token
+      // rows copied.  (What was seen complete stays complete.)
+      const int tile = (it.row0 - ctl->row_start[it.g]) / kPairN + ctl->tile_prefix[it.g];
+      const int wait_key = down_of_fused ? (1 << 30 | it.g) : tile;
+      if ((down_of_fused || (gathers && it.kind == 1)) && wait_key != ready_g) {
+        const uint32_t* counter = down_of_fused ? sec.done + it.g : tok.ready + tile;
+        const uint32_t target =
+            down_of_fused ? (uint32_t)(ctl->tile_prefix[it.g + 1] - ctl->tile_prefix[it.g]) * done_per_tile
+                          : (uint32_t)it.valid * (((uint32_t)H * 2u + kRowChunk - 1) / kRowChunk);
         unsigned long long t0 = 0;
         for (uint32_t spin = 0; ok; ++spin) {
           uint32_t seen;
-          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(sec.done + it.g) : "memory");
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
           if (seen >= target) break;
           if ((spin & 255u) == 255u) {
             if (*abort_flag) ok = false;
@@ -313,8 +346,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
           }
         }
         if (!ok) break;
-        ready_g = it.g;
-        // the rows were written through the generic proxy; the copies below read through the async proxy
+        ready_g = wait_key;
+        // (the intermediate rows were written through the generic proxy; the copies below read through the async proxy)
         asm volatile("fence.proxy.async;" ::: "memory");
       }
       const int n_mma = max(32, (it.valid + 31) & ~31);
@@ -346,6 +379,82 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
     if (!ok) {  // let copies already issued land before the CTA's shared memory is released
       const unsigned long long t0 = globaltimer();
       while (globaltimer() - t0 < 2000000ull) {
+      }
+    }
+  } else if (warp == kPairGatherWarp) {
+    // ------------------------------------------------------------ token rows of the group's experts
+    if (gathers && lane == 0 && !grp.withhold_loads) {
+      const uint32_t ring0 = tiles_base + kPairStages * kPairStage;
+      const uint32_t row_bytes = (uint32_t)H * 2u;
+      const int chunks = (int)((row_bytes + kRowChunk - 1) / kRowChunk);
+      // position in the group's rows: expert g, row r of it, chunk c; this CTA's next row is gridDim further
+      // (the rows of the first tiles are the epilogue warps')
+      int g = 0, r = (int)blockIdx.x, c = 0;
+      auto settle = [&]() {
+        for (;;) {
+          while (g < grp.n && r >= ctl->count[g]) r -= ctl->count[g++];
+          if (g >= grp.n || ctl->tile_prefix[g] + r / kPairN >= first_tiles) break;
+          r += (int)gridDim.x;
+        }
+      };
+      settle();
+      int issued = 0;
+      bool ok = true;
+      auto issue = [&]() {
+        const int slot = issued % kRowSlots;
+        const int row = ctl->row_start[g] + r;
+        const uint32_t off = (uint32_t)c * kRowChunk, bytes = min(kRowChunk, row_bytes - off);
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(tok.x) + (size_t)(__ldg(tok.perm + row) / tok.K) * row_bytes + off;
+        ctl->row_dst[slot] = reinterpret_cast<unsigned long long>(tok.xp) + (unsigned long long)row * row_bytes + off;
+        ctl->row_bytes[slot] = bytes;
+        ctl->row_tile[issued & 7] = ctl->tile_prefix[g] + r / kPairN;
+        const uint32_t bar = smem_u32(&ctl->row_full[slot]);
+        mbar_expect_tx(bar, bytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         ring0 + (uint32_t)slot * kRowChunk),
+                     "l"(src), "r"(bytes), "r"(bar)
+                     : "memory");
+        ++issued;
+        if (++c == chunks) {
+          c = 0;
+          r += (int)gridDim.x;
+          settle();
+        }
+      };
+      auto count_chunk = [&](int n) {  // chunk n is in global memory: visible device-wide, then counted
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __threadfence();
+        atomicAdd(tok.ready + ctl->row_tile[n & 7], 1u);
+      };
+      while (issued < kRowSlots - 1 && g < grp.n) issue();
+      int n = 0;
+      for (; ok && n < issued; ++n) {
+        const int slot = n % kRowSlots;
+        if (!mbar_wait(smem_u32(&ctl->row_full[slot]), (uint32_t)(n / kRowSlots) & 1u, abort_flag, status)) {
+          ok = false;
+          break;
+        }
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(ctl->row_dst[slot]),
+                     "r"(ring0 + (uint32_t)slot * kRowChunk), "r"(ctl->row_bytes[slot])
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        if (g < grp.n) {
+          // the slot the next copy lands in was read by the store before this one
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          issue();
+        }
+        if (n >= 2) {
+          asm volatile("cp.async.bulk.wait_group 2;" ::: "memory");
+          count_chunk(n - 2);
+        }
+      }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      if (ok)
+        for (int m = max(0, n - 2); m < n; ++m) count_chunk(m);
+      if (!ok) {  // let copies already issued land before the CTA's shared memory is released
+        const unsigned long long t0 = globaltimer();
+        while (globaltimer() - t0 < 2000000ull) {
+        }
       }
     }
   } else if (warp == kPairMmaWarp && lane == 0 && rank == 0) {
@@ -398,6 +507,40 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant_
   } else if (warp < kPairEpiWarps) {
     // ------------------------------------------------------------ epilogue (both CTAs)
     // warp w: TMEM lane quarter w mod 4 (32 of the CTA's 128 rows), every fourth 16-column chunk
+    if (gathers && !grp.withhold_loads) {
+      // These warps have nothing to do until the first item's MMAs are through: they copy the token
+      // rows of the tiles the first wave of items reads (one row per warp at a time, plain loads and
+      // stores), so that wave waits a few microseconds instead of for the gathering threads' ring.
+      const uint32_t row_bytes = (uint32_t)H * 2u;
+      const uint32_t chunks = (row_bytes + kRowChunk - 1) / kRowChunk;
+      const int W = (int)gridDim.x * kPairEpiWarps, w = (int)blockIdx.x * kPairEpiWarps + warp;
+      int before = 0;  // rows of the experts before g
+      for (int g = 0; g < grp.n && ctl->tile_prefix[g] < first_tiles; ++g) {
+        const int rows = min(ctl->count[g], (first_tiles - ctl->tile_prefix[g]) * kPairN);
+        for (int r = ((w - before) % W + W) % W; r < rows; r += W) {
+          const int row = ctl->row_start[g] + r;
+          const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(tok.x) +
+                                                            (size_t)(__ldg(tok.perm + row) / tok.K) * row_bytes);
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(tok.xp) + (size_t)row * row_bytes);
+          const int n16 = (int)(row_bytes >> 4);
+          for (int i0 = lane; i0 < n16; i0 += 32 * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (i0 + 32 * j < n16) v[j] = __ldg(src + i0 + 32 * j);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (i0 + 32 * j < n16) dst[i0 + 32 * j] = v[j];
+          }
+          // visible device-wide and to the async proxy of the items' copies, then counted
+          __threadfence();
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) atomicAdd(tok.ready + ctl->tile_prefix[g] + r / kPairN, chunks);
+        }
+        before += ctl->count[g];
+      }
+    }
     int local = 0;
     PairCursor cur;
     const int quarter = warp & 3, part = warp >> 2;
@@ -529,16 +672,24 @@ int launch_ffn_pair(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp,
   sec.tm_act2 = maps.hbuf[3];
   sec.out2 = y;
   sec.done = done;
+  PairTokens tok;
+  const bool gathers = kind != 2 && maps.token_source.perm != nullptr;
+  tok.x = maps.token_source.x;
+  tok.xp = maps.token_source.xp;
+  tok.perm = gathers ? maps.token_source.perm : nullptr;
+  tok.ready = maps.token_source.ready;
+  tok.K = maps.token_source.K;
+  if (gathers && tok.ready == nullptr) return OLED_ERR_INVALID_ARG;
   if (kind == 3) {
     if (done == nullptr) return OLED_ERR_INVALID_ARG;
     err = launch_pdl(ffn_pair_kernel<3>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w13, maps.xp[3], grp, offsets,
-                     (void*)hbuf, H, I, y_bf16, status, work_counter, timeline, timeline_slot, report, sec);
+                     (void*)hbuf, H, I, y_bf16, status, work_counter, timeline, timeline_slot, report, sec, tok);
   } else if (kind == 1)
     err = launch_pdl(ffn_pair_kernel<1>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w13, maps.xp[3], grp, offsets,
-                     (void*)hbuf, H, I, 0, status, work_counter, timeline, timeline_slot, report, sec);
+                     (void*)hbuf, H, I, 0, status, work_counter, timeline, timeline_slot, report, sec, tok);
   else
     err = launch_pdl(ffn_pair_kernel<2>, dim3(grid), dim3(kPairThreads), kPairSmem, st, maps.w2, maps.hbuf[3], grp,
-                     offsets, (void*)y, H, I, y_bf16, status, work_counter, timeline, timeline_slot, RouteReport{}, sec);
+                     offsets, (void*)y, H, I, y_bf16, status, work_counter, timeline, timeline_slot, RouteReport{}, sec, tok);
   return err == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
 

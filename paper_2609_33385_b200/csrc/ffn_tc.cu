@@ -1092,6 +1092,11 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
       return OLED_OK;
     cudaGetLastError();  // (a refused launch enqueues nothing)
     g_pairs_refused = true;
+    if (maps.token_source.perm != nullptr) {  // the one-CTA form reads the gathered copy
+      launch_gather(st, maps.token_source.x, maps.token_source.perm, maps.token_source.T, H, maps.token_source.K,
+                    maps.token_source.xp);
+      maps.token_source.perm = nullptr;
+    }
   }
   if (kind == 3 && grp.n_box > 32) {
     // (only reached when the pair launch was refused: the two launches of the one-CTA form, the
@@ -1153,6 +1158,19 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp_in
   }
   return cudaGetLastError() == cudaSuccess ? OLED_OK : OLED_ERR_CUDA;
 }
+
+bool ffn_tc_token_source_usable(const FfnTcMaps& maps, int H, int I) {
+  return maps.use_pairs && !g_pairs_refused && ffn_pair_usable(maps, 256, H, I);
+}
+void ffn_tc_set_token_source(FfnTcMaps* maps, const uint16_t* x, int T, const int32_t* perm, int K, uint16_t* xp) {
+  maps->token_source.perm = perm;
+  maps->token_source.K = K;
+  maps->token_source.T = T;
+  maps->token_source.x = x;
+  maps->token_source.xp = xp;
+  maps->token_source.ready = nullptr;
+}
+void ffn_tc_clear_token_source(FfnTcMaps* maps) { maps->token_source.perm = nullptr; }
 
 int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenSplit* split) {
   const bool direct = maps.fp8 && maps.e4m3_direct && (16 << box_index(max_count, 128)) <= 32 && split != nullptr &&

@@ -223,6 +223,18 @@ struct FfnTcMaps {
   CUtensorMap hbuf[5];   // [rows][I] bf16, box {64, 16<<i}
   bool fp8 = false;      // slots hold fp8 blobs: the weight maps are byte maps over the e4m3 codes
   bool use_pairs = true; // token tiles of 256 rows go to the CTA-pair kernel where it applies (OLED_OPT_FFN_PAIRS)
+  // The step made no gathered copy of the token rows (ffn_tc_set_token_source; perm == nullptr: it
+  // did): every gate/up launch copies its own experts' rows into xp while it runs (sorted row r is
+  // row perm[r] / K of x; CTA-pair kernel only).  Should a pair launch be refused, the gather kernel
+  // fills xp after all and the source is dropped.
+  struct TokenSource {
+    const int32_t* perm = nullptr;
+    int K = 0, T = 0;
+    const uint16_t* x = nullptr;
+    uint16_t* xp = nullptr;
+    uint32_t* ready = nullptr;  // per launch: one ZERO word per token tile of 256 rows (at most rows / 256 + experts)
+  };
+  mutable TokenSource token_source;
   const uint8_t* pool = nullptr;
   size_t slot_bytes = 0;
 };
@@ -247,6 +259,12 @@ int launch_ffn_tc(cudaStream_t st, const FfnTcMaps& maps, const FfnGroup& grp, i
                   StepTimeline* timeline, int timeline_slot, const RouteReport& report, uint32_t* done = nullptr,
                   const TokenSplit* split = nullptr);
 int ffn_tc_launches(const FfnTcMaps& maps, int max_count, int kind, const TokenSplit* split);
+// No gathered copy of the step's token rows exists: every FFN launch until
+// ffn_tc_clear_token_source must be one the CTA-pair kernel takes (token tile 256), and each gets
+// maps->token_source.ready set to zeroed words of its own.
+bool ffn_tc_token_source_usable(const FfnTcMaps& maps, int H, int I);
+void ffn_tc_set_token_source(FfnTcMaps* maps, const uint16_t* x, int T, const int32_t* perm, int K, uint16_t* xp);
+void ffn_tc_clear_token_source(FfnTcMaps* maps);
 bool ffn_tc_can_fuse(const FfnTcMaps& maps, int max_count);
 bool ffn_pair_can_fuse(const FfnTcMaps& maps, int max_count, int H, int I);  // kind 3 on CTA pairs
 // ---- ffn_pair.cu: the many-token form on CTA pairs (bf16 stores, token tiles of 256 rows,

@@ -92,6 +92,8 @@ struct oled_ctx {
   uint32_t* d_status = nullptr;
   uint32_t* d_work = nullptr;         // control block: work-item counters of the step's FFN launches
   uint32_t* d_done = nullptr;         // control block: [kFfnWorkCounters][E] completion counters of fused FFN launches
+  uint32_t* d_ready = nullptr;        // control block: [kFfnWorkCounters][ready_words] row-copy counters of FFN launches that gather
+  size_t ready_words = 0;             // token tiles of 256 rows a launch can have: max_tokens * K / 256 + E
   int32_t* d_seg = nullptr;           // control block, last: [kPermuteSegments][E] per-segment counts of many-token steps
   int work_next = 0;                  // next unused counter of the current layer execution
   bool ctrl_dirty = true;             // both control blocks must be cleared before the next gate launch
@@ -118,6 +120,7 @@ struct oled_ctx {
   bool timeline_on = false;    // OLED_OPT_TIMELINE
   bool fp8_direct = true;      // OLED_OPT_FP8_DIRECT
   bool l2_prefetch = true;     // OLED_OPT_L2_PREFETCH
+  bool gather_in_ffn = true;   // OLED_OPT_GATHER_IN_FFN
   cudaEvent_t ev_layer_done = nullptr;  // recorded behind a layer's last kernel (L2 prefetch of the next layer)
   StepTimeline* d_timeline = nullptr;
   bool y_bf16 = false;         // this step keeps the per-assignment outputs in bf16 (many tokens)
@@ -159,7 +162,8 @@ void select_ctrl(oled_ctx* ctx, int sel) {
   ctx->d_counts = reinterpret_cast<int32_t*>(b + E * sizeof(unsigned long long));
   ctx->d_work = reinterpret_cast<uint32_t*>(b + E * (sizeof(unsigned long long) + sizeof(int32_t)));
   ctx->d_done = ctx->d_work + kFfnWorkCounters;
-  ctx->d_seg = reinterpret_cast<int32_t*>(ctx->d_done + (size_t)kFfnWorkCounters * E);
+  ctx->d_ready = ctx->d_done + (size_t)kFfnWorkCounters * E;
+  ctx->d_seg = reinterpret_cast<int32_t*>(ctx->d_ready + (size_t)kFfnWorkCounters * ctx->ready_words);
 }
 
 template <typename T>
@@ -375,6 +379,9 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
   }
   if (grp.n <= 0) return OLED_OK;
   const int H = ctx->shape.hidden, I = ctx->shape.intermediate;
+  // (no gathered copy of the token rows exists: every launch of the step takes the token tile of 256
+  // rows, whatever its experts' counts, and gathers its own rows)
+  if (ctx->maps.token_source.perm != nullptr) max_count = std::max(max_count, 129);
   if (ctx->ffn_impl == 1) {
     if (before_down) OLED_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, before_down, 0));
     launch_ffn_simple(ctx->stream, grp, ctx->pool, ctx->slot_bytes, ctx->d_offsets, ctx->d_xp, ctx->d_hbuf,
@@ -399,10 +406,13 @@ int run_ffn_launches(oled_ctx* ctx, const FfnGroup& grp, int max_count, const in
       const int li = ctx->work_next % kFfnWorkCounters;
       uint32_t* work = ctx->d_work + li;
       uint32_t* done = ctx->d_done + (size_t)li * ctx->shape.n_experts;
+      uint32_t* ready = ctx->d_ready + (size_t)li * ctx->ready_words;
       if (ctx->work_next >= kFfnWorkCounters) {
         OLED_CUDA(ctx, cudaMemsetAsync(work, 0, sizeof(uint32_t), ctx->stream));
         OLED_CUDA(ctx, cudaMemsetAsync(done, 0, (size_t)ctx->shape.n_experts * sizeof(uint32_t), ctx->stream));
+        OLED_CUDA(ctx, cudaMemsetAsync(ready, 0, ctx->ready_words * sizeof(uint32_t), ctx->stream));
       }
+      ctx->maps.token_source.ready = ready;
       ctx->work_next += 1;
       const int rc = launch_ffn_tc(ctx->stream, ctx->maps, grp, max_count, kind, host_counts, ctx->d_offsets,
                                    ctx->d_hbuf, ctx->d_y, ctx->y_bf16 ? 1 : 0, H, I, ctx->n_sms, ctx->d_status, work,
@@ -557,8 +567,10 @@ int oled_create(const oled_model_shape* shape, const int32_t* cache_capacity, vo
 
   const size_t T = (size_t)s.max_tokens, E = (size_t)s.n_experts, K = (size_t)s.top_k;
   const size_t H = (size_t)s.hidden, I = (size_t)s.intermediate;
+  ctx->ready_words = T * K / 256 + E;
   ctx->ctrl_bytes = E * (sizeof(unsigned long long) + sizeof(int32_t)) + kFfnWorkCounters * sizeof(uint32_t) +
-                    (size_t)kFfnWorkCounters * E * sizeof(uint32_t) + (size_t)kPermuteSegments * E * sizeof(int32_t);
+                    (size_t)kFfnWorkCounters * (E + ctx->ready_words) * sizeof(uint32_t) +
+                    (size_t)kPermuteSegments * E * sizeof(int32_t);
   ctx->ctrl_bytes = (ctx->ctrl_bytes + 15) / 16 * 16;
   if ((rc = dev_alloc(ctx, &ctx->pool, (size_t)ctx->n_slots * ctx->slot_bytes)) != OLED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_ctrl[0], 2 * ctx->ctrl_bytes)) != OLED_OK) return fail(rc);
@@ -752,6 +764,16 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
                  ctx->d_logits, ctx->d_ids, ctx->d_gate, ctx->d_counts, ctx->d_scores, prev, tl, seg_counts, seg_tokens);
   }
   const bool fuse_gather = (size_t)T * K <= 4096;  // few rows per expert: one CTA per expert copies them
+  // Many rows per expert (every FFN launch of the step on CTA pairs, token tiles of 256 rows): no
+  // gather kernel, each gate/up launch copies its experts' token rows while its first items run.
+  const bool gather_in_ffn = !fuse_gather && ctx->gather_in_ffn && ctx->ffn_impl == 0 &&
+                             std::min<size_t>(T, 2 * (((size_t)T * K + E - 1) / E)) > 128 &&
+                             (reinterpret_cast<uintptr_t>(hidden) & 15u) == 0 &&  // (bulk copies of whole rows)
+                             ffn_tc_token_source_usable(ctx->maps, H, ctx->shape.intermediate);
+  if (gather_in_ffn)
+    ffn_tc_set_token_source(&ctx->maps, static_cast<const uint16_t*>(hidden), T, ctx->d_perm, K, ctx->d_xp);
+  else
+    ffn_tc_clear_token_source(&ctx->maps);
   NvtxRange nv_perm(ctx, "oled.step.2_permutation_counts");
   {
     ProfScope ps(ctx, OLED_KERNEL_PERMUTE, (uint64_t)T * K * 12 + (fuse_gather ? (uint64_t)T * K * H * 4 : 0), 0);
@@ -761,11 +783,11 @@ static int step_impl(oled_ctx* ctx, int32_t layer, const void* hidden, const flo
                    static_cast<const uint16_t*>(hidden), fuse_gather ? ctx->d_xp : nullptr, H, tl, ctx->step_split,
                    seg_counts, seg_tokens);
   }
-  if (!fuse_gather) {
+  if (!fuse_gather && !gather_in_ffn) {
     ProfScope ps(ctx, OLED_KERNEL_GATHER, (uint64_t)T * K * H * 4, 0);
     launch_gather(st, static_cast<const uint16_t*>(hidden), ctx->d_perm, T, H, K, ctx->d_xp);
   }
-  ctx->launches += fuse_gather ? 2 : 3;
+  ctx->launches += fuse_gather || gather_in_ffn ? 2 : 3;
   nv_perm.end();
   if (ctx->corrupt_perm) {
     launch_corrupt_perm(st, ctx->d_perm, T * K);
@@ -1228,6 +1250,9 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       return OLED_OK;
     case OLED_OPT_FFN_PAIRS:
       ctx->maps.use_pairs = value != 0;
+      return OLED_OK;
+    case OLED_OPT_GATHER_IN_FFN:
+      ctx->gather_in_ffn = value != 0;
       return OLED_OK;
     default:
       return OLED_ERR_INVALID_ARG;

@@ -194,6 +194,37 @@ def test_cta_pair_ffn_form_many_tokens(n):
             run.ctx.reset_cache()
         assert np.linalg.norm(outs[0] - outs[1]) <= 1e-3 * np.linalg.norm(outs[1])
         assert np.array_equal(outs[0], outs[2])   # the same items in the same arithmetic, one launch or two
+        # token rows gathered by the FFN launch itself (the default where it applies, n = 2100
+        # here) or by a gather kernel in front: the same operands
+        for fuse in (1, 0):
+            run.ctx.set_option(binding.OPT_FFN_PAIRS, 1)
+            run.ctx.set_option(binding.OPT_FUSE_FFN, fuse)
+            run.ctx.set_option(binding.OPT_GATHER_IN_FFN, 0)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, bits_to_dev(h_bits, run.device), c, out)
+            _check_step(run, 0, n, out, ref)
+            assert np.array_equal(outs[0], out.float().cpu().numpy().astype(np.float64))
+            run.ctx.reset_cache()
+    finally:
+        run.close()
+
+
+def test_gather_in_ffn_with_cache_misses():
+    """A many-token step with misses: the launches over the fetched experts gather their own token rows
+    as well (token tile 256 whatever their counts), ragged tiles included."""
+    from paper_2609_33385_b200.runner import bits_to_dev
+    n = 2100
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    run = _runner(w, capacity=[2], max_tokens=n)
+    ora = _oracle_for(run, [2])
+    try:
+        for seed in (9, 10):
+            h_bits, conf = synth.flat_tokens(w, n, seed)
+            ref = ora.denoise_step(0, h_bits, conf)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device), out)
+            _check_step(run, 0, n, out, ref)
+        assert run.ctx.stats().misses > 0
     finally:
         run.close()
 
