@@ -111,15 +111,23 @@ combine_bf16_wide_kernel(const uint16_t* __restrict__ y, const float* __restrict
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    for (int j = 0; j < K; ++j) {  // rank order
-      const uint4 p = *reinterpret_cast<const uint4*>(y + (size_t)s_r[j] * H + h);
-      const float g = s_g[j];
-      const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+    // four assignments' pieces are requested together, then accumulated in rank order
+    for (int j0 = 0; j0 < K; j0 += 4) {
+      uint4 p[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        acc[2 * i] = fmaf(g, __uint_as_float(w[i] << 16), acc[2 * i]);
-        acc[2 * i + 1] = fmaf(g, __uint_as_float(w[i] & 0xffff0000u), acc[2 * i + 1]);
-      }
+      for (int jj = 0; jj < 4; ++jj)
+        if (j0 + jj < K) p[jj] = *reinterpret_cast<const uint4*>(y + (size_t)s_r[j0 + jj] * H + h);
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj)
+        if (j0 + jj < K) {
+          const float g = s_g[j0 + jj];
+          const uint32_t w[4] = {p[jj].x, p[jj].y, p[jj].z, p[jj].w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            acc[2 * i] = fmaf(g, __uint_as_float(w[i] << 16), acc[2 * i]);
+            acc[2 * i + 1] = fmaf(g, __uint_as_float(w[i] & 0xffff0000u), acc[2 * i + 1]);
+          }
+        }
     }
     uint32_t o[4];
     __nv_bfloat162 ob[4];

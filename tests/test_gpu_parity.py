@@ -209,22 +209,37 @@ def test_cta_pair_ffn_form_many_tokens(n):
         run.close()
 
 
-def test_gather_in_ffn_with_cache_misses():
+@pytest.mark.parametrize("hidden", [512, 4608])
+def test_gather_in_ffn_with_cache_misses(hidden):
     """A many-token step with misses: the launches over the fetched experts gather their own token rows
-    as well (token tile 256 whatever their counts), ragged tiles included."""
-    from paper_2609_33385_b200.runner import bits_to_dev
+    as well (token tile 256 whatever their counts), ragged tiles included.  hidden 4608: a row is moved
+    as two pieces (8192 + 1024 bytes)."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
     n = 2100
-    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=512, intermediate=256)
+    # (weights scaled with the contraction length, so that the outputs stay of order one)
+    w = synth.tiny(n_layers=1, n_experts=4, top_k=2, hidden=hidden, intermediate=256,
+                   weight_std=0.05 * (512 / hidden) ** 0.5)
     run = _runner(w, capacity=[2], max_tokens=n)
     ora = _oracle_for(run, [2])
     try:
+        got = []
         for seed in (9, 10):
             h_bits, conf = synth.flat_tokens(w, n, seed)
             ref = ora.denoise_step(0, h_bits, conf)
             out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
             run.step(0, bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device), out)
             _check_step(run, 0, n, out, ref)
+            got.append(dev_to_bits(out).copy())
         assert run.ctx.stats().misses > 0
+        # the same two steps with a gather kernel in front: the same bits
+        run.ctx.reset_cache()
+        run.ctx.set_option(binding.OPT_GATHER_IN_FFN, 0)
+        for i, seed in enumerate((9, 10)):
+            h_bits, conf = synth.flat_tokens(w, n, seed)
+            out = torch.empty((n, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(0, bits_to_dev(h_bits, run.device), torch.from_numpy(conf).to(run.device), out)
+            assert np.array_equal(got[i], dev_to_bits(out))
     finally:
         run.close()
 
