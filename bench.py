@@ -48,6 +48,9 @@ NCU_TRAFFIC_RATIO = {
     # profiles/ffn_pair_kernel_cfg5_4096_tokens.md: 4096 tokens, H 4096, I 1536
     ("ffn_gate_up", "many_tokens"): (1944.0 + 100.7) / 1979.7,
     ("ffn_down", "many_tokens"): (909.4 + 264.2) / 1174.4,
+    # the one-launch form on CTA pairs, which also gathers its token rows (268 MB read and written
+    # on top of the projections' algorithmic bytes)
+    ("ffn_fused", "many_tokens"): (3180.0 + 631.6) / 3154.1,
 }
 
 
