@@ -256,7 +256,8 @@ int oled_residual_add(oled_ctx* ctx, const void* x, const void* r, void* y, size
  * execution had no miss runs its gate and permutation kernels (the HBM is idle then), the weights
  * of the first experts its FFN will stream - the residents activated at that previous execution,
  * adjacent iterations activating mostly the same experts (Sec. 3.3) - are called into L2 from
- * the side stream; 0 = off. */
+ * the side stream, provided that execution streamed at least 320 MB of experts (shorter streams
+ * were measured to lose); 2 = the same without that condition; 0 = off. */
 #define OLED_OPT_L2_PREFETCH 16
 /* OLED_OPT_GATHER_IN_FFN: 1 (default) = a many-token step whose FFN launches all run on CTA pairs
  * has no gather kernel: each gate/up launch copies its own experts' token rows into sorted order

@@ -119,7 +119,7 @@ struct oled_ctx {
   int ffn_impl = 0;
   bool timeline_on = false;    // OLED_OPT_TIMELINE
   bool fp8_direct = true;      // OLED_OPT_FP8_DIRECT
-  bool l2_prefetch = true;     // OLED_OPT_L2_PREFETCH
+  int l2_prefetch = 1;         // OLED_OPT_L2_PREFETCH (2: whatever the length of the expert stream)
   bool gather_in_ffn = true;   // OLED_OPT_GATHER_IN_FFN
   cudaEvent_t ev_layer_done = nullptr;  // recorded behind a layer's last kernel (L2 prefetch of the next layer)
   StepTimeline* d_timeline = nullptr;
@@ -1017,7 +1017,7 @@ static int prefetch_next_layer(oled_ctx* ctx, int32_t next) {
   size_t stream_bytes = 0;
   for (int32_t e = 0; e < ctx->shape.n_experts; ++e)
     if (N.last_counts[e] > 0) stream_bytes += (size_t)3 * ctx->shape.hidden * ctx->shape.intermediate * esz;
-  if (stream_bytes < 5 * kPrefetchBytes) return OLED_OK;
+  if (stream_bytes < 5 * kPrefetchBytes && ctx->l2_prefetch != 2) return OLED_OK;
   SlotList list;
   list.n = 0;
   const int cap = (int)std::max<size_t>(1, kPrefetchBytes / lead_bytes);
@@ -1246,7 +1246,7 @@ int oled_set_option(oled_ctx* ctx, int32_t option, int64_t value) {
       ctx->fp8_direct = value != 0;
       return OLED_OK;
     case OLED_OPT_L2_PREFETCH:
-      ctx->l2_prefetch = value != 0;
+      ctx->l2_prefetch = value;
       return OLED_OK;
     case OLED_OPT_FFN_PAIRS:
       ctx->maps.use_pairs = value != 0;

@@ -295,6 +295,33 @@ def test_iteration_entry_points_match_layer_by_layer_steps():
             r.close()
 
 
+def test_l2_prefetch_across_layers_changes_no_bit():
+    """OLED_OPT_L2_PREFETCH only calls weights into L2: with all experts resident (no miss, so the
+    prefetch kernel runs behind every layer; value 2 lifts the stream-length condition the tiny
+    shape would not meet) the iterations' outputs and statistics equal those with it off."""
+    from paper_2609_33385_b200 import binding
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=3, n_experts=8, top_k=2)
+    runs = [_runner(w, capacity=[8, 8, 8]) for _ in range(2)]
+    try:
+        runs[0].ctx.set_option(binding.OPT_L2_PREFETCH, 2)
+        runs[1].ctx.set_option(binding.OPT_L2_PREFETCH, 0)
+        dev = runs[0].device
+        for _, _, h_bits, conf in synth.denoise_inputs(w):
+            x, c = bits_to_dev(h_bits, dev), torch.from_numpy(conf).to(dev)
+            ys = []
+            for r in runs:
+                y = torch.empty((w.tokens, w.hidden), dtype=torch.bfloat16, device=dev)
+                r.ctx.denoise_iteration(x.data_ptr(), c.data_ptr(), w.tokens, y.data_ptr())
+                ys.append(dev_to_bits(y).copy())
+            assert np.array_equal(ys[0], ys[1])
+        assert runs[0].ctx.stats() == runs[1].ctx.stats()
+        assert runs[0].ctx.launch_count() > runs[1].ctx.launch_count()   # the prefetch kernel did run
+    finally:
+        for r in runs:
+            r.close()
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
     w = synth.tiny(n_layers=1)
