@@ -14,6 +14,8 @@
 //           epilogue hbuf[n, f] = bf16(silu(D_gate) * D_up)
 //   KIND 2: output rows c0 + 256 r .. + 255 for CTA r (two row blocks of Wd), epilogue y[n, c] = D
 // No TMA multicast: every CTA loads what lies in its own shared memory.
+// 19 warps per CTA: 16 epilogue warps, the TMA thread's, the MMA thread's, and one whose first thread
+// gathers token rows when the launch is asked to (PairTokens below); its lanes are idle otherwise.
 //
 // Protocol per pipeline stage (barriers at the same shared-memory offsets in both CTAs):
 //   full[s]   lives in the FIRST CTA: its TMA thread announces the bytes of both CTAs' copies
