@@ -175,6 +175,19 @@ def test_config5_shape_4096_tokens_zipf_bias():
         run.close()
 
 
+def test_config5_shape_half_residency():
+    """The same shape with room for 32 of the 64 experts: every step fetches experts, and the launches
+    over the fetched ones run on CTA pairs and gather their own token rows like the launch over the
+    residents (token tile 256 whatever an expert's count)."""
+    w = synth.config(4, blocks=2, residency=0.5)
+    run, ora = _setup(w)
+    try:
+        _replay(run, ora, 2, sample_layers={0}, min_tokens=128, rng=np.random.default_rng(5))
+        assert run.ctx.stats(0).misses > 0
+    finally:
+        run.close()
+
+
 @pytest.mark.parametrize("block_len", [1, 4])
 def test_config2_shape_short_blocks(block_len):
     """Block lengths 1 and 4 at the full layer shape (hidden 2048, 64 experts top-8, I 1024): most
