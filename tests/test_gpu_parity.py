@@ -145,6 +145,41 @@ def test_ragged_token_counts(n_tokens):
         run.close()
 
 
+@pytest.mark.parametrize("n_experts,n_tokens", [(64, 5), (64, 200), (64, 310), (128, 33), (128, 256), (128, 300)])
+def test_gate_with_64_and_128_experts(n_experts, n_tokens):
+    """The expert counts of the benchmark configurations at a small hidden size, with one, two and four
+    tokens per CTA of the few-token gate kernel (several passes over the experts per warp): logits,
+    ids, gate scores bit for bit; and the two layers as one iteration, whose second gate kernel
+    carries the first layer's combine."""
+    from paper_2609_33385_b200.runner import bits_to_dev, dev_to_bits
+    w = synth.tiny(n_layers=2, n_experts=n_experts, top_k=8, hidden=768, intermediate=128)
+    run = _runner(w, capacity=[n_experts // 2, n_experts // 2], max_tokens=n_tokens)
+    ora = _oracle_for(run, [n_experts // 2, n_experts // 2])
+    try:
+        h_bits, conf = synth.flat_tokens(w, n_tokens, 3)
+        c = torch.from_numpy(conf).to(run.device)
+        x = bits_to_dev(h_bits, run.device)
+        for layer in range(2):
+            out = torch.empty((n_tokens, w.hidden), dtype=torch.bfloat16, device=run.device)
+            run.step(layer, x, c, out)
+            ref = ora.denoise_step(layer, dev_to_bits(x), conf)
+            _check_step(run, layer, n_tokens, out, ref)
+            nxt = torch.empty_like(out)
+            run.ctx.residual_add(x.data_ptr(), out.data_ptr(), nxt.data_ptr(), x.numel())
+            x = nxt
+        # the same two layers as one iteration (the second gate kernel carries the first layer's combine)
+        run2 = _runner(w, capacity=[n_experts // 2, n_experts // 2], max_tokens=n_tokens)
+        try:
+            y = torch.empty((n_tokens, w.hidden), dtype=torch.bfloat16, device=run.device)
+            x0 = bits_to_dev(h_bits, run.device)
+            run2.ctx.denoise_iteration(x0.data_ptr(), c.data_ptr(), n_tokens, y.data_ptr())
+            assert np.array_equal(dev_to_bits(y), dev_to_bits(x))
+        finally:
+            run2.close()
+    finally:
+        run.close()
+
+
 @pytest.mark.parametrize("n", [700, 2100])
 def test_many_tokens_per_expert_multi_tile(n):
     """More than 256 rows for one expert: several N tiles per expert in both FFN kernels; the
